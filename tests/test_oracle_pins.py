@@ -1,0 +1,317 @@
+"""Pins of the fp64 oracle against things other than itself (CPU only).
+
+Each check compares the oracle with an independent statement of the same quantity:
+a hand-worked example, a dense N x N brute-force form written with numpy matrix
+products, a library routine (torch SDPA, torch elu), a closed form, or an invariant
+that a dropped term / wrong sign / wrong index / transposed operand would break.
+"""
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def rnd(shape, seed, scale=1.0):
+    return np.random.default_rng(seed).standard_normal(shape) * scale
+
+
+# ----------------------------------------------------------------------------- brute force
+def brute_window(q, k, v, w, scale):
+    """Full N x N logits, explicit band mask (-inf outside i-w < j <= i), row softmax."""
+    B, H, N, d = q.shape
+    i = np.arange(N)[:, None]
+    j = np.arange(N)[None, :]
+    allowed = (j <= i) & (j > i - w)
+    out = np.empty_like(q)
+    for b in range(B):
+        for h in range(H):
+            logits = (q[b, h] @ k[b, h].T) * scale
+            logits = np.where(allowed, logits, -np.inf)
+            logits = logits - logits.max(axis=1, keepdims=True)
+            p = np.exp(logits)
+            p = p / p.sum(axis=1, keepdims=True)
+            out[b, h] = p @ v[b, h]
+    return out
+
+
+def np_phi(x):
+    return np.where(x > 0, x + 1.0, np.exp(np.minimum(x, 0.0)))
+
+
+def brute_linear(q, k, v):
+    """Quadratic masked form ((phi(Q) phi(K)^T) * M) V / rowsum."""
+    B, H, N, d = q.shape
+    M = np.tril(np.ones((N, N)))
+    out = np.empty_like(q)
+    for b in range(B):
+        for h in range(H):
+            A = (np_phi(q[b, h]) @ np_phi(k[b, h]).T) * M
+            out[b, h] = (A @ v[b, h]) / A.sum(axis=1, keepdims=True)
+    return out
+
+
+# ----------------------------------------------------------------------------- golden
+def _golden():
+    with open(os.path.join(HERE, "golden", "hand_worked.json")) as f:
+        return json.load(f)
+
+
+def test_golden_window_hand_worked():
+    g = _golden()["window"]
+    q = np.array(g["q"])[None, None]
+    k = np.log(np.array(g["k_log_of"]))[None, None]
+    v = np.array(g["v"])[None, None]
+    for w, exp in g["expected"].items():
+        o = oracle.window_attn(q, k, v, int(w), scale=g["scale"])
+        np.testing.assert_allclose(o[0, 0], np.array(exp), rtol=0, atol=1e-14)
+
+
+def test_golden_linear_hand_worked():
+    g = _golden()["linear"]
+    fix = lambda rows: np.array([[(-math.log(2.0) if x == "-ln2" else x) for x in r] for r in rows])
+    q, k, v = fix(g["q"])[None, None], fix(g["k"])[None, None], fix(g["v"])[None, None]
+    S = np.zeros((1, 1, 2, 2))
+    z = np.zeros((1, 1, 2))
+    o = oracle.causal_linear_attn(q, k, v, S, z)
+    np.testing.assert_allclose(o[0, 0], np.array(g["expected"]), atol=1e-14)
+    np.testing.assert_allclose(S[0, 0], np.array(g["expected_S"]), atol=1e-14)
+    np.testing.assert_allclose(z[0, 0], np.array(g["expected_z"]), atol=1e-14)
+
+
+# ----------------------------------------------------------------------------- phi
+def test_phi_matches_library_elu_plus_one():
+    x = np.concatenate([np.linspace(-30, 30, 2001), [0.0, -0.0, 1e-300, -1e-300]])
+    ref = (torch.nn.functional.elu(torch.from_numpy(x)) + 1.0).numpy()
+    # the library forms (exp(x) - 1) + 1, which carries one rounding at magnitude 1
+    np.testing.assert_allclose(oracle.phi(x), ref, rtol=1e-15, atol=2.3e-16)
+
+
+def test_phi_properties():
+    assert oracle.phi(np.array([0.0]))[0] == 1.0
+    x = np.linspace(-20, 20, 4001)
+    y = oracle.phi(x)
+    assert (y > 0).all()
+    assert (np.diff(y) > 0).all()
+    np.testing.assert_allclose(y[x > 0], x[x > 0] + 1.0, rtol=1e-15)
+    np.testing.assert_allclose(y[x <= 0], np.exp(x[x <= 0]), rtol=1e-15)
+
+
+# ----------------------------------------------------------------------------- window
+@pytest.mark.parametrize("N,d", [(1, 4), (7, 3), (33, 8), (64, 16)])
+def test_window_equals_bruteforce_band_mask_all_w(N, d):
+    q, k, v = rnd((2, 2, N, d), 1), rnd((2, 2, N, d), 2), rnd((2, 2, N, d), 3)
+    for w in range(1, N + 3):
+        o = oracle.window_attn(q, k, v, w, scale=0.37)
+        np.testing.assert_allclose(o, brute_window(q, k, v, w, 0.37), rtol=1e-12, atol=1e-13)
+
+
+@pytest.mark.parametrize("w", [48, 49, 1000])
+def test_window_ge_N_is_full_causal_attention_library(w):
+    N, d = 48, 16
+    q, k, v = rnd((2, 3, N, d), 4), rnd((2, 3, N, d), 5), rnd((2, 3, N, d), 6)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v), is_causal=True).numpy()
+    o = oracle.window_attn(q, k, v, w)  # default scale 1/sqrt(d), same as the library's
+    np.testing.assert_allclose(o, ref, rtol=1e-12, atol=1e-13)
+
+
+def test_window_banded_matches_library_with_explicit_mask():
+    N, d, w = 40, 8, 7
+    q, k, v = rnd((1, 2, N, d), 7), rnd((1, 2, N, d), 8), rnd((1, 2, N, d), 9)
+    i = torch.arange(N)[:, None]
+    j = torch.arange(N)[None, :]
+    mask = (j <= i) & (j > i - w)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v), attn_mask=mask).numpy()
+    np.testing.assert_allclose(oracle.window_attn(q, k, v, w), ref, rtol=1e-12, atol=1e-13)
+
+
+def test_window_one_returns_values():
+    q, k, v = rnd((1, 2, 19, 5), 10), rnd((1, 2, 19, 5), 11), rnd((1, 2, 19, 5), 12)
+    assert np.array_equal(oracle.window_attn(q, k, v, 1), v)
+
+
+@pytest.mark.parametrize("zero", ["q", "k", "scale"])
+def test_window_uniform_logits_give_sliding_mean(zero):
+    N, d, w = 37, 6, 5
+    q, k, v = rnd((1, 1, N, d), 13), rnd((1, 1, N, d), 14), rnd((1, 1, N, d), 15)
+    scale = None
+    if zero == "q":
+        q = np.zeros_like(q)
+    elif zero == "k":
+        k = np.zeros_like(k)
+    else:
+        scale = 0.0
+    o = oracle.window_attn(q, k, v, w, scale=scale)
+    for i in range(N):
+        lo = max(0, i - w + 1)
+        np.testing.assert_allclose(o[0, 0, i], v[0, 0, lo:i + 1].mean(axis=0), rtol=1e-13, atol=1e-14)
+
+
+def test_window_constant_values_and_key_shift_invariance():
+    N, d, w = 50, 8, 9
+    q, k, v = rnd((1, 2, N, d), 16), rnd((1, 2, N, d), 17), rnd((1, 2, N, d), 18)
+    c = rnd((d,), 19)
+    vc = np.broadcast_to(c, v.shape).copy()
+    np.testing.assert_allclose(oracle.window_attn(q, k, vc, w), vc, rtol=1e-13)
+    u = rnd((d,), 20)
+    np.testing.assert_allclose(oracle.window_attn(q, k + u, v, w), oracle.window_attn(q, k, v, w),
+                               rtol=1e-10, atol=1e-12)
+
+
+def test_window_row_depends_only_on_its_window():
+    N, d, w = 40, 4, 6
+    q, k, v = rnd((1, 1, N, d), 21), rnd((1, 1, N, d), 22), rnd((1, 1, N, d), 23)
+    base = oracle.window_attn(q, k, v, w)
+    i = 20
+    for j in range(N):
+        k2, v2 = k.copy(), v.copy()
+        k2[0, 0, j] += 1.0
+        v2[0, 0, j] -= 2.0
+        changed = np.abs(oracle.window_attn(q, k2, v2, w)[0, 0, i] - base[0, 0, i]).max() > 1e-9
+        assert changed == (i - w < j <= i), (i, j)
+
+
+def test_window_needle_at_window_edge():
+    # One key with a huge logit: visible to row i exactly while it is inside the window.
+    N, d, w = 30, 4, 8
+    q = np.zeros((1, 1, N, d)); q[..., 0] = 1.0
+    k = np.zeros((1, 1, N, d)); k[0, 0, 5, 0] = 50.0
+    v = rnd((1, 1, N, d), 24)
+    o = oracle.window_attn(q, k, v, w, scale=1.0)
+    for i in range(N):
+        lo = max(0, i - w + 1)
+        if lo <= 5 <= i:
+            np.testing.assert_allclose(o[0, 0, i], v[0, 0, 5], atol=1e-12)
+        else:
+            np.testing.assert_allclose(o[0, 0, i], v[0, 0, lo:i + 1].mean(axis=0), atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- linear
+@pytest.mark.parametrize("N,d", [(1, 3), (9, 2), (40, 8), (64, 16)])
+def test_linear_prefix_sum_equals_quadratic_masked_form(N, d):
+    q, k, v = rnd((2, 2, N, d), 30), rnd((2, 2, N, d), 31), rnd((2, 2, N, d), 32)
+    np.testing.assert_allclose(oracle.causal_linear_attn(q, k, v), brute_linear(q, k, v),
+                               rtol=1e-12, atol=1e-13)
+
+
+def test_linear_first_row_is_first_value_and_K0_gives_cumulative_mean():
+    N, d = 25, 5
+    q, k, v = rnd((1, 2, N, d), 33), rnd((1, 2, N, d), 34), rnd((1, 2, N, d), 35)
+    o = oracle.causal_linear_attn(q, k, v)
+    np.testing.assert_allclose(o[:, :, 0], v[:, :, 0], rtol=1e-14)
+    o = oracle.causal_linear_attn(q, np.zeros_like(k), v)  # phi(0) = 1 -> plain running mean
+    cm = np.cumsum(v, axis=2) / np.arange(1, N + 1)[None, None, :, None]
+    np.testing.assert_allclose(o, cm, rtol=1e-13, atol=1e-14)
+
+
+def test_linear_constant_values_and_causality():
+    N, d = 30, 6
+    q, k, v = rnd((1, 1, N, d), 36), rnd((1, 1, N, d), 37), rnd((1, 1, N, d), 38)
+    c = rnd((d,), 39)
+    vc = np.broadcast_to(c, v.shape).copy()
+    np.testing.assert_allclose(oracle.causal_linear_attn(q, k, vc), vc, rtol=1e-13)
+    base = oracle.causal_linear_attn(q, k, v)
+    i = 12
+    for j in range(N):
+        k2, v2 = k.copy(), v.copy()
+        k2[0, 0, j] += 0.5
+        v2[0, 0, j] += 1.0
+        changed = np.abs(oracle.causal_linear_attn(q, k2, v2)[0, 0, i] - base[0, 0, i]).max() > 1e-9
+        assert changed == (j <= i)
+
+
+def test_linear_state_is_sum_of_outer_products_and_resumes():
+    N, d = 21, 4
+    q, k, v = rnd((1, 2, N, d), 40), rnd((1, 2, N, d), 41), rnd((1, 2, N, d), 42)
+    S = np.zeros((1, 2, d, d)); z = np.zeros((1, 2, d))
+    full = oracle.causal_linear_attn(q, k, v, S, z)
+    for h in range(2):
+        pk = np_phi(k[0, h])
+        np.testing.assert_allclose(S[0, h], pk.T @ v[0, h], rtol=1e-13)  # S[a][c] = sum_i phi(k_i)[a] v_i[c]
+        np.testing.assert_allclose(z[0, h], pk.sum(axis=0), rtol=1e-13)
+    # Splitting the sequence and carrying (S, z) gives the same rows.
+    S2 = np.zeros_like(S); z2 = np.zeros_like(z)
+    a = oracle.causal_linear_attn(q[:, :, :8], k[:, :, :8], v[:, :, :8], S2, z2)
+    b = oracle.causal_linear_attn(q[:, :, 8:], k[:, :, 8:], v[:, :, 8:], S2, z2)
+    np.testing.assert_allclose(np.concatenate([a, b], axis=2), full, rtol=1e-12)
+    np.testing.assert_allclose(S2, S, rtol=1e-13)
+
+
+def test_linear_differs_from_contract_before_cumsum_order():
+    # Contracting with phi(q_j) before the cumulative sum (the order in which the paper's
+    # PyTorch listing is printed) is a different, non-attention quantity; Algorithm 1 wins.
+    N, d = 12, 3
+    q, k, v = rnd((1, 1, N, d), 43), rnd((1, 1, N, d), 44), rnd((1, 1, N, d), 45)
+    pq, pk = np_phi(q[0, 0]), np_phi(k[0, 0])
+    num = np.cumsum(np.einsum("na,na,nc->nc", pq, pk, v[0, 0]), axis=0)
+    den = np.cumsum(np.einsum("na,na->n", pq, pk), axis=0)[:, None]
+    printed = num / den
+    o = oracle.causal_linear_attn(q, k, v)[0, 0]
+    assert np.abs(printed - o).max() > 1e-3
+    # ... while cumsum-then-contract is Algorithm 1 exactly.
+    A = np.cumsum(np.einsum("na,nc->nac", pk, v[0, 0]), axis=0)
+    Z = np.cumsum(pk, axis=0)
+    np.testing.assert_allclose(np.einsum("na,nac->nc", pq, A) / np.einsum("na,na->n", pq, Z)[:, None],
+                               o, rtol=1e-12)
+
+
+# ----------------------------------------------------------------------------- hybrid
+def test_default_head_split():
+    assert [oracle.default_h_sparse(H) for H in (2, 12, 16, 32)] == [1, 2, 3, 6]
+
+
+@pytest.mark.parametrize("h0", [0, 1, 2, 4])
+def test_hybrid_is_headwise_merge(h0):
+    B, H, N, d, w = 2, 4, 23, 8, 5
+    q, k, v = rnd((B, H, N, d), 50), rnd((B, H, N, d), 51), rnd((B, H, N, d), 52)
+    o = oracle.hybrid_attn(q, k, v, w, h_sparse=h0)
+    if h0 > 0:
+        np.testing.assert_array_equal(o[:, :h0], oracle.window_attn(q[:, :h0], k[:, :h0], v[:, :h0], w))
+        np.testing.assert_allclose(o[:, :h0], brute_window(q[:, :h0], k[:, :h0], v[:, :h0], w, d ** -0.5),
+                                   rtol=1e-12, atol=1e-13)
+    if h0 < H:
+        np.testing.assert_array_equal(o[:, h0:], oracle.causal_linear_attn(q[:, h0:], k[:, h0:], v[:, h0:]))
+        np.testing.assert_allclose(o[:, h0:], brute_linear(q[:, h0:], k[:, h0:], v[:, h0:]),
+                                   rtol=1e-12, atol=1e-13)
+
+
+# ----------------------------------------------------------------------------- decode
+@pytest.mark.parametrize("w", [1, 4, 16, 40])
+def test_decode_token_by_token_equals_full_sequence_rows(w):
+    B, H, N, d, h0 = 2, 3, 33, 4, 1
+    q, k, v = rnd((B, H, N, d), 60), rnd((B, H, N, d), 61), rnd((B, H, N, d), 62)
+    full_w = brute_window(q[:, :h0], k[:, :h0], v[:, :h0], w, d ** -0.5)
+    full_l = brute_linear(q[:, h0:], k[:, h0:], v[:, h0:])
+    st = oracle.DecodeState(B, H, d, w, h0)
+    for t in range(N):
+        o = oracle.decode_step(q[:, :, t], k[:, :, t], v[:, :, t], st)
+        np.testing.assert_allclose(o[:, :h0], full_w[:, :, t], rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(o[:, h0:], full_l[:, :, t], rtol=1e-11, atol=1e-12)
+    assert st.t == N
+
+
+@pytest.mark.parametrize("N0,w", [(5, 8), (8, 8), (21, 8), (30, 7)])
+def test_prefill_export_then_decode_equals_one_long_sequence(N0, w):
+    B, H, d, h0, steps = 1, 4, 4, 2, 13
+    N = N0 + steps
+    q, k, v = rnd((B, H, N, d), 63), rnd((B, H, N, d), 64), rnd((B, H, N, d), 65)
+    ref = np.concatenate([brute_window(q[:, :h0], k[:, :h0], v[:, :h0], w, d ** -0.5),
+                          brute_linear(q[:, h0:], k[:, h0:], v[:, h0:])], axis=1)
+    o, st = oracle.hybrid_attn(q[:, :, :N0], k[:, :, :N0], v[:, :, :N0], w, h_sparse=h0, export_state=True)
+    np.testing.assert_allclose(o, ref[:, :, :N0], rtol=1e-11, atol=1e-12)
+    assert st.t == N0
+    # ring placement: token j sits in slot j mod w
+    for j in range(max(0, N0 - w), N0):
+        np.testing.assert_array_equal(st.k_cache[:, :, j % w], k[:, :h0, j])
+        np.testing.assert_array_equal(st.v_cache[:, :, j % w], v[:, :h0, j])
+    for t in range(N0, N):
+        o = oracle.decode_step(q[:, :, t], k[:, :, t], v[:, :, t], st)
+        np.testing.assert_allclose(o, ref[:, :, t], rtol=1e-11, atol=1e-12)
