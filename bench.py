@@ -1,0 +1,311 @@
+#!/usr/bin/env python
+"""Benchmark of the hybrid attention layer on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+A step is one gformer_hybrid_attn call (all heads: windowed + linear, merged) on one batch of
+synthetic Q, K, V.  Default workload: the long-sequence layer B=1, H=32, N=32768, d=128,
+w=512, bf16 (6 windowed + 26 linear heads).  Every (batch, head) pair is an independent
+unit, so with N GPUs each rank runs its own batch element (weak scaling, no collective on
+the data path); rank 0 prints one JSON line.
+
+--impl reference times the fp64 CPU oracle on the host cores, on a bounded sample of the
+same workload (the first tokens of every head); it is a deliberately slow reference.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "hybrid_attention_tokens_per_s"
+UNIT = "tokens/s"
+# oracle samples: the first tokens of every head of the workload
+CPU_BASELINE_TOKENS = 32768  # cpu_baseline leg: about 10 s of fp64 work on 8 cores at d=128
+REFERENCE_STEP_TOKENS = 4096  # --impl reference: about 1 s per step
+
+WORKLOADS = {
+    "long32k": dict(B=1, H=32, N=32768, d=128, w=512, seed=2),
+    "gpt2s": dict(B=8, H=12, N=2048, d=64, w=128, seed=1),
+    "prefill4k": dict(B=64, H=16, N=4096, d=64, w=256, seed=3),
+}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def recorded_traffic(workload):
+    """DRAM bytes per launch from the committed ncu capture, if one is recorded."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            return json.load(f).get(workload)
+    return None
+
+
+def algorithmic_bytes(c):
+    """Read Q, K, V once and write O once (bf16)."""
+    return 4 * c["B"] * c["H"] * c["N"] * c["d"] * 2
+
+
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu_index = gpu_index
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()  # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1]))
+                smax.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def oracle_sample_rate(c, sample_tokens):
+    """Times the oracle on the first `sample_tokens` tokens of every head; tokens/s."""
+    import torch
+
+    import oracle
+    from paper_2412_19829_b200 import synth
+
+    n = min(c["N"], sample_tokens)
+    q, k, v = synth.qkv(c["B"], c["H"], n, c["d"], "bf16", c["seed"])
+    a = [t.to(torch.float64).numpy() for t in (q, k, v)]
+    h0 = oracle.default_h_sparse(c["H"])
+    t0 = time.perf_counter()
+    oracle.hybrid_attn(a[0], a[1], a[2], c["w"], h_sparse=h0)
+    dt = time.perf_counter() - t0
+    return c["B"] * n / dt, dt, n, oracle.num_threads()
+
+
+def run_reference(args, c, rank):
+    if rank != 0:
+        return
+    import oracle  # noqa: F401  (CPU oracle: the reference arm of this benchmark)
+
+    for _ in range(args.warmup):
+        oracle_sample_rate(c, REFERENCE_STEP_TOKENS)
+    times = []
+    n = cores = 0
+    for _ in range(args.steps):
+        _, dt, n, cores = oracle_sample_rate(c, REFERENCE_STEP_TOKENS)
+        times.append(dt)
+    mean = sum(times) / len(times)
+    value = c["B"] * n / mean
+    sample = f"first {n} tokens of each of the {c['B'] * c['H']} heads per step, fp64, OpenMP over heads"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, **{k: c[k] for k in ("B", "H", "N", "d", "w")},
+                   "h_sparse": oracle.default_h_sparse(c["H"]), "sampled_tokens": n},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, c, rank, world, local_rank):
+    import torch
+
+    from paper_2412_19829_b200 import binding as gf
+    from paper_2412_19829_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    h0 = gf.default_h_sparse(c["H"])
+    B, H, N, d, w = c["B"], c["H"], c["N"], c["d"], c["w"]
+
+    q, k, v = synth.qkv(B, H, N, d, "bf16", c["seed"] + 1000 * rank)
+    hq, hk, hv = [t.pin_memory() for t in (q, k, v)]
+    ho = torch.empty_like(hq).pin_memory()
+    dq, dk, dv = [t.cuda() for t in (hq, hk, hv)]
+    do = torch.empty_like(dq)
+    ws = gf.Workspace()
+    stream = torch.cuda.Stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        gf.hybrid_attn(dq, dk, dv, w, h_sparse=h0, out=do, ws=ws, stream=stream)
+
+    def step_e2e():
+        with torch.cuda.stream(stream):
+            dq.copy_(hq, non_blocking=True)
+            dk.copy_(hk, non_blocking=True)
+            dv.copy_(hv, non_blocking=True)
+        step()
+        with torch.cuda.stream(stream):
+            ho.copy_(do, non_blocking=True)
+
+    def timed(fn, steps):
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        evs[0].record(stream)
+        for i in range(steps):
+            fn()
+            evs[i + 1].record(stream)
+        stream.synchronize()
+        barrier()
+        total_ms = evs[0].elapsed_time(evs[-1])
+        per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
+        return total_ms, per
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    stream.synchronize()
+    if ws.last_device_status(stream) != gf.GF_OK:
+        raise SystemExit("device-side wait timed out during warm-up")
+
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
+    n0 = gf.launch_count()
+    total_ms, per = timed(step, args.steps)
+    launches = gf.launch_count() - n0
+    if sampler:
+        clocks = sampler.stop()
+    if ws.last_device_status(stream) != gf.GF_OK:
+        raise SystemExit("device-side wait timed out during the timed region")
+
+    for _ in range(2):
+        step_e2e()
+    e2e_ms, _ = timed(step_e2e, args.steps)
+
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms = t.tolist()
+
+    if rank == 0:
+        tokens = world * B * N * args.steps
+        value = tokens / (total_ms * 1e-3)
+        e2e_value = tokens / (e2e_ms * 1e-3)
+        peak, which = measured_peaks()
+        abytes = algorithmic_bytes(c)
+        mean_launch_s = (sum(per) / len(per)) * 1e-3
+        achieved = abytes / mean_launch_s / 1e9
+        tensor_bytes = B * H * N * d * 2
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "B": B, "H": H, "N": N, "d": d, "w": w, "h_sparse": h0,
+                       "global_batch": world * B, "seq_len": N,
+                       "parallelism": "replicas only (one batch element per GPU, no collective)",
+                       "l2": "inputs larger than L2 (Q+K+V = %.0f MB per step)" % (3 * tensor_bytes / 1e6)},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "traffic": recorded_traffic(args.workload),
+                         "peak_source": which + " copy bandwidth", "algorithmic_bytes": abytes,
+                         "kernel": "gformer_hybrid_attn launch (window + linear kernels, concurrent)",
+                         "tflops_algorithmic": algorithmic_flops(c, h0) / mean_launch_s / 1e12},
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * tensor_bytes,
+                    "d2h_bytes_per_step": tensor_bytes},
+            "gpu_launches": launches,
+            "clocks": clocks,
+            "step_ms_min": min(per), "step_ms_max": max(per),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            rate, dt, n, cores = oracle_sample_rate(c, CPU_BASELINE_TOKENS)
+            line["cpu_baseline"] = {
+                "value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"first {n} tokens of each of the {B * H} heads, {dt:.1f} s of fp64 CPU work"}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def algorithmic_flops(c, h0):
+    """Flops of the method itself: 4 d per (query, key) pair in the window, 4 d^2 per linear token."""
+    B, H, N, d, w = c["B"], c["H"], c["N"], c["d"], c["w"]
+    we = min(w, N)
+    pairs = N * we - we * (we - 1) // 2
+    return B * (h0 * 4 * d * pairs + (H - h0) * 4 * N * d * d)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="long32k", choices=sorted(WORKLOADS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    c = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, c, rank)
+    else:
+        run_ours(args, c, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

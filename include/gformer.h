@@ -1,0 +1,146 @@
+/*
+ * libgformer -- hybrid attention forward pass (GFormer) for NVIDIA B200 (sm_100a).
+ *
+ * The layer splits the H heads of Q, K, V into two groups (Sec. III-A): heads
+ * [0, h_sparse) run causal windowed softmax attention, heads [h_sparse, H) run
+ * causal linear attention; each head writes its own slot of the output.
+ *
+ * Conventions common to every entry point
+ *   - q, k, v, o and every state buffer are DEVICE pointers owned by the caller.  The
+ *     library never allocates, frees or keeps them.  Pointers must be 16-byte aligned.
+ *   - Logical tensor shape is [B, H, N, d]; `layout` says how it is stored:
+ *     GF_BHND = contiguous [B, H, N, d]; GF_BNHD = contiguous [B, N, H, d] (the order
+ *     the paper writes, Sec. III-A).  d is 64 or 128.
+ *   - dtype is the storage type of q, k, v, o and of the KV ring (GF_F32 or GF_BF16);
+ *     all accumulation is fp32; the linear state S, z is always fp32.
+ *   - Calls enqueue work on `cuda_stream` (a cudaStream_t cast to void*, NULL = the
+ *     legacy default stream) and return without synchronising.
+ *   - The return value is a gf_status.  Argument errors are found on the host before
+ *     anything is launched and leave every buffer untouched.  Nothing throws or aborts.
+ *   - `ws` is caller-provided device scratch of at least gformer_workspace_bytes(...)
+ *     bytes, 256-byte aligned; the tensor-core (bf16) kernels keep a device status word
+ *     there.  The library clears what it needs inside the call, so ws may hold anything
+ *     on entry, but two calls that run concurrently must not share one ws.
+ *   - o must not alias an input.
+ */
+#ifndef GFORMER_H_
+#define GFORMER_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GF_OK = 0,
+  GF_ERR_INVALID_ARG = 1, /* null/misaligned pointer, size out of range, aliasing */
+  GF_ERR_UNSUPPORTED = 2, /* valid request the library has no kernel for (e.g. d = 96) */
+  GF_ERR_WORKSPACE = 3,   /* ws missing or smaller than gformer_workspace_bytes */
+  GF_ERR_CUDA = 4,        /* a CUDA call or launch failed */
+  GF_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (see last_device_status) */
+} gf_status;
+
+typedef enum { GF_F32 = 0, GF_BF16 = 1 } gf_dtype;
+typedef enum { GF_BHND = 0, GF_BNHD = 1 } gf_layout;
+/* Feature map of the linear heads.  GF_PHI_ELU1: phi(x) = elu(x) + 1 (Sec. II-B). */
+typedef enum { GF_PHI_ELU1 = 0 } gf_phi;
+
+/* Process-wide knobs for tests and benchmarks (gformer_set_tuning). */
+typedef enum {
+  GF_TUNE_FORCE_SIMT = 0, /* 1: never take the tensor-core kernels (default 0)              */
+  GF_TUNE_LINEAR_SPLIT = 1 /* CTAs cooperating on one linear (b,h) chain: 0 = auto, 1, 2, 4 */
+} gf_tuning_key;
+
+/* Decode-time state of one batch (see gformer_decode_step).  The struct lives in host
+ * memory; the four pointers are device pointers owned by the caller. */
+typedef struct {
+  void* k_cache;   /* [B, h_sparse, w, d] dtype; ring: token j is in slot j mod w */
+  void* v_cache;   /* [B, h_sparse, w, d] dtype                                   */
+  float* S;        /* [B, H - h_sparse, d, d] fp32, S[a][c] = sum_j phi(k_j)[a] v_j[c] */
+  float* z;        /* [B, H - h_sparse, d]    fp32, z[a]    = sum_j phi(k_j)[a]        */
+  long long t;     /* tokens absorbed so far (whole batch in lock step)           */
+  int B, H, d, w, h_sparse;
+  int dtype;       /* gf_dtype of the ring                                         */
+} gf_decode_state;
+
+const char* gformer_status_string(int status);
+int gformer_version(void);
+
+/* Number of windowed heads used when a caller passes h_sparse < 0:
+ * max(1, round(3 H / 16)) -- 3 of 16 heads is the causal optimum reported in Sec. IV-D. */
+int gformer_default_h_sparse(int H);
+
+/* Sets a gf_tuning_key; returns GF_OK or GF_ERR_INVALID_ARG.  Not thread-safe against
+ * concurrent calls into the library. */
+int gformer_set_tuning(int key, int value);
+
+/* Number of kernels the library has launched in this process so far (all entry points,
+ * all streams).  For accounting in benchmarks. */
+unsigned long long gformer_launch_count(void);
+
+/* Scratch bytes the attention entry points need for this problem (never 0). */
+size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, int dtype);
+
+/* Synchronises `cuda_stream`, reads the device status word kept in ws and returns
+ * GF_OK, GF_ERR_TIMEOUT (a bounded wait inside a tensor-core kernel gave up; outputs of
+ * that call are undefined) or GF_ERR_CUDA.  ws must have been used by a previous call. */
+int gformer_last_device_status(void* ws, void* cuda_stream);
+
+/*
+ * Causal windowed softmax attention on all H heads (Eq. 1 restricted by the causal
+ * mask of Sec. II-A and the fixed left window of Sec. III-B):
+ *   o_i = sum_j p_ij v_j,  p_ij = softmax_j(scale * <q_i, k_j>),  j in [max(0, i-w+1), i].
+ * Token i attends to w keys, itself included; rows near the start see fewer.  w >= N is
+ * full causal attention.  scale <= 0 selects 1/sqrt(d).  1 <= w; N >= 1.
+ */
+int gformer_window_attn(const void* q, const void* k, const void* v, void* o,
+                        int B, int H, int N, int d, int w, float scale,
+                        int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Causal linear attention on all H heads (Algorithm 1, readout after the updates of
+ * step i; phi applied to raw q and k, no logit scale):
+ *   S_i = S_{i-1} + phi(k_i) v_i^T,  z_i = z_{i-1} + phi(k_i),
+ *   o_i = phi(q_i)^T S_i / <phi(q_i), z_i>.
+ * The phi(K)^T V outer products are accumulated by prefix sum, `chunk` rows at a time on
+ * the tensor-core path (0 = library default; otherwise 128).
+ * S_io [B,H,d,d] / z_io [B,H,d] (fp32, both or neither): when given they hold the state
+ * before token 0 on entry (zero them for a fresh sequence) and the state after token
+ * N-1 on return.
+ */
+int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void* o,
+                               int B, int H, int N, int d, int phi, int chunk,
+                               float* S_io, float* z_io,
+                               int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * The hybrid layer (Sec. III-A): heads [0, h_sparse) as gformer_window_attn, heads
+ * [h_sparse, H) as gformer_causal_linear_attn with a zero initial state; h_sparse < 0
+ * selects gformer_default_h_sparse(H).  Both groups are enqueued so that they overlap on
+ * the device.
+ * state_out (may be NULL): if given, its B, H, d, w, h_sparse, dtype must match the call
+ * and its buffers receive the decode state after the N tokens: the last min(N, w) keys
+ * and values of the windowed heads in ring slots j mod w, the final S and z of the linear
+ * heads, and t = N.
+ */
+int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o,
+                        int B, int H, int N, int d, int w, int h_sparse, float scale,
+                        int phi, int chunk, int dtype, int layout,
+                        gf_decode_state* state_out,
+                        void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * One autoregressive step for token index st->t: q, k, v, o are [B, H, d].  Windowed
+ * heads store k, v in ring slot t mod w and take the softmax over the min(t+1, w) cached
+ * keys (the window rule of Sec. III-B); linear heads run one iteration of Algorithm 1 on
+ * (S, z).  Updates the state buffers in place and increments st->t on success.  The
+ * result for token t equals row t of the full-sequence layer.
+ */
+int gformer_decode_step(const void* q, const void* k, const void* v, void* o,
+                        gf_decode_state* st, float scale, int phi, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GFORMER_H_ */

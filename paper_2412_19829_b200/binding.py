@@ -1,0 +1,241 @@
+"""ctypes binding of libgformer.so: same names as the C ABI, argument marshalling only.
+
+torch is used for device memory and streams; every step of the attention path runs in the
+library's kernels.  There is no CPU fallback: if the shared library is missing or a call
+returns a non-zero status, a GformerError is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+GF_OK, GF_ERR_INVALID_ARG, GF_ERR_UNSUPPORTED, GF_ERR_WORKSPACE, GF_ERR_CUDA, GF_ERR_TIMEOUT = range(6)
+GF_F32, GF_BF16 = 0, 1
+GF_BHND, GF_BNHD = 0, 1
+GF_PHI_ELU1 = 0
+GF_TUNE_FORCE_SIMT, GF_TUNE_LINEAR_SPLIT = 0, 1
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgformer.so")
+
+
+class GformerError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+class DecodeStateC(ctypes.Structure):
+    _fields_ = [("k_cache", ctypes.c_void_p), ("v_cache", ctypes.c_void_p),
+                ("S", ctypes.c_void_p), ("z", ctypes.c_void_p), ("t", ctypes.c_longlong),
+                ("B", ctypes.c_int), ("H", ctypes.c_int), ("d", ctypes.c_int), ("w", ctypes.c_int),
+                ("h_sparse", ctypes.c_int), ("dtype", ctypes.c_int)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libgformer.so (built in-tree by paper_2412_19829_b200.build); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is not built; run `python -m paper_2412_19829_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        L.gformer_status_string.restype = ctypes.c_char_p
+        L.gformer_status_string.argtypes = [i]
+        L.gformer_version.restype = i
+        L.gformer_launch_count.restype = ctypes.c_ulonglong
+        L.gformer_default_h_sparse.restype = i
+        L.gformer_default_h_sparse.argtypes = [i]
+        L.gformer_set_tuning.restype = i
+        L.gformer_set_tuning.argtypes = [i, i]
+        L.gformer_workspace_bytes.restype = sz
+        L.gformer_workspace_bytes.argtypes = [i] * 7
+        L.gformer_last_device_status.restype = i
+        L.gformer_last_device_status.argtypes = [vp, vp]
+        L.gformer_window_attn.restype = i
+        L.gformer_window_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp, sz, vp]
+        L.gformer_causal_linear_attn.restype = i
+        L.gformer_causal_linear_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, vp, i, i, vp, sz, vp]
+        L.gformer_hybrid_attn.restype = i
+        L.gformer_hybrid_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, i, i,
+                                          ctypes.POINTER(DecodeStateC), vp, sz, vp]
+        L.gformer_decode_step.restype = i
+        L.gformer_decode_step.argtypes = [vp, vp, vp, vp, ctypes.POINTER(DecodeStateC), f, i, vp]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().gformer_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return int(lib().gformer_version())
+
+
+def launch_count() -> int:
+    return int(lib().gformer_launch_count())
+
+
+def default_h_sparse(H: int) -> int:
+    return int(lib().gformer_default_h_sparse(int(H)))
+
+
+def set_tuning(key: int, value: int) -> None:
+    rc = lib().gformer_set_tuning(int(key), int(value))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_set_tuning")
+
+
+def workspace_bytes(B, H, N, d, w, h_sparse, dtype) -> int:
+    return int(lib().gformer_workspace_bytes(B, H, N, d, w, h_sparse, dtype))
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GF_F32
+    if t.dtype == torch.bfloat16:
+        return GF_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _stream_ptr(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _check_qkv(q, k, v):
+    for t in (q, k, v):
+        if not (t.is_cuda and t.is_contiguous()):
+            raise ValueError("q, k, v must be contiguous CUDA tensors")
+        if t.shape != q.shape or t.dtype != q.dtype:
+            raise ValueError("q, k, v must agree in shape and dtype")
+
+
+def _dims(q, layout):
+    if q.dim() != 4:
+        raise ValueError("expected a 4-D tensor")
+    if layout == GF_BNHD:
+        B, N, H, d = q.shape
+    else:
+        B, H, N, d = q.shape
+    return int(B), int(H), int(N), int(d)
+
+
+class Workspace:
+    """Caller-owned device scratch for the attention entry points."""
+
+    def __init__(self, nbytes: int = 256, device=None):
+        self.buf = torch.empty(max(int(nbytes), 256) + 256, dtype=torch.uint8,
+                               device=device if device is not None else "cuda")
+        off = (-self.buf.data_ptr()) % 256
+        self.ptr = self.buf.data_ptr() + off
+        self.nbytes = self.buf.numel() - off
+
+    def last_device_status(self, stream=None) -> int:
+        return int(lib().gformer_last_device_status(self.ptr, _stream_ptr(stream)))
+
+
+_default_ws: dict = {}
+
+
+def _ws_for(t: torch.Tensor, ws, need: int) -> Workspace:
+    if ws is not None:
+        return ws
+    key = t.device.index
+    cur = _default_ws.get(key)
+    if cur is None or cur.nbytes < need:
+        cur = Workspace(need, t.device)
+        _default_ws[key] = cur
+    return cur
+
+
+def window_attn(q, k, v, w: int, scale: float = 0.0, layout: int = GF_BHND, out=None, ws=None, stream=None):
+    """gformer_window_attn: causal softmax attention over the w most recent keys."""
+    _check_qkv(q, k, v)
+    B, H, N, d = _dims(q, layout)
+    o = torch.empty_like(q) if out is None else out
+    dt = _dtype_code(q)
+    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, H, dt))
+    rc = lib().gformer_window_attn(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, int(w),
+                                   float(scale), dt, layout, W.ptr, W.nbytes, _stream_ptr(stream))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_window_attn")
+    return o
+
+
+def causal_linear_attn(q, k, v, S=None, z=None, chunk: int = 0, layout: int = GF_BHND, out=None, ws=None,
+                       stream=None):
+    """gformer_causal_linear_attn: Algorithm 1 with phi = elu + 1; S, z (fp32) updated in place."""
+    _check_qkv(q, k, v)
+    B, H, N, d = _dims(q, layout)
+    o = torch.empty_like(q) if out is None else out
+    dt = _dtype_code(q)
+    if S is not None:
+        assert S.dtype == torch.float32 and S.is_contiguous() and tuple(S.shape) == (B, H, d, d)
+        assert z.dtype == torch.float32 and z.is_contiguous() and tuple(z.shape) == (B, H, d)
+    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, 1, 0, dt))
+    rc = lib().gformer_causal_linear_attn(
+        q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, GF_PHI_ELU1, int(chunk),
+        S.data_ptr() if S is not None else None, z.data_ptr() if z is not None else None,
+        dt, layout, W.ptr, W.nbytes, _stream_ptr(stream))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_causal_linear_attn")
+    return o
+
+
+class DecodeState:
+    """Device buffers of the decode state (ring KV cache, S, z) plus the host-side struct."""
+
+    def __init__(self, B, H, d, w, h_sparse, dtype=torch.bfloat16, device="cuda"):
+        H1 = H - h_sparse
+        self.k_cache = torch.zeros(B, max(h_sparse, 1), w, d, dtype=dtype, device=device)
+        self.v_cache = torch.zeros(B, max(h_sparse, 1), w, d, dtype=dtype, device=device)
+        self.S = torch.zeros(B, max(H1, 1), d, d, dtype=torch.float32, device=device)
+        self.z = torch.zeros(B, max(H1, 1), d, dtype=torch.float32, device=device)
+        self.c = DecodeStateC(self.k_cache.data_ptr(), self.v_cache.data_ptr(), self.S.data_ptr(),
+                              self.z.data_ptr(), 0, B, H, d, w, h_sparse,
+                              GF_F32 if dtype == torch.float32 else GF_BF16)
+
+    @property
+    def t(self) -> int:
+        return int(self.c.t)
+
+    @t.setter
+    def t(self, value: int):
+        self.c.t = int(value)
+
+
+def hybrid_attn(q, k, v, w: int, h_sparse: int = -1, scale: float = 0.0, chunk: int = 0,
+                layout: int = GF_BHND, state_out: DecodeState | None = None, out=None, ws=None, stream=None):
+    """gformer_hybrid_attn: heads [0, h_sparse) windowed, the rest linear, merged by head."""
+    _check_qkv(q, k, v)
+    B, H, N, d = _dims(q, layout)
+    o = torch.empty_like(q) if out is None else out
+    dt = _dtype_code(q)
+    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, h_sparse, dt))
+    rc = lib().gformer_hybrid_attn(
+        q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, int(w), int(h_sparse), float(scale),
+        GF_PHI_ELU1, int(chunk), dt, layout, ctypes.byref(state_out.c) if state_out is not None else None,
+        W.ptr, W.nbytes, _stream_ptr(stream))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_hybrid_attn")
+    return o
+
+
+def decode_step(q, k, v, st: DecodeState, scale: float = 0.0, out=None, stream=None):
+    """gformer_decode_step: q, k, v are [B, H, d]; st is advanced by one token."""
+    for t in (q, k, v):
+        if not (t.is_cuda and t.is_contiguous() and t.dim() == 3):
+            raise ValueError("q, k, v must be contiguous [B, H, d] CUDA tensors")
+    o = torch.empty_like(q) if out is None else out
+    rc = lib().gformer_decode_step(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), ctypes.byref(st.c),
+                                   float(scale), GF_PHI_ELU1, _stream_ptr(stream))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_decode_step")
+    return o

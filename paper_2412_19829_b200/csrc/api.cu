@@ -1,0 +1,274 @@
+// C ABI of libgformer: argument validation, path selection and launches.
+#include <math.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace gf {
+static std::atomic<unsigned long long> g_launches{0};
+void note_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+}  // namespace gf
+
+namespace {
+
+using gf::Strides;
+using gf::WsHeader;
+
+int g_force_simt = 0;
+int g_linear_split = 0;
+
+constexpr int kMaxDevices = 64;
+struct Fork {
+  cudaStream_t side = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  bool ready = false;
+};
+Fork g_fork[kMaxDevices];
+std::mutex g_fork_mutex;
+
+// Side stream + two events per device, created on first use; lets the two head groups of the
+// hybrid layer run concurrently while the caller sees a single-stream call.
+Fork* get_fork() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_fork_mutex);
+  Fork& f = g_fork[dev];
+  if (!f.ready) {
+    if (cudaStreamCreateWithFlags(&f.side, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&f.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&f.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    f.ready = true;
+  }
+  return &f;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool overlaps(const void* a, const void* b, size_t bytes) {
+  const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+  return x < y + bytes && y < x + bytes;
+}
+
+size_t elem_size(int dtype) { return dtype == GF_F32 ? 4 : 2; }
+
+int check_common(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
+                 int layout) {
+  if (!q || !k || !v || !o) return GF_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return GF_ERR_INVALID_ARG;
+  if (B < 1 || H < 1 || N < 1 || d < 1) return GF_ERR_INVALID_ARG;
+  if (dtype != GF_F32 && dtype != GF_BF16) return GF_ERR_INVALID_ARG;
+  if (layout != GF_BHND && layout != GF_BNHD) return GF_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return GF_ERR_UNSUPPORTED;
+  if ((long long)B * H > 65535LL * 65535LL || B > 65535 || H > 65535) return GF_ERR_UNSUPPORTED;
+  const size_t bytes = (size_t)B * H * N * d * elem_size(dtype);
+  if (overlaps(o, q, bytes) || overlaps(o, k, bytes) || overlaps(o, v, bytes)) return GF_ERR_INVALID_ARG;
+  return GF_OK;
+}
+
+int check_ws(void* ws, size_t ws_bytes, size_t need) {
+  if (!ws || ws_bytes < need) return GF_ERR_WORKSPACE;
+  if ((reinterpret_cast<uintptr_t>(ws) & 255u) != 0) return GF_ERR_INVALID_ARG;
+  return GF_OK;
+}
+
+int cuda_status(cudaError_t e) { return e == cudaSuccess ? GF_OK : GF_ERR_CUDA; }
+
+// Window heads [h_begin, h_begin+h_count) on `stream`.
+int run_window(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
+               float scale, int dtype, int layout, int h_begin, int h_count, WsHeader* ws,
+               cudaStream_t stream) {
+  if (h_count <= 0) return GF_OK;
+  const int w_eff = w > N ? N : w;  // keys before token 0 do not exist
+  if (!g_force_simt && gf::tc_window_supported(N, d, w_eff, dtype))
+    return cuda_status(
+        gf::launch_window_tc(q, k, v, o, B, H, N, d, w_eff, scale, layout, h_begin, h_count, ws, stream));
+  return cuda_status(gf::launch_window_simt(q, k, v, o, B, N, d, w_eff, scale, dtype,
+                                            gf::make_strides(layout, H, N, d), h_begin, h_count, stream));
+}
+
+int run_linear(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
+               int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init, WsHeader* ws,
+               cudaStream_t stream) {
+  if (h_count <= 0) return GF_OK;
+  if (!g_force_simt && gf::tc_linear_supported(N, d, dtype))
+    return cuda_status(gf::launch_linear_tc(q, k, v, o, B, H, N, d, layout, h_begin, h_count, S_io, z_io,
+                                            zero_init, g_linear_split, ws, stream));
+  return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d),
+                                            h_begin, h_count, S_io, z_io, zero_init, stream));
+}
+
+int clear_ws(void* ws, cudaStream_t stream) {
+  return cuda_status(cudaMemsetAsync(ws, 0, sizeof(WsHeader), stream));
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* gformer_status_string(int status) {
+  switch (status) {
+    case GF_OK: return "ok";
+    case GF_ERR_INVALID_ARG: return "invalid argument";
+    case GF_ERR_UNSUPPORTED: return "unsupported configuration";
+    case GF_ERR_WORKSPACE: return "workspace missing or too small";
+    case GF_ERR_CUDA: return "CUDA error";
+    case GF_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int gformer_version(void) { return 100; }
+
+unsigned long long gformer_launch_count(void) { return gf::g_launches.load(std::memory_order_relaxed); }
+
+int gformer_default_h_sparse(int H) {
+  if (H < 1) return 0;
+  int h0 = (int)floor(3.0 * H / 16.0 + 0.5);
+  if (h0 < 1) h0 = 1;
+  if (h0 > H) h0 = H;
+  return h0;
+}
+
+int gformer_set_tuning(int key, int value) {
+  switch (key) {
+    case GF_TUNE_FORCE_SIMT:
+      g_force_simt = value ? 1 : 0;
+      return GF_OK;
+    case GF_TUNE_LINEAR_SPLIT:
+      if (value != 0 && value != 1 && value != 2 && value != 4) return GF_ERR_INVALID_ARG;
+      g_linear_split = value;
+      return GF_OK;
+    default:
+      return GF_ERR_INVALID_ARG;
+  }
+}
+
+size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, int dtype) {
+  (void)B; (void)H; (void)N; (void)d; (void)w; (void)h_sparse; (void)dtype;
+  return sizeof(WsHeader);
+}
+
+int gformer_last_device_status(void* ws, void* cuda_stream) {
+  if (!ws) return GF_ERR_INVALID_ARG;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  WsHeader hdr;
+  if (cudaMemcpyAsync(&hdr, ws, sizeof(hdr), cudaMemcpyDeviceToHost, stream) != cudaSuccess) return GF_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return GF_ERR_CUDA;
+  return hdr.status == 0 ? GF_OK : GF_ERR_TIMEOUT;
+}
+
+int gformer_window_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
+                        float scale, int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
+  if (rc != GF_OK) return rc;
+  if (w < 1) return GF_ERR_INVALID_ARG;
+  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, H, dtype));
+  if (rc != GF_OK) return rc;
+  if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  rc = clear_ws(ws, stream);
+  if (rc != GF_OK) return rc;
+  return run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream);
+}
+
+int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                               int phi, int chunk, float* S_io, float* z_io, int dtype, int layout, void* ws,
+                               size_t ws_bytes, void* cuda_stream) {
+  int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
+  if (rc != GF_OK) return rc;
+  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  if (chunk != 0 && chunk != 128) return chunk < 0 || chunk % 64 ? GF_ERR_INVALID_ARG : GF_ERR_UNSUPPORTED;
+  if ((S_io == nullptr) != (z_io == nullptr)) return GF_ERR_INVALID_ARG;
+  if (S_io && (!aligned16(S_io) || !aligned16(z_io))) return GF_ERR_INVALID_ARG;
+  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, 1, 0, dtype));
+  if (rc != GF_OK) return rc;
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  rc = clear_ws(ws, stream);
+  if (rc != GF_OK) return rc;
+  return run_linear(q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, (WsHeader*)ws, stream);
+}
+
+int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
+                        int h_sparse, float scale, int phi, int chunk, int dtype, int layout,
+                        gf_decode_state* state_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+  int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
+  if (rc != GF_OK) return rc;
+  if (w < 1) return GF_ERR_INVALID_ARG;
+  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  if (chunk != 0 && chunk != 128) return chunk < 0 || chunk % 64 ? GF_ERR_INVALID_ARG : GF_ERR_UNSUPPORTED;
+  if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
+  if (h_sparse > H) return GF_ERR_INVALID_ARG;
+  const int h_lin = H - h_sparse;
+  if (state_out) {
+    gf_decode_state* s = state_out;
+    if (s->B != B || s->H != H || s->d != d || s->w != w || s->h_sparse != h_sparse || s->dtype != dtype)
+      return GF_ERR_INVALID_ARG;
+    if (h_sparse > 0 && (!s->k_cache || !s->v_cache || !aligned16(s->k_cache) || !aligned16(s->v_cache)))
+      return GF_ERR_INVALID_ARG;
+    if (h_lin > 0 && (!s->S || !s->z || !aligned16(s->S) || !aligned16(s->z))) return GF_ERR_INVALID_ARG;
+  }
+  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, h_sparse, dtype));
+  if (rc != GF_OK) return rc;
+  if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  rc = clear_ws(ws, stream);
+  if (rc != GF_OK) return rc;
+
+  float* S_out = state_out ? state_out->S : nullptr;
+  float* z_out = state_out ? state_out->z : nullptr;
+  const bool both = h_sparse > 0 && h_lin > 0;
+  Fork* f = both ? get_fork() : nullptr;
+  if (both && f == nullptr) return GF_ERR_CUDA;
+  if (both) {
+    // fork: the linear heads (the long serial chains) stay on the caller's stream, the
+    // windowed heads go to the side stream; join before returning control to the stream.
+    if (cudaEventRecord(f->fork, stream) != cudaSuccess) return GF_ERR_CUDA;
+    if (cudaStreamWaitEvent(f->side, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
+  }
+  rc = run_linear(q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, (WsHeader*)ws,
+                  stream);
+  cudaStream_t wstream = both ? f->side : stream;
+  int rc2 = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, wstream);
+  if (rc2 == GF_OK && state_out && h_sparse > 0)
+    rc2 = cuda_status(gf::launch_export_ring(k, v, state_out->k_cache, state_out->v_cache, B, N, d, w, dtype,
+                                             gf::make_strides(layout, H, N, d), h_sparse, wstream));
+  if (both) {
+    if (cudaEventRecord(f->join, f->side) != cudaSuccess) return GF_ERR_CUDA;
+    if (cudaStreamWaitEvent(stream, f->join, 0) != cudaSuccess) return GF_ERR_CUDA;
+  }
+  if (rc != GF_OK) return rc;
+  if (rc2 != GF_OK) return rc2;
+  if (state_out) state_out->t = N;
+  return GF_OK;
+}
+
+int gformer_decode_step(const void* q, const void* k, const void* v, void* o, gf_decode_state* st, float scale,
+                        int phi, void* cuda_stream) {
+  if (!q || !k || !v || !o || !st) return GF_ERR_INVALID_ARG;
+  if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return GF_ERR_INVALID_ARG;
+  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  if (st->B < 1 || st->H < 1 || st->w < 1 || st->h_sparse < 0 || st->h_sparse > st->H || st->t < 0)
+    return GF_ERR_INVALID_ARG;
+  if (st->dtype != GF_F32 && st->dtype != GF_BF16) return GF_ERR_INVALID_ARG;
+  if (st->d != 64 && st->d != 128) return GF_ERR_UNSUPPORTED;
+  if (st->B > 65535) return GF_ERR_UNSUPPORTED;
+  if ((size_t)st->w * sizeof(float) > 160 * 1024) return GF_ERR_UNSUPPORTED;
+  if (st->h_sparse > 0 &&
+      (!st->k_cache || !st->v_cache || !aligned16(st->k_cache) || !aligned16(st->v_cache)))
+    return GF_ERR_INVALID_ARG;
+  if (st->h_sparse < st->H && (!st->S || !st->z || !aligned16(st->S) || !aligned16(st->z)))
+    return GF_ERR_INVALID_ARG;
+  const size_t bytes = (size_t)st->B * st->H * st->d * elem_size(st->dtype);
+  if (overlaps(o, q, bytes) || overlaps(o, k, bytes) || overlaps(o, v, bytes)) return GF_ERR_INVALID_ARG;
+  if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)st->d);
+  cudaError_t e = gf::launch_decode_step(q, k, v, o, st->k_cache, st->v_cache, st->S, st->z, st->t, st->B, st->H,
+                                         st->d, st->w, st->h_sparse, scale, st->dtype, (cudaStream_t)cuda_stream);
+  if (e != cudaSuccess) return GF_ERR_CUDA;
+  st->t += 1;
+  return GF_OK;
+}
+
+}  // extern "C"

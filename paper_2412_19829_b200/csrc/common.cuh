@@ -1,0 +1,81 @@
+// Shared declarations of the libgformer CUDA sources (host-side launch interfaces and a
+// few device helpers).  Not part of the public ABI.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gformer.h"
+
+namespace gf {
+
+// Element strides of a logical [B, H, N, d] tensor (innermost stride is 1).
+struct Strides {
+  long long b, h, n;
+};
+
+inline Strides make_strides(int layout, int H, int N, int d) {
+  Strides s;
+  if (layout == GF_BNHD) {
+    s.b = (long long)N * H * d;
+    s.n = (long long)H * d;
+    s.h = d;
+  } else {
+    s.b = (long long)H * N * d;
+    s.h = (long long)N * d;
+    s.n = d;
+  }
+  return s;
+}
+
+// Layout of the first bytes of the caller's workspace.
+struct WsHeader {
+  unsigned int status;   // 0 = fine, else a code written by a kernel whose bounded wait expired
+  unsigned int where;    // which wait gave up (diagnostic)
+  unsigned int ticket;   // work counter of the persistent kernels
+  unsigned int pad[61];
+};
+static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
+
+// Counts kernel launches (reported by gformer_launch_count).
+void note_launch(int n = 1);
+
+// ---- SIMT (CUDA-core, fp32 arithmetic) path: any w, d in {64,128}, f32 or bf16 storage.
+// Heads [h_begin, h_begin + h_count) of the [B, H, N, d] tensors are processed.
+cudaError_t launch_window_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
+                               int w, float scale, int dtype, Strides st, int h_begin, int h_count,
+                               cudaStream_t stream);
+// S_io/z_io: [B, h_count, d, d] / [B, h_count, d] or null.  zero_init: ignore their contents on entry.
+cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
+                               int dtype, Strides st, int h_begin, int h_count, float* S_io, float* z_io,
+                               bool zero_init, cudaStream_t stream);
+cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void* v_cache, int B, int N, int d,
+                               int w, int dtype, Strides st, int h_sparse, cudaStream_t stream);
+cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
+                               void* v_cache, float* S, float* z, long long t, int B, int H, int d, int w,
+                               int h_sparse, float scale, int dtype, cudaStream_t stream);
+
+// ---- tensor-core (tcgen05 / TMEM / TMA) path: bf16 storage, d in {64,128}.
+bool tc_window_supported(int N, int d, int w, int dtype);
+bool tc_linear_supported(int N, int d, int dtype);
+cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                             int w, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
+                             cudaStream_t stream);
+cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                             int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
+                             int split, WsHeader* ws, cudaStream_t stream);
+
+// ---- device helpers
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) {
+  return __float2bfloat16_rn(x);
+}
+
+// phi(x) = elu(x) + 1 (Sec. II-B).
+__device__ __forceinline__ float phi_elu1(float x) { return x > 0.f ? x + 1.f : expf(x); }
+
+}  // namespace gf

@@ -1,0 +1,115 @@
+"""CPU-side checks of the C ABI: the library loads, exports what the header declares, and
+rejects bad arguments on the host before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import oracle
+from paper_2412_19829_b200 import binding as gf
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for fn in os.listdir(inc):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(gformer_\w+)\s*\(", text))
+    return sorted(names)
+
+
+def test_header_declares_the_four_entry_points():
+    names = declared_symbols()
+    for must in ("gformer_window_attn", "gformer_causal_linear_attn", "gformer_hybrid_attn",
+                 "gformer_decode_step", "gformer_workspace_bytes"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol():
+    L = gf.lib()
+    for name in declared_symbols():
+        assert hasattr(L, name), name
+
+
+def test_status_strings_and_version():
+    assert gf.version() >= 100
+    assert gf.status_string(gf.GF_OK) == "ok"
+    assert len({gf.status_string(i) for i in range(6)}) == 6
+
+
+def test_default_head_split_matches_oracle_reading():
+    for H in (1, 2, 3, 8, 12, 16, 24, 32, 40, 64, 96):
+        assert gf.default_h_sparse(H) == oracle.default_h_sparse(H)
+
+
+def test_workspace_bytes_nonzero():
+    assert gf.workspace_bytes(1, 32, 32768, 128, 512, 6, gf.GF_BF16) >= 256
+
+
+def test_tuning_rejects_unknown_keys():
+    L = gf.lib()
+    assert L.gformer_set_tuning(99, 1) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 3) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0) == gf.GF_OK
+
+
+FAKE = 0x10000  # a 16-byte-aligned non-null address; validation fails before it is ever used
+
+
+@pytest.mark.parametrize("kw,expect", [
+    (dict(q=0), gf.GF_ERR_INVALID_ARG),
+    (dict(q=FAKE + 4), gf.GF_ERR_INVALID_ARG),
+    (dict(B=0), gf.GF_ERR_INVALID_ARG),
+    (dict(N=0), gf.GF_ERR_INVALID_ARG),
+    (dict(w=0), gf.GF_ERR_INVALID_ARG),
+    (dict(d=96), gf.GF_ERR_UNSUPPORTED),
+    (dict(dtype=7), gf.GF_ERR_INVALID_ARG),
+    (dict(layout=5), gf.GF_ERR_INVALID_ARG),
+    (dict(o=FAKE), gf.GF_ERR_INVALID_ARG),          # o aliases q
+    (dict(ws=0), gf.GF_ERR_WORKSPACE),
+    (dict(ws_bytes=8), gf.GF_ERR_WORKSPACE),
+])
+def test_window_attn_argument_errors(kw, expect):
+    a = dict(q=FAKE, k=FAKE + (1 << 30), v=FAKE + (2 << 30), o=FAKE + (3 << 30), B=1, H=2, N=64, d=64, w=32,
+             scale=0.0, dtype=gf.GF_BF16, layout=gf.GF_BHND, ws=FAKE + (4 << 30), ws_bytes=4096)
+    a.update(kw)
+    rc = gf.lib().gformer_window_attn(a["q"], a["k"], a["v"], a["o"], a["B"], a["H"], a["N"], a["d"], a["w"],
+                                      a["scale"], a["dtype"], a["layout"], a["ws"], a["ws_bytes"], None)
+    assert rc == expect
+
+
+def test_hybrid_and_linear_argument_errors():
+    L = gf.lib()
+    q, k, v, o, ws = FAKE, FAKE + (1 << 30), FAKE + (2 << 30), FAKE + (3 << 30), FAKE + (4 << 30)
+    # h_sparse > H
+    assert L.gformer_hybrid_attn(q, k, v, o, 1, 4, 64, 64, 32, 5, 0.0, 0, 0, gf.GF_BF16, 0, None, ws, 4096,
+                                 None) == gf.GF_ERR_INVALID_ARG
+    # unknown feature map
+    assert L.gformer_hybrid_attn(q, k, v, o, 1, 4, 64, 64, 32, 1, 0.0, 3, 0, gf.GF_BF16, 0, None, ws, 4096,
+                                 None) == gf.GF_ERR_UNSUPPORTED
+    # chunk not a multiple of 64
+    assert L.gformer_causal_linear_attn(q, k, v, o, 1, 4, 64, 64, 0, 100, None, None, gf.GF_BF16, 0, ws, 4096,
+                                        None) == gf.GF_ERR_INVALID_ARG
+    # S without z
+    assert L.gformer_causal_linear_attn(q, k, v, o, 1, 4, 64, 64, 0, 0, FAKE + (5 << 30), None, gf.GF_BF16, 0,
+                                        ws, 4096, None) == gf.GF_ERR_INVALID_ARG
+    # state struct that disagrees with the call
+    st = gf.DecodeStateC(FAKE, FAKE, FAKE, FAKE, 0, 2, 4, 64, 32, 1, gf.GF_BF16)
+    assert L.gformer_hybrid_attn(q, k, v, o, 1, 4, 64, 64, 32, 1, 0.0, 0, 0, gf.GF_BF16, 0, ctypes.byref(st),
+                                 ws, 4096, None) == gf.GF_ERR_INVALID_ARG
+
+
+def test_decode_argument_errors():
+    L = gf.lib()
+    q, k, v, o = FAKE, FAKE + (1 << 30), FAKE + (2 << 30), FAKE + (3 << 30)
+    st = gf.DecodeStateC(FAKE, FAKE, FAKE, FAKE, 0, 2, 4, 96, 32, 1, gf.GF_BF16)
+    assert L.gformer_decode_step(q, k, v, o, ctypes.byref(st), 0.0, 0, None) == gf.GF_ERR_UNSUPPORTED
+    st = gf.DecodeStateC(0, FAKE, FAKE, FAKE, 0, 2, 4, 64, 32, 1, gf.GF_BF16)
+    assert L.gformer_decode_step(q, k, v, o, ctypes.byref(st), 0.0, 0, None) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_decode_step(q, k, v, o, None, 0.0, 0, None) == gf.GF_ERR_INVALID_ARG
+    assert st.t == 0

@@ -1,0 +1,328 @@
+"""GPU parity: libgformer (through the C ABI binding) against the fp64 oracle, element by
+element on the same seeded, storage-rounded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gates import assert_parity, errors, passes
+from paper_2412_19829_b200 import binding as gf
+from paper_2412_19829_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def f64(t):
+    return t.detach().cpu().to(torch.float64).numpy()
+
+
+def kind_of(dtype):
+    return "f32" if dtype == "f32" else "bf16"
+
+
+def dev(*ts):
+    return [t.cuda() for t in ts]
+
+
+@pytest.fixture(autouse=True)
+def _reset_tuning():
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 0)
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0)
+    yield
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 0)
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0)
+
+
+# ------------------------------------------------------------------ config 1: tiny fp32 hybrid
+def test_config1_tiny_fp32_hybrid():
+    c = synth.CONFIGS["tiny"]
+    q, k, v = synth.qkv(c["B"], c["H"], c["N"], c["d"], "f32", c["seed"])
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), c["w"])
+    o = gf.hybrid_attn(*dev(q, k, v), c["w"])
+    assert_parity(f64(o), ref, "f32", "config 1")
+
+
+# ------------------------------------------------------------------ window, CUDA-core path
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N,w,d", [(1, 1, 64), (63, 32, 64), (64, 64, 128), (65, 7, 64), (200, 100, 128),
+                                   (200, 1, 64), (130, 1000, 64), (257, 96, 128)])
+def test_window_simt(dtype, N, w, d):
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 1)
+    q, k, v = synth.qkv(2, 3, N, d, dtype, seed=100 + N + w, gain=1.0)
+    ref = oracle.window_attn(f64(q), f64(k), f64(v), w)
+    o = gf.window_attn(*dev(q, k, v), w)
+    assert_parity(f64(o), ref, kind_of(dtype), f"window simt N={N} w={w} d={d}")
+
+
+@pytest.mark.parametrize("force_simt", [1, 0])
+def test_window_bnhd_layout_and_custom_scale(force_simt):
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, force_simt)
+    B, H, N, d, w = 2, 3, 300, 64, 64
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=7, gain=1.0)
+    ref = oracle.window_attn(f64(q), f64(k), f64(v), w, scale=0.05)
+    qn, kn, vn = [t.permute(0, 2, 1, 3).contiguous().cuda() for t in (q, k, v)]
+    o = gf.window_attn(qn, kn, vn, w, scale=0.05, layout=gf.GF_BNHD)
+    assert_parity(f64(o.permute(0, 2, 1, 3)), ref, "bf16", "window bnhd")
+
+
+# ------------------------------------------------------------------ window, tensor-core path
+@pytest.mark.parametrize("N,w,d", [(128, 64, 64), (128, 128, 128), (300, 64, 128), (1000, 128, 64),
+                                   (1000, 512, 128), (1, 64, 64), (129, 192, 64), (640, 2048, 128),
+                                   (2048, 256, 64)])
+@pytest.mark.parametrize("gain", [None, 1.0])
+def test_window_tensor_core(N, w, d, gain):
+    q, k, v = synth.qkv(2, 2, N, d, "bf16", seed=200 + N + w, gain=gain)
+    ref = oracle.window_attn(f64(q), f64(k), f64(v), w)
+    ws = gf.Workspace()
+    o = gf.window_attn(*dev(q, k, v), w, ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    assert_parity(f64(o), ref, "bf16", f"window tc N={N} w={w} d={d}")
+
+
+def test_window_needle_at_window_edges_tensor_core():
+    # A key with a dominant logit: every row whose window holds it must return its value row,
+    # rows one past the window must not see it.
+    B, H, N, d, w = 1, 1, 700, 64, 128
+    for needle in (0, 127, 128, 300, 511):
+        q = torch.zeros(B, H, N, d)
+        q[..., 0] = 4.0
+        k = torch.zeros(B, H, N, d)
+        k[0, 0, needle, 0] = 64.0
+        v = synth.qkv(B, H, N, d, "bf16", seed=needle, gain=1.0)[2]
+        q, k = q.to(torch.bfloat16), k.to(torch.bfloat16)
+        ref = oracle.window_attn(f64(q), f64(k), f64(v), w, scale=1.0)
+        o = gf.window_attn(*dev(q, k, v), w, scale=1.0)
+        assert_parity(f64(o), ref, "bf16", f"needle {needle}")
+
+
+# ------------------------------------------------------------------ linear
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("N,d", [(1, 64), (17, 128), (130, 64), (300, 128)])
+def test_linear_simt(dtype, N, d):
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 1)
+    q, k, v = synth.qkv(2, 3, N, d, dtype, seed=300 + N, gain=1.0)
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v))
+    o = gf.causal_linear_attn(*dev(q, k, v))
+    assert_parity(f64(o), ref, kind_of(dtype), f"linear simt N={N} d={d}")
+
+
+@pytest.mark.parametrize("force_simt", [1, 0])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_linear_state_in_out_and_resume(force_simt, dtype):
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, force_simt)
+    B, H, N, d, cut = 2, 2, 333, 64, 200
+    q, k, v = synth.qkv(B, H, N, d, dtype, seed=11, gain=1.0)
+    S_ref = np.zeros((B, H, d, d)); z_ref = np.zeros((B, H, d))
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v), S_ref, z_ref)
+    S = torch.zeros(B, H, d, d, device="cuda"); z = torch.zeros(B, H, d, device="cuda")
+    qd, kd, vd = dev(q, k, v)
+    o1 = gf.causal_linear_attn(qd[:, :, :cut].contiguous(), kd[:, :, :cut].contiguous(),
+                               vd[:, :, :cut].contiguous(), S, z)
+    o2 = gf.causal_linear_attn(qd[:, :, cut:].contiguous(), kd[:, :, cut:].contiguous(),
+                               vd[:, :, cut:].contiguous(), S, z)
+    kind = kind_of(dtype)
+    assert_parity(f64(torch.cat([o1, o2], dim=2)), ref, kind, "linear resume")
+    tol = 1e-5 if (dtype == "f32" and force_simt) else 1e-2
+    assert errors(f64(S), S_ref)["rel_l2"] <= tol
+    assert errors(f64(z), z_ref)["rel_l2"] <= tol
+
+
+@pytest.mark.parametrize("N,d", [(128, 64), (128, 128), (300, 64), (1000, 128), (1, 128), (129, 64),
+                                 (4096, 128), (2048, 64)])
+@pytest.mark.parametrize("gain", [None, 1.0])
+def test_linear_tensor_core(N, d, gain):
+    q, k, v = synth.qkv(2, 2, N, d, "bf16", seed=400 + N, gain=gain)
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v))
+    ws = gf.Workspace()
+    o = gf.causal_linear_attn(*dev(q, k, v), ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    assert_parity(f64(o), ref, "bf16", f"linear tc N={N} d={d}")
+
+
+@pytest.mark.parametrize("split", [1, 2, 4])
+def test_linear_tensor_core_split_invariance(split):
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
+    q, k, v = synth.qkv(1, 3, 1500, 128, "bf16", seed=17, gain=1.0)
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v))
+    o = gf.causal_linear_attn(*dev(q, k, v))
+    assert_parity(f64(o), ref, "bf16", f"linear tc split={split}")
+
+
+def test_linear_bnhd_layout():
+    B, H, N, d = 2, 3, 260, 128
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=19, gain=1.0)
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v))
+    qn, kn, vn = [t.permute(0, 2, 1, 3).contiguous().cuda() for t in (q, k, v)]
+    o = gf.causal_linear_attn(qn, kn, vn, layout=gf.GF_BNHD)
+    assert_parity(f64(o.permute(0, 2, 1, 3)), ref, "bf16", "linear bnhd")
+
+
+# ------------------------------------------------------------------ hybrid merge
+@pytest.mark.parametrize("h0", [0, 1, 3, 4])
+def test_hybrid_merge_equals_pure_calls(h0):
+    B, H, N, d, w = 2, 4, 384, 64, 128
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=23, gain=1.0)
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0)
+    qd, kd, vd = dev(q, k, v)
+    o = gf.hybrid_attn(qd, kd, vd, w, h_sparse=h0)
+    assert_parity(f64(o), ref, "bf16", f"hybrid h0={h0}")
+    if h0 > 0:
+        ow = gf.window_attn(qd[:, :h0].contiguous(), kd[:, :h0].contiguous(), vd[:, :h0].contiguous(), w)
+        assert torch.equal(ow, o[:, :h0])
+    if h0 < H:
+        ol = gf.causal_linear_attn(qd[:, h0:].contiguous(), kd[:, h0:].contiguous(), vd[:, h0:].contiguous())
+        assert torch.equal(ol, o[:, h0:])
+
+
+def test_negative_controls_fail_the_gates():
+    # The gates must reject plausible wrong answers on the unscaled (stress) distribution.
+    B, H, N, d, w = 1, 4, 512, 64, 128
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=29, gain=1.0)
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=2)
+    assert not passes(np.zeros_like(ref), ref, "bf16")
+    assert not passes(f64(v), ref, "bf16")
+    for w_bad in (w - 1, w + 1):
+        wrong = oracle.hybrid_attn(f64(q), f64(k), f64(v), w_bad, h_sparse=2)
+        assert not passes(wrong, ref, "bf16")
+    o = gf.hybrid_attn(*dev(q, k, v), w, h_sparse=2)
+    assert passes(f64(o), ref, "bf16")
+
+
+def test_run_to_run_determinism():
+    c = dict(B=2, H=4, N=1024, d=128, w=256)
+    q, k, v = dev(*synth.qkv(c["B"], c["H"], c["N"], c["d"], "bf16", seed=31))
+    a = gf.hybrid_attn(q, k, v, c["w"])
+    b = gf.hybrid_attn(q, k, v, c["w"])
+    assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ config 2 (full tensors)
+def test_config2_gpt2_small_full():
+    c = synth.CONFIGS["gpt2s"]
+    q, k, v = synth.qkv(c["B"], c["H"], c["N"], c["d"], "bf16", c["seed"])
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), c["w"])
+    ws = gf.Workspace()
+    o = gf.hybrid_attn(*dev(q, k, v), c["w"], ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    assert_parity(f64(o), ref, "bf16", "config 2")
+
+
+# ------------------------------------------------------------------ config 3 (full size on the GPU,
+# oracle on sampled heads: every head is an independent unit, so a head-by-head check is exact)
+def test_config3_long_sequence_sampled_heads():
+    c = synth.CONFIGS["long32k"]
+    q, k, v = synth.qkv(c["B"], c["H"], c["N"], c["d"], "bf16", c["seed"])
+    h0 = gf.default_h_sparse(c["H"])
+    assert h0 == 6
+    ws = gf.Workspace()
+    o = gf.hybrid_attn(*dev(q, k, v), c["w"], ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    assert torch.isfinite(o.float()).all()
+    wh = [0, h0 - 1]
+    ref_w = oracle.window_attn(f64(q[:, wh]), f64(k[:, wh]), f64(v[:, wh]), c["w"])
+    assert_parity(f64(o[:, wh]), ref_w, "bf16", "config 3 window heads")
+    lh = [h0, c["H"] - 1]
+    ref_l = oracle.causal_linear_attn(f64(q[:, lh]), f64(k[:, lh]), f64(v[:, lh]))
+    assert_parity(f64(o[:, lh]), ref_l, "bf16", "config 3 linear heads")
+
+
+# ------------------------------------------------------------------ decode
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d,w,h0", [(64, 16, 1), (128, 40, 2), (64, 300, 3), (64, 8, 0)])
+def test_decode_from_scratch_equals_full_sequence(dtype, d, w, h0):
+    B, H, T = 2, 3, 50
+    q, k, v = synth.qkv(B, H, T, d, dtype, seed=41, gain=1.0)
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0)
+    st = gf.DecodeState(B, H, d, w, h0, dtype=synth.torch_dtype(dtype))
+    qd, kd, vd = dev(q, k, v)
+    outs = []
+    for t in range(T):
+        outs.append(gf.decode_step(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(),
+                                   vd[:, :, t].contiguous(), st))
+    assert st.t == T
+    got = torch.stack(outs, dim=2)
+    assert_parity(f64(got), ref, kind_of(dtype), f"decode d={d} w={w}")
+
+
+@pytest.mark.parametrize("N0,w", [(100, 128), (128, 128), (333, 128), (40, 64)])
+def test_prefill_export_then_decode(N0, w):
+    B, H, d, h0, steps = 2, 4, 64, 2, 20
+    N = N0 + steps
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=43, gain=1.0)
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0)
+    qd, kd, vd = dev(q, k, v)
+    st = gf.DecodeState(B, H, d, w, h0)
+    o = gf.hybrid_attn(qd[:, :, :N0].contiguous(), kd[:, :, :N0].contiguous(), vd[:, :, :N0].contiguous(), w,
+                       h_sparse=h0, state_out=st)
+    assert st.t == N0
+    assert_parity(f64(o), ref[:, :, :N0], "bf16", "prefill")
+    # ring placement is exact (a copy): token j in slot j mod w
+    for j in range(max(0, N0 - w), N0):
+        assert torch.equal(st.k_cache[:, :, j % w], kd[:, :h0, j])
+        assert torch.equal(st.v_cache[:, :, j % w], vd[:, :h0, j])
+    outs = [gf.decode_step(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous(), st)
+            for t in range(N0, N)]
+    assert_parity(f64(torch.stack(outs, dim=2)), ref[:, :, N0:], "bf16", "decode after prefill")
+
+
+def test_decode_state_copy_resumes_identically():
+    B, H, d, w, h0 = 2, 4, 64, 32, 1
+    q, k, v = dev(*synth.qkv(B, H, 40, d, "bf16", seed=47, gain=1.0))
+    st = gf.DecodeState(B, H, d, w, h0)
+    for t in range(30):
+        gf.decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), st)
+    st2 = gf.DecodeState(B, H, d, w, h0)
+    for name in ("k_cache", "v_cache", "S", "z"):
+        getattr(st2, name).copy_(getattr(st, name))
+    st2.t = st.t
+    for t in range(30, 40):
+        a = gf.decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), st)
+        b = gf.decode_step(q[:, :, t].contiguous(), k[:, :, t].contiguous(), v[:, :, t].contiguous(), st2)
+        assert torch.equal(a, b)
+
+
+def test_config4_prefill_and_decode_sampled_batch():
+    c = synth.CONFIGS["decode"]
+    B, H, N, d, w, steps = c["B"], c["H"], c["N"], c["d"], c["w"], 64  # 64 of the 256 steps checked
+    h0 = gf.default_h_sparse(H)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", c["seed"])
+    tq, tk, tv = synth.decode_tokens(steps, B, H, d, "bf16", c["seed"])
+    st = gf.DecodeState(B, H, d, w, h0)
+    o = gf.hybrid_attn(*dev(q, k, v), w, state_out=st).cpu()
+    tqd, tkd, tvd = dev(tq, tk, tv)
+    outs = torch.stack([gf.decode_step(tqd[s], tkd[s], tvd[s], st) for s in range(steps)]).cpu()
+    bs = [0, B - 1]  # batch elements are independent: check two of them exactly
+    ref, ost = oracle.hybrid_attn(f64(q[bs]), f64(k[bs]), f64(v[bs]), w, h_sparse=h0, export_state=True)
+    assert_parity(f64(o[bs]), ref, "bf16", "config 4 prefill")
+    for s in range(steps):
+        r = oracle.decode_step(f64(tq[s][bs]), f64(tk[s][bs]), f64(tv[s][bs]), ost)
+        assert_parity(f64(outs[s][bs]), r, "bf16", f"config 4 decode step {s}")
+
+
+# ------------------------------------------------------------------ config 5 sweep
+@pytest.mark.parametrize("idx", list(range(32)))
+def test_config5_sweep_point(idx):
+    p = synth.sweep_points()[idx]
+    B, H, N, d, w = p["B"], p["H"], p["N"], p["d"], p["w"]
+    h0 = gf.default_h_sparse(H)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", p["seed"])
+    ws = gf.Workspace()
+    o = gf.hybrid_attn(*dev(q, k, v), w, ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    assert torch.isfinite(o.float()).all()
+    b = B - 1
+    # windowed head: rows depend on at most w keys, so the head of the sequence and an interior
+    # slice that starts w-1 tokens early are both exact sub-problems
+    n_head = min(N, 2048)
+    ref = oracle.window_attn(f64(q[b:b + 1, :1, :n_head]), f64(k[b:b + 1, :1, :n_head]),
+                             f64(v[b:b + 1, :1, :n_head]), w)
+    assert_parity(f64(o[b:b + 1, :1, :n_head]), ref, "bf16", "sweep window head rows")
+    if N > 2048:
+        lo = N - 1024 - (w - 1)
+        ref = oracle.window_attn(f64(q[b:b + 1, 2:3, lo:]), f64(k[b:b + 1, 2:3, lo:]), f64(v[b:b + 1, 2:3, lo:]), w)
+        assert_parity(f64(o[b:b + 1, 2:3, N - 1024:]), ref[:, :, w - 1:], "bf16", "sweep window tail rows")
+    # linear head: the whole chain of one head (its last rows depend on every token)
+    hl = H - 1
+    ref = oracle.causal_linear_attn(f64(q[b:b + 1, hl:hl + 1]), f64(k[b:b + 1, hl:hl + 1]),
+                                    f64(v[b:b + 1, hl:hl + 1]))
+    assert_parity(f64(o[b:b + 1, hl:hl + 1]), ref, "bf16", "sweep linear head")
