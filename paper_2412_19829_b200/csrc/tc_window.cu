@@ -1,7 +1,291 @@
-// placeholder until the tcgen05 window kernel lands
+// Windowed causal softmax attention on the tensor cores (bf16 in, fp32 accumulate).
+//
+// One CTA = one tile of 128 query rows of one (batch, head).  The keys a tile can see,
+// [i0 - w + 1, i0 + 127], are walked in 128-key tiles aligned to the query grid:
+//   S = Q K^T      tcgen05.mma, A and B from shared memory (K-major), S (128x128 fp32) in TMEM
+//   P = softmax    one thread per query row reads its S row from TMEM, masks (causal edge on
+//                  the diagonal tile, window edge on the leftmost ones), exponentiates against a
+//                  running reference maximum and writes P as bf16 back over S in TMEM
+//   O += P V       tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
+// O stays in TMEM across key tiles; it is rescaled only when a row's maximum moves by more than
+// 2^8 (lazy rescaling), which with bounded logits is rare.  Final rows are divided by the softmax
+// denominator, packed to bf16 and written with a TMA store.
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = softmax/epilogue.
+// TMEM use is 256 columns and shared memory under 113 KB so that two CTAs share an SM: while one
+// is in its softmax the other owns the tensor core.
 #include "common.cuh"
+#include "sm100.cuh"
+
 namespace gf {
-bool tc_window_supported(int, int, int, int) { return false; }
-cudaError_t launch_window_tc(const void*, const void*, const void*, void*, int, int, int, int, int, float, int,
-                             int, int, WsHeader*, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+using namespace sm100;
+
+constexpr int kThreads = 192;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+template <int D>
+struct WinSmem {
+  static constexpr int kTile = 128 * D * 2;  // bytes of one 128 x D bf16 tile
+  static constexpr int kQ = 0;
+  static constexpr int kK = kTile;
+  static constexpr int kV = 2 * kTile;
+  static constexpr int kBytes = 3 * kTile + 1024;  // + alignment slack
+};
+
+struct WinParams {
+  int N, w, tiles_back;  // tiles_back = number of key tiles before the diagonal one
+  float scale_log2;
+  int h_begin;
+  unsigned int* status;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kThreads, 2)
+window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
+                 const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
+                 const WinParams p) {
+  extern __shared__ uint8_t raw_smem[];
+  uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw_smem) + 1023) & ~(uintptr_t)1023);
+  uint8_t* sQ = sm + WinSmem<D>::kQ;
+  uint8_t* sK = sm + WinSmem<D>::kK;
+  uint8_t* sV = sm + WinSmem<D>::kV;
+  __shared__ __align__(8) uint64_t q_full, k_full, k_empty, v_full, v_empty, s_full, p_full, pv_done;
+  __shared__ uint32_t tmem_base_s;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int qt = blockIdx.x, h = p.h_begin + blockIdx.y, b = blockIdx.z;
+  const int i0 = qt * 128;
+  const int t_first = (qt - p.tiles_back) > 0 ? (qt - p.tiles_back) : 0;
+  const int n_tiles = qt - t_first + 1;
+
+  if (tid == 0) {
+    mbar_init(&q_full, 1);
+    mbar_init(&k_full, 1);
+    mbar_init(&k_empty, 1);
+    mbar_init(&v_full, 1);
+    mbar_init(&v_empty, 1);
+    mbar_init(&s_full, 1);
+    mbar_init(&p_full, 128);
+    mbar_init(&pv_done, 1);
+    mbar_fence_init();
+    tma_prefetch_desc(&mq);
+    tma_prefetch_desc(&mk);
+    tma_prefetch_desc(&mv);
+    tma_prefetch_desc(&mo);
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_base_s, 256);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = tmem_base_s;
+  const uint32_t tS = tmem;        // 128 columns: S, later P (bf16 pairs in the first 64)
+  const uint32_t tO = tmem + 128;  // D columns
+
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (elect_one()) {
+      mbar_arrive_expect_tx(&q_full, WinSmem<D>::kTile);
+      for (int c = 0; c < D / 64; ++c) tma_load_4d(sQ + c * 16384, &mq, &q_full, c * 64, i0, h, b);
+      for (int it = 0; it < n_tiles; ++it) {
+        const int j0 = (t_first + it) * 128;
+        if (!mbar_wait(&k_empty, (it + 1) & 1, p.status, 10)) break;
+        mbar_arrive_expect_tx(&k_full, WinSmem<D>::kTile);
+        for (int c = 0; c < D / 64; ++c) tma_load_4d(sK + c * 16384, &mk, &k_full, c * 64, j0, h, b);
+        if (!mbar_wait(&v_empty, (it + 1) & 1, p.status, 11)) break;
+        mbar_arrive_expect_tx(&v_full, WinSmem<D>::kTile);
+        for (int c = 0; c < D / 64; ++c) tma_load_4d(sV + c * 16384, &mv, &v_full, c * 64, j0, h, b);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (elect_one()) {
+      constexpr uint32_t idesc_qk = umma_idesc_bf16(128, 128, false, false);
+      constexpr uint32_t idesc_pv = umma_idesc_bf16(128, D, false, true);
+      bool ok = mbar_wait(&q_full, 0, p.status, 20);
+      for (int it = 0; it < n_tiles && ok; ++it) {
+        if (!mbar_wait(&k_full, it & 1, p.status, 21)) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+          umma_ss(tS, umma_smem_desc(smem_u32(sQ) + off, 16, 1024), umma_smem_desc(smem_u32(sK) + off, 16, 1024),
+                  idesc_qk, ks > 0);
+        }
+        umma_commit(&k_empty);
+        umma_commit(&s_full);
+        if (!mbar_wait(&p_full, it & 1, p.status, 22)) break;
+        if (!mbar_wait(&v_full, it & 1, p.status, 23)) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          umma_ts(tO, tS + ks * 8, umma_smem_desc(smem_u32(sV) + ks * 2048, 16384, 1024), idesc_pv,
+                  (it > 0) || (ks > 0));
+        }
+        umma_commit(&v_empty);
+        umma_commit(&pv_done);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------ softmax + epilogue
+    const int quarter = warp & 3;  // TMEM lane quarter this warp may touch
+    const int r = quarter * 32 + lane;
+    const int i = i0 + r;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    float m_ref = -INFINITY;  // reference maximum the stored O and l are relative to
+    float l = 0.f;
+    bool ok = true;
+    for (int it = 0; it < n_tiles; ++it) {
+      const int j0 = (t_first + it) * 128;
+      if (!mbar_wait(&s_full, it & 1, p.status, 30)) { ok = false; break; }
+      tc_fence_after_sync();
+      uint32_t sreg[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, sreg[c]);
+      tmem_wait_ld();
+      // valid key columns of this row in this tile: [lo, hi]
+      int lo = i - p.w + 1 - j0;
+      if (lo < 0) lo = 0;
+      int hi = i - j0;
+      if (hi > 127) hi = 127;
+      const bool full = (lo == 0) && (hi == 127);
+      float mt = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          float s = __uint_as_float(sreg[c][j]) * p.scale_log2;
+          if (!full) {
+            const int col = c * 32 + j;
+            if (col < lo || col > hi) s = -INFINITY;
+          }
+          sreg[c][j] = __float_as_uint(s);
+          mt = fmaxf(mt, s);
+        }
+      }
+      // lazy rescale of what has been accumulated so far
+      float alpha = 1.f;
+      bool need = false;
+      if (mt > m_ref + kRescaleThreshold) {  // also true for the first finite maximum
+        need = (m_ref != -INFINITY);         // nothing accumulated yet otherwise (O row and l are 0)
+        alpha = need ? exp2f(m_ref - mt) : 1.f;
+        m_ref = mt;
+        l *= alpha;
+      }
+      if (it > 0) {
+        if (__any_sync(0xffffffffu, need)) {
+          if (!mbar_wait(&pv_done, (it - 1) & 1, p.status, 31)) { ok = false; break; }
+          tc_fence_after_sync();
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t oreg[32];
+            tmem_ld32(tO + lane_off + c * 32, oreg);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) oreg[j] = __float_as_uint(__uint_as_float(oreg[j]) * alpha);
+            tmem_st32(tO + lane_off + c * 32, oreg);
+          }
+          tmem_wait_st();
+        }
+      }
+      const float mref_safe = (m_ref == -INFINITY) ? 0.f : m_ref;
+      float lsum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float p0 = exp2f(__uint_as_float(sreg[c][2 * j]) - mref_safe);
+          const float p1 = exp2f(__uint_as_float(sreg[c][2 * j + 1]) - mref_safe);
+          lsum += p0 + p1;
+          pk[j] = pack_bf16(p0, p1);
+        }
+        tmem_st16(tS + lane_off + c * 16, pk);
+      }
+      l += lsum;
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(&p_full);
+    }
+    // epilogue: O / l -> bf16 -> shared (swizzled, Q's buffer is free by now) -> TMA store
+    if (ok) ok = mbar_wait(&pv_done, (n_tiles - 1) & 1, p.status, 32);
+    tc_fence_after_sync();
+    if (ok) {
+      const float inv = 1.f / l;
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t oreg[32];
+        tmem_ld32(tO + lane_off + c * 32, oreg);
+        tmem_wait_ld();
+        uint8_t* box = sQ + (c >> 1) * 16384;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {  // 4 chunks of 8 columns
+          uint4 val;
+          val.x = pack_bf16(__uint_as_float(oreg[8 * g + 0]) * inv, __uint_as_float(oreg[8 * g + 1]) * inv);
+          val.y = pack_bf16(__uint_as_float(oreg[8 * g + 2]) * inv, __uint_as_float(oreg[8 * g + 3]) * inv);
+          val.z = pack_bf16(__uint_as_float(oreg[8 * g + 4]) * inv, __uint_as_float(oreg[8 * g + 5]) * inv);
+          val.w = pack_bf16(__uint_as_float(oreg[8 * g + 6]) * inv, __uint_as_float(oreg[8 * g + 7]) * inv);
+          const uint32_t col = (c & 1) * 32 + g * 8;
+          *reinterpret_cast<uint4*>(box + swz128_offset(r, col)) = val;
+        }
+      }
+      fence_proxy_async_smem();
+    }
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    if (ok && warp == 2 && elect_one()) {
+      for (int c = 0; c < D / 64; ++c) tma_store_4d(&mo, sQ + c * 16384, c * 64, i0, h, b);
+      tma_store_commit();
+      tma_store_wait_read<0>();
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 256);
+}
+
+}  // namespace
+
+bool tc_window_supported(int N, int d, int w, int dtype) {
+  (void)N;
+  (void)w;
+  return dtype == GF_BF16 && (d == 64 || d == 128);
+}
+
+cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                             int w, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
+                             cudaStream_t stream) {
+  if (h_count <= 0) return cudaSuccess;
+  CUtensorMap mq, mk, mv, mo;
+  if (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128) ||
+      !make_qkv_tensor_map(&mv, v, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mo, o, B, H, N, d, layout, 128))
+    return cudaErrorInvalidValue;
+  WinParams p;
+  p.N = N;
+  p.w = w;
+  p.tiles_back = (w - 1 + 127) / 128;
+  p.scale_log2 = scale * kLog2e;
+  p.h_begin = h_begin;
+  p.status = &ws->status;
+  dim3 grid((N + 127) / 128, h_count, B);
+  cudaError_t e;
+  if (d == 64) {
+    auto kern = window_tc_kernel<64>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, WinSmem<64>::kBytes);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, WinSmem<64>::kBytes, stream>>>(mq, mk, mv, mo, p);
+  } else {
+    auto kern = window_tc_kernel<128>;
+    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, WinSmem<128>::kBytes);
+    if (e != cudaSuccess) return e;
+    kern<<<grid, kThreads, WinSmem<128>::kBytes, stream>>>(mq, mk, mv, mo, p);
+  }
+  note_launch();
+  return cudaGetLastError();
+}
+
 }  // namespace gf
