@@ -39,34 +39,35 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+// One attempt; the hardware may park the thread for up to `hint_ns` while the phase is pending,
+// so a waiting warp does not burn issue slots that the working warps need.
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred P;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 P, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, P;\n\t}\n"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
       : "memory");
   return ok != 0;
 }
 
-// Spin budget of one wait, in SM clock cycles (about one second).
-constexpr long long kWaitCycles = 2000000000LL;
+constexpr uint32_t kWaitHintNs = 1000000u;  // per attempt: 1 ms
+constexpr int kWaitAttempts = 2000;         // about two seconds in total
 
-// Bounded wait.  Returns false after kWaitCycles; the first thread to give up records
+// Bounded wait.  Returns false when the budget is spent; the first thread to give up records
 // (status=1, where) in the two words at `status`.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, unsigned int* status,
                                           unsigned int where) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
   const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity)) {
-    if (clock64() - t0 > kWaitCycles) {
-      if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
-      return false;
-    }
+  for (int it = 0; it < kWaitAttempts; ++it) {
+    if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
+    if (clock64() - t0 > 4000000000LL) break;
   }
-  return true;
+  if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
+  return false;
 }
 
 // ---------------------------------------------------------------- fences

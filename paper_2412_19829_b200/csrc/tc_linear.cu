@@ -12,9 +12,11 @@
 //   warp 1       MMA issuer
 //   warps 2-5    "P group": masks/packs P in TMEM, converts S to bf16 for the next chunk's
 //                readout, divides and stores O (one thread per row / TMEM lane)
-//   warps 6-13   "phi group": applies phi to Q (result goes to TMEM as the A operand of MMA1/MMA2,
-//                together with the per-row dot product with z) and to K (in place in shared
-//                memory, with its column sums for z)
+//   warps 6-13   "phi(Q) group": applies phi to Q; the result goes to TMEM as the A operand of
+//                MMA1/MMA2, together with the per-row dot product with z_{c-1}
+//   warps 14-21  "phi(K) group": applies phi to K in place in shared memory and adds its column
+//                sums to z
+//   warp 22      stores O tiles (staged in the dead V buffer) with TMA
 // TMEM (D=128): P 128 | O 128 | S 128 | phi(Q) 2 x 64 columns = 512.
 // Every wait is bounded; on expiry the kernel records a status word and drains.
 #include "common.cuh"
@@ -25,7 +27,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 448;
+constexpr int kThreads = 736;  // 23 warps, 88 registers each
 constexpr float kLog2e = 1.4426950408889634f;
 
 template <int D>
@@ -46,8 +48,6 @@ struct LinCfg {
 
 struct LinParams {
   int N, h_begin, h_count;
-  Strides st;            // element strides of o
-  __nv_bfloat16* o;
   float* S_io;           // [B, h_count, D, D] or null
   float* z_io;           // [B, h_count, D] or null
   int zero_init;
@@ -57,10 +57,26 @@ struct LinParams {
 struct LinBarriers {
   uint64_t q_full, q_land_free;
   uint64_t k_full[2], v_full[2], k_free[2], v_free[2];
-  uint64_t qphi_full[2], kphi_full[2], qphi_free[2];
+  uint64_t qphi_full[2], kphi_full[2], qphi_free[2], qz_free[2];
   uint64_t p_full, s_full, o_full, mma2_done;
-  uint64_t pm_full, s_loaded, sb_full, o_free;
+  uint64_t pm_full, s_loaded, sb_full, o_free, o_staged;
 };
+
+// Developer instrumentation (compiled only with -DGF_PROFILE): per-role time stamps of the first
+// chunks of CTA (0,0), read back with gformer_debug_read_profile.
+#ifdef GF_PROFILE
+__device__ unsigned long long g_prof[4][64][8];
+__device__ __forceinline__ void prof_stamp(int role, int c, int ev) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && c < 64) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    g_prof[role][c][ev] = t;
+  }
+}
+#define PROF(role, c, ev) prof_stamp(role, c, ev)
+#else
+#define PROF(role, c, ev)
+#endif
 
 // Named barrier over `n` threads that also ORs a predicate, so that a timed-out wait makes the
 // whole group leave its loop together (nobody is left behind at a barrier).
@@ -77,12 +93,28 @@ __device__ __forceinline__ bool named_bar_or(int id, int n, bool pred) {
   return r != 0;
 }
 
-__device__ __forceinline__ float phi_fast(float x) { return x > 0.f ? x + 1.f : exp2f(x * kLog2e); }
+// phi(x) = elu(x) + 1 = max(x, 0) + exp(min(x, 0)) on two packed bf16 values (branch free; the
+// result is needed in bf16 anyway).  log2(e) is split in two bf16 terms so that the exponent
+// argument carries only the rounding of one bf16 product.
+__device__ __forceinline__ uint32_t phi_bf16x2(uint32_t w) {
+  const __nv_bfloat162 x = *reinterpret_cast<const __nv_bfloat162*>(&w);
+  const __nv_bfloat162 zero = __float2bfloat162_rn(0.f);
+  const __nv_bfloat162 l2e_hi = __float2bfloat162_rn(1.4453125f);
+  const __nv_bfloat162 l2e_lo = __float2bfloat162_rn(kLog2e - 1.4453125f);
+  const __nv_bfloat162 t = __hmin2(__hfma2(x, l2e_lo, __hmul2(x, l2e_hi)), zero);
+  uint32_t e;  // native packed exponential (the header's h2exp2 goes through two fp32 ex2 + converts)
+  asm("ex2.approx.ftz.bf16x2 %0, %1;" : "=r"(e) : "r"(*reinterpret_cast<const uint32_t*>(&t)));
+  const __nv_bfloat162 f = __hadd2(__hmax2(x, zero), *reinterpret_cast<const __nv_bfloat162*>(&e));
+  return *reinterpret_cast<const uint32_t*>(&f);
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
-                 const __grid_constant__ CUtensorMap mv, const LinParams p) {
+                 const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
+                 const LinParams p) {
   using C = LinCfg<D>;
   extern __shared__ uint8_t raw_smem[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw_smem) + 1023) & ~(uintptr_t)1023);
@@ -91,8 +123,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint8_t* sV = sm + C::kV;
   uint8_t* sSb = sm + C::kSb;
   __shared__ __align__(8) LinBarriers bar;
-  __shared__ __align__(16) float zs[2][D];       // z before chunk c is zs[c & 1]
-  __shared__ float qz[2][2][128];                // [chunk parity][column half][row]
+  __shared__ __align__(16) float zs[4][D];  // z before chunk c is zs[c & 3]
+  __shared__ float qz[2][2][128];           // [chunk parity][column half][row]
+  __shared__ int z_ready;                   // chunks whose column sums are in zs (monotonic)
   __shared__ uint32_t tmem_base_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -112,6 +145,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(&bar.qphi_full[s], 8);
       mbar_init(&bar.kphi_full[s], 8);
       mbar_init(&bar.qphi_free[s], 1);
+      mbar_init(&bar.qz_free[s], 128);
     }
     mbar_init(&bar.p_full, 1);
     mbar_init(&bar.s_full, 1);
@@ -121,10 +155,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.s_loaded, 128);
     mbar_init(&bar.sb_full, 128);
     mbar_init(&bar.o_free, 128);
+    mbar_init(&bar.o_staged, 128);
+    z_ready = -1;
     mbar_fence_init();
     tma_prefetch_desc(&mq);
     tma_prefetch_desc(&mk);
     tma_prefetch_desc(&mv);
+    tma_prefetch_desc(&mo);
   }
   if (warp == 1) {
     tmem_alloc(&tmem_base_s, C::kTmemCols);
@@ -140,14 +177,17 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     if (elect_one()) {
       for (int c = 0; c < nch; ++c) {
         const int s = c & 1, n0 = c * 128;
-        if (c >= 1 && !mbar_wait(&bar.q_land_free, (c - 1) & 1, p.status, 100)) break;
-        mbar_arrive_expect_tx(&bar.q_full, C::kTile);
-        for (int x = 0; x < D / 64; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, h, b);
         if (c >= 2 && !mbar_wait(&bar.k_free[s], ((c >> 1) + 1) & 1, p.status, 101)) break;
+        PROF(0, c, 1);
         mbar_arrive_expect_tx(&bar.k_full[s], C::kTile);
         for (int x = 0; x < D / 64; ++x)
           tma_load_4d(sK + s * C::kTile + x * C::kBoxBytes, &mk, &bar.k_full[s], x * 64, n0, h, b);
+        if (c >= 1 && !mbar_wait(&bar.q_land_free, (c - 1) & 1, p.status, 100)) break;
+        PROF(0, c, 0);
+        mbar_arrive_expect_tx(&bar.q_full, C::kTile);
+        for (int x = 0; x < D / 64; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, h, b);
         if (c >= 2 && !mbar_wait(&bar.v_free[s], ((c >> 1) + 1) & 1, p.status, 102)) break;
+        PROF(0, c, 2);
         mbar_arrive_expect_tx(&bar.v_full[s], C::kTile);
         for (int x = 0; x < D / 64; ++x)
           tma_load_4d(sV + s * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[s], x * 64, n0, h, b);
@@ -167,6 +207,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         const uint32_t tq = tmem + C::tQ + s * (D / 2);
         if (!mbar_wait(&bar.qphi_full[s], ph2, p.status, 200)) break;
         if (!mbar_wait(&bar.kphi_full[s], ph2, p.status, 201)) break;
+        PROF(1, c, 0);
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
@@ -175,6 +216,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         umma_commit(&bar.p_full);
         if (!mbar_wait(&bar.v_full[s], ph2, p.status, 202)) break;
         if (!mbar_wait(&bar.s_loaded, c & 1, p.status, 203)) break;
+        PROF(1, c, 1);
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
@@ -184,6 +226,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         umma_commit(&bar.k_free[s]);
         if (!mbar_wait(&bar.sb_full, c & 1, p.status, 204)) break;
         if (c >= 1 && !mbar_wait(&bar.o_free, (c - 1) & 1, p.status, 205)) break;
+        PROF(1, c, 2);
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
@@ -192,13 +235,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         umma_commit(&bar.mma2_done);
         umma_commit(&bar.qphi_free[s]);
         if (!mbar_wait(&bar.pm_full, c & 1, p.status, 206)) break;
+        PROF(1, c, 3);
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks)
           umma_ts(tmem + C::tO, tmem + C::tP + ks * 8, umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
                   id_o, true);
         umma_commit(&bar.o_full);
-        umma_commit(&bar.v_free[s]);
       }
     }
   } else if (warp < 6) {
@@ -237,133 +280,160 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     }
     for (int c = 0; c < nch; ++c) {
       const int s = c & 1;
-      const int i = c * 128 + r;
       // ---- P: causal mask inside the chunk, row sum, bf16 back into TMEM
       if (!mbar_wait(&bar.qphi_full[s], (c >> 1) & 1, p.status, 300)) break;
+      const float qzr = qz[s][0][r] + qz[s][1][r];
+      mbar_arrive(&bar.qz_free[s]);
       if (!mbar_wait(&bar.p_full, c & 1, p.status, 301)) break;
+      if (tid == 64) PROF(2, c, 0);
       tc_fence_after_sync();
       float rowsum = 0.f;
 #pragma unroll
       for (int cc = 0; cc < 4; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
-        tmem_wait_ld();
+        // 32-column block cc of this warp's rows [32 q, 32 q + 32): all kept left of the
+        // diagonal block, all dropped right of it, triangular on it (warp-uniform choice)
         uint32_t pk[16];
+        if (cc > quarter) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const int col = cc * 32 + 2 * j;
-          const float p0 = (col <= r) ? __uint_as_float(v[2 * j]) : 0.f;
-          const float p1 = (col + 1 <= r) ? __uint_as_float(v[2 * j + 1]) : 0.f;
-          rowsum += p0 + p1;
-          pk[j] = pack_bf16(p0, p1);
+          for (int j = 0; j < 16; ++j) pk[j] = 0u;
+        } else {
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
+          tmem_wait_ld();
+          const bool diag = (cc == quarter);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            const float p0 = (!diag || 2 * j <= lane) ? __uint_as_float(v[2 * j]) : 0.f;
+            const float p1 = (!diag || 2 * j + 1 <= lane) ? __uint_as_float(v[2 * j + 1]) : 0.f;
+            rowsum += p0 + p1;
+            pk[j] = pack_bf16(p0, p1);
+          }
         }
         tmem_st16(tmem + C::tP + lane_off + cc * 16, pk);
       }
-      const float den = rowsum + qz[s][0][r] + qz[s][1][r];
+      const float den = rowsum + qzr;
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(&bar.pm_full);
-      // ---- S: fp32 master stays in TMEM; refresh the bf16 copy used by the next chunk's readout
+      if (tid == 64) PROF(2, c, 1);
+      // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old bf16
+      //      copy, stream the new one into shared memory for the next chunk
       if (!mbar_wait(&bar.s_full, c & 1, p.status, 302)) break;
+      if (tid == 64) PROF(2, c, 2);
+      if (!mbar_wait(&bar.mma2_done, c & 1, p.status, 303)) break;
+      if (tid == 64) PROF(2, c, 3);
       tc_fence_after_sync();
-      uint32_t sp[D / 2];
       const bool last = (c == nch - 1);
 #pragma unroll
       for (int cc = 0; cc < D / 32; ++cc) {
         uint32_t v[32];
         tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
         tmem_wait_ld();
+        if (s_row) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j)
-          sp[cc * 16 + j] = pack_bf16(__uint_as_float(v[2 * j]), __uint_as_float(v[2 * j + 1]));
-        if (last && p.S_io != nullptr && s_row) {
-          float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
+          for (int g = 0; g < 4; ++g) {
+            uint4 val;
+            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+            *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+          }
+          if (last && p.S_io != nullptr) {
+            float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
 #pragma unroll
-          for (int j = 0; j < 32; j += 4)
-            *reinterpret_cast<float4*>(dst + j) =
-                make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                            __uint_as_float(v[j + 3]));
+            for (int j = 0; j < 32; j += 4)
+              *reinterpret_cast<float4*>(dst + j) =
+                  make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
+                              __uint_as_float(v[j + 3]));
+          }
         }
       }
       tc_fence_before_sync();
       mbar_arrive(&bar.s_loaded);
-      if (!mbar_wait(&bar.mma2_done, c & 1, p.status, 303)) break;  // readout of chunk c has consumed Sb
-      if (s_row) {
-#pragma unroll
-        for (int g = 0; g < D / 8; ++g) {
-          uint4 val = make_uint4(sp[4 * g], sp[4 * g + 1], sp[4 * g + 2], sp[4 * g + 3]);
-          *reinterpret_cast<uint4*>(sSb + (g >> 3) * C::kSbBox + swz128_offset(r, (g & 7) * 8)) = val;
-        }
-      }
       fence_proxy_async_smem();
       mbar_arrive(&bar.sb_full);
-      // ---- O: divide by the denominator, bf16, store
+      if (tid == 64) PROF(2, c, 5);
+      // ---- O: divide by the denominator, bf16, stage for the TMA store
       if (!mbar_wait(&bar.o_full, c & 1, p.status, 304)) break;
+      if (tid == 64) PROF(2, c, 6);
       tc_fence_after_sync();
       const float inv = 1.f / den;
-      __nv_bfloat16* orow = p.o + (long long)b * p.st.b + (long long)h * p.st.h + (long long)i * p.st.n;
+      uint8_t* stage = sV + s * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
 #pragma unroll
       for (int cc = 0; cc < D / 32; ++cc) {
         uint32_t v[32];
         tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
         tmem_wait_ld();
-        if (i < p.N) {
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 val;
-            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
-            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
-            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
-            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4*>(orow + cc * 32 + g * 8) = val;
-          }
+        for (int g = 0; g < 4; ++g) {
+          uint4 val;
+          val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
+          val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
+          val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
+          val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
+          *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
         }
       }
       tc_fence_before_sync();
       mbar_arrive(&bar.o_free);
+      fence_proxy_async_smem();
+      mbar_arrive(&bar.o_staged);
+      if (tid == 64) PROF(2, c, 7);
     }
-  } else {
-    // ================================================================ phi group (8 warps)
-    const int tt = tid - 6 * 32;          // 0..255
+  } else if (warp < 14) {
+    // ================================================================ phi(Q) group (8 warps)
     const int quarter = warp & 3;         // TMEM lane quarter of this warp
-    const int half = (warp - 6) >> 2;     // which half of the head dimension this warp handles for Q
+    const int half = (warp - 6) >> 2;     // which half of the head dimension this warp handles
     const int r = quarter * 32 + lane;    // Q row
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per thread
-    if (tt < D) zs[0][tt] = (p.z_io != nullptr && !p.zero_init) ? p.z_io[sidx * D + tt] : 0.f;
-    asm volatile("bar.sync 2, 256;" ::: "memory");
     for (int c = 0; c < nch; ++c) {
       const int s = c & 1;
-      // ---- Q: phi, pack into TMEM as the A operand, dot with z_{c-1}
       bool ok = mbar_wait(&bar.q_full, c & 1, p.status, 400);
+      if (tid == 192) PROF(3, c, 0);
       if (ok && c >= 2) {
-        ok = mbar_wait(&bar.qphi_free[s], ((c >> 1) + 1) & 1, p.status, 401) &&
-             mbar_wait(&bar.pm_full, c & 1, p.status, 402);  // qz[s] of chunk c-2 has been read
+        ok = mbar_wait(&bar.qphi_free[s], ((c >> 1) + 1) & 1, p.status, 401) &&  // phi(Q) buffer s is free
+             mbar_wait(&bar.qz_free[s], ((c >> 1) + 1) & 1, p.status, 402);      // qz[s] of chunk c-2 was read
       }
+      // z before this chunk = column sums of chunks < c, published by the phi(K) group
+      if (ok) {
+        const long long t0 = clock64();
+        while (*reinterpret_cast<volatile int*>(&z_ready) < c) {
+          if (clock64() - t0 > 4000000000LL) {
+            if (atomicCAS(p.status, 0u, 1u) == 0u) p.status[1] = 403;
+            ok = false;
+            break;
+          }
+          __nanosleep(32);
+        }
+        __threadfence_block();
+      }
+      if (tid == 192) PROF(3, c, 1);
       tc_fence_after_sync();
       if (ok) {
         uint32_t pk[kChunksPerHalf * 4];
-        float dot = 0.f;
-        const float* zc = zs[s];
+        float dot[2] = {0.f, 0.f};
+        const float* zc = zs[c & 3];
 #pragma unroll
         for (int g = 0; g < kChunksPerHalf; ++g) {
           const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
           const int box = gl >> 3, cin = gl & 7;
           const uint4 rawv = *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
           const uint32_t w4[4] = {rawv.x, rawv.y, rawv.z, rawv.w};
+          const float4 za = *reinterpret_cast<const float4*>(zc + gl * 8);
+          const float4 zb = *reinterpret_cast<const float4*>(zc + gl * 8 + 4);
+          const float zv[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float x0 = __uint_as_float(w4[e] << 16);
-            const float x1 = __uint_as_float(w4[e] & 0xffff0000u);
-            const float f0 = phi_fast(x0), f1 = phi_fast(x1);
-            const uint32_t pkv = pack_bf16(f0, f1);
+            const uint32_t pkv = phi_bf16x2(w4[e]);
             pk[g * 4 + e] = pkv;
             // the dot product uses the rounded values the tensor core will see
-            dot = fmaf(__uint_as_float(pkv << 16), zc[gl * 8 + 2 * e], dot);
-            dot = fmaf(__uint_as_float(pkv & 0xffff0000u), zc[gl * 8 + 2 * e + 1], dot);
+            dot[e & 1] = fmaf(bf16_lo(pkv), zv[2 * e], dot[e & 1]);
+            dot[e & 1] = fmaf(bf16_hi(pkv), zv[2 * e + 1], dot[e & 1]);
           }
         }
-        qz[s][half][r] = dot;
+        qz[s][half][r] = dot[0] + dot[1];
         if constexpr (D == 128) {
           uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
           tmem_st32(tmem + C::tQ + s * (D / 2) + lane_off + half * 32, pk32);
@@ -378,34 +448,55 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           mbar_arrive(&bar.q_land_free);
         }
       }
-      if (named_bar_or(2, 256, !ok)) break;
-      // ---- K: phi in place (rows past N become 0), column sums -> z_c
-      ok = mbar_wait(&bar.k_full[s], (c >> 1) & 1, p.status, 403);
+      if (tid == 192) PROF(3, c, 2);
+      if (__any_sync(0xffffffffu, !ok)) break;
+    }
+  } else if (warp < 22) {
+    // ================================================================ phi(K) group (8 warps)
+    const int tt = tid - 14 * 32;  // 0..255
+    if (tt < D) zs[0][tt] = (p.z_io != nullptr && !p.zero_init) ? p.z_io[sidx * D + tt] : 0.f;
+    asm volatile("bar.sync 3, 256;" ::: "memory");
+    if (tt == 0) {
+      __threadfence_block();
+      *reinterpret_cast<volatile int*>(&z_ready) = 0;  // zs[0] holds the initial z
+    }
+    for (int c = 0; c < nch; ++c) {
+      const int s = c & 1;
+      const bool ok = mbar_wait(&bar.k_full[s], (c >> 1) & 1, p.status, 410);
+      if (tt == 0) PROF(3, c, 4);
       if (ok && tt < 2 * D) {
-        const int cc = tt >> 4;        // logical 16-byte column chunk 0 .. D/8-1
+        const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
         const int box = cc >> 3, cin = cc & 7;
         uint8_t* kb = sK + s * C::kTile + box * C::kBoxBytes;
         float cs[8];
 #pragma unroll
         for (int e = 0; e < 8; ++e) cs[e] = 0.f;
+        // all loads first, then branch-free arithmetic, then all stores (the tile is updated in place)
+        uint4 rawv[8];
 #pragma unroll
         for (int k8 = 0; k8 < 8; ++k8) {
           const int row = (tt & 15) + 16 * k8;
-          uint4* ptr = reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
-          const uint4 rawv = *ptr;
-          const uint32_t w4[4] = {rawv.x, rawv.y, rawv.z, rawv.w};
-          uint32_t o4[4];
-          const bool valid = (c * 128 + row) < p.N;
+          rawv[k8] = *reinterpret_cast<const uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
+        }
+#pragma unroll
+        for (int k8 = 0; k8 < 8; ++k8) {
+          const int row = (tt & 15) + 16 * k8;
+          const uint32_t keep = ((c * 128 + row) < p.N) ? 0xffffffffu : 0u;  // rows past N must not enter S, z
+          uint32_t w4[4] = {rawv[k8].x, rawv[k8].y, rawv[k8].z, rawv[k8].w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            const float f0 = valid ? phi_fast(__uint_as_float(w4[e] << 16)) : 0.f;
-            const float f1 = valid ? phi_fast(__uint_as_float(w4[e] & 0xffff0000u)) : 0.f;
-            o4[e] = pack_bf16(f0, f1);
-            cs[2 * e] += __uint_as_float(o4[e] << 16);
-            cs[2 * e + 1] += __uint_as_float(o4[e] & 0xffff0000u);
+            w4[e] = phi_bf16x2(w4[e]) & keep;
+            cs[2 * e] += bf16_lo(w4[e]);
+            cs[2 * e + 1] += bf16_hi(w4[e]);
           }
-          *ptr = make_uint4(o4[0], o4[1], o4[2], o4[3]);
+          rawv[k8] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
         }
+#pragma unroll
+        for (int k8 = 0; k8 < 8; ++k8) {
+          const int row = (tt & 15) + 16 * k8;
+          *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k8];
+        }
+        fence_proxy_async_smem();
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
 #pragma unroll
@@ -413,15 +504,33 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         }
         if ((tt & 15) == 0) {
 #pragma unroll
-          for (int e = 0; e < 8; ++e) zs[s ^ 1][cc * 8 + e] = zs[s][cc * 8 + e] + cs[e];
+          for (int e = 0; e < 8; ++e) zs[(c + 1) & 3][cc * 8 + e] = zs[c & 3][cc * 8 + e] + cs[e];
         }
-        fence_proxy_async_smem();
       }
       __syncwarp();
       if (ok && lane == 0) mbar_arrive(&bar.kphi_full[s]);
-      if (named_bar_or(2, 256, !ok)) break;
+      if (tt == 0) PROF(3, c, 5);
+      if (named_bar_or(3, 256, !ok)) break;
+      if (tt == 0) {
+        __threadfence_block();
+        *reinterpret_cast<volatile int*>(&z_ready) = c + 1;
+      }
     }
-    if (p.z_io != nullptr && tt < D) p.z_io[sidx * D + tt] = zs[nch & 1][tt];
+    if (p.z_io != nullptr && tt < D) p.z_io[sidx * D + tt] = zs[nch & 3][tt];
+  } else {
+    // ================================================================ O store warp
+    if (elect_one()) {
+      for (int c = 0; c < nch; ++c) {
+        const int s = c & 1;
+        if (!mbar_wait(&bar.o_staged, c & 1, p.status, 500)) break;
+        for (int x = 0; x < D / 64; ++x)
+          tma_store_4d(&mo, sV + s * C::kTile + x * C::kBoxBytes, x * 64, c * 128, h, b);
+        tma_store_commit();
+        tma_store_wait_read<0>();
+        mbar_arrive(&bar.v_free[s]);  // the staging buffer may take V of chunk c+2
+      }
+      tma_store_wait_all<0>();
+    }
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -429,6 +538,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 }
 
 }  // namespace
+
+#ifdef GF_PROFILE
+extern "C" int gformer_debug_read_profile(unsigned long long* host_dst) {
+  return (int)cudaMemcpyFromSymbol(host_dst, g_prof, sizeof(g_prof));
+}
+#endif
 
 bool tc_linear_supported(int N, int d, int dtype) {
   (void)N;
@@ -440,16 +555,14 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
                              int split, WsHeader* ws, cudaStream_t stream) {
   (void)split;
   if (h_count <= 0) return cudaSuccess;
-  CUtensorMap mq, mk, mv;
+  CUtensorMap mq, mk, mv, mo;
   if (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128) ||
-      !make_qkv_tensor_map(&mv, v, B, H, N, d, layout, 128))
+      !make_qkv_tensor_map(&mv, v, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mo, o, B, H, N, d, layout, 128))
     return cudaErrorInvalidValue;
   LinParams p;
   p.N = N;
   p.h_begin = h_begin;
   p.h_count = h_count;
-  p.st = make_strides(layout, H, N, d);
-  p.o = (__nv_bfloat16*)o;
   p.S_io = S_io;
   p.z_io = z_io;
   p.zero_init = zero_init ? 1 : 0;
@@ -460,12 +573,12 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
     auto kern = linear_tc_kernel<64>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, LinCfg<64>::kBytes);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, LinCfg<64>::kBytes, stream>>>(mq, mk, mv, p);
+    kern<<<grid, kThreads, LinCfg<64>::kBytes, stream>>>(mq, mk, mv, mo, p);
   } else {
     auto kern = linear_tc_kernel<128>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, LinCfg<128>::kBytes);
     if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, LinCfg<128>::kBytes, stream>>>(mq, mk, mv, p);
+    kern<<<grid, kThreads, LinCfg<128>::kBytes, stream>>>(mq, mk, mv, mo, p);
   }
   note_launch();
   return cudaGetLastError();
