@@ -180,7 +180,7 @@ def run_ours(args, c, rank, world, local_rank):
     ho = torch.empty_like(hq).pin_memory()
     dq, dk, dv = [t.cuda() for t in (hq, hk, hv)]
     do = torch.empty_like(dq)
-    ws = gf.Workspace()
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
     stream = torch.cuda.Stream()
 
     def barrier():

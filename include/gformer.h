@@ -19,8 +19,10 @@
  *     anything is launched and leave every buffer untouched.  Nothing throws or aborts.
  *   - `ws` is caller-provided device scratch of at least gformer_workspace_bytes(...)
  *     bytes, 256-byte aligned; the tensor-core (bf16) kernels keep a device status word
- *     there.  The library clears what it needs inside the call, so ws may hold anything
- *     on entry, but two calls that run concurrently must not share one ws.
+ *     there, and the linear-attention kernel the per-segment states and flags through
+ *     which the CTAs that share one (batch, head) chain hand the running state on.  The
+ *     library clears what it needs inside the call, so ws may hold anything on entry, but
+ *     two calls that run concurrently must not share one ws.
  *   - o must not alias an input.
  */
 #ifndef GFORMER_H_
@@ -49,7 +51,7 @@ typedef enum { GF_PHI_ELU1 = 0 } gf_phi;
 /* Process-wide knobs for tests and benchmarks (gformer_set_tuning). */
 typedef enum {
   GF_TUNE_FORCE_SIMT = 0, /* 1: never take the tensor-core kernels (default 0)              */
-  GF_TUNE_LINEAR_SPLIT = 1 /* CTAs cooperating on one linear (b,h) chain: 0 = auto, 1, 2, 4 */
+  GF_TUNE_LINEAR_SPLIT = 1 /* 128-row chunks per sequence segment of a linear chain: 0 = auto    */
 } gf_tuning_key;
 
 /* Decode-time state of one batch (see gformer_decode_step).  The struct lives in host

@@ -137,6 +137,11 @@ class Workspace:
         self.ptr = self.buf.data_ptr() + off
         self.nbytes = self.buf.numel() - off
 
+    @classmethod
+    def for_problem(cls, B, H, N, d, w=1, h_sparse=0, dtype=GF_BF16, device=None):
+        """Scratch sized by gformer_workspace_bytes for this problem."""
+        return cls(workspace_bytes(B, H, N, d, w, h_sparse, dtype), device)
+
     def last_device_status(self, stream=None) -> int:
         return int(lib().gformer_last_device_status(self.ptr, _stream_ptr(stream)))
 

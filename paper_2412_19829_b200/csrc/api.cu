@@ -138,7 +138,7 @@ int gformer_set_tuning(int key, int value) {
       g_force_simt = value ? 1 : 0;
       return GF_OK;
     case GF_TUNE_LINEAR_SPLIT:
-      if (value != 0 && value != 1 && value != 2 && value != 4) return GF_ERR_INVALID_ARG;
+      if (value < 0 || value > 4096) return GF_ERR_INVALID_ARG;
       g_linear_split = value;
       return GF_OK;
     default:
@@ -147,8 +147,15 @@ int gformer_set_tuning(int key, int value) {
 }
 
 size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, int dtype) {
-  (void)B; (void)H; (void)N; (void)d; (void)w; (void)h_sparse; (void)dtype;
-  return sizeof(WsHeader);
+  (void)w;
+  size_t bytes = sizeof(WsHeader);
+  if (B < 1 || H < 1 || N < 1) return bytes;
+  if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
+  if (h_sparse > H) h_sparse = H;
+  const int h_lin = H - h_sparse;
+  if (h_lin > 0 && !g_force_simt && gf::tc_linear_supported(N, d, dtype))
+    bytes += gf::linear_tc_workspace_bytes(B * h_lin, N, d, g_linear_split);
+  return bytes;
 }
 
 int gformer_last_device_status(void* ws, void* cuda_stream) {

@@ -7,7 +7,16 @@
 //   O   = Qc Sb_{c-1}  (+)  Pm V_c      (MMA2, MMA3)  Sb = bf16 copy of S in shared memory
 //   den = rowsum(Pm) + Qc z_{c-1},  z_c = z_{c-1} + colsum(Kc)      (fp32, CUDA cores)
 //   out = O / den
-// One CTA walks one (batch, head) chain.  Warp roles:
+// A (batch, head) chain is cut into segments of L chunks; a work item is one segment.  CTAs are
+// persistent and take items round-robin in an order in which a segment's predecessor always has
+// a smaller index, so the CTA that owns it is already running.  For an item the CTA
+//   (A) accumulates the segment's own state contribution dS = sum Kc^T V, dz = sum colsum(Kc)
+//       (K, V only; skipped for a chain's last segment and when a chain is a single segment),
+//   (B) waits for the inclusive state of the previous segment in global scratch (bounded
+//       spin), publishes its own inclusive state = previous + dS and raises its flag,
+//   (C) walks its chunks with the full pipeline starting from the previous segment's state
+//       (K and V come from L2 this second time).
+// Warp roles:
 //   warp 0       TMA producer (raw Q, K, V tiles; K and V double buffered)
 //   warp 1       MMA issuer
 //   warps 2-5    "P group": masks/packs P in TMEM, converts S to bf16 for the next chunk's
@@ -29,6 +38,7 @@ using namespace sm100;
 
 constexpr int kThreads = 736;  // 23 warps, 88 registers each
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr int kFlagStride = 32;  // one flag per 128-byte line
 
 template <int D>
 struct LinCfg {
@@ -44,23 +54,84 @@ struct LinCfg {
   // TMEM columns
   static constexpr uint32_t tP = 0, tO = 128, tS = 128 + D, tQ = 128 + 2 * D;  // tQ: 2 x D/2
   static constexpr uint32_t kTmemCols = 512;
+  // One published state: S then z.  S is stored [column/4][128 rows][4] so that the threads of a
+  // warp (one row each, the TMEM lane order) touch consecutive 16-byte pieces.
+  static constexpr int kStateZ = 128 * D;
+  static constexpr int kStateFloats = 128 * D + D;
 };
 
 struct LinParams {
-  int N, h_begin, h_count;
+  int N, nch, h_begin, h_count, nchains;
+  int L, G, nitems;      // chunks per segment, segments per chain, nchains * G
   float* S_io;           // [B, h_count, D, D] or null
   float* z_io;           // [B, h_count, D] or null
   int zero_init;
-  unsigned int* status;
+  unsigned int* status;  // two words: status, where
+  unsigned int* flags;   // [nchains * G] x kFlagStride: 1 once the segment's inclusive state is in `prefix`
+  float* prefix;         // [nchains * G][D*D + D]
 };
+
+struct LinItem {
+  int g, chain, b, hl, h, c_begin, nC, nA;
+  bool last_seg;
+};
+
+__device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
+  LinItem it;
+  it.g = item / p.nchains;
+  it.chain = item - it.g * p.nchains;
+  it.b = it.chain / p.h_count;
+  it.hl = it.chain - it.b * p.h_count;
+  it.h = p.h_begin + it.hl;
+  it.c_begin = it.g * p.L;
+  const int c_end = (it.c_begin + p.L < p.nch) ? it.c_begin + p.L : p.nch;
+  it.nC = c_end - it.c_begin;
+  it.last_seg = (it.g == p.G - 1);
+  it.nA = it.last_seg ? 0 : it.nC;  // the last segment's contribution is needed by nobody
+  return it;
+}
 
 struct LinBarriers {
   uint64_t q_full, q_land_free;
   uint64_t k_full[2], v_full[2], k_free[2], v_free[2];
   uint64_t qphi_full[2], kphi_full[2], qphi_free[2], qz_free[2];
-  uint64_t p_full, s_full, o_full, mma2_done;
+  uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, prev_ready;
   uint64_t pm_full, s_loaded, sb_full, o_free, o_staged;
 };
+
+// Bounded poll of a monotonic counter in shared memory.
+__device__ __forceinline__ bool wait_epoch(const int* counter, int target, unsigned int* status,
+                                           unsigned int where) {
+  const volatile int* c = counter;
+  if (*c >= target) { __threadfence_block(); return true; }
+  const long long t0 = clock64();
+  while (*c < target) {
+    if (clock64() - t0 > 4000000000LL) {
+      if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
+      return false;
+    }
+    __nanosleep(20);
+  }
+  __threadfence_block();
+  return true;
+}
+
+// Bounded poll of a flag in global memory written by another CTA (acquire).
+__device__ __forceinline__ bool wait_flag(const unsigned int* flag, unsigned int* status, unsigned int where) {
+  unsigned int v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+  if (v != 0u) return true;
+  const long long t0 = clock64();
+  while (true) {
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v != 0u) return true;
+    if (clock64() - t0 > 4000000000LL) {
+      if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
+      return false;
+    }
+    __nanosleep(100);
+  }
+}
 
 // Developer instrumentation (compiled only with -DGF_PROFILE): per-role time stamps of the first
 // chunks of CTA (0,0), read back with gformer_debug_read_profile.
@@ -73,9 +144,19 @@ __device__ __forceinline__ void prof_stamp(int role, int c, int ev) {
     g_prof[role][c][ev] = t;
   }
 }
+__device__ unsigned long long g_prof2[64][8];  // per CTA: hand-over time line of its first item
+__device__ __forceinline__ void prof2_stamp(int ev) {
+  if (blockIdx.x < 64) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    g_prof2[blockIdx.x][ev] = t;
+  }
+}
 #define PROF(role, c, ev) prof_stamp(role, c, ev)
+#define PROF2(cond, ev) do { if (cond) prof2_stamp(ev); } while (0)
 #else
 #define PROF(role, c, ev)
+#define PROF2(cond, ev)
 #endif
 
 // Named barrier over `n` threads that also ORs a predicate, so that a timed-out wait makes the
@@ -110,6 +191,70 @@ __device__ __forceinline__ uint32_t phi_bf16x2(uint32_t w) {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// Critical path of the segment hand-over, run by the 16 phi warps (4 per TMEM lane quarter, each
+// thread one row x 32 columns): inclusive state of this segment = inclusive state of the previous
+// one (global scratch, or the caller's initial state for the first segment) + this segment's own
+// contribution (still in TMEM after pass A).  One batch of loads, one batch of stores, a fence and
+// an arrival; the flag itself is raised by the store warp once every warp has arrived.
+template <int D>
+__device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinItem& it, LinBarriers& bar,
+                                                  uint32_t tmem, int warp, int lane, uint32_t a_parity,
+                                                  uint32_t item_parity) {
+  using C = LinCfg<D>;
+  const int quarter = warp & 3, colq = (warp - 6) >> 2;  // colq 0..3: which 32 columns (D=128) / 16 (D=64)
+  const int r = quarter * 32 + lane;
+  constexpr int W = D / 4;  // columns per thread
+  const long long slot = (long long)it.chain * p.G + it.g;
+  bool ok = mbar_wait(&bar.a_done, a_parity, p.status, 600);
+  tc_fence_after_sync();
+  PROF2(warp == 6 && lane == 0 && a_parity == 0, 0);
+  // one thread of the CTA (store warp) polls the previous segment's flag for everybody
+  ok = ok && mbar_wait(&bar.prev_ready, item_parity, p.status, 601);
+  PROF2(warp == 6 && lane == 0 && a_parity == 0, 1);
+  if (ok) {
+    uint32_t ds[W];
+    if constexpr (D == 128) {
+      uint32_t(&d32)[32] = *reinterpret_cast<uint32_t(*)[32]>(ds);
+      tmem_ld32(tmem + C::tS + ((uint32_t)(quarter * 32) << 16) + colq * 32, d32);
+    } else {
+      tmem_ld16(tmem + C::tS + ((uint32_t)(quarter * 32) << 16) + colq * 16, ds);
+    }
+    if (r < D) {
+      const float* Sin = nullptr;
+      long long sin_stride = 1;  // in float4 units between consecutive column groups of one row
+      if (it.g > 0) {
+        Sin = p.prefix + (slot - 1) * C::kStateFloats + ((long long)(colq * (W / 4)) * 128 + r) * 4;
+        sin_stride = 128;
+      } else if (p.S_io != nullptr && !p.zero_init) {
+        Sin = p.S_io + (((long long)it.b * p.h_count + it.hl) * D + r) * D + colq * W;  // caller's row-major state
+      }
+      float4 in[W / 4];
+#pragma unroll
+      for (int j = 0; j < W / 4; ++j)
+        in[j] = (Sin != nullptr) ? __ldcg(reinterpret_cast<const float4*>(Sin) + j * sin_stride)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+      tmem_wait_ld();
+      PROF2(warp == 6 && lane == 0 && a_parity == 0, 2);
+      float* Sout = p.prefix + slot * C::kStateFloats + ((long long)(colq * (W / 4)) * 128 + r) * 4;
+#pragma unroll
+      for (int j = 0; j < W / 4; ++j)
+        __stcg(reinterpret_cast<float4*>(Sout) + j * 128,
+               make_float4(in[j].x + __uint_as_float(ds[4 * j]), in[j].y + __uint_as_float(ds[4 * j + 1]),
+                           in[j].z + __uint_as_float(ds[4 * j + 2]), in[j].w + __uint_as_float(ds[4 * j + 3])));
+    } else {
+      tmem_wait_ld();
+    }
+    // No per-thread gpu-scope fence here (hundreds of sequentially consistent fences at once cost
+    // microseconds): the arrival below releases these stores at CTA scope to the store warp, whose
+    // single st.release.gpu on the flag then publishes them (release is cumulative).
+    tc_fence_before_sync();
+    PROF2(warp == 6 && lane == 0 && a_parity == 0, 3);
+  }
+  __syncwarp();
+  if (ok && lane == 0) mbar_arrive(&bar.pub_done);
+  return ok;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
@@ -123,16 +268,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint8_t* sV = sm + C::kV;
   uint8_t* sSb = sm + C::kSb;
   __shared__ __align__(8) LinBarriers bar;
-  __shared__ __align__(16) float zs[4][D];  // z before chunk c is zs[c & 3]
+  __shared__ __align__(16) float zs[8][D];  // running z, one buffer per "version" (index & 7)
   __shared__ float qz[2][2][128];           // [chunk parity][column half][row]
-  __shared__ int z_ready;                   // chunks whose column sums are in zs (monotonic)
+  __shared__ int z_epoch;                   // newest complete version of z (monotonic)
   __shared__ uint32_t tmem_base_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int hl = blockIdx.x, b = blockIdx.y;
-  const int h = p.h_begin + hl;
-  const int nch = (p.N + 127) / 128;
-  const long long sidx = (long long)b * p.h_count + hl;
 
   if (tid == 0) {
     mbar_init(&bar.q_full, 1);
@@ -151,12 +292,15 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.s_full, 1);
     mbar_init(&bar.o_full, 1);
     mbar_init(&bar.mma2_done, 1);
+    mbar_init(&bar.a_done, 1);
+    mbar_init(&bar.pub_done, 20);  // 16 phi warps + 4 P-group warps
+    mbar_init(&bar.prev_ready, 1);
     mbar_init(&bar.pm_full, 128);
     mbar_init(&bar.s_loaded, 128);
     mbar_init(&bar.sb_full, 128);
     mbar_init(&bar.o_free, 128);
     mbar_init(&bar.o_staged, 128);
-    z_ready = -1;
+    z_epoch = -1;
     mbar_fence_init();
     tma_prefetch_desc(&mq);
     tma_prefetch_desc(&mk);
@@ -172,25 +316,40 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   tc_fence_after_sync();
   const uint32_t tmem = tmem_base_s;
 
+  // Versions of z: an item that starts at version v uses v (zero) .. v+nA (its own dz),
+  // v+nA+1 (state before its first chunk) .. v+nA+1+nC (state after its last chunk).
+  // Every role steps through the same item list and keeps its own running counters.
+
   if (warp == 0) {
     // ================================================================ TMA producer
     if (elect_one()) {
-      for (int c = 0; c < nch; ++c) {
-        const int s = c & 1, n0 = c * 128;
-        if (c >= 2 && !mbar_wait(&bar.k_free[s], ((c >> 1) + 1) & 1, p.status, 101)) break;
-        PROF(0, c, 1);
-        mbar_arrive_expect_tx(&bar.k_full[s], C::kTile);
-        for (int x = 0; x < D / 64; ++x)
-          tma_load_4d(sK + s * C::kTile + x * C::kBoxBytes, &mk, &bar.k_full[s], x * 64, n0, h, b);
-        if (c >= 1 && !mbar_wait(&bar.q_land_free, (c - 1) & 1, p.status, 100)) break;
-        PROF(0, c, 0);
-        mbar_arrive_expect_tx(&bar.q_full, C::kTile);
-        for (int x = 0; x < D / 64; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, h, b);
-        if (c >= 2 && !mbar_wait(&bar.v_free[s], ((c >> 1) + 1) & 1, p.status, 102)) break;
-        PROF(0, c, 2);
-        mbar_arrive_expect_tx(&bar.v_full[s], C::kTile);
-        for (int x = 0; x < D / 64; ++x)
-          tma_load_4d(sV + s * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[s], x * 64, n0, h, b);
+      uint32_t nkv = 0, nq = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
+        const LinItem it = decode_item(p, item);
+        for (int pass = (it.nA > 0 ? 0 : 1); pass < 2 && ok; ++pass) {
+          for (int j = 0; j < it.nC; ++j) {
+            const int s = nkv & 1, n0 = (it.c_begin + j) * 128;
+            const uint32_t par = ((nkv >> 1) + 1) & 1;
+            if (nkv >= 2 && !mbar_wait(&bar.k_free[s], par, p.status, 101)) { ok = false; break; }
+            mbar_arrive_expect_tx(&bar.k_full[s], C::kTile);
+            for (int x = 0; x < D / 64; ++x)
+              tma_load_4d(sK + s * C::kTile + x * C::kBoxBytes, &mk, &bar.k_full[s], x * 64, n0, it.h, it.b);
+            if (pass == 1) {
+              if (nq >= 1 && !mbar_wait(&bar.q_land_free, (nq - 1) & 1, p.status, 100)) { ok = false; break; }
+              PROF(0, nq, 0);
+              mbar_arrive_expect_tx(&bar.q_full, C::kTile);
+              for (int x = 0; x < D / 64; ++x)
+                tma_load_4d(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, it.h, it.b);
+              ++nq;
+            }
+            if (nkv >= 2 && !mbar_wait(&bar.v_free[s], par, p.status, 102)) { ok = false; break; }
+            mbar_arrive_expect_tx(&bar.v_full[s], C::kTile);
+            for (int x = 0; x < D / 64; ++x)
+              tma_load_4d(sV + s * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[s], x * 64, n0, it.h, it.b);
+            ++nkv;
+          }
+        }
       }
     }
   } else if (warp == 1) {
@@ -200,48 +359,96 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       constexpr uint32_t id_s = umma_idesc_bf16(128, D, true, true);      // S += Kc^T V
       constexpr uint32_t id_o = umma_idesc_bf16(128, D, false, true);     // O  = Qc Sb,  O += Pm V
       constexpr uint32_t kLboA = (D == 128) ? C::kBoxBytes : 0;           // D=64: rows 64..127 of S mirror 0..63
-      for (int c = 0; c < nch; ++c) {
-        const int s = c & 1;
-        const uint32_t ph2 = (c >> 1) & 1;
-        const uint32_t kbase = smem_u32(sK) + s * C::kTile, vbase = smem_u32(sV) + s * C::kTile;
-        const uint32_t tq = tmem + C::tQ + s * (D / 2);
-        if (!mbar_wait(&bar.qphi_full[s], ph2, p.status, 200)) break;
-        if (!mbar_wait(&bar.kphi_full[s], ph2, p.status, 201)) break;
-        PROF(1, c, 0);
-        tc_fence_after_sync();
+      uint32_t nkv = 0, nq = 0, n_sl = 0, n_sb = 0, n_of = 0, n_pm = 0;
+      bool ok = true, first_item = true;
+      for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
+        const LinItem it = decode_item(p, item);
+        if (!first_item) {
+          // the previous item's last S conversion has read TMEM and written Sb: consume its phases
+          ok = mbar_wait(&bar.s_loaded, n_sl & 1, p.status, 210) && mbar_wait(&bar.sb_full, n_sb & 1, p.status, 211);
+          ++n_sl;
+          ++n_sb;
+          if (!ok) break;
+        }
+        first_item = false;
+        if (it.nA > 0) {
+          // ---- pass A: dS = sum Kc^T V over the segment, from zero
+          for (int j = 0; j < it.nA; ++j) {
+            const int s = nkv & 1;
+            const uint32_t ph2 = (nkv >> 1) & 1;
+            const uint32_t kbase = smem_u32(sK) + s * C::kTile, vbase = smem_u32(sV) + s * C::kTile;
+            if (!mbar_wait(&bar.kphi_full[s], ph2, p.status, 220) || !mbar_wait(&bar.v_full[s], ph2, p.status, 221)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after_sync();
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-          umma_ts(tmem + C::tP, tq + ks * 8,
-                  umma_smem_desc(kbase + (ks >> 2) * C::kBoxBytes + (ks & 3) * 32, 16, 1024), id_p, ks > 0);
-        umma_commit(&bar.p_full);
-        if (!mbar_wait(&bar.v_full[s], ph2, p.status, 202)) break;
-        if (!mbar_wait(&bar.s_loaded, c & 1, p.status, 203)) break;
-        PROF(1, c, 1);
-        tc_fence_after_sync();
+            for (int ks = 0; ks < 8; ++ks)
+              umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
+                      umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, (j > 0) || (ks > 0));
+            umma_commit(&bar.k_free[s]);
+            umma_commit(&bar.v_free[s]);
+            ++nkv;
+          }
+          if (!ok) break;
+          umma_commit(&bar.a_done);
+        }
+        // ---- pass C
+        for (int j = 0; j < it.nC; ++j) {
+          const int s = nkv & 1, sq = nq & 1;
+          const uint32_t ph2 = (nkv >> 1) & 1, phq = (nq >> 1) & 1;
+          const uint32_t kbase = smem_u32(sK) + s * C::kTile, vbase = smem_u32(sV) + s * C::kTile;
+          const uint32_t tq = tmem + C::tQ + sq * (D / 2);
+          if (!mbar_wait(&bar.qphi_full[sq], phq, p.status, 200) || !mbar_wait(&bar.kphi_full[s], ph2, p.status, 201)) {
+            ok = false;
+            break;
+          }
+          PROF(1, nq, 0);
+          tc_fence_after_sync();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
-                  umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, true);
-        umma_commit(&bar.s_full);
-        umma_commit(&bar.k_free[s]);
-        if (!mbar_wait(&bar.sb_full, c & 1, p.status, 204)) break;
-        if (c >= 1 && !mbar_wait(&bar.o_free, (c - 1) & 1, p.status, 205)) break;
-        PROF(1, c, 2);
-        tc_fence_after_sync();
+          for (int ks = 0; ks < D / 16; ++ks)
+            umma_ts(tmem + C::tP, tq + ks * 8,
+                    umma_smem_desc(kbase + (ks >> 2) * C::kBoxBytes + (ks & 3) * 32, 16, 1024), id_p, ks > 0);
+          umma_commit(&bar.p_full);
+          if (!mbar_wait(&bar.v_full[s], ph2, p.status, 202) || !mbar_wait(&bar.s_loaded, n_sl & 1, p.status, 203)) {
+            ok = false;
+            break;
+          }
+          ++n_sl;
+          PROF(1, nq, 1);
+          tc_fence_after_sync();
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-          umma_ts(tmem + C::tO, tq + ks * 8, umma_smem_desc(smem_u32(sSb) + ks * 2048, C::kSbBox, 1024), id_o,
-                  ks > 0);
-        umma_commit(&bar.mma2_done);
-        umma_commit(&bar.qphi_free[s]);
-        if (!mbar_wait(&bar.pm_full, c & 1, p.status, 206)) break;
-        PROF(1, c, 3);
-        tc_fence_after_sync();
+          for (int ks = 0; ks < 8; ++ks)
+            umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
+                    umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, true);
+          umma_commit(&bar.s_full);
+          umma_commit(&bar.k_free[s]);
+          if (!mbar_wait(&bar.sb_full, n_sb & 1, p.status, 204)) { ok = false; break; }
+          ++n_sb;
+          if (nq >= 1) {
+            if (!mbar_wait(&bar.o_free, n_of & 1, p.status, 205)) { ok = false; break; }
+            ++n_of;
+          }
+          PROF(1, nq, 2);
+          tc_fence_after_sync();
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks)
-          umma_ts(tmem + C::tO, tmem + C::tP + ks * 8, umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
-                  id_o, true);
-        umma_commit(&bar.o_full);
+          for (int ks = 0; ks < D / 16; ++ks)
+            umma_ts(tmem + C::tO, tq + ks * 8, umma_smem_desc(smem_u32(sSb) + ks * 2048, C::kSbBox, 1024), id_o,
+                    ks > 0);
+          umma_commit(&bar.mma2_done);
+          umma_commit(&bar.qphi_free[sq]);
+          if (!mbar_wait(&bar.pm_full, n_pm & 1, p.status, 206)) { ok = false; break; }
+          ++n_pm;
+          PROF(1, nq, 3);
+          tc_fence_after_sync();
+#pragma unroll
+          for (int ks = 0; ks < 8; ++ks)
+            umma_ts(tmem + C::tO, tmem + C::tP + ks * 8, umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
+                    id_o, true);
+          umma_commit(&bar.o_full);
+          ++nkv;
+          ++nq;
+        }
       }
     }
   } else if (warp < 6) {
@@ -250,136 +457,197 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const bool s_row = r < D;  // rows of S are feature indices a < D
-    // ---- initial state: S (fp32) into TMEM, its bf16 copy into shared memory
-    {
-      const float* Sin = (p.S_io != nullptr && !p.zero_init) ? p.S_io + (sidx * D + r) * D : nullptr;
-#pragma unroll
-      for (int cc = 0; cc < D / 32; ++cc) {
-        uint32_t v[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = (Sin != nullptr && s_row) ? __float_as_uint(Sin[cc * 32 + j]) : 0u;
-        tmem_st32(tmem + C::tS + lane_off + cc * 32, v);
-        if (s_row) {
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 val;
-            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-            const uint32_t col = (cc & 1) * 32 + g * 8;
-            *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, col)) = val;
-          }
-        }
+    uint32_t nkv = 0, nq = 0, n_a = 0, n_items = 0;
+    int zv = 0;  // z version at which the current item starts
+    bool ok = true;
+    for (int item = blockIdx.x; item < p.nitems; item += gridDim.x) {
+      const LinItem it = decode_item(p, item);
+      const long long sidx = (long long)it.b * p.h_count + it.hl;
+      // ---- state hand-over.  The phi warps add this segment's contribution to the previous
+      //      segment's inclusive state and publish it (the chain's critical path); this group
+      //      publishes z the same way and loads the previous state as the start of pass C.
+      const long long slot = (long long)it.chain * p.G + it.g;
+      if (it.nA > 0) {
+        ok = mbar_wait(&bar.a_done, n_a & 1, p.status, 310);
+        tc_fence_after_sync();
       }
-      tmem_wait_st();
-      fence_proxy_async_smem();
-      tc_fence_before_sync();
-      mbar_arrive(&bar.s_loaded);
-      mbar_arrive(&bar.sb_full);
-    }
-    for (int c = 0; c < nch; ++c) {
-      const int s = c & 1;
-      // ---- P: causal mask inside the chunk, row sum, bf16 back into TMEM
-      if (!mbar_wait(&bar.qphi_full[s], (c >> 1) & 1, p.status, 300)) break;
-      const float qzr = qz[s][0][r] + qz[s][1][r];
-      mbar_arrive(&bar.qz_free[s]);
-      if (!mbar_wait(&bar.p_full, c & 1, p.status, 301)) break;
-      if (tid == 64) PROF(2, c, 0);
-      tc_fence_after_sync();
-      float rowsum = 0.f;
+      ok = ok && wait_epoch(&z_epoch, zv + it.nA, p.status, 311);
+      ok = ok && mbar_wait(&bar.prev_ready, n_items & 1, p.status, 312);
+      ++n_items;
+      if (named_bar_or(1, 128, !ok)) break;
+      {
+        if (s_row) {
+          float zin = 0.f;
+          if (it.g > 0) zin = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
+          else if (p.z_io != nullptr && !p.zero_init) zin = p.z_io[sidx * D + r];
+          if (it.nA > 0) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, zin + zs[(zv + it.nA) & 7][r]);
+          zs[(zv + it.nA + 1) & 7][r] = zin;
+        }
+        if (it.nA > 0) {
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bar.pub_done);
+          PROF2(tid == 64 && zv == 0, 5);
+          // the phi warps read dS from TMEM: do not overwrite it before they are done
+          ok = mbar_wait(&bar.pub_done, n_a & 1, p.status, 313);
+          ++n_a;
+          tc_fence_after_sync();
+        }
+        const float* Sin = nullptr;
+        long long sin_stride = 1;  // float4 units between consecutive column groups of one row
+        if (it.g > 0) {
+          Sin = p.prefix + (slot - 1) * C::kStateFloats + (long long)r * 4;
+          sin_stride = 128;
+        } else if (p.S_io != nullptr && !p.zero_init) {
+          Sin = p.S_io + (sidx * D + r) * D;  // caller's row-major state
+        }
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        // 32-column block cc of this warp's rows [32 q, 32 q + 32): all kept left of the
-        // diagonal block, all dropped right of it, triangular on it (warp-uniform choice)
-        uint32_t pk[16];
-        if (cc > quarter) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) pk[j] = 0u;
-        } else {
+        for (int cc = 0; cc < D / 32; ++cc) {
           uint32_t v[32];
-          tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
-          tmem_wait_ld();
-          const bool diag = (cc == quarter);
 #pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            const float p0 = (!diag || 2 * j <= lane) ? __uint_as_float(v[2 * j]) : 0.f;
-            const float p1 = (!diag || 2 * j + 1 <= lane) ? __uint_as_float(v[2 * j + 1]) : 0.f;
-            rowsum += p0 + p1;
-            pk[j] = pack_bf16(p0, p1);
+          for (int j = 0; j < 32; j += 4) {
+            float4 in = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (Sin != nullptr && s_row)
+              in = __ldcg(reinterpret_cast<const float4*>(Sin) + (cc * 8 + j / 4) * sin_stride);
+            v[j] = __float_as_uint(in.x);
+            v[j + 1] = __float_as_uint(in.y);
+            v[j + 2] = __float_as_uint(in.z);
+            v[j + 3] = __float_as_uint(in.w);
+          }
+          tmem_st32(tmem + C::tS + lane_off + cc * 32, v);
+          if (s_row) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 val;
+              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+              const uint32_t col = (cc & 1) * 32 + g * 8;
+              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, col)) = val;
+            }
           }
         }
-        tmem_st16(tmem + C::tP + lane_off + cc * 16, pk);
+        tmem_wait_st();
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        if (named_bar_or(1, 128, !ok)) break;
+        if (tid == 64) {
+          __threadfence_block();
+          *reinterpret_cast<volatile int*>(&z_epoch) = zv + it.nA + 1;
+          PROF2(zv == 0, 6);
+        }
+        mbar_arrive(&bar.s_loaded);
+        mbar_arrive(&bar.sb_full);
       }
-      const float den = rowsum + qzr;
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(&bar.pm_full);
-      if (tid == 64) PROF(2, c, 1);
-      // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old bf16
-      //      copy, stream the new one into shared memory for the next chunk
-      if (!mbar_wait(&bar.s_full, c & 1, p.status, 302)) break;
-      if (tid == 64) PROF(2, c, 2);
-      if (!mbar_wait(&bar.mma2_done, c & 1, p.status, 303)) break;
-      if (tid == 64) PROF(2, c, 3);
-      tc_fence_after_sync();
-      const bool last = (c == nch - 1);
+      nkv += it.nA;
+      // ---- pass C
+      for (int j = 0; j < it.nC; ++j) {
+        const int s = nkv & 1, sq = nq & 1;
+        // ---- P: causal mask inside the chunk, row sum, bf16 back into TMEM
+        if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
+        const float qzr = qz[sq][0][r] + qz[sq][1][r];
+        mbar_arrive(&bar.qz_free[sq]);
+        if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
+        if (tid == 64) PROF(2, nq, 0);
+        tc_fence_after_sync();
+        float rowsum = 0.f;
 #pragma unroll
-      for (int cc = 0; cc < D / 32; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
-        tmem_wait_ld();
-        if (s_row) {
+        for (int cc = 0; cc < 4; ++cc) {
+          // 32-column block cc of this warp's rows [32 q, 32 q + 32): all kept left of the
+          // diagonal block, all dropped right of it, triangular on it (warp-uniform choice)
+          uint32_t pk[16];
+          if (cc > quarter) {
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+          } else {
+            uint32_t v[32];
+            tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
+            tmem_wait_ld();
+            const bool diag = (cc == quarter);
+#pragma unroll
+            for (int jj = 0; jj < 16; ++jj) {
+              const float p0 = (!diag || 2 * jj <= lane) ? __uint_as_float(v[2 * jj]) : 0.f;
+              const float p1 = (!diag || 2 * jj + 1 <= lane) ? __uint_as_float(v[2 * jj + 1]) : 0.f;
+              rowsum += p0 + p1;
+              pk[jj] = pack_bf16(p0, p1);
+            }
+          }
+          tmem_st16(tmem + C::tP + lane_off + cc * 16, pk);
+        }
+        const float den = rowsum + qzr;
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(&bar.pm_full);
+        if (tid == 64) PROF(2, nq, 1);
+        // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
+        //      bf16 copy, stream the new one into shared memory for the next chunk
+        if (!mbar_wait(&bar.s_full, nq & 1, p.status, 302)) { ok = false; break; }
+        if (tid == 64) PROF(2, nq, 2);
+        if (!mbar_wait(&bar.mma2_done, nq & 1, p.status, 303)) { ok = false; break; }
+        if (tid == 64) PROF(2, nq, 3);
+        tc_fence_after_sync();
+        const bool write_final = it.last_seg && (j == it.nC - 1) && p.S_io != nullptr;
+#pragma unroll
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
+          tmem_wait_ld();
+          if (s_row) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 val;
+              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+            }
+            if (write_final) {
+              float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
+#pragma unroll
+              for (int jj = 0; jj < 32; jj += 4)
+                *reinterpret_cast<float4*>(dst + jj) =
+                    make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
+                                __uint_as_float(v[jj + 3]));
+            }
+          }
+        }
+        tc_fence_before_sync();
+        mbar_arrive(&bar.s_loaded);
+        fence_proxy_async_smem();
+        mbar_arrive(&bar.sb_full);
+        if (tid == 64) PROF(2, nq, 5);
+        // ---- O: divide by the denominator, bf16, stage for the TMA store
+        if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304)) { ok = false; break; }
+        if (tid == 64) PROF(2, nq, 6);
+        tc_fence_after_sync();
+        const float inv = 1.f / den;
+        uint8_t* stage = sV + s * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
+#pragma unroll
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
+          tmem_wait_ld();
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             uint4 val;
-            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-            *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-          }
-          if (last && p.S_io != nullptr) {
-            float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
-#pragma unroll
-            for (int j = 0; j < 32; j += 4)
-              *reinterpret_cast<float4*>(dst + j) =
-                  make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                              __uint_as_float(v[j + 3]));
+            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
+            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
+            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
+            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
+            *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
           }
         }
+        tc_fence_before_sync();
+        mbar_arrive(&bar.o_free);
+        fence_proxy_async_smem();
+        mbar_arrive(&bar.o_staged);
+        if (tid == 64) PROF(2, nq, 7);
+        ++nkv;
+        ++nq;
       }
-      tc_fence_before_sync();
-      mbar_arrive(&bar.s_loaded);
-      fence_proxy_async_smem();
-      mbar_arrive(&bar.sb_full);
-      if (tid == 64) PROF(2, c, 5);
-      // ---- O: divide by the denominator, bf16, stage for the TMA store
-      if (!mbar_wait(&bar.o_full, c & 1, p.status, 304)) break;
-      if (tid == 64) PROF(2, c, 6);
-      tc_fence_after_sync();
-      const float inv = 1.f / den;
-      uint8_t* stage = sV + s * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
-#pragma unroll
-      for (int cc = 0; cc < D / 32; ++cc) {
-        uint32_t v[32];
-        tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
-        tmem_wait_ld();
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          uint4 val;
-          val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
-          val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
-          val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
-          val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-          *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-        }
-      }
-      tc_fence_before_sync();
-      mbar_arrive(&bar.o_free);
-      fence_proxy_async_smem();
-      mbar_arrive(&bar.o_staged);
-      if (tid == 64) PROF(2, c, 7);
+      if (!ok) break;
+      zv += it.nA + it.nC + 2;
     }
   } else if (warp < 14) {
     // ================================================================ phi(Q) group (8 warps)
@@ -388,148 +656,203 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int r = quarter * 32 + lane;    // Q row
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per thread
-    for (int c = 0; c < nch; ++c) {
-      const int s = c & 1;
-      bool ok = mbar_wait(&bar.q_full, c & 1, p.status, 400);
-      if (tid == 192) PROF(3, c, 0);
-      if (ok && c >= 2) {
-        ok = mbar_wait(&bar.qphi_free[s], ((c >> 1) + 1) & 1, p.status, 401) &&  // phi(Q) buffer s is free
-             mbar_wait(&bar.qz_free[s], ((c >> 1) + 1) & 1, p.status, 402);      // qz[s] of chunk c-2 was read
+    uint32_t nq = 0, n_a = 0, n_items = 0;
+    int zv = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
+      const LinItem it = decode_item(p, item);
+      if (it.nA > 0) {
+        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, n_items & 1);
+        ++n_a;
+        ok = !__any_sync(0xffffffffu, !ok);
+        if (!ok) break;
       }
-      // z before this chunk = column sums of chunks < c, published by the phi(K) group
-      if (ok) {
-        const long long t0 = clock64();
-        while (*reinterpret_cast<volatile int*>(&z_ready) < c) {
-          if (clock64() - t0 > 4000000000LL) {
-            if (atomicCAS(p.status, 0u, 1u) == 0u) p.status[1] = 403;
-            ok = false;
-            break;
-          }
-          __nanosleep(32);
+      ++n_items;
+      for (int j = 0; j < it.nC; ++j) {
+        const int sq = nq & 1;
+        const int ver = zv + it.nA + 1 + j;  // z before this chunk
+        ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
+        if (tid == 192) PROF(3, nq, 0);
+        if (ok && nq >= 2) {
+          const uint32_t par = ((nq >> 1) + 1) & 1;
+          ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // phi(Q) buffer sq is free
+               mbar_wait(&bar.qz_free[sq], par, p.status, 402);      // qz[sq] of two chunks ago was read
         }
-        __threadfence_block();
-      }
-      if (tid == 192) PROF(3, c, 1);
-      tc_fence_after_sync();
-      if (ok) {
-        uint32_t pk[kChunksPerHalf * 4];
-        float dot[2] = {0.f, 0.f};
-        const float* zc = zs[c & 3];
+        ok = ok && wait_epoch(&z_epoch, ver, p.status, 403);
+        if (tid == 192) PROF(3, nq, 1);
+        tc_fence_after_sync();
+        if (ok) {
+          uint32_t pk[kChunksPerHalf * 4];
+          float dot[2] = {0.f, 0.f};
+          const float* zc = zs[ver & 7];
 #pragma unroll
-        for (int g = 0; g < kChunksPerHalf; ++g) {
-          const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
-          const int box = gl >> 3, cin = gl & 7;
-          const uint4 rawv = *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
-          const uint32_t w4[4] = {rawv.x, rawv.y, rawv.z, rawv.w};
-          const float4 za = *reinterpret_cast<const float4*>(zc + gl * 8);
-          const float4 zb = *reinterpret_cast<const float4*>(zc + gl * 8 + 4);
-          const float zv[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+          for (int g = 0; g < kChunksPerHalf; ++g) {
+            const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
+            const int box = gl >> 3, cin = gl & 7;
+            const uint4 rawv =
+                *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
+            const uint32_t w4[4] = {rawv.x, rawv.y, rawv.z, rawv.w};
+            const float4 za = *reinterpret_cast<const float4*>(zc + gl * 8);
+            const float4 zb = *reinterpret_cast<const float4*>(zc + gl * 8 + 4);
+            const float zvv[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const uint32_t pkv = phi_bf16x2(w4[e]);
-            pk[g * 4 + e] = pkv;
-            // the dot product uses the rounded values the tensor core will see
-            dot[e & 1] = fmaf(bf16_lo(pkv), zv[2 * e], dot[e & 1]);
-            dot[e & 1] = fmaf(bf16_hi(pkv), zv[2 * e + 1], dot[e & 1]);
+            for (int e = 0; e < 4; ++e) {
+              const uint32_t pkv = phi_bf16x2(w4[e]);
+              pk[g * 4 + e] = pkv;
+              // the dot product uses the rounded values the tensor core will see
+              dot[e & 1] = fmaf(bf16_lo(pkv), zvv[2 * e], dot[e & 1]);
+              dot[e & 1] = fmaf(bf16_hi(pkv), zvv[2 * e + 1], dot[e & 1]);
+            }
+          }
+          qz[sq][half][r] = dot[0] + dot[1];
+          if constexpr (D == 128) {
+            uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
+            tmem_st32(tmem + C::tQ + sq * (D / 2) + lane_off + half * 32, pk32);
+          } else {
+            tmem_st16(tmem + C::tQ + sq * (D / 2) + lane_off + half * 16, pk);
+          }
+          tmem_wait_st();
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            mbar_arrive(&bar.qphi_full[sq]);
+            mbar_arrive(&bar.q_land_free);
           }
         }
-        qz[s][half][r] = dot[0] + dot[1];
-        if constexpr (D == 128) {
-          uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
-          tmem_st32(tmem + C::tQ + s * (D / 2) + lane_off + half * 32, pk32);
-        } else {
-          tmem_st16(tmem + C::tQ + s * (D / 2) + lane_off + half * 16, pk);
-        }
-        tmem_wait_st();
-        tc_fence_before_sync();
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(&bar.qphi_full[s]);
-          mbar_arrive(&bar.q_land_free);
-        }
+        if (tid == 192) PROF(3, nq, 2);
+        ok = !__any_sync(0xffffffffu, !ok);
+        if (!ok) break;
+        ++nq;
       }
-      if (tid == 192) PROF(3, c, 2);
-      if (__any_sync(0xffffffffu, !ok)) break;
+      zv += it.nA + it.nC + 2;
     }
   } else if (warp < 22) {
     // ================================================================ phi(K) group (8 warps)
     const int tt = tid - 14 * 32;  // 0..255
-    if (tt < D) zs[0][tt] = (p.z_io != nullptr && !p.zero_init) ? p.z_io[sidx * D + tt] : 0.f;
-    asm volatile("bar.sync 3, 256;" ::: "memory");
-    if (tt == 0) {
-      __threadfence_block();
-      *reinterpret_cast<volatile int*>(&z_ready) = 0;  // zs[0] holds the initial z
-    }
-    for (int c = 0; c < nch; ++c) {
-      const int s = c & 1;
-      const bool ok = mbar_wait(&bar.k_full[s], (c >> 1) & 1, p.status, 410);
-      if (tt == 0) PROF(3, c, 4);
-      if (ok && tt < 2 * D) {
-        const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
-        const int box = cc >> 3, cin = cc & 7;
-        uint8_t* kb = sK + s * C::kTile + box * C::kBoxBytes;
-        float cs[8];
-#pragma unroll
-        for (int e = 0; e < 8; ++e) cs[e] = 0.f;
-        // all loads first, then branch-free arithmetic, then all stores (the tile is updated in place)
-        uint4 rawv[8];
-#pragma unroll
-        for (int k8 = 0; k8 < 8; ++k8) {
-          const int row = (tt & 15) + 16 * k8;
-          rawv[k8] = *reinterpret_cast<const uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
-        }
-#pragma unroll
-        for (int k8 = 0; k8 < 8; ++k8) {
-          const int row = (tt & 15) + 16 * k8;
-          const uint32_t keep = ((c * 128 + row) < p.N) ? 0xffffffffu : 0u;  // rows past N must not enter S, z
-          uint32_t w4[4] = {rawv[k8].x, rawv[k8].y, rawv[k8].z, rawv[k8].w};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            w4[e] = phi_bf16x2(w4[e]) & keep;
-            cs[2 * e] += bf16_lo(w4[e]);
-            cs[2 * e + 1] += bf16_hi(w4[e]);
-          }
-          rawv[k8] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-        }
-#pragma unroll
-        for (int k8 = 0; k8 < 8; ++k8) {
-          const int row = (tt & 15) + 16 * k8;
-          *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k8];
-        }
-        fence_proxy_async_smem();
-#pragma unroll
-        for (int e = 0; e < 8; ++e) {
-#pragma unroll
-          for (int off = 8; off > 0; off >>= 1) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], off);
-        }
-        if ((tt & 15) == 0) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) zs[(c + 1) & 3][cc * 8 + e] = zs[c & 3][cc * 8 + e] + cs[e];
-        }
-      }
-      __syncwarp();
-      if (ok && lane == 0) mbar_arrive(&bar.kphi_full[s]);
-      if (tt == 0) PROF(3, c, 5);
-      if (named_bar_or(3, 256, !ok)) break;
+    uint32_t nkv = 0, n_a = 0, n_items = 0;
+    int zv = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
+      const LinItem it = decode_item(p, item);
+      // version zv: zero (start of the segment's own column sums)
+      if (tt < D) zs[zv & 7][tt] = 0.f;
+      if (named_bar_or(3, 256, false)) break;
       if (tt == 0) {
         __threadfence_block();
-        *reinterpret_cast<volatile int*>(&z_ready) = c + 1;
+        *reinterpret_cast<volatile int*>(&z_epoch) = zv;
       }
+      for (int pass = (it.nA > 0 ? 0 : 1); pass < 2 && ok; ++pass) {
+        // pass C starts from the state before the segment, written by the P group
+        if (pass == 1) {
+          if (it.nA > 0) {
+            ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, n_items & 1);  // column quarters 2, 3
+            ++n_a;
+            if (named_bar_or(3, 256, !ok)) { ok = false; break; }
+          }
+          ok = wait_epoch(&z_epoch, zv + it.nA + 1, p.status, 411);
+        }
+        for (int j = 0; j < it.nC; ++j) {
+          const int s = nkv & 1;
+          const int ver = (pass == 0) ? zv + j : zv + it.nA + 1 + j;  // version read; ver + 1 is written
+          const int n0 = (it.c_begin + j) * 128;
+          ok = ok && mbar_wait(&bar.k_full[s], (nkv >> 1) & 1, p.status, 410);
+          if (tt == 0 && pass == 1) PROF(3, nkv, 4);
+          if (ok && tt < 2 * D) {
+            const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
+            const int box = cc >> 3, cin = cc & 7;
+            uint8_t* kb = sK + s * C::kTile + box * C::kBoxBytes;
+            float cs[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) cs[e] = 0.f;
+            // all loads first, then branch-free arithmetic, then all stores (the tile is updated in place)
+            uint4 rawv[8];
+#pragma unroll
+            for (int k8 = 0; k8 < 8; ++k8) {
+              const int row = (tt & 15) + 16 * k8;
+              rawv[k8] = *reinterpret_cast<const uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
+            }
+#pragma unroll
+            for (int k8 = 0; k8 < 8; ++k8) {
+              const int row = (tt & 15) + 16 * k8;
+              const uint32_t keep = ((n0 + row) < p.N) ? 0xffffffffu : 0u;  // rows past N must not enter S, z
+              uint32_t w4[4] = {rawv[k8].x, rawv[k8].y, rawv[k8].z, rawv[k8].w};
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                w4[e] = phi_bf16x2(w4[e]) & keep;
+                cs[2 * e] += bf16_lo(w4[e]);
+                cs[2 * e + 1] += bf16_hi(w4[e]);
+              }
+              rawv[k8] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+            }
+#pragma unroll
+            for (int k8 = 0; k8 < 8; ++k8) {
+              const int row = (tt & 15) + 16 * k8;
+              *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k8];
+            }
+            fence_proxy_async_smem();
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+#pragma unroll
+              for (int off = 8; off > 0; off >>= 1) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], off);
+            }
+            if ((tt & 15) == 0) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) zs[(ver + 1) & 7][cc * 8 + e] = zs[ver & 7][cc * 8 + e] + cs[e];
+            }
+          }
+          __syncwarp();
+          if (ok && lane == 0) mbar_arrive(&bar.kphi_full[s]);
+          if (tt == 0 && pass == 1) PROF(3, nkv, 5);
+          if (named_bar_or(3, 256, !ok)) { ok = false; break; }
+          if (tt == 0) {
+            __threadfence_block();
+            *reinterpret_cast<volatile int*>(&z_epoch) = ver + 1;
+          }
+          ++nkv;
+        }
+      }
+      ++n_items;
+      if (ok && it.last_seg && p.z_io != nullptr && tt < D)
+        p.z_io[((long long)it.b * p.h_count + it.hl) * D + tt] = zs[(zv + it.nA + 1 + it.nC) & 7][tt];
+      zv += it.nA + it.nC + 2;
     }
-    if (p.z_io != nullptr && tt < D) p.z_io[sidx * D + tt] = zs[nch & 3][tt];
   } else {
     // ================================================================ O store warp
     if (elect_one()) {
-      for (int c = 0; c < nch; ++c) {
-        const int s = c & 1;
-        if (!mbar_wait(&bar.o_staged, c & 1, p.status, 500)) break;
-        for (int x = 0; x < D / 64; ++x)
-          tma_store_4d(&mo, sV + s * C::kTile + x * C::kBoxBytes, x * 64, c * 128, h, b);
-        tma_store_commit();
-        tma_store_wait_read<0>();
-        mbar_arrive(&bar.v_free[s]);  // the staging buffer may take V of chunk c+2
+      uint32_t nkv = 0, nq = 0, n_a = 0;
+      bool ok = true;
+      for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
+        const LinItem it = decode_item(p, item);
+        nkv += it.nA;
+        // one poller per CTA: hundreds of threads spinning on a handful of L2 lines slow the whole chain
+        if (it.g > 0 && !wait_flag(p.flags + ((long long)it.chain * p.G + it.g - 1) * kFlagStride, p.status, 511)) {
+          ok = false;
+          break;
+        }
+        mbar_arrive(&bar.prev_ready);
+        if (it.nA > 0) {
+          // every warp of the hand-over has written and fenced its part of the inclusive state
+          if (!mbar_wait(&bar.pub_done, n_a & 1, p.status, 510)) { ok = false; break; }
+          PROF2(n_a == 0, 4);
+          ++n_a;
+          const unsigned int one = 1u;
+          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.flags + ((long long)it.chain * p.G + it.g) * kFlagStride), "r"(one)
+                       : "memory");
+        }
+        for (int j = 0; j < it.nC; ++j) {
+          const int s = nkv & 1;
+          if (!mbar_wait(&bar.o_staged, nq & 1, p.status, 500)) { ok = false; break; }
+          for (int x = 0; x < D / 64; ++x)
+            tma_store_4d(&mo, sV + s * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b);
+          tma_store_commit();
+          tma_store_wait_read<0>();
+          mbar_arrive(&bar.v_free[s]);  // the staging buffer may take the V tile two uses later
+          ++nkv;
+          ++nq;
+        }
       }
       tma_store_wait_all<0>();
+      PROF2(true, 7);
     }
   }
   tc_fence_before_sync();
@@ -540,6 +863,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 }  // namespace
 
 #ifdef GF_PROFILE
+extern "C" int gformer_debug_read_profile2(unsigned long long* host_dst) {
+  return (int)cudaMemcpyFromSymbol(host_dst, g_prof2, sizeof(g_prof2));
+}
 extern "C" int gformer_debug_read_profile(unsigned long long* host_dst) {
   return (int)cudaMemcpyFromSymbol(host_dst, g_prof, sizeof(g_prof));
 }
@@ -550,10 +876,36 @@ bool tc_linear_supported(int N, int d, int dtype) {
   return dtype == GF_BF16 && (d == 64 || d == 128);
 }
 
+// Segmentation of the chains: chunks per segment L and segments per chain G.
+void linear_tc_plan(int nchains, int N, int split, int* L_out, int* G_out) {
+  const int nch = (N + 127) / 128;
+  int L;
+  if (split > 0) {
+    L = split;
+  } else if (nchains >= 120 || nch <= 8) {
+    L = nch;  // enough chains to fill the machine (or nothing to cut): one segment per chain
+  } else {
+    L = 8;
+    // keep at least ~2 items per SM, but never segments shorter than 4 chunks
+    while (L > 4 && (long long)nchains * ((nch + L - 1) / L) < 296) L -= 1;
+  }
+  if (L > nch) L = nch;
+  if (L < 1) L = 1;
+  *L_out = L;
+  *G_out = (nch + L - 1) / L;
+}
+
+size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
+  int L, G;
+  linear_tc_plan(nchains, N, split, &L, &G);
+  if (G <= 1) return 0;
+  const size_t flags = (size_t)nchains * G * kFlagStride * sizeof(unsigned int);
+  return flags + (size_t)nchains * G * ((size_t)128 * d + d) * sizeof(float);
+}
+
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
                              int split, WsHeader* ws, cudaStream_t stream) {
-  (void)split;
   if (h_count <= 0) return cudaSuccess;
   CUtensorMap mq, mk, mv, mo;
   if (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128) ||
@@ -561,14 +913,30 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
     return cudaErrorInvalidValue;
   LinParams p;
   p.N = N;
+  p.nch = (N + 127) / 128;
   p.h_begin = h_begin;
   p.h_count = h_count;
+  p.nchains = B * h_count;
+  linear_tc_plan(p.nchains, N, split, &p.L, &p.G);
+  p.nitems = p.nchains * p.G;
   p.S_io = S_io;
   p.z_io = z_io;
   p.zero_init = zero_init ? 1 : 0;
   p.status = &ws->status;
-  dim3 grid(h_count, B);
+  uint8_t* scratch = reinterpret_cast<uint8_t*>(ws) + sizeof(WsHeader);
+  const size_t flag_bytes = (size_t)p.nchains * p.G * kFlagStride * sizeof(unsigned int);
+  p.flags = reinterpret_cast<unsigned int*>(scratch);
+  p.prefix = reinterpret_cast<float*>(scratch + flag_bytes);
   cudaError_t e;
+  if (p.G > 1) {
+    e = cudaMemsetAsync(p.flags, 0, flag_bytes, stream);
+    if (e != cudaSuccess) return e;
+  }
+  int dev = 0, sms = 0;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  // One CTA per SM at most: every CTA must be resident for the segment hand-over to make progress.
+  dim3 grid(p.nitems < sms ? p.nitems : sms);
   if (d == 64) {
     auto kern = linear_tc_kernel<64>;
     e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, LinCfg<64>::kBytes);

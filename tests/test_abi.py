@@ -54,7 +54,7 @@ def test_workspace_bytes_nonzero():
 def test_tuning_rejects_unknown_keys():
     L = gf.lib()
     assert L.gformer_set_tuning(99, 1) == gf.GF_ERR_INVALID_ARG
-    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 3) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, -1) == gf.GF_ERR_INVALID_ARG
     assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0) == gf.GF_OK
 
 

@@ -73,7 +73,7 @@ def test_window_bnhd_layout_and_custom_scale(force_simt):
 def test_window_tensor_core(N, w, d, gain):
     q, k, v = synth.qkv(2, 2, N, d, "bf16", seed=200 + N + w, gain=gain)
     ref = oracle.window_attn(f64(q), f64(k), f64(v), w)
-    ws = gf.Workspace()
+    ws = gf.Workspace.for_problem(2, 2, N, d, w, 2)
     o = gf.window_attn(*dev(q, k, v), w, ws=ws)
     assert ws.last_device_status() == gf.GF_OK
     assert_parity(f64(o), ref, "bf16", f"window tc N={N} w={w} d={d}")
@@ -133,7 +133,7 @@ def test_linear_state_in_out_and_resume(force_simt, dtype):
 def test_linear_tensor_core(N, d, gain):
     q, k, v = synth.qkv(2, 2, N, d, "bf16", seed=400 + N, gain=gain)
     ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v))
-    ws = gf.Workspace()
+    ws = gf.Workspace.for_problem(2, 2, N, d)
     o = gf.causal_linear_attn(*dev(q, k, v), ws=ws)
     assert ws.last_device_status() == gf.GF_OK
     assert_parity(f64(o), ref, "bf16", f"linear tc N={N} d={d}")
@@ -201,7 +201,7 @@ def test_config2_gpt2_small_full():
     c = synth.CONFIGS["gpt2s"]
     q, k, v = synth.qkv(c["B"], c["H"], c["N"], c["d"], "bf16", c["seed"])
     ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), c["w"])
-    ws = gf.Workspace()
+    ws = gf.Workspace.for_problem(c["B"], c["H"], c["N"], c["d"], c["w"], -1)
     o = gf.hybrid_attn(*dev(q, k, v), c["w"], ws=ws)
     assert ws.last_device_status() == gf.GF_OK
     assert_parity(f64(o), ref, "bf16", "config 2")
@@ -214,7 +214,7 @@ def test_config3_long_sequence_sampled_heads():
     q, k, v = synth.qkv(c["B"], c["H"], c["N"], c["d"], "bf16", c["seed"])
     h0 = gf.default_h_sparse(c["H"])
     assert h0 == 6
-    ws = gf.Workspace()
+    ws = gf.Workspace.for_problem(c["B"], c["H"], c["N"], c["d"], c["w"], -1)
     o = gf.hybrid_attn(*dev(q, k, v), c["w"], ws=ws).cpu()
     assert ws.last_device_status() == gf.GF_OK
     assert torch.isfinite(o.float()).all()
@@ -306,7 +306,7 @@ def test_config5_sweep_point(idx):
     B, H, N, d, w = p["B"], p["H"], p["N"], p["d"], p["w"]
     h0 = gf.default_h_sparse(H)
     q, k, v = synth.qkv(B, H, N, d, "bf16", p["seed"])
-    ws = gf.Workspace()
+    ws = gf.Workspace.for_problem(B, H, N, d, w, -1)
     o = gf.hybrid_attn(*dev(q, k, v), w, ws=ws).cpu()
     assert ws.last_device_status() == gf.GF_OK
     assert torch.isfinite(o.float()).all()
