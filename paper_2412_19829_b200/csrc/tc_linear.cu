@@ -10,12 +10,15 @@
 // A (batch, head) chain is cut into segments of L chunks; a work item is one segment.  CTAs are
 // persistent and take items round-robin in an order in which a segment's predecessor always has
 // a smaller index, so the CTA that owns it is already running.  For an item the CTA
-//   (A) accumulates the segment's own state contribution dS = sum Kc^T V, dz = sum colsum(Kc)
-//       (K, V only; skipped for a chain's last segment and when a chain is a single segment),
-//   (B) waits for the inclusive state of the previous segment in global scratch (bounded
-//       spin), publishes its own inclusive state = previous + dS and raises its flag,
-//   (C) walks its chunks with the full pipeline starting from the previous segment's state
-//       (K and V come from L2 this second time).
+//   (A) applies phi to the segment's K tiles once, parks the results in the rows of the OUTPUT
+//       tensor that this segment will later overwrite (no extra scratch, and the lines are still
+//       in L2 when pass C reads them back), keeps the running column sums of phi(K) in shared
+//       memory, and accumulates the segment's own state contribution dS = sum Kc^T V (not for a
+//       chain's last segment, whose contribution nobody needs),
+//   (B) waits for the inclusive state of the previous segment in global scratch (one bounded
+//       poller per CTA), publishes its own inclusive state = previous + dS and raises its flag,
+//   (C) walks its chunks with the full pipeline starting from the previous segment's state,
+//       reading phi(K) back instead of K, so every exponential of the layer is computed once.
 // Warp roles:
 //   warp 0       TMA producer (raw Q, K, V tiles; K and V double buffered)
 //   warp 1       MMA issuer
@@ -23,9 +26,11 @@
 //                readout, divides and stores O (one thread per row / TMEM lane)
 //   warps 6-13   "phi(Q) group": applies phi to Q; the result goes to TMEM as the A operand of
 //                MMA1/MMA2, together with the per-row dot product with z_{c-1}
-//   warps 14-21  "phi(K) group": applies phi to K in place in shared memory and adds its column
-//                sums to z
-//   warp 22      stores O tiles (staged in the dead V buffer) with TMA
+//   warps 14-21  "phi(K) group" (pass A): applies phi to K in place in shared memory and keeps the
+//                cumulative column sums
+//   warp 22      TMA stores: parks phi(K) tiles (pass A), stores O tiles staged in the dead V
+//                buffer (pass C)
+//   warp 23      polls the previous segment's flag and raises this segment's flag
 // TMEM (D=128): P 128 | O 128 | S 128 | phi(Q) 2 x 64 columns = 512.
 // Every wait is bounded; on expiry the kernel records a status word and drains.
 #include "common.cuh"
@@ -36,7 +41,8 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 736;  // 23 warps, 88 registers each
+constexpr int kThreads = 768;  // 24 warps, 80 registers each
+constexpr int kMaxL = 8;       // chunks per segment (bounded by the per-segment z history kept in shared memory)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kFlagStride = 32;  // one flag per 128-byte line
 
@@ -72,8 +78,8 @@ struct LinParams {
 };
 
 struct LinItem {
-  int g, chain, b, hl, h, c_begin, nC, nA;
-  bool last_seg;
+  int g, chain, b, hl, h, c_begin, nC;
+  bool last_seg, need_dS;
 };
 
 __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
@@ -87,15 +93,15 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
   const int c_end = (it.c_begin + p.L < p.nch) ? it.c_begin + p.L : p.nch;
   it.nC = c_end - it.c_begin;
   it.last_seg = (it.g == p.G - 1);
-  it.nA = it.last_seg ? 0 : it.nC;  // the last segment's contribution is needed by nobody
+  it.need_dS = !it.last_seg;  // the last segment's contribution is needed by nobody
   return it;
 }
 
 struct LinBarriers {
   uint64_t q_full, q_land_free;
-  uint64_t k_full[2], v_full[2], k_free[2], v_free[2];
+  uint64_t k_full[2], ka_full[2], v_full[2], k_free[2], v_free[2];  // ka_full: K tiles of pass A, k_full: of pass C
   uint64_t qphi_full[2], kphi_full[2], qphi_free[2], qz_free[2];
-  uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, prev_ready;
+  uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, prev_ready, park_done;
   uint64_t pm_full, s_loaded, sb_full, o_free, o_staged;
 };
 
@@ -268,9 +274,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint8_t* sV = sm + C::kV;
   uint8_t* sSb = sm + C::kSb;
   __shared__ __align__(8) LinBarriers bar;
-  __shared__ __align__(16) float zs[8][D];  // running z, one buffer per "version" (index & 7)
-  __shared__ float qz[2][2][128];           // [chunk parity][column half][row]
-  __shared__ int z_epoch;                   // newest complete version of z (monotonic)
+  // per item parity: zcum[j] = column sums of phi(K) over the first j chunks of the segment,
+  // zin = z before the segment
+  __shared__ __align__(16) float zcum[2][kMaxL + 1][D];
+  __shared__ __align__(16) float zin[2][D];
+  __shared__ float qz[2][2][128];  // [chunk parity][column half][row]
+  __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
+  __shared__ int zin_epoch;        // items whose zin is in place (monotonic)
   __shared__ uint32_t tmem_base_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -280,8 +290,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.q_land_free, 8);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar.k_full[s], 1);
+      mbar_init(&bar.ka_full[s], 1);
       mbar_init(&bar.v_full[s], 1);
-      mbar_init(&bar.k_free[s], 1);
+      mbar_init(&bar.k_free[s], 2);
       mbar_init(&bar.v_free[s], 1);
       mbar_init(&bar.qphi_full[s], 8);
       mbar_init(&bar.kphi_full[s], 8);
@@ -295,12 +306,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.a_done, 1);
     mbar_init(&bar.pub_done, 20);  // 16 phi warps + 4 P-group warps
     mbar_init(&bar.prev_ready, 1);
+    mbar_init(&bar.park_done, 1);
     mbar_init(&bar.pm_full, 128);
     mbar_init(&bar.s_loaded, 128);
     mbar_init(&bar.sb_full, 128);
     mbar_init(&bar.o_free, 128);
     mbar_init(&bar.o_staged, 128);
-    z_epoch = -1;
+    ka_epoch = 0;
+    zin_epoch = 0;
     mbar_fence_init();
     tma_prefetch_desc(&mq);
     tma_prefetch_desc(&mk);
@@ -316,25 +329,30 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   tc_fence_after_sync();
   const uint32_t tmem = tmem_base_s;
 
-  // Versions of z: an item that starts at version v uses v (zero) .. v+nA (its own dz),
-  // v+nA+1 (state before its first chunk) .. v+nA+1+nC (state after its last chunk).
-  // Every role steps through the same item list and keeps its own running counters.
+  // Every role walks the same item list and keeps its own running counters: nk / nv = K / V tiles
+  // that went through the two-stage rings so far (stage = count & 1, phase = count >> 1), nq =
+  // pass-C chunks so far, na = pass-A tiles so far.
 
   if (warp == 0) {
     // ================================================================ TMA producer
     if (elect_one()) {
-      uint32_t nkv = 0, nq = 0;
+      // a waiter may only use a parity wait on a barrier whose every phase it observes, so the K
+      // tiles of the two passes complete on different barriers (phi(K) group / MMA issuer)
+      uint32_t nk = 0, nv = 0, nq = 0, n_items = 0;
       bool ok = true;
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
-        for (int pass = (it.nA > 0 ? 0 : 1); pass < 2 && ok; ++pass) {
+        for (int pass = 0; pass < 2 && ok; ++pass) {
+          if (pass == 1 && !mbar_wait(&bar.park_done, n_items & 1, p.status, 103)) { ok = false; break; }
           for (int j = 0; j < it.nC; ++j) {
-            const int s = nkv & 1, n0 = (it.c_begin + j) * 128;
-            const uint32_t par = ((nkv >> 1) + 1) & 1;
-            if (nkv >= 2 && !mbar_wait(&bar.k_free[s], par, p.status, 101)) { ok = false; break; }
-            mbar_arrive_expect_tx(&bar.k_full[s], C::kTile);
-            for (int x = 0; x < D / 64; ++x)
-              tma_load_4d(sK + s * C::kTile + x * C::kBoxBytes, &mk, &bar.k_full[s], x * 64, n0, it.h, it.b);
+            const int n0 = (it.c_begin + j) * 128;
+            const int sk = nk & 1;
+            if (nk >= 2 && !mbar_wait(&bar.k_free[sk], ((nk >> 1) + 1) & 1, p.status, 101)) { ok = false; break; }
+            uint64_t* kbar = (pass == 0) ? &bar.ka_full[sk] : &bar.k_full[sk];
+            mbar_arrive_expect_tx(kbar, C::kTile);
+            for (int x = 0; x < D / 64; ++x)  // pass C reads back the phi(K) tile parked in the output rows
+              tma_load_4d(sK + sk * C::kTile + x * C::kBoxBytes, pass == 0 ? &mk : &mo, kbar, x * 64, n0, it.h, it.b);
+            ++nk;
             if (pass == 1) {
               if (nq >= 1 && !mbar_wait(&bar.q_land_free, (nq - 1) & 1, p.status, 100)) { ok = false; break; }
               PROF(0, nq, 0);
@@ -343,13 +361,17 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                 tma_load_4d(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, it.h, it.b);
               ++nq;
             }
-            if (nkv >= 2 && !mbar_wait(&bar.v_free[s], par, p.status, 102)) { ok = false; break; }
-            mbar_arrive_expect_tx(&bar.v_full[s], C::kTile);
-            for (int x = 0; x < D / 64; ++x)
-              tma_load_4d(sV + s * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[s], x * 64, n0, it.h, it.b);
-            ++nkv;
+            if (pass == 1 || it.need_dS) {
+              const int sv = nv & 1;
+              if (nv >= 2 && !mbar_wait(&bar.v_free[sv], ((nv >> 1) + 1) & 1, p.status, 102)) { ok = false; break; }
+              mbar_arrive_expect_tx(&bar.v_full[sv], C::kTile);
+              for (int x = 0; x < D / 64; ++x)
+                tma_load_4d(sV + sv * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[sv], x * 64, n0, it.h, it.b);
+              ++nv;
+            }
           }
         }
+        ++n_items;
       }
     }
   } else if (warp == 1) {
@@ -359,7 +381,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       constexpr uint32_t id_s = umma_idesc_bf16(128, D, true, true);      // S += Kc^T V
       constexpr uint32_t id_o = umma_idesc_bf16(128, D, false, true);     // O  = Qc Sb,  O += Pm V
       constexpr uint32_t kLboA = (D == 128) ? C::kBoxBytes : 0;           // D=64: rows 64..127 of S mirror 0..63
-      uint32_t nkv = 0, nq = 0, n_sl = 0, n_sb = 0, n_of = 0, n_pm = 0;
+      uint32_t nk = 0, nv = 0, nq = 0, n_sl = 0, n_sb = 0, n_of = 0, n_pm = 0;
+      uint32_t n_kphi[2] = {0, 0}, n_kc[2] = {0, 0};
       bool ok = true, first_item = true;
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
@@ -371,38 +394,41 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (!ok) break;
         }
         first_item = false;
-        if (it.nA > 0) {
-          // ---- pass A: dS = sum Kc^T V over the segment, from zero
-          for (int j = 0; j < it.nA; ++j) {
-            const int s = nkv & 1;
-            const uint32_t ph2 = (nkv >> 1) & 1;
-            const uint32_t kbase = smem_u32(sK) + s * C::kTile, vbase = smem_u32(sV) + s * C::kTile;
-            if (!mbar_wait(&bar.kphi_full[s], ph2, p.status, 220) || !mbar_wait(&bar.v_full[s], ph2, p.status, 221)) {
-              ok = false;
-              break;
-            }
+        // ---- pass A: dS = sum Kc^T V over the segment, from zero (only if somebody needs it)
+        for (int j = 0; j < it.nC; ++j) {
+          const int sk = nk & 1;
+          if (!mbar_wait(&bar.kphi_full[sk], n_kphi[sk] & 1, p.status, 220)) { ok = false; break; }
+          ++n_kphi[sk];
+          if (it.need_dS) {
+            const int sv = nv & 1;
+            const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
+            if (!mbar_wait(&bar.v_full[sv], (nv >> 1) & 1, p.status, 221)) { ok = false; break; }
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
               umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
                       umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, (j > 0) || (ks > 0));
-            umma_commit(&bar.k_free[s]);
-            umma_commit(&bar.v_free[s]);
-            ++nkv;
+            umma_commit(&bar.k_free[sk]);  // second arrival: the store warp, once the tile is parked
+            umma_commit(&bar.v_free[sv]);
+            ++nv;
+          } else {
+            mbar_arrive(&bar.k_free[sk]);
           }
-          if (!ok) break;
-          umma_commit(&bar.a_done);
+          ++nk;
         }
+        if (!ok) break;
+        if (it.need_dS) umma_commit(&bar.a_done);
         // ---- pass C
         for (int j = 0; j < it.nC; ++j) {
-          const int s = nkv & 1, sq = nq & 1;
-          const uint32_t ph2 = (nkv >> 1) & 1, phq = (nq >> 1) & 1;
-          const uint32_t kbase = smem_u32(sK) + s * C::kTile, vbase = smem_u32(sV) + s * C::kTile;
+          const int sk = nk & 1, sv = nv & 1, sq = nq & 1;
+          const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
           const uint32_t tq = tmem + C::tQ + sq * (D / 2);
-          if (!mbar_wait(&bar.qphi_full[sq], phq, p.status, 200) || !mbar_wait(&bar.kphi_full[s], ph2, p.status, 201)) {
+          if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 200) ||
+              !mbar_wait(&bar.k_full[sk], n_kc[sk] & 1, p.status, 201)) {
             ok = false;
             break;
           }
+          ++n_kc[sk];
           PROF(1, nq, 0);
           tc_fence_after_sync();
 #pragma unroll
@@ -410,7 +436,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             umma_ts(tmem + C::tP, tq + ks * 8,
                     umma_smem_desc(kbase + (ks >> 2) * C::kBoxBytes + (ks & 3) * 32, 16, 1024), id_p, ks > 0);
           umma_commit(&bar.p_full);
-          if (!mbar_wait(&bar.v_full[s], ph2, p.status, 202) || !mbar_wait(&bar.s_loaded, n_sl & 1, p.status, 203)) {
+          if (!mbar_wait(&bar.v_full[sv], (nv >> 1) & 1, p.status, 202) ||
+              !mbar_wait(&bar.s_loaded, n_sl & 1, p.status, 203)) {
             ok = false;
             break;
           }
@@ -422,7 +449,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
                     umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, true);
           umma_commit(&bar.s_full);
-          umma_commit(&bar.k_free[s]);
+          umma_commit(&bar.k_free[sk]);
+          mbar_arrive(&bar.k_free[sk]);  // nothing else holds the tile in this pass
           if (!mbar_wait(&bar.sb_full, n_sb & 1, p.status, 204)) { ok = false; break; }
           ++n_sb;
           if (nq >= 1) {
@@ -446,7 +474,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             umma_ts(tmem + C::tO, tmem + C::tP + ks * 8, umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
                     id_o, true);
           umma_commit(&bar.o_full);
-          ++nkv;
+          ++nk;
+          ++nv;
           ++nq;
         }
       }
@@ -457,36 +486,38 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const bool s_row = r < D;  // rows of S are feature indices a < D
-    uint32_t nkv = 0, nq = 0, n_a = 0, n_items = 0;
-    int zv = 0;  // z version at which the current item starts
+    uint32_t nv = 0, nq = 0, n_a = 0, n_items = 0;
+    int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
       const long long sidx = (long long)it.b * p.h_count + it.hl;
+      const int ip = n_items & 1;
       // ---- state hand-over.  The phi warps add this segment's contribution to the previous
       //      segment's inclusive state and publish it (the chain's critical path); this group
       //      publishes z the same way and loads the previous state as the start of pass C.
       const long long slot = (long long)it.chain * p.G + it.g;
-      if (it.nA > 0) {
+      na += it.nC;
+      if (it.need_dS) {
         ok = mbar_wait(&bar.a_done, n_a & 1, p.status, 310);
         tc_fence_after_sync();
       }
-      ok = ok && wait_epoch(&z_epoch, zv + it.nA, p.status, 311);
+      ok = ok && wait_epoch(&ka_epoch, na, p.status, 311);
       ok = ok && mbar_wait(&bar.prev_ready, n_items & 1, p.status, 312);
-      ++n_items;
       if (named_bar_or(1, 128, !ok)) break;
       {
         if (s_row) {
-          float zin = 0.f;
-          if (it.g > 0) zin = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
-          else if (p.z_io != nullptr && !p.zero_init) zin = p.z_io[sidx * D + r];
-          if (it.nA > 0) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, zin + zs[(zv + it.nA) & 7][r]);
-          zs[(zv + it.nA + 1) & 7][r] = zin;
+          float z0 = 0.f;
+          if (it.g > 0) z0 = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
+          else if (p.z_io != nullptr && !p.zero_init) z0 = p.z_io[sidx * D + r];
+          if (it.need_dS) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, z0 + zcum[ip][it.nC][r]);
+          if (it.last_seg && p.z_io != nullptr) p.z_io[sidx * D + r] = z0 + zcum[ip][it.nC][r];
+          zin[ip][r] = z0;
         }
-        if (it.nA > 0) {
+        if (it.need_dS) {
           __syncwarp();
           if (lane == 0) mbar_arrive(&bar.pub_done);
-          PROF2(tid == 64 && zv == 0, 5);
+          PROF2(tid == 64 && n_items == 0, 5);
           // the phi warps read dS from TMEM: do not overwrite it before they are done
           ok = mbar_wait(&bar.pub_done, n_a & 1, p.status, 313);
           ++n_a;
@@ -533,16 +564,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (named_bar_or(1, 128, !ok)) break;
         if (tid == 64) {
           __threadfence_block();
-          *reinterpret_cast<volatile int*>(&z_epoch) = zv + it.nA + 1;
-          PROF2(zv == 0, 6);
+          *reinterpret_cast<volatile int*>(&zin_epoch) = (int)n_items + 1;
+          PROF2(n_items == 0, 6);
         }
         mbar_arrive(&bar.s_loaded);
         mbar_arrive(&bar.sb_full);
       }
-      nkv += it.nA;
+      if (it.need_dS) nv += it.nC;
       // ---- pass C
       for (int j = 0; j < it.nC; ++j) {
-        const int s = nkv & 1, sq = nq & 1;
+        const int sv = nv & 1, sq = nq & 1;
         // ---- P: causal mask inside the chunk, row sum, bf16 back into TMEM
         if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
         const float qzr = qz[sq][0][r] + qz[sq][1][r];
@@ -622,7 +653,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (tid == 64) PROF(2, nq, 6);
         tc_fence_after_sync();
         const float inv = 1.f / den;
-        uint8_t* stage = sV + s * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
+        uint8_t* stage = sV + sv * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
 #pragma unroll
         for (int cc = 0; cc < D / 32; ++cc) {
           uint32_t v[32];
@@ -643,11 +674,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         fence_proxy_async_smem();
         mbar_arrive(&bar.o_staged);
         if (tid == 64) PROF(2, nq, 7);
-        ++nkv;
+        ++nv;
         ++nq;
       }
       if (!ok) break;
-      zv += it.nA + it.nC + 2;
+      ++n_items;
     }
   } else if (warp < 14) {
     // ================================================================ phi(Q) group (8 warps)
@@ -657,20 +688,22 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per thread
     uint32_t nq = 0, n_a = 0, n_items = 0;
-    int zv = 0;
+    int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
-      if (it.nA > 0) {
+      const int ip = n_items & 1;
+      na += it.nC;
+      if (it.need_dS) {
         ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, n_items & 1);
         ++n_a;
         ok = !__any_sync(0xffffffffu, !ok);
         if (!ok) break;
       }
-      ++n_items;
-      for (int j = 0; j < it.nC; ++j) {
+      // z before chunk j = zin (state before the segment) + zcum[j] (this segment's first j chunks)
+      ok = wait_epoch(&zin_epoch, (int)n_items + 1, p.status, 403) && wait_epoch(&ka_epoch, na, p.status, 404);
+      for (int j = 0; j < it.nC && ok; ++j) {
         const int sq = nq & 1;
-        const int ver = zv + it.nA + 1 + j;  // z before this chunk
         ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
         if (tid == 192) PROF(3, nq, 0);
         if (ok && nq >= 2) {
@@ -678,13 +711,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // phi(Q) buffer sq is free
                mbar_wait(&bar.qz_free[sq], par, p.status, 402);      // qz[sq] of two chunks ago was read
         }
-        ok = ok && wait_epoch(&z_epoch, ver, p.status, 403);
         if (tid == 192) PROF(3, nq, 1);
         tc_fence_after_sync();
         if (ok) {
           uint32_t pk[kChunksPerHalf * 4];
           float dot[2] = {0.f, 0.f};
-          const float* zc = zs[ver & 7];
+          const float* za_base = zin[ip];
+          const float* zb_base = zcum[ip][j];
 #pragma unroll
           for (int g = 0; g < kChunksPerHalf; ++g) {
             const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
@@ -692,9 +725,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             const uint4 rawv =
                 *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
             const uint32_t w4[4] = {rawv.x, rawv.y, rawv.z, rawv.w};
-            const float4 za = *reinterpret_cast<const float4*>(zc + gl * 8);
-            const float4 zb = *reinterpret_cast<const float4*>(zc + gl * 8 + 4);
-            const float zvv[8] = {za.x, za.y, za.z, za.w, zb.x, zb.y, zb.z, zb.w};
+            const float4 a0 = *reinterpret_cast<const float4*>(za_base + gl * 8);
+            const float4 a1 = *reinterpret_cast<const float4*>(za_base + gl * 8 + 4);
+            const float4 b0 = *reinterpret_cast<const float4*>(zb_base + gl * 8);
+            const float4 b1 = *reinterpret_cast<const float4*>(zb_base + gl * 8 + 4);
+            const float zvv[8] = {a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w,
+                                  a1.x + b1.x, a1.y + b1.y, a1.z + b1.z, a1.w + b1.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
               const uint32_t pkv = phi_bf16x2(w4[e]);
@@ -721,138 +757,154 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         }
         if (tid == 192) PROF(3, nq, 2);
         ok = !__any_sync(0xffffffffu, !ok);
-        if (!ok) break;
         ++nq;
       }
-      zv += it.nA + it.nC + 2;
+      ++n_items;
     }
   } else if (warp < 22) {
-    // ================================================================ phi(K) group (8 warps)
+    // ================================================================ phi(K) group (8 warps, pass A)
     const int tt = tid - 14 * 32;  // 0..255
-    uint32_t nkv = 0, n_a = 0, n_items = 0;
-    int zv = 0;
+    uint32_t nk = 0, n_a = 0, n_items = 0;
+    uint32_t n_ka[2] = {0, 0};
+    int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
-      // version zv: zero (start of the segment's own column sums)
-      if (tt < D) zs[zv & 7][tt] = 0.f;
+      const int ip = n_items & 1;
+      if (tt < D) zcum[ip][0][tt] = 0.f;
       if (named_bar_or(3, 256, false)) break;
-      if (tt == 0) {
-        __threadfence_block();
-        *reinterpret_cast<volatile int*>(&z_epoch) = zv;
+      for (int j = 0; j < it.nC; ++j) {
+        const int sk = nk & 1;
+        const int n0 = (it.c_begin + j) * 128;
+        ok = ok && mbar_wait(&bar.ka_full[sk], n_ka[sk] & 1, p.status, 410);
+        ++n_ka[sk];
+        if (tt == 0) PROF(3, na, 4);
+        if (ok && tt < 2 * D) {
+          const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
+          const int box = cc >> 3, cin = cc & 7;
+          uint8_t* kb = sK + sk * C::kTile + box * C::kBoxBytes;
+          float cs[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) cs[e] = 0.f;
+          // all loads first, then branch-free arithmetic, then all stores (the tile is updated in place)
+          uint4 rawv[8];
+#pragma unroll
+          for (int k8 = 0; k8 < 8; ++k8) {
+            const int row = (tt & 15) + 16 * k8;
+            rawv[k8] = *reinterpret_cast<const uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
+          }
+#pragma unroll
+          for (int k8 = 0; k8 < 8; ++k8) {
+            const int row = (tt & 15) + 16 * k8;
+            const uint32_t keep = ((n0 + row) < p.N) ? 0xffffffffu : 0u;  // rows past N must not enter S, z
+            uint32_t w4[4] = {rawv[k8].x, rawv[k8].y, rawv[k8].z, rawv[k8].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              w4[e] = phi_bf16x2(w4[e]) & keep;
+              cs[2 * e] += bf16_lo(w4[e]);
+              cs[2 * e + 1] += bf16_hi(w4[e]);
+            }
+            rawv[k8] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          }
+#pragma unroll
+          for (int k8 = 0; k8 < 8; ++k8) {
+            const int row = (tt & 15) + 16 * k8;
+            *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k8];
+          }
+          fence_proxy_async_smem();
+#pragma unroll
+          for (int e = 0; e < 8; ++e) {
+#pragma unroll
+            for (int off = 8; off > 0; off >>= 1) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], off);
+          }
+          if ((tt & 15) == 0) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) zcum[ip][j + 1][cc * 8 + e] = zcum[ip][j][cc * 8 + e] + cs[e];
+          }
+        }
+        __syncwarp();
+        if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);
+        if (tt == 0) PROF(3, na, 5);
+        if (named_bar_or(3, 256, !ok)) { ok = false; break; }
+        ++na;
+        if (tt == 0) {
+          __threadfence_block();
+          *reinterpret_cast<volatile int*>(&ka_epoch) = na;
+        }
+        ++nk;
       }
-      for (int pass = (it.nA > 0 ? 0 : 1); pass < 2 && ok; ++pass) {
-        // pass C starts from the state before the segment, written by the P group
-        if (pass == 1) {
-          if (it.nA > 0) {
-            ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, n_items & 1);  // column quarters 2, 3
-            ++n_a;
-            if (named_bar_or(3, 256, !ok)) { ok = false; break; }
-          }
-          ok = wait_epoch(&z_epoch, zv + it.nA + 1, p.status, 411);
-        }
-        for (int j = 0; j < it.nC; ++j) {
-          const int s = nkv & 1;
-          const int ver = (pass == 0) ? zv + j : zv + it.nA + 1 + j;  // version read; ver + 1 is written
-          const int n0 = (it.c_begin + j) * 128;
-          ok = ok && mbar_wait(&bar.k_full[s], (nkv >> 1) & 1, p.status, 410);
-          if (tt == 0 && pass == 1) PROF(3, nkv, 4);
-          if (ok && tt < 2 * D) {
-            const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
-            const int box = cc >> 3, cin = cc & 7;
-            uint8_t* kb = sK + s * C::kTile + box * C::kBoxBytes;
-            float cs[8];
-#pragma unroll
-            for (int e = 0; e < 8; ++e) cs[e] = 0.f;
-            // all loads first, then branch-free arithmetic, then all stores (the tile is updated in place)
-            uint4 rawv[8];
-#pragma unroll
-            for (int k8 = 0; k8 < 8; ++k8) {
-              const int row = (tt & 15) + 16 * k8;
-              rawv[k8] = *reinterpret_cast<const uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
-            }
-#pragma unroll
-            for (int k8 = 0; k8 < 8; ++k8) {
-              const int row = (tt & 15) + 16 * k8;
-              const uint32_t keep = ((n0 + row) < p.N) ? 0xffffffffu : 0u;  // rows past N must not enter S, z
-              uint32_t w4[4] = {rawv[k8].x, rawv[k8].y, rawv[k8].z, rawv[k8].w};
-#pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                w4[e] = phi_bf16x2(w4[e]) & keep;
-                cs[2 * e] += bf16_lo(w4[e]);
-                cs[2 * e + 1] += bf16_hi(w4[e]);
-              }
-              rawv[k8] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-            }
-#pragma unroll
-            for (int k8 = 0; k8 < 8; ++k8) {
-              const int row = (tt & 15) + 16 * k8;
-              *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k8];
-            }
-            fence_proxy_async_smem();
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-#pragma unroll
-              for (int off = 8; off > 0; off >>= 1) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], off);
-            }
-            if ((tt & 15) == 0) {
-#pragma unroll
-              for (int e = 0; e < 8; ++e) zs[(ver + 1) & 7][cc * 8 + e] = zs[ver & 7][cc * 8 + e] + cs[e];
-            }
-          }
-          __syncwarp();
-          if (ok && lane == 0) mbar_arrive(&bar.kphi_full[s]);
-          if (tt == 0 && pass == 1) PROF(3, nkv, 5);
-          if (named_bar_or(3, 256, !ok)) { ok = false; break; }
-          if (tt == 0) {
-            __threadfence_block();
-            *reinterpret_cast<volatile int*>(&z_epoch) = ver + 1;
-          }
-          ++nkv;
-        }
+      if (!ok) break;
+      nk += it.nC;  // the K ring also carries the pass-C tiles
+      if (it.need_dS) {
+        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, n_items & 1);  // column quarters 2, 3
+        ++n_a;
+        if (named_bar_or(3, 256, !ok)) break;
       }
       ++n_items;
-      if (ok && it.last_seg && p.z_io != nullptr && tt < D)
-        p.z_io[((long long)it.b * p.h_count + it.hl) * D + tt] = zs[(zv + it.nA + 1 + it.nC) & 7][tt];
-      zv += it.nA + it.nC + 2;
     }
-  } else {
-    // ================================================================ O store warp
+  } else if (warp == 22) {
+    // ================================================================ TMA store warp
     if (elect_one()) {
-      uint32_t nkv = 0, nq = 0, n_a = 0;
+      uint32_t nk = 0, nv = 0, nq = 0;
+      uint32_t n_kphi[2] = {0, 0};
       bool ok = true;
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
-        nkv += it.nA;
-        // one poller per CTA: hundreds of threads spinning on a handful of L2 lines slow the whole chain
-        if (it.g > 0 && !wait_flag(p.flags + ((long long)it.chain * p.G + it.g - 1) * kFlagStride, p.status, 511)) {
-          ok = false;
-          break;
-        }
-        mbar_arrive(&bar.prev_ready);
-        if (it.nA > 0) {
-          // every warp of the hand-over has written and fenced its part of the inclusive state
-          if (!mbar_wait(&bar.pub_done, n_a & 1, p.status, 510)) { ok = false; break; }
-          PROF2(n_a == 0, 4);
-          ++n_a;
-          const unsigned int one = 1u;
-          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.flags + ((long long)it.chain * p.G + it.g) * kFlagStride), "r"(one)
-                       : "memory");
-        }
+        // ---- pass A: park phi(K) tiles in the output rows of their chunk
         for (int j = 0; j < it.nC; ++j) {
-          const int s = nkv & 1;
-          if (!mbar_wait(&bar.o_staged, nq & 1, p.status, 500)) { ok = false; break; }
+          const int sk = nk & 1;
+          if (!mbar_wait(&bar.kphi_full[sk], n_kphi[sk] & 1, p.status, 520)) { ok = false; break; }
+          ++n_kphi[sk];
           for (int x = 0; x < D / 64; ++x)
-            tma_store_4d(&mo, sV + s * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b);
+            tma_store_4d(&mo, sK + sk * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b);
           tma_store_commit();
           tma_store_wait_read<0>();
-          mbar_arrive(&bar.v_free[s]);  // the staging buffer may take the V tile two uses later
-          ++nkv;
+          mbar_arrive(&bar.k_free[sk]);
+          ++nk;
+        }
+        if (!ok) break;
+        tma_store_wait_all<0>();  // parked tiles are in memory before pass C asks for them
+        mbar_arrive(&bar.park_done);
+        nk += it.nC;
+        if (it.need_dS) nv += it.nC;
+        // ---- pass C: O tiles
+        for (int j = 0; j < it.nC; ++j) {
+          const int sv = nv & 1;
+          if (!mbar_wait(&bar.o_staged, nq & 1, p.status, 500)) { ok = false; break; }
+          for (int x = 0; x < D / 64; ++x)
+            tma_store_4d(&mo, sV + sv * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b);
+          tma_store_commit();
+          tma_store_wait_read<0>();
+          mbar_arrive(&bar.v_free[sv]);  // the staging buffer may take the V tile two uses later
+          ++nv;
           ++nq;
         }
       }
       tma_store_wait_all<0>();
       PROF2(true, 7);
+    }
+  } else {
+    // ================================================================ flag warp
+    if (elect_one()) {
+      uint32_t n_a = 0;
+      int n_items = 0;
+      for (int item = blockIdx.x; item < p.nitems; item += gridDim.x, ++n_items) {
+        const LinItem it = decode_item(p, item);
+        const long long slot = (long long)it.chain * p.G + it.g;
+        // stay at most one item ahead of the hand-over (prev_ready is waited on by item parity)
+        if (n_items > 0 && !wait_epoch(&zin_epoch, n_items, p.status, 512)) break;
+        // one poller per CTA: hundreds of threads spinning on a handful of L2 lines slow the whole chain
+        if (it.g > 0 && !wait_flag(p.flags + (slot - 1) * kFlagStride, p.status, 511)) break;
+        mbar_arrive(&bar.prev_ready);
+        if (it.need_dS) {
+          // every warp of the hand-over has written its part of the inclusive state
+          if (!mbar_wait(&bar.pub_done, n_a & 1, p.status, 510)) break;
+          PROF2(n_a == 0, 4);
+          ++n_a;
+          const unsigned int one = 1u;
+          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.flags + slot * kFlagStride), "r"(one) : "memory");
+        }
+      }
     }
   }
   tc_fence_before_sync();
@@ -882,13 +934,12 @@ void linear_tc_plan(int nchains, int N, int split, int* L_out, int* G_out) {
   int L;
   if (split > 0) {
     L = split;
-  } else if (nchains >= 120 || nch <= 8) {
-    L = nch;  // enough chains to fill the machine (or nothing to cut): one segment per chain
   } else {
-    L = 8;
+    L = kMaxL;
     // keep at least ~2 items per SM, but never segments shorter than 4 chunks
     while (L > 4 && (long long)nchains * ((nch + L - 1) / L) < 296) L -= 1;
   }
+  if (L > kMaxL) L = kMaxL;
   if (L > nch) L = nch;
   if (L < 1) L = 1;
   *L_out = L;
@@ -898,7 +949,6 @@ void linear_tc_plan(int nchains, int N, int split, int* L_out, int* G_out) {
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
   int L, G;
   linear_tc_plan(nchains, N, split, &L, &G);
-  if (G <= 1) return 0;
   const size_t flags = (size_t)nchains * G * kFlagStride * sizeof(unsigned int);
   return flags + (size_t)nchains * G * ((size_t)128 * d + d) * sizeof(float);
 }
@@ -928,10 +978,8 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   p.flags = reinterpret_cast<unsigned int*>(scratch);
   p.prefix = reinterpret_cast<float*>(scratch + flag_bytes);
   cudaError_t e;
-  if (p.G > 1) {
-    e = cudaMemsetAsync(p.flags, 0, flag_bytes, stream);
-    if (e != cudaSuccess) return e;
-  }
+  e = cudaMemsetAsync(p.flags, 0, flag_bytes, stream);
+  if (e != cudaSuccess) return e;
   int dev = 0, sms = 0;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
   if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
