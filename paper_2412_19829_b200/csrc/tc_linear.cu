@@ -22,12 +22,13 @@
 // Warp roles:
 //   warp 0       TMA producer (raw Q, K, V tiles; K and V double buffered)
 //   warp 1       MMA issuer
-//   warps 2-5    "P group": masks/packs P in TMEM, converts S to bf16 for the next chunk's
-//                readout, divides and stores O (one thread per row / TMEM lane)
-//   warps 6-13   "phi(Q) group": applies phi to Q; the result goes to TMEM as the A operand of
-//                MMA1/MMA2, together with the per-row dot product with z_{c-1}
-//   warps 14-21  "phi(K) group" (pass A): applies phi to K in place in shared memory and keeps the
-//                cumulative column sums
+//   warps 2-5    "P group": masks/packs P in TMEM and forms the denominators (one thread per row)
+//   warps 6-13   "Q group": pass C: applies phi to Q; the result goes to TMEM as the A operand of
+//                MMA1/MMA2, together with the per-row dot product with z_{c-1};
+//                pass A: transforms half of every K tile
+//   warps 14-21  "K group": pass A: applies phi to the other half of every K tile (in place in
+//                shared memory) and keeps the cumulative column sums; pass C: converts S to bf16
+//                for the next chunk's readout, divides O and stages it for the store
 //   warp 22      TMA stores: parks phi(K) tiles (pass A), stores O tiles staged in the dead V
 //                buffer (pass C)
 //   warp 23      polls the previous segment's flag and raises this segment's flag
@@ -101,8 +102,8 @@ struct LinBarriers {
   uint64_t q_full, q_land_free;
   uint64_t k_full[2], ka_full[2], v_full[2], k_free[2], v_free[2];  // ka_full: K tiles of pass A, k_full: of pass C
   uint64_t qphi_full[2], kphi_full[2], qphi_free[2], qz_free[2];
-  uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, prev_ready, park_done;
-  uint64_t pm_full, s_loaded, sb_full, o_free, o_staged;
+  uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done;
+  uint64_t pm_full, den_full[2], s_loaded, sb_full, o_free, o_staged[2];
 };
 
 // Bounded poll of a monotonic counter in shared memory.
@@ -197,6 +198,45 @@ __device__ __forceinline__ uint32_t phi_bf16x2(uint32_t w) {
 __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
+// phi on rows {lane16 + 16 k8 : k8 in [k8_begin, k8_begin + 4)} x one 16-byte column chunk of a K
+// tile, in place, plus the column sums of those rows reduced over the 16 lanes that share the
+// column chunk (result valid in the lane with lane16 == 0).  Rows at or past n_valid become 0.
+__device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane16, int k8_begin, int n_valid,
+                                                 float (&cs)[8]) {
+#pragma unroll
+  for (int e = 0; e < 8; ++e) cs[e] = 0.f;
+  uint4 rawv[4];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int row = lane16 + 16 * (k8_begin + k);
+    rawv[k] = *reinterpret_cast<const uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int row = lane16 + 16 * (k8_begin + k);
+    const uint32_t keep = (row < n_valid) ? 0xffffffffu : 0u;
+    uint32_t w4[4] = {rawv[k].x, rawv[k].y, rawv[k].z, rawv[k].w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      w4[e] = phi_bf16x2(w4[e]) & keep;
+      cs[2 * e] += bf16_lo(w4[e]);
+      cs[2 * e + 1] += bf16_hi(w4[e]);
+    }
+    rawv[k] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+  }
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int row = lane16 + 16 * (k8_begin + k);
+    *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k];
+  }
+  fence_proxy_async_smem();
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+#pragma unroll
+    for (int off = 8; off > 0; off >>= 1) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], off);
+  }
+}
+
 // Critical path of the segment hand-over, run by the 16 phi warps (4 per TMEM lane quarter, each
 // thread one row x 32 columns): inclusive state of this segment = inclusive state of the previous
 // one (global scratch, or the caller's initial state for the first segment) + this segment's own
@@ -205,7 +245,7 @@ __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w 
 template <int D>
 __device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinItem& it, LinBarriers& bar,
                                                   uint32_t tmem, int warp, int lane, uint32_t a_parity,
-                                                  uint32_t item_parity) {
+                                                  const int* prev_epoch, int item_number) {
   using C = LinCfg<D>;
   const int quarter = warp & 3, colq = (warp - 6) >> 2;  // colq 0..3: which 32 columns (D=128) / 16 (D=64)
   const int r = quarter * 32 + lane;
@@ -214,8 +254,8 @@ __device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinI
   bool ok = mbar_wait(&bar.a_done, a_parity, p.status, 600);
   tc_fence_after_sync();
   PROF2(warp == 6 && lane == 0 && a_parity == 0, 0);
-  // one thread of the CTA (store warp) polls the previous segment's flag for everybody
-  ok = ok && mbar_wait(&bar.prev_ready, item_parity, p.status, 601);
+  // one thread of the CTA (flag warp) polls the previous segment's flag for everybody
+  ok = ok && wait_epoch(prev_epoch, item_number + 1, p.status, 601);
   PROF2(warp == 6 && lane == 0 && a_parity == 0, 1);
   if (ok) {
     uint32_t ds[W];
@@ -279,8 +319,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   __shared__ __align__(16) float zcum[2][kMaxL + 1][D];
   __shared__ __align__(16) float zin[2][D];
   __shared__ float qz[2][2][128];  // [chunk parity][column half][row]
+  __shared__ float den_s[2][128];  // [chunk parity][row]: denominators, P group -> K group
+  __shared__ float zpart[2][2][D]; // [tile parity][row half][column]: column sums of one K tile
   __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
   __shared__ int zin_epoch;        // items whose zin is in place (monotonic)
+  __shared__ int prev_epoch;       // items whose predecessor state has been seen in global memory (monotonic)
   __shared__ uint32_t tmem_base_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -295,7 +338,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(&bar.k_free[s], 2);
       mbar_init(&bar.v_free[s], 1);
       mbar_init(&bar.qphi_full[s], 8);
-      mbar_init(&bar.kphi_full[s], 8);
+      mbar_init(&bar.kphi_full[s], 16);
       mbar_init(&bar.qphi_free[s], 1);
       mbar_init(&bar.qz_free[s], 128);
     }
@@ -305,15 +348,18 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.mma2_done, 1);
     mbar_init(&bar.a_done, 1);
     mbar_init(&bar.pub_done, 20);  // 16 phi warps + 4 P-group warps
-    mbar_init(&bar.prev_ready, 1);
     mbar_init(&bar.park_done, 1);
     mbar_init(&bar.pm_full, 128);
-    mbar_init(&bar.s_loaded, 128);
-    mbar_init(&bar.sb_full, 128);
-    mbar_init(&bar.o_free, 128);
-    mbar_init(&bar.o_staged, 128);
+    mbar_init(&bar.den_full[0], 128);
+    mbar_init(&bar.den_full[1], 128);
+    mbar_init(&bar.s_loaded, 256);
+    mbar_init(&bar.sb_full, 256);
+    mbar_init(&bar.o_free, 256);
+    mbar_init(&bar.o_staged[0], 256);
+    mbar_init(&bar.o_staged[1], 256);
     ka_epoch = 0;
     zin_epoch = 0;
+    prev_epoch = 0;
     mbar_fence_init();
     tma_prefetch_desc(&mq);
     tma_prefetch_desc(&mk);
@@ -485,96 +531,41 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const bool s_row = r < D;  // rows of S are feature indices a < D
-    uint32_t nv = 0, nq = 0, n_a = 0, n_items = 0;
+    uint32_t nq = 0, n_items = 0;
     int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
       const long long sidx = (long long)it.b * p.h_count + it.hl;
       const int ip = n_items & 1;
-      // ---- state hand-over.  The phi warps add this segment's contribution to the previous
-      //      segment's inclusive state and publish it (the chain's critical path); this group
-      //      publishes z the same way and loads the previous state as the start of pass C.
       const long long slot = (long long)it.chain * p.G + it.g;
+      // ---- hand-over of z: previous segment's inclusive z in, this segment's inclusive z out
       na += it.nC;
-      if (it.need_dS) {
-        ok = mbar_wait(&bar.a_done, n_a & 1, p.status, 310);
-        tc_fence_after_sync();
-      }
-      ok = ok && wait_epoch(&ka_epoch, na, p.status, 311);
-      ok = ok && mbar_wait(&bar.prev_ready, n_items & 1, p.status, 312);
+      ok = wait_epoch(&ka_epoch, na, p.status, 311);
+      ok = ok && wait_epoch(&prev_epoch, (int)n_items + 1, p.status, 312);
       if (named_bar_or(1, 128, !ok)) break;
-      {
-        if (s_row) {
-          float z0 = 0.f;
-          if (it.g > 0) z0 = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
-          else if (p.z_io != nullptr && !p.zero_init) z0 = p.z_io[sidx * D + r];
-          if (it.need_dS) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, z0 + zcum[ip][it.nC][r]);
-          if (it.last_seg && p.z_io != nullptr) p.z_io[sidx * D + r] = z0 + zcum[ip][it.nC][r];
-          zin[ip][r] = z0;
-        }
-        if (it.need_dS) {
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bar.pub_done);
-          PROF2(tid == 64 && n_items == 0, 5);
-          // the phi warps read dS from TMEM: do not overwrite it before they are done
-          ok = mbar_wait(&bar.pub_done, n_a & 1, p.status, 313);
-          ++n_a;
-          tc_fence_after_sync();
-        }
-        const float* Sin = nullptr;
-        long long sin_stride = 1;  // float4 units between consecutive column groups of one row
-        if (it.g > 0) {
-          Sin = p.prefix + (slot - 1) * C::kStateFloats + (long long)r * 4;
-          sin_stride = 128;
-        } else if (p.S_io != nullptr && !p.zero_init) {
-          Sin = p.S_io + (sidx * D + r) * D;  // caller's row-major state
-        }
-#pragma unroll
-        for (int cc = 0; cc < D / 32; ++cc) {
-          uint32_t v[32];
-#pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            float4 in = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (Sin != nullptr && s_row)
-              in = __ldcg(reinterpret_cast<const float4*>(Sin) + (cc * 8 + j / 4) * sin_stride);
-            v[j] = __float_as_uint(in.x);
-            v[j + 1] = __float_as_uint(in.y);
-            v[j + 2] = __float_as_uint(in.z);
-            v[j + 3] = __float_as_uint(in.w);
-          }
-          tmem_st32(tmem + C::tS + lane_off + cc * 32, v);
-          if (s_row) {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              uint4 val;
-              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-              const uint32_t col = (cc & 1) * 32 + g * 8;
-              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, col)) = val;
-            }
-          }
-        }
-        tmem_wait_st();
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        if (named_bar_or(1, 128, !ok)) break;
-        if (tid == 64) {
-          __threadfence_block();
-          *reinterpret_cast<volatile int*>(&zin_epoch) = (int)n_items + 1;
-          PROF2(n_items == 0, 6);
-        }
-        mbar_arrive(&bar.s_loaded);
-        mbar_arrive(&bar.sb_full);
+      if (r < D) {
+        float z0 = 0.f;
+        if (it.g > 0) z0 = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
+        else if (p.z_io != nullptr && !p.zero_init) z0 = p.z_io[sidx * D + r];
+        if (it.need_dS) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, z0 + zcum[ip][it.nC][r]);
+        if (it.last_seg && p.z_io != nullptr) p.z_io[sidx * D + r] = z0 + zcum[ip][it.nC][r];
+        zin[ip][r] = z0;
       }
-      if (it.need_dS) nv += it.nC;
-      // ---- pass C
+      if (it.need_dS) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar.pub_done);
+        PROF2(tid == 64 && n_items == 0, 5);
+      }
+      if (named_bar_or(1, 128, false)) break;
+      if (tid == 64) {
+        __threadfence_block();
+        *reinterpret_cast<volatile int*>(&zin_epoch) = (int)n_items + 1;
+        PROF2(n_items == 0, 6);
+      }
+      // ---- pass C: causal mask inside the chunk, row sum, bf16 back into TMEM, denominator
       for (int j = 0; j < it.nC; ++j) {
-        const int sv = nv & 1, sq = nq & 1;
-        // ---- P: causal mask inside the chunk, row sum, bf16 back into TMEM
+        const int sq = nq & 1;
         if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
         const float qzr = qz[sq][0][r] + qz[sq][1][r];
         mbar_arrive(&bar.qz_free[sq]);
@@ -605,76 +596,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           }
           tmem_st16(tmem + C::tP + lane_off + cc * 16, pk);
         }
-        const float den = rowsum + qzr;
+        den_s[sq][r] = rowsum + qzr;
+        mbar_arrive(&bar.den_full[sq]);
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(&bar.pm_full);
         if (tid == 64) PROF(2, nq, 1);
-        // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
-        //      bf16 copy, stream the new one into shared memory for the next chunk
-        if (!mbar_wait(&bar.s_full, nq & 1, p.status, 302)) { ok = false; break; }
-        if (tid == 64) PROF(2, nq, 2);
-        if (!mbar_wait(&bar.mma2_done, nq & 1, p.status, 303)) { ok = false; break; }
-        if (tid == 64) PROF(2, nq, 3);
-        tc_fence_after_sync();
-        const bool write_final = it.last_seg && (j == it.nC - 1) && p.S_io != nullptr;
-#pragma unroll
-        for (int cc = 0; cc < D / 32; ++cc) {
-          uint32_t v[32];
-          tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
-          tmem_wait_ld();
-          if (s_row) {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              uint4 val;
-              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-            }
-            if (write_final) {
-              float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
-#pragma unroll
-              for (int jj = 0; jj < 32; jj += 4)
-                *reinterpret_cast<float4*>(dst + jj) =
-                    make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
-                                __uint_as_float(v[jj + 3]));
-            }
-          }
-        }
-        tc_fence_before_sync();
-        mbar_arrive(&bar.s_loaded);
-        fence_proxy_async_smem();
-        mbar_arrive(&bar.sb_full);
-        if (tid == 64) PROF(2, nq, 5);
-        // ---- O: divide by the denominator, bf16, stage for the TMA store
-        if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304)) { ok = false; break; }
-        if (tid == 64) PROF(2, nq, 6);
-        tc_fence_after_sync();
-        const float inv = 1.f / den;
-        uint8_t* stage = sV + sv * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
-#pragma unroll
-        for (int cc = 0; cc < D / 32; ++cc) {
-          uint32_t v[32];
-          tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
-          tmem_wait_ld();
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 val;
-            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
-            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
-            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
-            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-          }
-        }
-        tc_fence_before_sync();
-        mbar_arrive(&bar.o_free);
-        fence_proxy_async_smem();
-        mbar_arrive(&bar.o_staged);
-        if (tid == 64) PROF(2, nq, 7);
-        ++nv;
         ++nq;
       }
       if (!ok) break;
@@ -687,15 +614,41 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int r = quarter * 32 + lane;    // Q row
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per thread
-    uint32_t nq = 0, n_a = 0, n_items = 0;
+    uint32_t nq = 0, nk = 0, n_a = 0, n_items = 0;
+    uint32_t n_ka[2] = {0, 0};
     int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
       const int ip = n_items & 1;
       na += it.nC;
+      // ---- pass A: rows 64..127 (by sixteens) of every K tile
+      {
+        const int tt = tid - 6 * 32;
+        for (int j = 0; j < it.nC; ++j) {
+          const int sk = nk & 1;
+          ok = ok && mbar_wait(&bar.ka_full[sk], n_ka[sk] & 1, p.status, 420);
+          ++n_ka[sk];
+          if (ok && tt < 2 * D) {
+            const int cc = tt >> 4;
+            float cs[8];
+            transform_k_rows(sK + sk * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, 4,
+                             p.N - (it.c_begin + j) * 128, cs);
+            if ((tt & 15) == 0) {
+#pragma unroll
+              for (int e = 0; e < 8; ++e) zpart[j & 1][1][cc * 8 + e] = cs[e];
+            }
+          }
+          __syncwarp();
+          if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);
+          if (named_bar_or(4, 512, !ok)) { ok = false; break; }
+          ++nk;
+        }
+        if (!ok) break;
+        nk += it.nC;
+      }
       if (it.need_dS) {
-        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, n_items & 1);
+        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);
         ++n_a;
         ok = !__any_sync(0xffffffffu, !ok);
         if (!ok) break;
@@ -762,70 +715,46 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       ++n_items;
     }
   } else if (warp < 22) {
-    // ================================================================ phi(K) group (8 warps, pass A)
-    const int tt = tid - 14 * 32;  // 0..255
-    uint32_t nk = 0, n_a = 0, n_items = 0;
+    // ================================================================ K group (8 warps)
+    const int tt = tid - 14 * 32;         // 0..255
+    const int quarter = warp & 3;         // TMEM lane quarter of this warp
+    const int colh = (warp - 14) >> 2;    // which half of the columns this warp handles in pass C
+    const int r = quarter * 32 + lane;
+    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
+    const bool s_row = r < D;             // rows of S are feature indices a < D
+    constexpr int EC = D / 64;            // 32-column blocks per thread in pass C
+    uint32_t nk = 0, nv = 0, nq = 0, n_a = 0, n_items = 0;
     uint32_t n_ka[2] = {0, 0};
     int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
+      const long long sidx = (long long)it.b * p.h_count + it.hl;
+      const long long slot = (long long)it.chain * p.G + it.g;
       const int ip = n_items & 1;
       if (tt < D) zcum[ip][0][tt] = 0.f;
-      if (named_bar_or(3, 256, false)) break;
+      // ---- pass A: rows 0..63 (by sixteens) of every K tile, cumulative column sums
       for (int j = 0; j < it.nC; ++j) {
         const int sk = nk & 1;
-        const int n0 = (it.c_begin + j) * 128;
         ok = ok && mbar_wait(&bar.ka_full[sk], n_ka[sk] & 1, p.status, 410);
         ++n_ka[sk];
         if (tt == 0) PROF(3, na, 4);
         if (ok && tt < 2 * D) {
           const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
-          const int box = cc >> 3, cin = cc & 7;
-          uint8_t* kb = sK + sk * C::kTile + box * C::kBoxBytes;
           float cs[8];
-#pragma unroll
-          for (int e = 0; e < 8; ++e) cs[e] = 0.f;
-          // all loads first, then branch-free arithmetic, then all stores (the tile is updated in place)
-          uint4 rawv[8];
-#pragma unroll
-          for (int k8 = 0; k8 < 8; ++k8) {
-            const int row = (tt & 15) + 16 * k8;
-            rawv[k8] = *reinterpret_cast<const uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4));
-          }
-#pragma unroll
-          for (int k8 = 0; k8 < 8; ++k8) {
-            const int row = (tt & 15) + 16 * k8;
-            const uint32_t keep = ((n0 + row) < p.N) ? 0xffffffffu : 0u;  // rows past N must not enter S, z
-            uint32_t w4[4] = {rawv[k8].x, rawv[k8].y, rawv[k8].z, rawv[k8].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              w4[e] = phi_bf16x2(w4[e]) & keep;
-              cs[2 * e] += bf16_lo(w4[e]);
-              cs[2 * e + 1] += bf16_hi(w4[e]);
-            }
-            rawv[k8] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-          }
-#pragma unroll
-          for (int k8 = 0; k8 < 8; ++k8) {
-            const int row = (tt & 15) + 16 * k8;
-            *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k8];
-          }
-          fence_proxy_async_smem();
-#pragma unroll
-          for (int e = 0; e < 8; ++e) {
-#pragma unroll
-            for (int off = 8; off > 0; off >>= 1) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], off);
-          }
+          transform_k_rows(sK + sk * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, 0,
+                           p.N - (it.c_begin + j) * 128, cs);
           if ((tt & 15) == 0) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) zcum[ip][j + 1][cc * 8 + e] = zcum[ip][j][cc * 8 + e] + cs[e];
+            for (int e = 0; e < 8; ++e) zpart[j & 1][0][cc * 8 + e] = cs[e];
           }
         }
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);
         if (tt == 0) PROF(3, na, 5);
-        if (named_bar_or(3, 256, !ok)) { ok = false; break; }
+        if (named_bar_or(4, 512, !ok)) { ok = false; break; }  // both halves of the tile are done
+        if (tt < D) zcum[ip][j + 1][tt] = zcum[ip][j][tt] + (zpart[j & 1][0][tt] + zpart[j & 1][1][tt]);
+        if (named_bar_or(3, 256, false)) { ok = false; break; }
         ++na;
         if (tt == 0) {
           __threadfence_block();
@@ -835,18 +764,144 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       }
       if (!ok) break;
       nk += it.nC;  // the K ring also carries the pass-C tiles
+      // ---- hand-over of S: publish (with the Q group), then load the state before the segment
       if (it.need_dS) {
-        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, n_items & 1);  // column quarters 2, 3
+        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);  // column quarters 2, 3
+        // all 16 phi warps read dS from TMEM: do not overwrite it before they are done
+        ok = ok && mbar_wait(&bar.pub_done, n_a & 1, p.status, 413);
         ++n_a;
-        if (named_bar_or(3, 256, !ok)) break;
+        tc_fence_after_sync();
+        nv += it.nC;
+      } else {
+        ok = wait_epoch(&prev_epoch, (int)n_items + 1, p.status, 414);
       }
+      if (named_bar_or(3, 256, !ok)) break;
+      {
+        const float* Sin = nullptr;
+        long long sin_stride = 1;  // float4 units between consecutive column groups of one row
+        if (it.g > 0) {
+          Sin = p.prefix + (slot - 1) * C::kStateFloats + (long long)r * 4;
+          sin_stride = 128;
+        } else if (p.S_io != nullptr && !p.zero_init) {
+          Sin = p.S_io + (sidx * D + r) * D;  // caller's row-major state
+        }
+#pragma unroll
+        for (int e = 0; e < EC; ++e) {
+          const int cc = colh * EC + e;
+          uint32_t v[32];
+#pragma unroll
+          for (int jj = 0; jj < 32; jj += 4) {
+            float4 in = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (Sin != nullptr && s_row)
+              in = __ldcg(reinterpret_cast<const float4*>(Sin) + (cc * 8 + jj / 4) * sin_stride);
+            v[jj] = __float_as_uint(in.x);
+            v[jj + 1] = __float_as_uint(in.y);
+            v[jj + 2] = __float_as_uint(in.z);
+            v[jj + 3] = __float_as_uint(in.w);
+          }
+          tmem_st32(tmem + C::tS + lane_off + cc * 32, v);
+          if (s_row) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 val;
+              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+            }
+          }
+        }
+        tmem_wait_st();
+        fence_proxy_async_smem();
+        tc_fence_before_sync();
+        mbar_arrive(&bar.s_loaded);
+        mbar_arrive(&bar.sb_full);
+      }
+      // ---- pass C
+      for (int j = 0; j < it.nC; ++j) {
+        const int sv = nv & 1, sq = nq & 1;
+        // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
+        //      bf16 copy, stream the new one into shared memory for the next chunk
+        if (!mbar_wait(&bar.s_full, nq & 1, p.status, 302) || !mbar_wait(&bar.mma2_done, nq & 1, p.status, 303)) {
+          ok = false;
+          break;
+        }
+        if (tt == 0) PROF(2, nq, 2);
+        tc_fence_after_sync();
+        const bool write_final = it.last_seg && (j == it.nC - 1) && p.S_io != nullptr;
+#pragma unroll
+        for (int e = 0; e < EC; ++e) {
+          const int cc = colh * EC + e;
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
+          tmem_wait_ld();
+          if (s_row) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 val;
+              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+            }
+            if (write_final) {
+              float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
+#pragma unroll
+              for (int jj = 0; jj < 32; jj += 4)
+                *reinterpret_cast<float4*>(dst + jj) =
+                    make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
+                                __uint_as_float(v[jj + 3]));
+            }
+          }
+        }
+        tc_fence_before_sync();
+        mbar_arrive(&bar.s_loaded);
+        fence_proxy_async_smem();
+        mbar_arrive(&bar.sb_full);
+        if (tt == 0) PROF(2, nq, 5);
+        // ---- O: divide by the denominator, bf16, stage for the TMA store
+        if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304) || !mbar_wait(&bar.den_full[sq], (nq >> 1) & 1, p.status, 305)) {
+          ok = false;
+          break;
+        }
+        if (tt == 0) PROF(2, nq, 6);
+        tc_fence_after_sync();
+        const float inv = 1.f / den_s[sq][r];
+        uint8_t* stage = sV + sv * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
+#pragma unroll
+        for (int e = 0; e < EC; ++e) {
+          const int cc = colh * EC + e;
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            uint4 val;
+            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
+            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
+            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
+            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
+            *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+          }
+        }
+        tc_fence_before_sync();
+        mbar_arrive(&bar.o_free);
+        fence_proxy_async_smem();
+        mbar_arrive(&bar.o_staged[sv]);
+        if (tt == 0) PROF(2, nq, 7);
+        ++nv;
+        ++nq;
+      }
+      if (!ok) break;
       ++n_items;
     }
   } else if (warp == 22) {
     // ================================================================ TMA store warp
     if (elect_one()) {
       uint32_t nk = 0, nv = 0, nq = 0;
-      uint32_t n_kphi[2] = {0, 0};
+      uint32_t n_kphi[2] = {0, 0}, n_os[2] = {0, 0};
       bool ok = true;
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
@@ -870,7 +925,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         // ---- pass C: O tiles
         for (int j = 0; j < it.nC; ++j) {
           const int sv = nv & 1;
-          if (!mbar_wait(&bar.o_staged, nq & 1, p.status, 500)) { ok = false; break; }
+          if (!mbar_wait(&bar.o_staged[sv], n_os[sv] & 1, p.status, 500)) { ok = false; break; }
+          ++n_os[sv];
           for (int x = 0; x < D / 64; ++x)
             tma_store_4d(&mo, sV + sv * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b);
           tma_store_commit();
@@ -891,11 +947,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       for (int item = blockIdx.x; item < p.nitems; item += gridDim.x, ++n_items) {
         const LinItem it = decode_item(p, item);
         const long long slot = (long long)it.chain * p.G + it.g;
-        // stay at most one item ahead of the hand-over (prev_ready is waited on by item parity)
-        if (n_items > 0 && !wait_epoch(&zin_epoch, n_items, p.status, 512)) break;
         // one poller per CTA: hundreds of threads spinning on a handful of L2 lines slow the whole chain
         if (it.g > 0 && !wait_flag(p.flags + (slot - 1) * kFlagStride, p.status, 511)) break;
-        mbar_arrive(&bar.prev_ready);
+        __threadfence_block();
+        *reinterpret_cast<volatile int*>(&prev_epoch) = n_items + 1;
         if (it.need_dS) {
           // every warp of the hand-over has written its part of the inclusive state
           if (!mbar_wait(&bar.pub_done, n_a & 1, p.status, 510)) break;
