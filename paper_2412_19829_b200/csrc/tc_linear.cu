@@ -22,13 +22,16 @@
 // Warp roles:
 //   warp 0       TMA producer (raw Q, K, V tiles; K and V double buffered)
 //   warp 1       MMA issuer
-//   warps 2-5    "P group": masks/packs P in TMEM and forms the denominators (one thread per row)
+//   warps 2-5    "row group" (one thread per row): loads the state before the segment; pass C:
+//                converts S to bf16 for the next chunk's readout, divides O by the denominator
+//                and stages it for the store
 //   warps 6-13   "Q group": pass C: applies phi to Q; the result goes to TMEM as the A operand of
 //                MMA1/MMA2, together with the per-row dot product with z_{c-1};
 //                pass A: transforms half of every K tile
 //   warps 14-21  "K group": pass A: applies phi to the other half of every K tile (in place in
-//                shared memory) and keeps the cumulative column sums; pass C: converts S to bf16
-//                for the next chunk's readout, divides O and stages it for the store
+//                shared memory) and keeps the cumulative column sums; pass C: masks/packs P in
+//                TMEM (two warps per TMEM lane quarter, half of the key columns each) and forms
+//                the row sums for the denominators
 //   warp 22      TMA stores: parks phi(K) tiles (pass A), stores O tiles staged in the dead V
 //                buffer (pass C)
 //   warp 23      polls the previous segment's flag and raises this segment's flag
@@ -319,7 +322,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   __shared__ __align__(16) float zcum[2][kMaxL + 1][D];
   __shared__ __align__(16) float zin[2][D];
   __shared__ float qz[2][2][128];  // [chunk parity][column half][row]
-  __shared__ float den_s[2][128];  // [chunk parity][row]: denominators, P group -> K group
+  __shared__ float den_s[2][2][128];  // [chunk parity][column half][row]: partial denominators, K group -> row group
   __shared__ float zpart[2][2][D]; // [tile parity][row half][column]: column sums of one K tile
   __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
   __shared__ int zin_epoch;        // items whose zin is in place (monotonic)
@@ -349,14 +352,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.a_done, 1);
     mbar_init(&bar.pub_done, 20);  // 16 phi warps + 4 P-group warps
     mbar_init(&bar.park_done, 1);
-    mbar_init(&bar.pm_full, 128);
-    mbar_init(&bar.den_full[0], 128);
-    mbar_init(&bar.den_full[1], 128);
-    mbar_init(&bar.s_loaded, 256);
-    mbar_init(&bar.sb_full, 256);
-    mbar_init(&bar.o_free, 256);
-    mbar_init(&bar.o_staged[0], 256);
-    mbar_init(&bar.o_staged[1], 256);
+    mbar_init(&bar.pm_full, 256);
+    mbar_init(&bar.den_full[0], 256);
+    mbar_init(&bar.den_full[1], 256);
+    mbar_init(&bar.s_loaded, 128);
+    mbar_init(&bar.sb_full, 128);
+    mbar_init(&bar.o_free, 128);
+    mbar_init(&bar.o_staged[0], 128);
+    mbar_init(&bar.o_staged[1], 128);
     ka_epoch = 0;
     zin_epoch = 0;
     prev_epoch = 0;
@@ -517,7 +520,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           tc_fence_after_sync();
 #pragma unroll
           for (int ks = 0; ks < 8; ++ks)
-            umma_ts(tmem + C::tO, tmem + C::tP + ks * 8, umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
+            umma_ts(tmem + C::tO, tmem + C::tP + (ks >> 2) * 64 + (ks & 3) * 8,
+                    umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
                     id_o, true);
           umma_commit(&bar.o_full);
           ++nk;
@@ -527,11 +531,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       }
     }
   } else if (warp < 6) {
-    // ================================================================ P group (one thread per row)
+    // ================================================================ row group (one thread per row)
     const int quarter = warp & 3;
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    uint32_t nq = 0, n_items = 0;
+    const bool s_row = r < D;  // rows of S are feature indices a < D
+    uint32_t nv = 0, nq = 0, n_a = 0, n_items = 0;
     int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems; item += gridDim.x) {
@@ -544,7 +549,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       ok = wait_epoch(&ka_epoch, na, p.status, 311);
       ok = ok && wait_epoch(&prev_epoch, (int)n_items + 1, p.status, 312);
       if (named_bar_or(1, 128, !ok)) break;
-      if (r < D) {
+      if (s_row) {
         float z0 = 0.f;
         if (it.g > 0) z0 = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
         else if (p.z_io != nullptr && !p.zero_init) z0 = p.z_io[sidx * D + r];
@@ -563,45 +568,128 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         *reinterpret_cast<volatile int*>(&zin_epoch) = (int)n_items + 1;
         PROF2(n_items == 0, 6);
       }
-      // ---- pass C: causal mask inside the chunk, row sum, bf16 back into TMEM, denominator
-      for (int j = 0; j < it.nC; ++j) {
-        const int sq = nq & 1;
-        if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
-        const float qzr = qz[sq][0][r] + qz[sq][1][r];
-        mbar_arrive(&bar.qz_free[sq]);
-        if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
-        if (tid == 64) PROF(2, nq, 0);
+      // ---- hand-over of S: the 16 phi warps publish the inclusive state (they read dS from TMEM:
+      //      do not overwrite it before they are done); this group loads the state before the segment
+      if (it.need_dS) {
+        ok = mbar_wait(&bar.pub_done, n_a & 1, p.status, 313);
+        ++n_a;
         tc_fence_after_sync();
-        float rowsum = 0.f;
+        nv += it.nC;
+      }
+      {
+        const float* Sin = nullptr;
+        long long sin_stride = 1;  // float4 units between consecutive column groups of one row
+        if (it.g > 0) {
+          Sin = p.prefix + (slot - 1) * C::kStateFloats + (long long)r * 4;
+          sin_stride = 128;
+        } else if (p.S_io != nullptr && !p.zero_init) {
+          Sin = p.S_io + (sidx * D + r) * D;  // caller's row-major state
+        }
 #pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          // 32-column block cc of this warp's rows [32 q, 32 q + 32): all kept left of the
-          // diagonal block, all dropped right of it, triangular on it (warp-uniform choice)
-          uint32_t pk[16];
-          if (cc > quarter) {
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
-          } else {
-            uint32_t v[32];
-            tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
-            tmem_wait_ld();
-            const bool diag = (cc == quarter);
+          for (int jj = 0; jj < 32; jj += 4) {
+            float4 in = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (Sin != nullptr && s_row)
+              in = __ldcg(reinterpret_cast<const float4*>(Sin) + (cc * 8 + jj / 4) * sin_stride);
+            v[jj] = __float_as_uint(in.x);
+            v[jj + 1] = __float_as_uint(in.y);
+            v[jj + 2] = __float_as_uint(in.z);
+            v[jj + 3] = __float_as_uint(in.w);
+          }
+          tmem_st32(tmem + C::tS + lane_off + cc * 32, v);
+          if (s_row) {
 #pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-              const float p0 = (!diag || 2 * jj <= lane) ? __uint_as_float(v[2 * jj]) : 0.f;
-              const float p1 = (!diag || 2 * jj + 1 <= lane) ? __uint_as_float(v[2 * jj + 1]) : 0.f;
-              rowsum += p0 + p1;
-              pk[jj] = pack_bf16(p0, p1);
+            for (int g = 0; g < 4; ++g) {
+              uint4 val;
+              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
             }
           }
-          tmem_st16(tmem + C::tP + lane_off + cc * 16, pk);
         }
-        den_s[sq][r] = rowsum + qzr;
-        mbar_arrive(&bar.den_full[sq]);
         tmem_wait_st();
+        fence_proxy_async_smem();
         tc_fence_before_sync();
-        mbar_arrive(&bar.pm_full);
-        if (tid == 64) PROF(2, nq, 1);
+        mbar_arrive(&bar.s_loaded);
+        mbar_arrive(&bar.sb_full);
+      }
+      // ---- pass C
+      for (int j = 0; j < it.nC; ++j) {
+        const int sv = nv & 1, sq = nq & 1;
+        // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
+        //      bf16 copy, stream the new one into shared memory for the next chunk
+        if (!mbar_wait(&bar.s_full, nq & 1, p.status, 302) || !mbar_wait(&bar.mma2_done, nq & 1, p.status, 303)) {
+          ok = false;
+          break;
+        }
+        if (tid == 64) PROF(2, nq, 2);
+        tc_fence_after_sync();
+        const bool write_final = it.last_seg && (j == it.nC - 1) && p.S_io != nullptr;
+#pragma unroll
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
+          tmem_wait_ld();
+          if (s_row) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              uint4 val;
+              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+            }
+            if (write_final) {
+              float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
+#pragma unroll
+              for (int jj = 0; jj < 32; jj += 4)
+                *reinterpret_cast<float4*>(dst + jj) =
+                    make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
+                                __uint_as_float(v[jj + 3]));
+            }
+          }
+        }
+        tc_fence_before_sync();
+        mbar_arrive(&bar.s_loaded);
+        fence_proxy_async_smem();
+        mbar_arrive(&bar.sb_full);
+        if (tid == 64) PROF(2, nq, 5);
+        // ---- O: divide by the denominator, bf16, stage for the TMA store
+        if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304) ||
+            !mbar_wait(&bar.den_full[sq], (nq >> 1) & 1, p.status, 305)) {
+          ok = false;
+          break;
+        }
+        if (tid == 64) PROF(2, nq, 6);
+        tc_fence_after_sync();
+        const float inv = 1.f / (den_s[sq][0][r] + den_s[sq][1][r]);
+        uint8_t* stage = sV + sv * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
+#pragma unroll
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
+          tmem_wait_ld();
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            uint4 val;
+            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
+            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
+            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
+            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
+            *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+          }
+        }
+        tc_fence_before_sync();
+        mbar_arrive(&bar.o_free);
+        fence_proxy_async_smem();
+        mbar_arrive(&bar.o_staged[sv]);
+        if (tid == 64) PROF(2, nq, 7);
+        ++nv;
         ++nq;
       }
       if (!ok) break;
@@ -721,16 +809,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int colh = (warp - 14) >> 2;    // which half of the columns this warp handles in pass C
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    const bool s_row = r < D;             // rows of S are feature indices a < D
-    constexpr int EC = D / 64;            // 32-column blocks per thread in pass C
-    uint32_t nk = 0, nv = 0, nq = 0, n_a = 0, n_items = 0;
+    uint32_t nk = 0, nq = 0, n_a = 0, n_items = 0;
     uint32_t n_ka[2] = {0, 0};
     int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
-      const long long sidx = (long long)it.b * p.h_count + it.hl;
-      const long long slot = (long long)it.chain * p.G + it.g;
       const int ip = n_items & 1;
       if (tt < D) zcum[ip][0][tt] = 0.f;
       // ---- pass A: rows 0..63 (by sixteens) of every K tile, cumulative column sums
@@ -764,134 +848,57 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       }
       if (!ok) break;
       nk += it.nC;  // the K ring also carries the pass-C tiles
-      // ---- hand-over of S: publish (with the Q group), then load the state before the segment
+      // ---- hand-over of S: publish the inclusive state together with the Q group
       if (it.need_dS) {
         ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);  // column quarters 2, 3
-        // all 16 phi warps read dS from TMEM: do not overwrite it before they are done
-        ok = ok && mbar_wait(&bar.pub_done, n_a & 1, p.status, 413);
         ++n_a;
-        tc_fence_after_sync();
-        nv += it.nC;
-      } else {
-        ok = wait_epoch(&prev_epoch, (int)n_items + 1, p.status, 414);
       }
       if (named_bar_or(3, 256, !ok)) break;
-      {
-        const float* Sin = nullptr;
-        long long sin_stride = 1;  // float4 units between consecutive column groups of one row
-        if (it.g > 0) {
-          Sin = p.prefix + (slot - 1) * C::kStateFloats + (long long)r * 4;
-          sin_stride = 128;
-        } else if (p.S_io != nullptr && !p.zero_init) {
-          Sin = p.S_io + (sidx * D + r) * D;  // caller's row-major state
-        }
-#pragma unroll
-        for (int e = 0; e < EC; ++e) {
-          const int cc = colh * EC + e;
-          uint32_t v[32];
-#pragma unroll
-          for (int jj = 0; jj < 32; jj += 4) {
-            float4 in = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (Sin != nullptr && s_row)
-              in = __ldcg(reinterpret_cast<const float4*>(Sin) + (cc * 8 + jj / 4) * sin_stride);
-            v[jj] = __float_as_uint(in.x);
-            v[jj + 1] = __float_as_uint(in.y);
-            v[jj + 2] = __float_as_uint(in.z);
-            v[jj + 3] = __float_as_uint(in.w);
-          }
-          tmem_st32(tmem + C::tS + lane_off + cc * 32, v);
-          if (s_row) {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              uint4 val;
-              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-            }
-          }
-        }
-        tmem_wait_st();
-        fence_proxy_async_smem();
-        tc_fence_before_sync();
-        mbar_arrive(&bar.s_loaded);
-        mbar_arrive(&bar.sb_full);
-      }
-      // ---- pass C
+      // ---- pass C: causal mask inside the chunk, bf16 back into TMEM, partial denominators.
+      //      This warp owns rows [32 q, 32 q + 32) x key columns [64 colh, 64 colh + 64).
       for (int j = 0; j < it.nC; ++j) {
-        const int sv = nv & 1, sq = nq & 1;
-        // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
-        //      bf16 copy, stream the new one into shared memory for the next chunk
-        if (!mbar_wait(&bar.s_full, nq & 1, p.status, 302) || !mbar_wait(&bar.mma2_done, nq & 1, p.status, 303)) {
-          ok = false;
-          break;
+        const int sq = nq & 1;
+        if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
+        float part = 0.f;
+        if (colh == 0) {
+          part = qz[sq][0][r] + qz[sq][1][r];
+          mbar_arrive(&bar.qz_free[sq]);
         }
-        if (tt == 0) PROF(2, nq, 2);
+        if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
+        if (tt == 0) PROF(2, nq, 0);
         tc_fence_after_sync();
-        const bool write_final = it.last_seg && (j == it.nC - 1) && p.S_io != nullptr;
 #pragma unroll
-        for (int e = 0; e < EC; ++e) {
-          const int cc = colh * EC + e;
-          uint32_t v[32];
-          tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
-          tmem_wait_ld();
-          if (s_row) {
+        for (int e = 0; e < 2; ++e) {
+          // 32-column block cc: all kept left of the diagonal block, all dropped right of it,
+          // triangular on it (warp-uniform choice)
+          const int cc = 2 * colh + e;
+          uint32_t pk[16];
+          if (cc > quarter) {
 #pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              uint4 val;
-              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-            }
-            if (write_final) {
-              float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
+            for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+          } else {
+            uint32_t v[32];
+            tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
+            tmem_wait_ld();
+            const bool diag = (cc == quarter);
 #pragma unroll
-              for (int jj = 0; jj < 32; jj += 4)
-                *reinterpret_cast<float4*>(dst + jj) =
-                    make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
-                                __uint_as_float(v[jj + 3]));
+            for (int jj = 0; jj < 16; ++jj) {
+              const float p0 = (!diag || 2 * jj <= lane) ? __uint_as_float(v[2 * jj]) : 0.f;
+              const float p1 = (!diag || 2 * jj + 1 <= lane) ? __uint_as_float(v[2 * jj + 1]) : 0.f;
+              part += p0 + p1;
+              pk[jj] = pack_bf16(p0, p1);
             }
           }
+          // packed P stays inside this warp's own fp32 columns (keys 64h..64h+63 -> columns 64h..64h+31),
+          // so the two warps of a lane quarter never touch each other's unread input
+          tmem_st16(tmem + C::tP + lane_off + colh * 64 + e * 16, pk);
         }
+        den_s[sq][colh][r] = part;
+        mbar_arrive(&bar.den_full[sq]);
+        tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive(&bar.s_loaded);
-        fence_proxy_async_smem();
-        mbar_arrive(&bar.sb_full);
-        if (tt == 0) PROF(2, nq, 5);
-        // ---- O: divide by the denominator, bf16, stage for the TMA store
-        if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304) || !mbar_wait(&bar.den_full[sq], (nq >> 1) & 1, p.status, 305)) {
-          ok = false;
-          break;
-        }
-        if (tt == 0) PROF(2, nq, 6);
-        tc_fence_after_sync();
-        const float inv = 1.f / den_s[sq][r];
-        uint8_t* stage = sV + sv * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
-#pragma unroll
-        for (int e = 0; e < EC; ++e) {
-          const int cc = colh * EC + e;
-          uint32_t v[32];
-          tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
-          tmem_wait_ld();
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            uint4 val;
-            val.x = pack_bf16(__uint_as_float(v[8 * g + 0]) * inv, __uint_as_float(v[8 * g + 1]) * inv);
-            val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
-            val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
-            val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-          }
-        }
-        tc_fence_before_sync();
-        mbar_arrive(&bar.o_free);
-        fence_proxy_async_smem();
-        mbar_arrive(&bar.o_staged[sv]);
-        if (tt == 0) PROF(2, nq, 7);
-        ++nv;
+        mbar_arrive(&bar.pm_full);
+        if (tt == 0) PROF(2, nq, 1);
         ++nq;
       }
       if (!ok) break;
