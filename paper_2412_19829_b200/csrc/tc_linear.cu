@@ -104,7 +104,7 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
 struct LinBarriers {
   uint64_t q_full, q_land_free;
   uint64_t k_full[2], ka_full[2], v_full[2], k_free[2], v_free[2];  // ka_full: K tiles of pass A, k_full: of pass C
-  uint64_t qphi_full[2], kphi_full[2], qphi_free[2], qz_free[2];
+  uint64_t qphi_full[2], kphi_full[2], qphi_free[2];
   uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done;
   uint64_t pm_full, den_full[2], s_loaded, sb_full, o_free, o_staged[2];
 };
@@ -321,7 +321,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   // zin = z before the segment
   __shared__ __align__(16) float zcum[2][kMaxL + 1][D];
   __shared__ __align__(16) float zin[2][D];
-  __shared__ float qz[2][2][128];  // [chunk parity][column half][row]
   __shared__ float den_s[2][2][128];  // [chunk parity][column half][row]: partial denominators, K group -> row group
   __shared__ float zpart[2][2][D]; // [tile parity][row half][column]: column sums of one K tile
   __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
@@ -343,7 +342,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       mbar_init(&bar.qphi_full[s], 8);
       mbar_init(&bar.kphi_full[s], 16);
       mbar_init(&bar.qphi_free[s], 1);
-      mbar_init(&bar.qz_free[s], 128);
     }
     mbar_init(&bar.p_full, 1);
     mbar_init(&bar.s_full, 1);
@@ -389,6 +387,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       // tiles of the two passes complete on different barriers (phi(K) group / MMA issuer)
       uint32_t nk = 0, nv = 0, nq = 0, n_items = 0;
       bool ok = true;
+      // K, Q and the second read of V are streamed once; the first read of V (and the parked phi(K)
+      // tiles) come back within the same item and should stay in L2 until then
+      const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
         for (int pass = 0; pass < 2 && ok; ++pass) {
@@ -398,16 +399,18 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             const int sk = nk & 1;
             if (nk >= 2 && !mbar_wait(&bar.k_free[sk], ((nk >> 1) + 1) & 1, p.status, 101)) { ok = false; break; }
             uint64_t* kbar = (pass == 0) ? &bar.ka_full[sk] : &bar.k_full[sk];
+            if (pass == 0) PROF(0, nk - nq, 1);
             mbar_arrive_expect_tx(kbar, C::kTile);
             for (int x = 0; x < D / 64; ++x)  // pass C reads back the phi(K) tile parked in the output rows
-              tma_load_4d(sK + sk * C::kTile + x * C::kBoxBytes, pass == 0 ? &mk : &mo, kbar, x * 64, n0, it.h, it.b);
+              tma_load_4d_hint(sK + sk * C::kTile + x * C::kBoxBytes, pass == 0 ? &mk : &mo, kbar, x * 64, n0, it.h, it.b,
+                               pol_stream);
             ++nk;
             if (pass == 1) {
               if (nq >= 1 && !mbar_wait(&bar.q_land_free, (nq - 1) & 1, p.status, 100)) { ok = false; break; }
               PROF(0, nq, 0);
               mbar_arrive_expect_tx(&bar.q_full, C::kTile);
               for (int x = 0; x < D / 64; ++x)
-                tma_load_4d(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, it.h, it.b);
+                tma_load_4d_hint(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, it.h, it.b, pol_stream);
               ++nq;
             }
             if (pass == 1 || it.need_dS) {
@@ -415,7 +418,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               if (nv >= 2 && !mbar_wait(&bar.v_free[sv], ((nv >> 1) + 1) & 1, p.status, 102)) { ok = false; break; }
               mbar_arrive_expect_tx(&bar.v_full[sv], C::kTile);
               for (int x = 0; x < D / 64; ++x)
-                tma_load_4d(sV + sv * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[sv], x * 64, n0, it.h, it.b);
+                tma_load_4d_hint(sV + sv * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[sv], x * 64, n0, it.h, it.b,
+                                 pass == 0 ? pol_keep : pol_stream);
               ++nv;
             }
           }
@@ -448,6 +452,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           const int sk = nk & 1;
           if (!mbar_wait(&bar.kphi_full[sk], n_kphi[sk] & 1, p.status, 220)) { ok = false; break; }
           ++n_kphi[sk];
+          PROF(1, nk - nq, 4);
           if (it.need_dS) {
             const int sv = nv & 1;
             const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
@@ -457,6 +462,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             for (int ks = 0; ks < 8; ++ks)
               umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
                       umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, (j > 0) || (ks > 0));
+            PROF(1, nk - nq, 5);
             umma_commit(&bar.k_free[sk]);  // second arrival: the store warp, once the tile is parked
             umma_commit(&bar.v_free[sv]);
             ++nv;
@@ -708,7 +714,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
-      const int ip = n_items & 1;
       na += it.nC;
       // ---- pass A: rows 64..127 (by sixteens) of every K tile
       {
@@ -741,47 +746,36 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         ok = !__any_sync(0xffffffffu, !ok);
         if (!ok) break;
       }
-      // z before chunk j = zin (state before the segment) + zcum[j] (this segment's first j chunks)
-      ok = wait_epoch(&zin_epoch, (int)n_items + 1, p.status, 403) && wait_epoch(&ka_epoch, na, p.status, 404);
       for (int j = 0; j < it.nC && ok; ++j) {
         const int sq = nq & 1;
         ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
         if (tid == 192) PROF(3, nq, 0);
         if (ok && nq >= 2) {
           const uint32_t par = ((nq >> 1) + 1) & 1;
-          ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // phi(Q) buffer sq is free
-               mbar_wait(&bar.qz_free[sq], par, p.status, 402);      // qz[sq] of two chunks ago was read
+          ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // MMA1/MMA2 of two chunks ago are done with it
+               mbar_wait(&bar.den_full[sq], par, p.status, 402);     // ... and so is the K group's dot product
         }
         if (tid == 192) PROF(3, nq, 1);
         tc_fence_after_sync();
         if (ok) {
+          // copy the raw row half out of the landing buffer and hand the buffer back at once, so
+          // that the next Q tile is in flight while this one is transformed
           uint32_t pk[kChunksPerHalf * 4];
-          float dot[2] = {0.f, 0.f};
-          const float* za_base = zin[ip];
-          const float* zb_base = zcum[ip][j];
 #pragma unroll
           for (int g = 0; g < kChunksPerHalf; ++g) {
             const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
             const int box = gl >> 3, cin = gl & 7;
             const uint4 rawv =
                 *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
-            const uint32_t w4[4] = {rawv.x, rawv.y, rawv.z, rawv.w};
-            const float4 a0 = *reinterpret_cast<const float4*>(za_base + gl * 8);
-            const float4 a1 = *reinterpret_cast<const float4*>(za_base + gl * 8 + 4);
-            const float4 b0 = *reinterpret_cast<const float4*>(zb_base + gl * 8);
-            const float4 b1 = *reinterpret_cast<const float4*>(zb_base + gl * 8 + 4);
-            const float zvv[8] = {a0.x + b0.x, a0.y + b0.y, a0.z + b0.z, a0.w + b0.w,
-                                  a1.x + b1.x, a1.y + b1.y, a1.z + b1.z, a1.w + b1.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const uint32_t pkv = phi_bf16x2(w4[e]);
-              pk[g * 4 + e] = pkv;
-              // the dot product uses the rounded values the tensor core will see
-              dot[e & 1] = fmaf(bf16_lo(pkv), zvv[2 * e], dot[e & 1]);
-              dot[e & 1] = fmaf(bf16_hi(pkv), zvv[2 * e + 1], dot[e & 1]);
-            }
+            pk[g * 4 + 0] = rawv.x;
+            pk[g * 4 + 1] = rawv.y;
+            pk[g * 4 + 2] = rawv.z;
+            pk[g * 4 + 3] = rawv.w;
           }
-          qz[sq][half][r] = dot[0] + dot[1];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bar.q_land_free);
+#pragma unroll
+          for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
           if constexpr (D == 128) {
             uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
             tmem_st32(tmem + C::tQ + sq * (D / 2) + lane_off + half * 32, pk32);
@@ -791,10 +785,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           tmem_wait_st();
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) {
-            mbar_arrive(&bar.qphi_full[sq]);
-            mbar_arrive(&bar.q_land_free);
-          }
+          if (lane == 0) mbar_arrive(&bar.qphi_full[sq]);
         }
         if (tid == 192) PROF(3, nq, 2);
         ok = !__any_sync(0xffffffffu, !ok);
@@ -853,16 +844,40 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);  // column quarters 2, 3
         ++n_a;
       }
+      ok = ok && wait_epoch(&zin_epoch, (int)n_items + 1, p.status, 415);
       if (named_bar_or(3, 256, !ok)) break;
       // ---- pass C: causal mask inside the chunk, bf16 back into TMEM, partial denominators.
       //      This warp owns rows [32 q, 32 q + 32) x key columns [64 colh, 64 colh + 64).
       for (int j = 0; j < it.nC; ++j) {
         const int sq = nq & 1;
         if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
-        float part = 0.f;
-        if (colh == 0) {
-          part = qz[sq][0][r] + qz[sq][1][r];
-          mbar_arrive(&bar.qz_free[sq]);
+        tc_fence_after_sync();
+        // phi(q_i) . z_{c-1} over this warp's half of the head dimension, from the phi(Q) operand in
+        // TMEM (the rounded values the tensor core sees); z before chunk j = zin + zcum[j]
+        float part;
+        {
+          constexpr int W = D / 4;  // packed words per half row
+          uint32_t qw[W];
+          if constexpr (D == 128) {
+            uint32_t(&q32)[32] = *reinterpret_cast<uint32_t(*)[32]>(qw);
+            tmem_ld32(tmem + C::tQ + sq * (D / 2) + lane_off + colh * 32, q32);
+          } else {
+            tmem_ld16(tmem + C::tQ + sq * (D / 2) + lane_off + colh * 16, qw);
+          }
+          tmem_wait_ld();
+          const float* za = zin[ip] + colh * (D / 2);
+          const float* zb = zcum[ip][j] + colh * (D / 2);
+          float d0 = 0.f, d1 = 0.f;
+#pragma unroll
+          for (int w = 0; w < W; w += 2) {
+            const float4 a = *reinterpret_cast<const float4*>(za + 2 * w);
+            const float4 b = *reinterpret_cast<const float4*>(zb + 2 * w);
+            d0 = fmaf(bf16_lo(qw[w]), a.x + b.x, d0);
+            d1 = fmaf(bf16_hi(qw[w]), a.y + b.y, d1);
+            d0 = fmaf(bf16_lo(qw[w + 1]), a.z + b.z, d0);
+            d1 = fmaf(bf16_hi(qw[w + 1]), a.w + b.w, d1);
+          }
+          part = d0 + d1;
         }
         if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
         if (tt == 0) PROF(2, nq, 0);
@@ -910,6 +925,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       uint32_t nk = 0, nv = 0, nq = 0;
       uint32_t n_kphi[2] = {0, 0}, n_os[2] = {0, 0};
       bool ok = true;
+      const uint64_t pol_keep = l2_policy_evict_last();  // parked phi(K) tiles are read back by pass C
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
         // ---- pass A: park phi(K) tiles in the output rows of their chunk
@@ -918,9 +934,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (!mbar_wait(&bar.kphi_full[sk], n_kphi[sk] & 1, p.status, 520)) { ok = false; break; }
           ++n_kphi[sk];
           for (int x = 0; x < D / 64; ++x)
-            tma_store_4d(&mo, sK + sk * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b);
+            tma_store_4d_hint(&mo, sK + sk * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b,
+                              pol_keep);
           tma_store_commit();
           tma_store_wait_read<0>();
+          PROF(0, nk - nq, 3);
           mbar_arrive(&bar.k_free[sk]);
           ++nk;
         }
