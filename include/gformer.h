@@ -119,8 +119,8 @@ int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void
 /*
  * The hybrid layer (Sec. III-A): heads [0, h_sparse) as gformer_window_attn, heads
  * [h_sparse, H) as gformer_causal_linear_attn with a zero initial state; h_sparse < 0
- * selects gformer_default_h_sparse(H).  Both groups are enqueued so that they overlap on
- * the device.
+ * selects gformer_default_h_sparse(H).  The two groups overlap on the device when the
+ * linear heads alone do not fill it; otherwise they run back to back on `cuda_stream`.
  * state_out (may be NULL): if given, its B, H, d, w, h_sparse, dtype must match the call
  * and its buffers receive the decode state after the N tokens: the last min(N, w) keys
  * and values of the windowed heads in ring slots j mod w, the final S and z of the linear

@@ -226,7 +226,17 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
 
   float* S_out = state_out ? state_out->S : nullptr;
   float* z_out = state_out ? state_out->z : nullptr;
-  const bool both = h_sparse > 0 && h_lin > 0;
+  // The two head groups run side by side on two streams while the persistent linear kernel leaves
+  // SMs free; once it fills the machine (one CTA per SM, whose segment hand-over needs every CTA
+  // resident) the windowed heads follow it on the same stream instead of competing for SMs.
+  bool both = h_sparse > 0 && h_lin > 0;
+  if (both && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
+    int L = 0, G = 0, dev = 0, sms = 0;
+    gf::linear_tc_plan(B * h_lin, N, g_linear_split, &L, &G);
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return GF_ERR_CUDA;
+    if ((long long)B * h_lin * G >= sms) both = false;
+  }
   Fork* f = both ? get_fork() : nullptr;
   if (both && f == nullptr) return GF_ERR_CUDA;
   if (both) {

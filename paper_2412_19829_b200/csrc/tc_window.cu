@@ -26,6 +26,12 @@ constexpr int kThreads = 192;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
+__device__ __forceinline__ float ex2_approx(float x) {  // 2^x, flushes denormals, 2^-inf = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 template <int D>
 struct WinSmem {
   static constexpr int kTile = 128 * D * 2;  // bytes of one 128 x D bf16 tile
@@ -144,30 +150,35 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       const int j0 = (t_first + it) * 128;
       if (!mbar_wait(&s_full, it & 1, p.status, 30)) { ok = false; break; }
       tc_fence_after_sync();
-      uint32_t sreg[4][32];
-#pragma unroll
-      for (int c = 0; c < 4; ++c) tmem_ld32(tS + lane_off + c * 32, sreg[c]);
-      tmem_wait_ld();
-      // valid key columns of this row in this tile: [lo, hi]
+      // valid key columns of this row in this tile: [lo, hi]; of this warp's 32 rows: between
+      // [lo_w, hi_w + 31] (all rows see at least) and [lo_w + 31, hi_w] ... classified per 32-column
+      // block so that fully masked blocks cost nothing and fully visible ones need no per-element test
       int lo = i - p.w + 1 - j0;
-      if (lo < 0) lo = 0;
       int hi = i - j0;
-      if (hi > 127) hi = 127;
-      const bool full = (lo == 0) && (hi == 127);
-      float mt = -INFINITY;
+      const int lo_first = (i0 + quarter * 32) - p.w + 1 - j0;  // lo of the warp's first row (last row: +31)
+      const int hi_first = (i0 + quarter * 32) - j0;            // hi of the warp's first row (last row: +31)
+      // pass 1: row maximum of the raw scores (scale > 0, so it commutes with the maximum)
+      float mraw = -INFINITY;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
+        const int c0 = c * 32, c1 = c * 32 + 31;
+        if (c1 < lo_first || c0 > hi_first + 31) continue;  // masked for every row of the warp
+        uint32_t sr[32];
+        tmem_ld32(tS + lane_off + c0, sr);
+        tmem_wait_ld();
+        const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);  // visible to every row of the warp
+        if (inside) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          float s = __uint_as_float(sreg[c][j]) * p.scale_log2;
-          if (!full) {
-            const int col = c * 32 + j;
-            if (col < lo || col > hi) s = -INFINITY;
+          for (int j = 0; j < 32; ++j) mraw = fmaxf(mraw, __uint_as_float(sr[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int col = c0 + j;
+            if (col >= lo && col <= hi) mraw = fmaxf(mraw, __uint_as_float(sr[j]));
           }
-          sreg[c][j] = __float_as_uint(s);
-          mt = fmaxf(mt, s);
         }
       }
+      const float mt = mraw * p.scale_log2;
       // lazy rescale of what has been accumulated so far
       float alpha = 1.f;
       bool need = false;
@@ -193,17 +204,35 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           tmem_wait_st();
         }
       }
-      const float mref_safe = (m_ref == -INFINITY) ? 0.f : m_ref;
+      // pass 2: p = 2^(s * scale_log2 - m_ref), bf16, back over S (block c of P lands in columns
+      // [16 c, 16 c + 16), which only covers S blocks that have already been consumed)
+      const float neg_mref = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float lsum = 0.f;
 #pragma unroll
       for (int c = 0; c < 4; ++c) {
+        const int c0 = c * 32, c1 = c * 32 + 31;
         uint32_t pk[16];
+        if (c1 < lo_first || c0 > hi_first + 31) {
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          const float p0 = exp2f(__uint_as_float(sreg[c][2 * j]) - mref_safe);
-          const float p1 = exp2f(__uint_as_float(sreg[c][2 * j + 1]) - mref_safe);
-          lsum += p0 + p1;
-          pk[j] = pack_bf16(p0, p1);
+          for (int j = 0; j < 16; ++j) pk[j] = 0u;
+        } else {
+          uint32_t sr[32];
+          tmem_ld32(tS + lane_off + c0, sr);
+          tmem_wait_ld();
+          const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) {
+            float a0 = fmaf(__uint_as_float(sr[2 * j]), p.scale_log2, neg_mref);
+            float a1 = fmaf(__uint_as_float(sr[2 * j + 1]), p.scale_log2, neg_mref);
+            if (!inside) {
+              const int col = c0 + 2 * j;
+              if (col < lo || col > hi) a0 = -INFINITY;
+              if (col + 1 < lo || col + 1 > hi) a1 = -INFINITY;
+            }
+            const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
+            lsum += p0 + p1;
+            pk[j] = pack_bf16(p0, p1);
+          }
         }
         tmem_st16(tS + lane_off + c * 16, pk);
       }
