@@ -117,6 +117,35 @@ int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void
                                int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * gformer_causal_linear_attn for callers that cannot allocate device memory (no counterpart
+ * in the paper; it exists for the deployment, not for the method).
+ *
+ * Who needs it: code that receives tensors and a stream but does not own an allocator --
+ * a plug-in inside a framework whose memory pool holds the whole device, a capture-time or
+ * real-time path in which cudaMalloc and the synchronisation it implies are off limits.  Such
+ * a caller has nowhere to get the `ws` scratch the linear-attention kernel uses for the
+ * states its thread blocks pass from one sequence segment to the next.
+ *
+ * This entry point takes that scratch from a fixed array of gformer_noalloc_scratch_bytes()
+ * = 8 MiB that is part of the library image (each GPU that loads the library keeps it until
+ * the process exits).  It allocates and frees nothing, in CUDA or on the host side of any
+ * framework.  Arguments, results and status codes are those of gformer_causal_linear_attn;
+ * in addition GF_ERR_WORKSPACE is returned, before anything is launched or written, when
+ * gformer_workspace_bytes(B, H, N, d, 1, 0, dtype) exceeds the array (for d = 128 that is
+ * about 120 sequence segments of 1024 tokens in total, e.g. B*H = 4 chains of 8192 tokens).
+ *
+ * The first call on a device looks up the array's device address; make that call once
+ * outside any stream capture.  All calls share the one array: it still holds the previous
+ * call's contents on entry (the kernel clears the words it relies on), and two calls whose
+ * kernels overlap on the GPU -- different streams, or different host threads -- race on it.
+ */
+size_t gformer_noalloc_scratch_bytes(void);
+int gformer_causal_linear_attn_noalloc(const void* q, const void* k, const void* v, void* o,
+                                       int B, int H, int N, int d, int phi, int chunk,
+                                       float* S_io, float* z_io, int dtype, int layout,
+                                       void* cuda_stream);
+
+/*
  * The hybrid layer (Sec. III-A): heads [0, h_sparse) as gformer_window_attn, heads
  * [h_sparse, H) as gformer_causal_linear_attn with a zero initial state; h_sparse < 0
  * selects gformer_default_h_sparse(H).  The two groups overlap on the device when the

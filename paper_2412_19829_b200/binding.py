@@ -61,6 +61,9 @@ def lib() -> ctypes.CDLL:
         L.gformer_window_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp, sz, vp]
         L.gformer_causal_linear_attn.restype = i
         L.gformer_causal_linear_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, vp, i, i, vp, sz, vp]
+        L.gformer_noalloc_scratch_bytes.restype = sz
+        L.gformer_causal_linear_attn_noalloc.restype = i
+        L.gformer_causal_linear_attn_noalloc.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, vp, i, i, vp]
         L.gformer_hybrid_attn.restype = i
         L.gformer_hybrid_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, i, i,
                                           ctypes.POINTER(DecodeStateC), vp, sz, vp]
@@ -192,6 +195,21 @@ def causal_linear_attn(q, k, v, S=None, z=None, chunk: int = 0, layout: int = GF
     if rc != GF_OK:
         raise GformerError(rc, "gformer_causal_linear_attn")
     return o
+
+
+def causal_linear_attn_noalloc(q, k, v, out, S=None, z=None, chunk: int = 0, layout: int = GF_BHND, stream=None):
+    """gformer_causal_linear_attn_noalloc: same result as causal_linear_attn, but the kernel's scratch
+    is the fixed array inside the library, so nothing is allocated here or there.  The caller brings
+    the output tensor; problems whose scratch exceeds the array raise GformerError(GF_ERR_WORKSPACE)."""
+    _check_qkv(q, k, v)
+    B, H, N, d = _dims(q, layout)
+    rc = lib().gformer_causal_linear_attn_noalloc(
+        q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(), B, H, N, d, GF_PHI_ELU1, int(chunk),
+        S.data_ptr() if S is not None else None, z.data_ptr() if z is not None else None,
+        _dtype_code(q), layout, _stream_ptr(stream))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_causal_linear_attn_noalloc")
+    return out
 
 
 class DecodeState:
