@@ -157,28 +157,34 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       int hi = i - j0;
       const int lo_first = (i0 + quarter * 32) - p.w + 1 - j0;  // lo of the warp's first row (last row: +31)
       const int hi_first = (i0 + quarter * 32) - j0;            // hi of the warp's first row (last row: +31)
-      // pass 1: row maximum of the raw scores (scale > 0, so it commutes with the maximum)
-      float mraw = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int c0 = c * 32, c1 = c * 32 + 31;
+      // Two sweeps over the row (maximum, then exponentials), 64 columns per TMEM round trip: the
+      // scores stay in TMEM between the sweeps, so only 64 of them are live in registers at a time.
+      float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+  #pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int c0 = hh * 64, c1 = hh * 64 + 63;
         if (c1 < lo_first || c0 > hi_first + 31) continue;  // masked for every row of the warp
-        uint32_t sr[32];
-        tmem_ld32(tS + lane_off + c0, sr);
+        uint32_t sa[32], sb[32];
+        tmem_ld32(tS + lane_off + c0, sa);
+        tmem_ld32(tS + lane_off + c0 + 32, sb);
         tmem_wait_ld();
         const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);  // visible to every row of the warp
         if (inside) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) mraw = fmaxf(mraw, __uint_as_float(sr[j]));
+  #pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(sa[j]));
+            mx[(j + 2) & 3] = fmaxf(mx[(j + 2) & 3], __uint_as_float(sb[j]));
+          }
         } else {
-#pragma unroll
+  #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const int col = c0 + j;
-            if (col >= lo && col <= hi) mraw = fmaxf(mraw, __uint_as_float(sr[j]));
+            if (col >= lo && col <= hi) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(sa[j]));
+            if (col + 32 >= lo && col + 32 <= hi) mx[(j + 2) & 3] = fmaxf(mx[(j + 2) & 3], __uint_as_float(sb[j]));
           }
         }
       }
-      const float mt = mraw * p.scale_log2;
+      const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;  // scale > 0
       // lazy rescale of what has been accumulated so far
       float alpha = 1.f;
       bool need = false;
@@ -192,50 +198,68 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (__any_sync(0xffffffffu, need)) {
           if (!mbar_wait(&pv_done, (it - 1) & 1, p.status, 31)) { ok = false; break; }
           tc_fence_after_sync();
-#pragma unroll
+  #pragma unroll
           for (int c = 0; c < D / 32; ++c) {
             uint32_t oreg[32];
             tmem_ld32(tO + lane_off + c * 32, oreg);
             tmem_wait_ld();
-#pragma unroll
+  #pragma unroll
             for (int j = 0; j < 32; ++j) oreg[j] = __float_as_uint(__uint_as_float(oreg[j]) * alpha);
             tmem_st32(tO + lane_off + c * 32, oreg);
           }
           tmem_wait_st();
         }
       }
-      // pass 2: p = 2^(s * scale_log2 - m_ref), bf16, back over S (block c of P lands in columns
-      // [16 c, 16 c + 16), which only covers S blocks that have already been consumed)
+      // p = 2^(s * scale_log2 - m_ref), bf16, back over S: the 64 scores of half hh become 32 packed
+      // columns at [32 hh, 32 hh + 32), inside columns this thread has already consumed
       const float neg_mref = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      float lsum = 0.f;
-#pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        const int c0 = c * 32, c1 = c * 32 + 31;
-        uint32_t pk[16];
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+  #pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        const int c0 = hh * 64, c1 = hh * 64 + 63;
+        uint32_t pk[32];
         if (c1 < lo_first || c0 > hi_first + 31) {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) pk[j] = 0u;
+  #pragma unroll
+          for (int j = 0; j < 32; ++j) pk[j] = 0u;
         } else {
-          uint32_t sr[32];
-          tmem_ld32(tS + lane_off + c0, sr);
+          uint32_t sa[32], sb[32];
+          tmem_ld32(tS + lane_off + c0, sa);
+          tmem_ld32(tS + lane_off + c0 + 32, sb);
           tmem_wait_ld();
           const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) {
-            float a0 = fmaf(__uint_as_float(sr[2 * j]), p.scale_log2, neg_mref);
-            float a1 = fmaf(__uint_as_float(sr[2 * j + 1]), p.scale_log2, neg_mref);
-            if (!inside) {
+          if (inside) {  // the common case, kept free of any masking arithmetic
+  #pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const float p0 = ex2_approx(fmaf(__uint_as_float(sa[2 * j]), p.scale_log2, neg_mref));
+              const float p1 = ex2_approx(fmaf(__uint_as_float(sa[2 * j + 1]), p.scale_log2, neg_mref));
+              const float p2 = ex2_approx(fmaf(__uint_as_float(sb[2 * j]), p.scale_log2, neg_mref));
+              const float p3 = ex2_approx(fmaf(__uint_as_float(sb[2 * j + 1]), p.scale_log2, neg_mref));
+              ls[j & 3] += (p0 + p1) + (p2 + p3);
+              pk[j] = pack_bf16(p0, p1);
+              pk[16 + j] = pack_bf16(p2, p3);
+            }
+          } else {
+  #pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              float a0 = fmaf(__uint_as_float(sa[2 * j]), p.scale_log2, neg_mref);
+              float a1 = fmaf(__uint_as_float(sa[2 * j + 1]), p.scale_log2, neg_mref);
+              float b0 = fmaf(__uint_as_float(sb[2 * j]), p.scale_log2, neg_mref);
+              float b1 = fmaf(__uint_as_float(sb[2 * j + 1]), p.scale_log2, neg_mref);
               const int col = c0 + 2 * j;
               if (col < lo || col > hi) a0 = -INFINITY;
               if (col + 1 < lo || col + 1 > hi) a1 = -INFINITY;
+              if (col + 32 < lo || col + 32 > hi) b0 = -INFINITY;
+              if (col + 33 < lo || col + 33 > hi) b1 = -INFINITY;
+              const float p0 = ex2_approx(a0), p1 = ex2_approx(a1), p2 = ex2_approx(b0), p3 = ex2_approx(b1);
+              ls[j & 3] += (p0 + p1) + (p2 + p3);
+              pk[j] = pack_bf16(p0, p1);
+              pk[16 + j] = pack_bf16(p2, p3);
             }
-            const float p0 = ex2_approx(a0), p1 = ex2_approx(a1);
-            lsum += p0 + p1;
-            pk[j] = pack_bf16(p0, p1);
           }
         }
-        tmem_st16(tS + lane_off + c * 16, pk);
+        tmem_st32(tS + lane_off + hh * 32, pk);
       }
+      const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
       l += lsum;
       tmem_wait_st();
       tc_fence_before_sync();
