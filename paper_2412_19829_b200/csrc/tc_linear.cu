@@ -72,7 +72,8 @@ struct LinCfg {
 
 struct LinParams {
   int N, nch, h_begin, h_count, nchains;
-  int L, G, nitems;      // chunks per segment, segments per chain, nchains * G
+  int G, nitems;         // segments per chain, nchains * G
+  int seg_base, seg_rem; // the first seg_rem segments of a chain have seg_base + 1 chunks, the others seg_base
   float* S_io;           // [B, h_count, D, D] or null
   float* z_io;           // [B, h_count, D] or null
   int zero_init;
@@ -93,9 +94,8 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
   it.b = it.chain / p.h_count;
   it.hl = it.chain - it.b * p.h_count;
   it.h = p.h_begin + it.hl;
-  it.c_begin = it.g * p.L;
-  const int c_end = (it.c_begin + p.L < p.nch) ? it.c_begin + p.L : p.nch;
-  it.nC = c_end - it.c_begin;
+  it.c_begin = it.g * p.seg_base + (it.g < p.seg_rem ? it.g : p.seg_rem);
+  it.nC = p.seg_base + (it.g < p.seg_rem ? 1 : 0);
   it.last_seg = (it.g == p.G - 1);
   it.need_dS = !it.last_seg;  // the last segment's contribution is needed by nobody
   return it;
@@ -162,11 +162,21 @@ __device__ __forceinline__ void prof2_stamp(int ev) {
     g_prof2[blockIdx.x][ev] = t;
   }
 }
+__device__ unsigned long long g_prof3[160][8][8];  // per CTA, per item of that CTA: phase time line
+__device__ __forceinline__ void prof3_stamp(unsigned int n_item, int ev) {
+  if (blockIdx.x < 160 && n_item < 8) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    g_prof3[blockIdx.x][n_item][ev] = t;
+  }
+}
 #define PROF(role, c, ev) prof_stamp(role, c, ev)
 #define PROF2(cond, ev) do { if (cond) prof2_stamp(ev); } while (0)
+#define PROF3(n, ev) prof3_stamp(n, ev)
 #else
 #define PROF(role, c, ev)
 #define PROF2(cond, ev)
+#define PROF3(n, ev)
 #endif
 
 // Named barrier over `n` threads that also ORs a predicate, so that a timed-out wait makes the
@@ -394,6 +404,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         const LinItem it = decode_item(p, item);
         for (int pass = 0; pass < 2 && ok; ++pass) {
           if (pass == 1 && !mbar_wait(&bar.park_done, n_items & 1, p.status, 103)) { ok = false; break; }
+          PROF3(n_items, pass);
           for (int j = 0; j < it.nC; ++j) {
             const int n0 = (it.c_begin + j) * 128;
             const int sk = nk & 1;
@@ -437,7 +448,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       uint32_t nk = 0, nv = 0, nq = 0, n_sl = 0, n_sb = 0, n_of = 0, n_pm = 0;
       uint32_t n_kphi[2] = {0, 0}, n_kc[2] = {0, 0};
       bool ok = true, first_item = true;
-      for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
+      [[maybe_unused]] uint32_t n_items = 0;
+      for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x, ++n_items) {
         const LinItem it = decode_item(p, item);
         if (!first_item) {
           // the previous item's last S conversion has read TMEM and written Sb: consume its phases
@@ -485,6 +497,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           }
           ++n_kc[sk];
           PROF(1, nq, 0);
+          if (j == 0) PROF3(n_items, 4);
           tc_fence_after_sync();
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
@@ -923,6 +936,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     // ================================================================ TMA store warp
     if (elect_one()) {
       uint32_t nk = 0, nv = 0, nq = 0;
+      [[maybe_unused]] uint32_t n_items = 0;
       uint32_t n_kphi[2] = {0, 0}, n_os[2] = {0, 0};
       bool ok = true;
       const uint64_t pol_keep = l2_policy_evict_last();  // parked phi(K) tiles are read back by pass C
@@ -960,6 +974,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           ++nv;
           ++nq;
         }
+        PROF3(n_items, 5);
+        ++n_items;
       }
       tma_store_wait_all<0>();
       PROF2(true, 7);
@@ -976,6 +992,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (it.g > 0 && !wait_flag(p.flags + (slot - 1) * kFlagStride, p.status, 511)) break;
         __threadfence_block();
         *reinterpret_cast<volatile int*>(&prev_epoch) = n_items + 1;
+        PROF3(n_items, 2);
         if (it.need_dS) {
           // every warp of the hand-over has written its part of the inclusive state
           if (!mbar_wait(&bar.pub_done, n_a & 1, p.status, 510)) break;
@@ -983,6 +1000,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           ++n_a;
           const unsigned int one = 1u;
           asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.flags + slot * kFlagStride), "r"(one) : "memory");
+          PROF3(n_items, 3);
         }
       }
     }
@@ -998,6 +1016,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 extern "C" int gformer_debug_read_profile2(unsigned long long* host_dst) {
   return (int)cudaMemcpyFromSymbol(host_dst, g_prof2, sizeof(g_prof2));
 }
+extern "C" int gformer_debug_read_profile3(unsigned long long* host_dst) {
+  return (int)cudaMemcpyFromSymbol(host_dst, g_prof3, sizeof(g_prof3));
+}
 extern "C" int gformer_debug_read_profile(unsigned long long* host_dst) {
   return (int)cudaMemcpyFromSymbol(host_dst, g_prof, sizeof(g_prof));
 }
@@ -1008,22 +1029,37 @@ bool tc_linear_supported(int N, int d, int dtype) {
   return dtype == GF_BF16 && (d == 64 || d == 128);
 }
 
-// Segmentation of the chains: chunks per segment L and segments per chain G.
+// Segmentation of the chains: G segments per chain, their lengths differing by one chunk at most
+// (the longest has *L_out chunks).  CTAs take items round-robin, so the kernel lasts about
+// ceil(items / CTAs) rounds of one item each: among the segment counts that keep segments between
+// 4 and kMaxL chunks, take the one with the least rounds x (chunks per item + the fixed cost of a
+// hand-over, about 0.7 chunk).  The plan must not depend on the device that is current when the
+// workspace size is asked for, so it assumes the 148 SMs of a B200.
 void linear_tc_plan(int nchains, int N, int split, int* L_out, int* G_out) {
   const int nch = (N + 127) / 128;
-  int L;
+  int G;
   if (split > 0) {
-    L = split;
+    const int L = split > kMaxL ? kMaxL : split;
+    G = (nch + L - 1) / L;
   } else {
-    L = kMaxL;
-    // keep at least ~2 items per SM, but never segments shorter than 4 chunks
-    while (L > 4 && (long long)nchains * ((nch + L - 1) / L) < 296) L -= 1;
+    constexpr int kPlanSMs = 148;
+    const int g_min = (nch + kMaxL - 1) / kMaxL;
+    int g_max = (nch + 3) / 4;
+    if (g_max < g_min) g_max = g_min;
+    G = g_min;
+    double best = 1e300;
+    for (int g = g_min; g <= g_max; ++g) {
+      const long long rounds = ((long long)nchains * g + kPlanSMs - 1) / kPlanSMs;
+      const double cost = (double)rounds * ((double)nch / g + 0.7);
+      if (cost < best * (1.0 - 1e-9)) {
+        best = cost;
+        G = g;
+      }
+    }
   }
-  if (L > kMaxL) L = kMaxL;
-  if (L > nch) L = nch;
-  if (L < 1) L = 1;
-  *L_out = L;
-  *G_out = (nch + L - 1) / L;
+  if (G < 1) G = 1;
+  *G_out = G;
+  *L_out = (nch + G - 1) / G;
 }
 
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
@@ -1047,7 +1083,10 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   p.h_begin = h_begin;
   p.h_count = h_count;
   p.nchains = B * h_count;
-  linear_tc_plan(p.nchains, N, split, &p.L, &p.G);
+  int L_max = 0;
+  linear_tc_plan(p.nchains, N, split, &L_max, &p.G);
+  p.seg_base = p.nch / p.G;
+  p.seg_rem = p.nch % p.G;
   p.nitems = p.nchains * p.G;
   p.S_io = S_io;
   p.z_io = z_io;
