@@ -212,8 +212,8 @@ __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 // phi on rows {lane16 + 16 k8 : k8 in [k8_begin, k8_begin + 4)} x one 16-byte column chunk of a K
-// tile, in place, plus the column sums of those rows reduced over the 16 lanes that share the
-// column chunk (result valid in the lane with lane16 == 0).  Rows at or past n_valid become 0.
+// tile, in place, plus this thread's share of the column sums of those rows (to be reduced over
+// the 16 lanes that share the column chunk).  Rows at or past n_valid become 0.
 __device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane16, int k8_begin, int n_valid,
                                                  float (&cs)[8]) {
 #pragma unroll
@@ -243,6 +243,10 @@ __device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane1
     *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k];
   }
   fence_proxy_async_smem();
+}
+
+// Column sums of transform_k_rows reduced over the 16 lanes that share a column chunk.
+__device__ __forceinline__ void reduce_column_sums(float (&cs)[8]) {
 #pragma unroll
   for (int e = 0; e < 8; ++e) {
 #pragma unroll
@@ -714,222 +718,190 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       if (!ok) break;
       ++n_items;
     }
-  } else if (warp < 14) {
-    // ================================================================ phi(Q) group (8 warps)
-    const int quarter = warp & 3;         // TMEM lane quarter of this warp
-    const int half = (warp - 6) >> 2;     // which half of the head dimension this warp handles
-    const int r = quarter * 32 + lane;    // Q row
+  } else if (warp < 22) {
+    // ================================================================ phi warps: Q group (warps 6-13), K group (14-21)
+    // Pass A and the hand-over of S are common to the two groups (one copy of the code); in pass
+    // C the Q group applies phi to Q and the K group masks P.
+    const bool kgrp = warp >= 14;
+    const int tt = kgrp ? tid - 14 * 32 : tid - 6 * 32;  // 0..255 within the group
+    const int quarter = warp & 3;                        // TMEM lane quarter of this warp
+    const int half = ((warp - 6) >> 2) & 1;  // Q group: half of the head dimension; K group: half of the key columns
+    const int colh = half;
+    const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per thread
+    constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per Q-group thread
     uint32_t nq = 0, nk = 0, n_a = 0, n_items = 0;
     uint32_t n_ka[2] = {0, 0};
     int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
-      na += it.nC;
-      // ---- pass A: rows 64..127 (by sixteens) of every K tile
-      {
-        const int tt = tid - 6 * 32;
-        for (int j = 0; j < it.nC; ++j) {
-          const int sk = nk & 1;
-          ok = ok && mbar_wait(&bar.ka_full[sk], n_ka[sk] & 1, p.status, 420);
-          ++n_ka[sk];
-          if (ok && tt < 2 * D) {
-            const int cc = tt >> 4;
-            float cs[8];
-            transform_k_rows(sK + sk * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, 4,
-                             p.N - (it.c_begin + j) * 128, cs);
-            if ((tt & 15) == 0) {
-#pragma unroll
-              for (int e = 0; e < 8; ++e) zpart[j & 1][1][cc * 8 + e] = cs[e];
-            }
-          }
-          __syncwarp();
-          if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);
-          if (named_bar_or(4, 512, !ok)) { ok = false; break; }
-          ++nk;
-        }
-        if (!ok) break;
-        nk += it.nC;
-      }
-      if (it.need_dS) {
-        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);
-        ++n_a;
-        ok = !__any_sync(0xffffffffu, !ok);
-        if (!ok) break;
-      }
-      for (int j = 0; j < it.nC && ok; ++j) {
-        const int sq = nq & 1;
-        ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
-        if (tid == 192) PROF(3, nq, 0);
-        if (ok && nq >= 2) {
-          const uint32_t par = ((nq >> 1) + 1) & 1;
-          ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // MMA1/MMA2 of two chunks ago are done with it
-               mbar_wait(&bar.den_full[sq], par, p.status, 402);     // ... and so is the K group's dot product
-        }
-        if (tid == 192) PROF(3, nq, 1);
-        tc_fence_after_sync();
-        if (ok) {
-          // copy the raw row half out of the landing buffer and hand the buffer back at once, so
-          // that the next Q tile is in flight while this one is transformed
-          uint32_t pk[kChunksPerHalf * 4];
-#pragma unroll
-          for (int g = 0; g < kChunksPerHalf; ++g) {
-            const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
-            const int box = gl >> 3, cin = gl & 7;
-            const uint4 rawv =
-                *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
-            pk[g * 4 + 0] = rawv.x;
-            pk[g * 4 + 1] = rawv.y;
-            pk[g * 4 + 2] = rawv.z;
-            pk[g * 4 + 3] = rawv.w;
-          }
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bar.q_land_free);
-#pragma unroll
-          for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
-          if constexpr (D == 128) {
-            uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
-            tmem_st32(tmem + C::tQ + sq * (D / 2) + lane_off + half * 32, pk32);
-          } else {
-            tmem_st16(tmem + C::tQ + sq * (D / 2) + lane_off + half * 16, pk);
-          }
-          tmem_wait_st();
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bar.qphi_full[sq]);
-        }
-        if (tid == 192) PROF(3, nq, 2);
-        ok = !__any_sync(0xffffffffu, !ok);
-        ++nq;
-      }
-      ++n_items;
-    }
-  } else if (warp < 22) {
-    // ================================================================ K group (8 warps)
-    const int tt = tid - 14 * 32;         // 0..255
-    const int quarter = warp & 3;         // TMEM lane quarter of this warp
-    const int colh = (warp - 14) >> 2;    // which half of the columns this warp handles in pass C
-    const int r = quarter * 32 + lane;
-    const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    uint32_t nk = 0, nq = 0, n_a = 0, n_items = 0;
-    uint32_t n_ka[2] = {0, 0};
-    int na = 0;
-    bool ok = true;
-    for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
-      const LinItem it = decode_item(p, item);
       const int ip = n_items & 1;
-      if (tt < D) zcum[ip][0][tt] = 0.f;
-      // ---- pass A: rows 0..63 (by sixteens) of every K tile, cumulative column sums
+      if (kgrp && tt < D) zcum[ip][0][tt] = 0.f;
+      // ---- pass A: the K group takes rows 0..63 (by sixteens) of every K tile, the Q group rows
+      //      64..127; the K group also keeps the cumulative column sums
       for (int j = 0; j < it.nC; ++j) {
         const int sk = nk & 1;
         ok = ok && mbar_wait(&bar.ka_full[sk], n_ka[sk] & 1, p.status, 410);
         ++n_ka[sk];
-        if (tt == 0) PROF(3, na, 4);
-        if (ok && tt < 2 * D) {
-          const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
-          float cs[8];
-          transform_k_rows(sK + sk * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, 0,
+        if (tid == 14 * 32) PROF(3, na, 4);
+        const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
+        float cs[8];
+        if (ok && tt < 2 * D)
+          transform_k_rows(sK + sk * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
                            p.N - (it.c_begin + j) * 128, cs);
+        __syncwarp();
+        if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);  // the tile may go to the tensor core and be parked
+        if (tid == 14 * 32) PROF(3, na, 5);
+        if (ok && tt < 2 * D) {
+          reduce_column_sums(cs);
           if ((tt & 15) == 0) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) zpart[j & 1][0][cc * 8 + e] = cs[e];
+            for (int e = 0; e < 8; ++e) zpart[j & 1][kgrp ? 0 : 1][cc * 8 + e] = cs[e];
           }
         }
-        __syncwarp();
-        if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);
-        if (tt == 0) PROF(3, na, 5);
         if (named_bar_or(4, 512, !ok)) { ok = false; break; }  // both halves of the tile are done
-        if (tt < D) zcum[ip][j + 1][tt] = zcum[ip][j][tt] + (zpart[j & 1][0][tt] + zpart[j & 1][1][tt]);
-        if (named_bar_or(3, 256, false)) { ok = false; break; }
-        ++na;
-        if (tt == 0) {
-          __threadfence_block();
-          *reinterpret_cast<volatile int*>(&ka_epoch) = na;
+        if (kgrp) {
+          if (tt < D) zcum[ip][j + 1][tt] = zcum[ip][j][tt] + (zpart[j & 1][0][tt] + zpart[j & 1][1][tt]);
+          if (named_bar_or(3, 256, false)) { ok = false; break; }
+          ++na;
+          if (tt == 0) {
+            __threadfence_block();
+            *reinterpret_cast<volatile int*>(&ka_epoch) = na;
+          }
         }
         ++nk;
       }
       if (!ok) break;
       nk += it.nC;  // the K ring also carries the pass-C tiles
-      // ---- hand-over of S: publish the inclusive state together with the Q group
+      // ---- hand-over of S: the two groups publish the inclusive state (column quarters 0, 1 / 2, 3)
       if (it.need_dS) {
-        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);  // column quarters 2, 3
+        ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);
         ++n_a;
       }
-      ok = ok && wait_epoch(&zin_epoch, (int)n_items + 1, p.status, 415);
-      if (named_bar_or(3, 256, !ok)) break;
-      // ---- pass C: causal mask inside the chunk, bf16 back into TMEM, partial denominators.
-      //      This warp owns rows [32 q, 32 q + 32) x key columns [64 colh, 64 colh + 64).
-      for (int j = 0; j < it.nC; ++j) {
-        const int sq = nq & 1;
-        if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
-        tc_fence_after_sync();
-        // phi(q_i) . z_{c-1} over this warp's half of the head dimension, from the phi(Q) operand in
-        // TMEM (the rounded values the tensor core sees); z before chunk j = zin + zcum[j]
-        float part;
-        {
-          constexpr int W = D / 4;  // packed words per half row
-          uint32_t qw[W];
-          if constexpr (D == 128) {
-            uint32_t(&q32)[32] = *reinterpret_cast<uint32_t(*)[32]>(qw);
-            tmem_ld32(tmem + C::tQ + sq * (D / 2) + lane_off + colh * 32, q32);
-          } else {
-            tmem_ld16(tmem + C::tQ + sq * (D / 2) + lane_off + colh * 16, qw);
-          }
-          tmem_wait_ld();
-          const float* za = zin[ip] + colh * (D / 2);
-          const float* zb = zcum[ip][j] + colh * (D / 2);
-          float d0 = 0.f, d1 = 0.f;
-#pragma unroll
-          for (int w = 0; w < W; w += 2) {
-            const float4 a = *reinterpret_cast<const float4*>(za + 2 * w);
-            const float4 b = *reinterpret_cast<const float4*>(zb + 2 * w);
-            d0 = fmaf(bf16_lo(qw[w]), a.x + b.x, d0);
-            d1 = fmaf(bf16_hi(qw[w]), a.y + b.y, d1);
-            d0 = fmaf(bf16_lo(qw[w + 1]), a.z + b.z, d0);
-            d1 = fmaf(bf16_hi(qw[w + 1]), a.w + b.w, d1);
-          }
-          part = d0 + d1;
-        }
-        if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
-        if (tt == 0) PROF(2, nq, 0);
-        tc_fence_after_sync();
-#pragma unroll
-        for (int e = 0; e < 2; ++e) {
-          // 32-column block cc: all kept left of the diagonal block, all dropped right of it,
-          // triangular on it (warp-uniform choice)
-          const int cc = 2 * colh + e;
-          uint32_t pk[16];
-          if (cc > quarter) {
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
-          } else {
-            uint32_t v[32];
-            tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
-            tmem_wait_ld();
-            const bool diag = (cc == quarter);
-#pragma unroll
-            for (int jj = 0; jj < 16; ++jj) {
-              const float p0 = (!diag || 2 * jj <= lane) ? __uint_as_float(v[2 * jj]) : 0.f;
-              const float p1 = (!diag || 2 * jj + 1 <= lane) ? __uint_as_float(v[2 * jj + 1]) : 0.f;
-              part += p0 + p1;
-              pk[jj] = pack_bf16(p0, p1);
+      if (kgrp) {
+        ok = ok && wait_epoch(&zin_epoch, (int)n_items + 1, p.status, 415);
+        if (named_bar_or(3, 256, !ok)) break;
+        // ---- pass C: causal mask inside the chunk, bf16 back into TMEM, partial denominators.
+        //      This warp owns rows [32 q, 32 q + 32) x key columns [64 colh, 64 colh + 64).
+        for (int j = 0; j < it.nC; ++j) {
+          const int sq = nq & 1;
+          if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
+          tc_fence_after_sync();
+          // phi(q_i) . z_{c-1} over this warp's half of the head dimension, from the phi(Q) operand in
+          // TMEM (the rounded values the tensor core sees); z before chunk j = zin + zcum[j]
+          float part;
+          {
+            constexpr int W = D / 4;  // packed words per half row
+            uint32_t qw[W];
+            if constexpr (D == 128) {
+              uint32_t(&q32)[32] = *reinterpret_cast<uint32_t(*)[32]>(qw);
+              tmem_ld32(tmem + C::tQ + sq * (D / 2) + lane_off + colh * 32, q32);
+            } else {
+              tmem_ld16(tmem + C::tQ + sq * (D / 2) + lane_off + colh * 16, qw);
             }
+            tmem_wait_ld();
+            const float* za = zin[ip] + colh * (D / 2);
+            const float* zb = zcum[ip][j] + colh * (D / 2);
+            float d0 = 0.f, d1 = 0.f;
+  #pragma unroll
+            for (int w = 0; w < W; w += 2) {
+              const float4 a = *reinterpret_cast<const float4*>(za + 2 * w);
+              const float4 b = *reinterpret_cast<const float4*>(zb + 2 * w);
+              d0 = fmaf(bf16_lo(qw[w]), a.x + b.x, d0);
+              d1 = fmaf(bf16_hi(qw[w]), a.y + b.y, d1);
+              d0 = fmaf(bf16_lo(qw[w + 1]), a.z + b.z, d0);
+              d1 = fmaf(bf16_hi(qw[w + 1]), a.w + b.w, d1);
+            }
+            part = d0 + d1;
           }
-          // packed P stays inside this warp's own fp32 columns (keys 64h..64h+63 -> columns 64h..64h+31),
-          // so the two warps of a lane quarter never touch each other's unread input
-          tmem_st16(tmem + C::tP + lane_off + colh * 64 + e * 16, pk);
+          if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
+          if (tt == 0) PROF(2, nq, 0);
+          tc_fence_after_sync();
+  #pragma unroll
+          for (int e = 0; e < 2; ++e) {
+            // 32-column block cc: all kept left of the diagonal block, all dropped right of it,
+            // triangular on it (warp-uniform choice)
+            const int cc = 2 * colh + e;
+            uint32_t pk[16];
+            if (cc > quarter) {
+  #pragma unroll
+              for (int jj = 0; jj < 16; ++jj) pk[jj] = 0u;
+            } else {
+              uint32_t v[32];
+              tmem_ld32(tmem + C::tP + lane_off + cc * 32, v);
+              tmem_wait_ld();
+              const bool diag = (cc == quarter);
+  #pragma unroll
+              for (int jj = 0; jj < 16; ++jj) {
+                const float p0 = (!diag || 2 * jj <= lane) ? __uint_as_float(v[2 * jj]) : 0.f;
+                const float p1 = (!diag || 2 * jj + 1 <= lane) ? __uint_as_float(v[2 * jj + 1]) : 0.f;
+                part += p0 + p1;
+                pk[jj] = pack_bf16(p0, p1);
+              }
+            }
+            // packed P stays inside this warp's own fp32 columns (keys 64h..64h+63 -> columns 64h..64h+31),
+            // so the two warps of a lane quarter never touch each other's unread input
+            tmem_st16(tmem + C::tP + lane_off + colh * 64 + e * 16, pk);
+          }
+          den_s[sq][colh][r] = part;
+          mbar_arrive(&bar.den_full[sq]);
+          tmem_wait_st();
+          tc_fence_before_sync();
+          mbar_arrive(&bar.pm_full);
+          if (tt == 0) PROF(2, nq, 1);
+          ++nq;
         }
-        den_s[sq][colh][r] = part;
-        mbar_arrive(&bar.den_full[sq]);
-        tmem_wait_st();
-        tc_fence_before_sync();
-        mbar_arrive(&bar.pm_full);
-        if (tt == 0) PROF(2, nq, 1);
-        ++nq;
+        if (!ok) break;
+      } else {
+        ok = !__any_sync(0xffffffffu, !ok);
+        if (!ok) break;
+        for (int j = 0; j < it.nC && ok; ++j) {
+          const int sq = nq & 1;
+          ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
+          if (tid == 192) PROF(3, nq, 0);
+          if (ok && nq >= 2) {
+            const uint32_t par = ((nq >> 1) + 1) & 1;
+            ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // MMA1/MMA2 of two chunks ago are done with it
+                 mbar_wait(&bar.den_full[sq], par, p.status, 402);     // ... and so is the K group's dot product
+          }
+          if (tid == 192) PROF(3, nq, 1);
+          tc_fence_after_sync();
+          if (ok) {
+            // copy the raw row half out of the landing buffer and hand the buffer back at once, so
+            // that the next Q tile is in flight while this one is transformed
+            uint32_t pk[kChunksPerHalf * 4];
+  #pragma unroll
+            for (int g = 0; g < kChunksPerHalf; ++g) {
+              const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
+              const int box = gl >> 3, cin = gl & 7;
+              const uint4 rawv =
+                  *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
+              pk[g * 4 + 0] = rawv.x;
+              pk[g * 4 + 1] = rawv.y;
+              pk[g * 4 + 2] = rawv.z;
+              pk[g * 4 + 3] = rawv.w;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar.q_land_free);
+  #pragma unroll
+            for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
+            if constexpr (D == 128) {
+              uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
+              tmem_st32(tmem + C::tQ + sq * (D / 2) + lane_off + half * 32, pk32);
+            } else {
+              tmem_st16(tmem + C::tQ + sq * (D / 2) + lane_off + half * 16, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bar.qphi_full[sq]);
+          }
+          if (tid == 192) PROF(3, nq, 2);
+          ok = !__any_sync(0xffffffffu, !ok);
+          ++nq;
+        }
       }
-      if (!ok) break;
       ++n_items;
     }
   } else if (warp == 22) {
