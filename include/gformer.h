@@ -51,7 +51,10 @@ typedef enum { GF_PHI_ELU1 = 0 } gf_phi;
 /* Process-wide knobs for tests and benchmarks (gformer_set_tuning). */
 typedef enum {
   GF_TUNE_FORCE_SIMT = 0, /* 1: never take the tensor-core kernels (default 0)              */
-  GF_TUNE_LINEAR_SPLIT = 1 /* 128-row chunks per sequence segment of a linear chain: 0 = auto    */
+  GF_TUNE_LINEAR_SPLIT = 1, /* 128-row chunks per sequence segment of a linear chain: 0 = auto   */
+  GF_TUNE_LINEAR_CTAS = 2   /* gformer_hybrid_attn: CTAs of the persistent linear-attention kernel
+                               when it shares the GPU with the windowed heads; 0 = auto, else an
+                               upper bound in [1, 65535] (the SM count bounds it too)              */
 } gf_tuning_key;
 
 /* Decode-time state of one batch (see gformer_decode_step).  The struct lives in host

@@ -15,7 +15,7 @@ GF_OK, GF_ERR_INVALID_ARG, GF_ERR_UNSUPPORTED, GF_ERR_WORKSPACE, GF_ERR_CUDA, GF
 GF_F32, GF_BF16 = 0, 1
 GF_BHND, GF_BNHD = 0, 1
 GF_PHI_ELU1 = 0
-GF_TUNE_FORCE_SIMT, GF_TUNE_LINEAR_SPLIT = 0, 1
+GF_TUNE_FORCE_SIMT, GF_TUNE_LINEAR_SPLIT, GF_TUNE_LINEAR_CTAS = 0, 1, 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgformer.so")

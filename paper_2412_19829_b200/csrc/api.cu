@@ -19,11 +19,12 @@ using gf::WsHeader;
 
 int g_force_simt = 0;
 int g_linear_split = 0;
+int g_linear_ctas = 0;
 
 constexpr int kMaxDevices = 64;
 struct Fork {
-  cudaStream_t side = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaStream_t side = nullptr, first = nullptr;  // lowest / highest stream priority
+  cudaEvent_t fork = nullptr, join = nullptr, join_first = nullptr;
   bool ready = false;
 };
 Fork g_fork[kMaxDevices];
@@ -37,7 +38,13 @@ Fork* get_fork() {
   std::lock_guard<std::mutex> lock(g_fork_mutex);
   Fork& f = g_fork[dev];
   if (!f.ready) {
-    if (cudaStreamCreateWithFlags(&f.side, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    // lowest priority: where the two kernels compete for an SM, the persistent linear kernel
+    // (whose CTAs wait for one another) is placed first
+    int prio_least = 0, prio_greatest = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&f.side, cudaStreamNonBlocking, prio_least) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithPriority(&f.first, cudaStreamNonBlocking, prio_greatest) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&f.join_first, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&f.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&f.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     f.ready = true;
@@ -90,12 +97,12 @@ int run_window(const void* q, const void* k, const void* v, void* o, int B, int 
 }
 
 int run_linear(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
-               int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init, WsHeader* ws,
-               cudaStream_t stream) {
+               int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init, int max_ctas,
+               WsHeader* ws, cudaStream_t stream) {
   if (h_count <= 0) return GF_OK;
   if (!g_force_simt && gf::tc_linear_supported(N, d, dtype))
     return cuda_status(gf::launch_linear_tc(q, k, v, o, B, H, N, d, layout, h_begin, h_count, S_io, z_io,
-                                            zero_init, g_linear_split, ws, stream));
+                                            zero_init, g_linear_split, max_ctas, ws, stream));
   return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d),
                                             h_begin, h_count, S_io, z_io, zero_init, stream));
 }
@@ -140,6 +147,10 @@ int gformer_set_tuning(int key, int value) {
     case GF_TUNE_LINEAR_SPLIT:
       if (value < 0 || value > 4096) return GF_ERR_INVALID_ARG;
       g_linear_split = value;
+      return GF_OK;
+    case GF_TUNE_LINEAR_CTAS:
+      if (value < 0 || value > 65535) return GF_ERR_INVALID_ARG;
+      g_linear_ctas = value;
       return GF_OK;
     default:
       return GF_ERR_INVALID_ARG;
@@ -195,7 +206,7 @@ int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   rc = clear_ws(ws, stream);
   if (rc != GF_OK) return rc;
-  return run_linear(q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, (WsHeader*)ws, stream);
+  return run_linear(q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, 0, (WsHeader*)ws, stream);
 }
 
 int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
@@ -226,16 +237,21 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
 
   float* S_out = state_out ? state_out->S : nullptr;
   float* z_out = state_out ? state_out->z : nullptr;
-  // The two head groups run side by side on two streams while the persistent linear kernel leaves
-  // SMs free; once it fills the machine (one CTA per SM, whose segment hand-over needs every CTA
-  // resident) the windowed heads follow it on the same stream instead of competing for SMs.
-  bool both = h_sparse > 0 && h_lin > 0;
+  // The two head groups run side by side on two streams.  The persistent linear kernel holds one
+  // CTA per SM it uses.  When it has work for every SM it still takes them all (measured on a
+  // B200, leaving some to the windowed heads from the start was no faster and less steady), on a
+  // stream of the highest priority; the windowed heads' short-lived CTAs then fill the SMs that
+  // linear CTAs leave at different times towards the end.
+  const bool both = h_sparse > 0 && h_lin > 0;
+  int lin_ctas = 0;
   if (both && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
     int L = 0, G = 0, dev = 0, sms = 0;
-    gf::linear_tc_plan(B * h_lin, N, g_linear_split, &L, &G);
+    gf::linear_tc_plan(B * h_lin, N, g_linear_split, 0, &L, &G);
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return GF_ERR_CUDA;
-    if ((long long)B * h_lin * G >= sms) both = false;
+    if ((long long)B * h_lin * G >= sms) {
+      lin_ctas = (g_linear_ctas > 0 && g_linear_ctas < sms) ? g_linear_ctas : sms;
+    }
   }
   Fork* f = both ? get_fork() : nullptr;
   if (both && f == nullptr) return GF_ERR_CUDA;
@@ -245,8 +261,16 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
     if (cudaEventRecord(f->fork, stream) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(f->side, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
   }
-  rc = run_linear(q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, (WsHeader*)ws,
-                  stream);
+  // When the two kernels compete for SMs the linear one goes to a stream of the highest priority
+  // (the caller's stream may well have the lowest, like the side stream).
+  const bool lin_first = both && lin_ctas > 0;
+  if (lin_first && cudaStreamWaitEvent(f->first, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
+  rc = run_linear(q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, lin_ctas,
+                  (WsHeader*)ws, lin_first ? f->first : stream);
+  if (lin_first) {
+    if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
+    if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
+  }
   cudaStream_t wstream = both ? f->side : stream;
   int rc2 = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, wstream);
   if (rc2 == GF_OK && state_out && h_sparse > 0)

@@ -62,13 +62,14 @@ bool tc_linear_supported(int N, int d, int dtype);
 cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int w, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
                              cudaStream_t stream);
-// Segmentation used by the tensor-core linear kernel (split: 0 = automatic, else chunks per segment)
-// and the scratch it needs beyond the workspace header.
-void linear_tc_plan(int nchains, int N, int split, int* chunks_per_segment, int* segments_per_chain);
+// Segmentation used by the tensor-core linear kernel (split: 0 = automatic, else chunks per segment;
+// ctas: CTAs the kernel will run with, 0 = one per SM of a B200) and the scratch it needs beyond
+// the workspace header (sized for the largest segment count the plan may pick for any ctas).
+void linear_tc_plan(int nchains, int N, int split, int ctas, int* chunks_per_segment, int* segments_per_chain);
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split);
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                             int split, WsHeader* ws, cudaStream_t stream);
+                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream);
 
 // ---- device helpers
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -1006,18 +1006,34 @@ bool tc_linear_supported(int N, int d, int dtype) {
 // ceil(items / CTAs) rounds of one item each: among the segment counts that keep segments between
 // 4 and kMaxL chunks, take the one with the least rounds x (chunks per item + the fixed cost of a
 // hand-over, about 0.7 chunk).  The plan must not depend on the device that is current when the
-// workspace size is asked for, so it assumes the 148 SMs of a B200.
-void linear_tc_plan(int nchains, int N, int split, int* L_out, int* G_out) {
+// workspace size is asked for, so without a CTA count it assumes the 148 SMs of a B200.
+namespace {
+// Range of segment counts the automatic plan chooses from.
+void plan_range(int nchains, int nch, int* g_min_out, int* g_max_out) {
+  const int g_min = (nch + kMaxL - 1) / kMaxL;
+  int g_max = (nch + 3) / 4;
+  // long chains in numbers: stay within a quarter more segments than the minimum (the scratch
+  // grows with the segment count); few chains: as many segments as it takes to fill the GPU
+  int cap = (5 * g_min + 3) / 4;
+  const int fill = (296 + nchains - 1) / nchains;
+  if (cap < fill) cap = fill;
+  if (g_max > cap) g_max = cap;
+  if (g_max < g_min) g_max = g_min;
+  *g_min_out = g_min;
+  *g_max_out = g_max;
+}
+}  // namespace
+
+void linear_tc_plan(int nchains, int N, int split, int ctas, int* L_out, int* G_out) {
   const int nch = (N + 127) / 128;
   int G;
   if (split > 0) {
     const int L = split > kMaxL ? kMaxL : split;
     G = (nch + L - 1) / L;
   } else {
-    constexpr int kPlanSMs = 148;
-    const int g_min = (nch + kMaxL - 1) / kMaxL;
-    int g_max = (nch + 3) / 4;
-    if (g_max < g_min) g_max = g_min;
+    const int kPlanSMs = ctas > 0 ? ctas : 148;
+    int g_min, g_max;
+    plan_range(nchains, nch, &g_min, &g_max);
     G = g_min;
     double best = 1e300;
     for (int g = g_min; g <= g_max; ++g) {
@@ -1036,14 +1052,18 @@ void linear_tc_plan(int nchains, int N, int split, int* L_out, int* G_out) {
 
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
   int L, G;
-  linear_tc_plan(nchains, N, split, &L, &G);
+  linear_tc_plan(nchains, N, split, 0, &L, &G);
+  if (split <= 0) {
+    int g_min;
+    plan_range(nchains, (N + 127) / 128, &g_min, &G);
+  }
   const size_t flags = (size_t)nchains * G * kFlagStride * sizeof(unsigned int);
   return flags + (size_t)nchains * G * ((size_t)128 * d + d) * sizeof(float);
 }
 
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                             int split, WsHeader* ws, cudaStream_t stream) {
+                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream) {
   if (h_count <= 0) return cudaSuccess;
   CUtensorMap mq, mk, mv, mo;
   if (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128) ||
@@ -1055,8 +1075,15 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   p.h_begin = h_begin;
   p.h_count = h_count;
   p.nchains = B * h_count;
+  int dev = 0, sms = 0;
+  cudaError_t e;
+  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  // One CTA per SM at most: every CTA must be resident for the segment hand-over to make progress.
+  // (max_ctas > 0 leaves SMs to a kernel running beside this one.)
+  if (max_ctas > 0 && max_ctas < sms) sms = max_ctas;
   int L_max = 0;
-  linear_tc_plan(p.nchains, N, split, &L_max, &p.G);
+  linear_tc_plan(p.nchains, N, split, sms, &L_max, &p.G);
   p.seg_base = p.nch / p.G;
   p.seg_rem = p.nch % p.G;
   p.nitems = p.nchains * p.G;
@@ -1068,13 +1095,8 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   const size_t flag_bytes = (size_t)p.nchains * p.G * kFlagStride * sizeof(unsigned int);
   p.flags = reinterpret_cast<unsigned int*>(scratch);
   p.prefix = reinterpret_cast<float*>(scratch + flag_bytes);
-  cudaError_t e;
   e = cudaMemsetAsync(p.flags, 0, flag_bytes, stream);
   if (e != cudaSuccess) return e;
-  int dev = 0, sms = 0;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-  // One CTA per SM at most: every CTA must be resident for the segment hand-over to make progress.
   dim3 grid(p.nitems < sms ? p.nitems : sms);
   if (d == 64) {
     auto kern = linear_tc_kernel<64>;

@@ -56,6 +56,21 @@ def test_tuning_rejects_unknown_keys():
     assert L.gformer_set_tuning(99, 1) == gf.GF_ERR_INVALID_ARG
     assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, -1) == gf.GF_ERR_INVALID_ARG
     assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0) == gf.GF_OK
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_CTAS, -1) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_CTAS, 70000) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_CTAS, 0) == gf.GF_OK
+
+
+def test_workspace_covers_every_plan():
+    # the scratch is sized for the largest segment count the plan may choose, whatever CTA count
+    # the launch ends up with: it never shrinks when the chunks-per-segment knob is left on auto
+    auto = gf.workspace_bytes(1, 32, 32768, 128, 512, 6, gf.GF_BF16)
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 8)
+    try:
+        fixed = gf.workspace_bytes(1, 32, 32768, 128, 512, 6, gf.GF_BF16)
+    finally:
+        gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0)
+    assert auto >= fixed
 
 
 FAKE = 0x10000  # a 16-byte-aligned non-null address; validation fails before it is ever used
