@@ -102,7 +102,7 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
 }
 
 struct LinBarriers {
-  uint64_t q_full, q_land_free;
+  uint64_t q_full;
   uint64_t k_full[2], ka_full[2], v_full[2], k_free[2], v_free[2];  // ka_full: K tiles of pass A, k_full: of pass C
   uint64_t qphi_full[2], kphi_full[2], qphi_free[2];
   uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done;
@@ -170,6 +170,34 @@ __device__ __forceinline__ void prof3_stamp(unsigned int n_item, int ev) {
     g_prof3[blockIdx.x][n_item][ev] = t;
   }
 }
+// time spent in every bounded wait, per CTA and wait site (the `where` code), first warp of each role
+__device__ unsigned long long g_wait[160][1024];
+__device__ __forceinline__ void wait_account(unsigned int where, long long t0) {
+  const int w = threadIdx.x >> 5;
+  if ((threadIdx.x & 31) == 0 && ((0x00C04047u >> w) & 1u) && blockIdx.x < 160 && where < 1024)
+    g_wait[blockIdx.x][where] += (unsigned long long)(clock64() - t0);
+}
+__device__ __forceinline__ bool prof_mbar_wait(uint64_t* b, uint32_t par, unsigned int* st, unsigned int where) {
+  const long long t0 = clock64();
+  const bool ok = mbar_wait(b, par, st, where);
+  wait_account(where, t0);
+  return ok;
+}
+__device__ __forceinline__ bool prof_wait_epoch(const int* c, int target, unsigned int* st, unsigned int where) {
+  const long long t0 = clock64();
+  const bool ok = wait_epoch(c, target, st, where);
+  wait_account(where, t0);
+  return ok;
+}
+__device__ __forceinline__ bool prof_wait_flag(const unsigned int* f, unsigned int* st, unsigned int where) {
+  const long long t0 = clock64();
+  const bool ok = wait_flag(f, st, where);
+  wait_account(where, t0);
+  return ok;
+}
+#define mbar_wait prof_mbar_wait
+#define wait_epoch prof_wait_epoch
+#define wait_flag prof_wait_flag
 #define PROF(role, c, ev) prof_stamp(role, c, ev)
 #define PROF2(cond, ev) do { if (cond) prof2_stamp(ev); } while (0)
 #define PROF3(n, ev) prof3_stamp(n, ev)
@@ -340,13 +368,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
   __shared__ int zin_epoch;        // items whose zin is in place (monotonic)
   __shared__ int prev_epoch;       // items whose predecessor state has been seen in global memory (monotonic)
+  __shared__ int q_copied;         // Q-group warps that have copied their part of a Q tile out of the landing buffer (monotonic)
   __shared__ uint32_t tmem_base_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
     mbar_init(&bar.q_full, 1);
-    mbar_init(&bar.q_land_free, 8);
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar.k_full[s], 1);
       mbar_init(&bar.ka_full[s], 1);
@@ -375,6 +403,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     ka_epoch = 0;
     zin_epoch = 0;
     prev_epoch = 0;
+    q_copied = 0;
     mbar_fence_init();
     tma_prefetch_desc(&mq);
     tma_prefetch_desc(&mk);
@@ -420,14 +449,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               tma_load_4d_hint(sK + sk * C::kTile + x * C::kBoxBytes, pass == 0 ? &mk : &mo, kbar, x * 64, n0, it.h, it.b,
                                pol_stream);
             ++nk;
-            if (pass == 1) {
-              if (nq >= 1 && !mbar_wait(&bar.q_land_free, (nq - 1) & 1, p.status, 100)) { ok = false; break; }
-              PROF(0, nq, 0);
-              mbar_arrive_expect_tx(&bar.q_full, C::kTile);
-              for (int x = 0; x < D / 64; ++x)
-                tma_load_4d_hint(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n0, it.h, it.b, pol_stream);
-              ++nq;
-            }
+            if (pass == 1) ++nq;
             if (pass == 1 || it.need_dS) {
               const int sv = nv & 1;
               if (nv >= 2 && !mbar_wait(&bar.v_free[sv], ((nv >> 1) + 1) & 1, p.status, 102)) { ok = false; break; }
@@ -734,6 +756,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     uint32_t n_ka[2] = {0, 0};
     int na = 0;
     bool ok = true;
+    if (tid == 6 * 32 && (int)blockIdx.x < p.nitems) {
+      // the very first Q tile; every later one is requested by the warp that frees the landing buffer
+      const LinItem first = decode_item(p, blockIdx.x);
+      mbar_arrive_expect_tx(&bar.q_full, C::kTile);
+      for (int x = 0; x < D / 64; ++x)
+        tma_load_4d_hint(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, first.c_begin * 128, first.h, first.b,
+                         l2_policy_evict_first());
+    }
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
       const int ip = n_items & 1;
@@ -860,18 +890,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           const int sq = nq & 1;
           ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
           if (tid == 192) PROF(3, nq, 0);
-          if (ok && nq >= 2) {
-            const uint32_t par = ((nq >> 1) + 1) & 1;
-            ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // MMA1/MMA2 of two chunks ago are done with it
-                 mbar_wait(&bar.den_full[sq], par, p.status, 402);     // ... and so is the K group's dot product
-          }
-          if (tid == 192) PROF(3, nq, 1);
-          tc_fence_after_sync();
           if (ok) {
-            // copy the raw row half out of the landing buffer and hand the buffer back at once, so
-            // that the next Q tile is in flight while this one is transformed
+            // copy the raw row half out of the landing buffer; the last warp to have done so
+            // starts the load of the next Q tile at once (the next chunk's, or the first one of
+            // this CTA's next item), so that it is in flight while this one is transformed
             uint32_t pk[kChunksPerHalf * 4];
-  #pragma unroll
+#pragma unroll
             for (int g = 0; g < kChunksPerHalf; ++g) {
               const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
               const int box = gl >> 3, cin = gl & 7;
@@ -883,19 +907,50 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               pk[g * 4 + 3] = rawv.w;
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(&bar.q_land_free);
-  #pragma unroll
-            for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
-            if constexpr (D == 128) {
-              uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
-              tmem_st32(tmem + C::tQ + sq * (D / 2) + lane_off + half * 32, pk32);
-            } else {
-              tmem_st16(tmem + C::tQ + sq * (D / 2) + lane_off + half * 16, pk);
+            if (lane == 0) {
+              __threadfence_block();
+              const int before = atomicAdd(&q_copied, 1);
+              if ((before & 7) == 7) {
+                int n_item = item, n_chunk = it.c_begin + j + 1;
+                LinItem nx = it;
+                if (j + 1 == it.nC) {
+                  n_item = item + gridDim.x;
+                  if (n_item < p.nitems) {
+                    nx = decode_item(p, n_item);
+                    n_chunk = nx.c_begin;
+                  }
+                }
+                if (n_item < p.nitems) {
+                  __threadfence_block();
+                  fence_proxy_async_smem();
+                  mbar_arrive_expect_tx(&bar.q_full, C::kTile);
+                  for (int x = 0; x < D / 64; ++x)
+                    tma_load_4d_hint(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n_chunk * 128, nx.h, nx.b,
+                                     l2_policy_evict_first());
+                }
+              }
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&bar.qphi_full[sq]);
+#pragma unroll
+            for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
+            if (nq >= 2) {
+              const uint32_t par = ((nq >> 1) + 1) & 1;
+              ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // MMA1/MMA2 of two chunks ago are done with it
+                   mbar_wait(&bar.den_full[sq], par, p.status, 402);     // ... and so is the K group's dot product
+            }
+            if (tid == 192) PROF(3, nq, 1);
+            tc_fence_after_sync();
+            if (ok) {
+              if constexpr (D == 128) {
+                uint32_t(&pk32)[32] = *reinterpret_cast<uint32_t(*)[32]>(pk);
+                tmem_st32(tmem + C::tQ + sq * (D / 2) + lane_off + half * 32, pk32);
+              } else {
+                tmem_st16(tmem + C::tQ + sq * (D / 2) + lane_off + half * 16, pk);
+              }
+              tmem_wait_st();
+              tc_fence_before_sync();
+              __syncwarp();
+              if (lane == 0) mbar_arrive(&bar.qphi_full[sq]);
+            }
           }
           if (tid == 192) PROF(3, nq, 2);
           ok = !__any_sync(0xffffffffu, !ok);
@@ -987,6 +1042,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 #ifdef GF_PROFILE
 extern "C" int gformer_debug_read_profile2(unsigned long long* host_dst) {
   return (int)cudaMemcpyFromSymbol(host_dst, g_prof2, sizeof(g_prof2));
+}
+extern "C" int gformer_debug_read_waits(unsigned long long* host_dst) {
+  return (int)cudaMemcpyFromSymbol(host_dst, g_wait, sizeof(g_wait));
+}
+extern "C" int gformer_debug_reset_waits() {
+  static unsigned long long zeros[160 * 1024];
+  return (int)cudaMemcpyToSymbol(g_wait, zeros, sizeof(g_wait));
 }
 extern "C" int gformer_debug_read_profile3(unsigned long long* host_dst) {
   return (int)cudaMemcpyFromSymbol(host_dst, g_prof3, sizeof(g_prof3));
