@@ -107,8 +107,13 @@ int run_linear(const void* q, const void* k, const void* v, void* o, int B, int 
                                             h_begin, h_count, S_io, z_io, zero_init, stream));
 }
 
-int clear_ws(void* ws, cudaStream_t stream) {
-  return cuda_status(cudaMemsetAsync(ws, 0, sizeof(WsHeader), stream));
+// Zeroes the workspace header and, for a call that runs the tensor-core linear kernel on n_lin
+// chains, the hand-over flags behind it: one memset, ahead of everything the call launches.
+int clear_ws(void* ws, cudaStream_t stream, int n_lin = 0, int N = 0, int d = 0, int dtype = GF_BF16) {
+  size_t bytes = sizeof(WsHeader);
+  if (n_lin > 0 && !g_force_simt && gf::tc_linear_supported(N, d, dtype))
+    bytes += gf::linear_tc_flag_bytes(n_lin, N, g_linear_split);
+  return cuda_status(cudaMemsetAsync(ws, 0, bytes, stream));
 }
 
 }  // namespace
@@ -204,7 +209,7 @@ int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void
   rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, 1, 0, dtype));
   if (rc != GF_OK) return rc;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  rc = clear_ws(ws, stream);
+  rc = clear_ws(ws, stream, B * H, N, d, dtype);
   if (rc != GF_OK) return rc;
   return run_linear(q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, 0, (WsHeader*)ws, stream);
 }
@@ -232,7 +237,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  rc = clear_ws(ws, stream);
+  rc = clear_ws(ws, stream, B * h_lin, N, d, dtype);
   if (rc != GF_OK) return rc;
 
   float* S_out = state_out ? state_out->S : nullptr;

@@ -67,6 +67,9 @@ cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* 
 // the workspace header (sized for the largest segment count the plan may pick for any ctas).
 void linear_tc_plan(int nchains, int N, int split, int ctas, int* chunks_per_segment, int* segments_per_chain);
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split);
+// Bytes at the start of that scratch (right after the workspace header) that must be zero when the
+// kernel starts: the hand-over flags.  The caller clears them (together with the header).
+size_t linear_tc_flag_bytes(int nchains, int N, int split);
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
                              int split, int max_ctas, WsHeader* ws, cudaStream_t stream);

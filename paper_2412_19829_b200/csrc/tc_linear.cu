@@ -1112,15 +1112,26 @@ void linear_tc_plan(int nchains, int N, int split, int ctas, int* L_out, int* G_
   *L_out = (nch + G - 1) / G;
 }
 
-size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
+namespace {
+// Largest segment count the plan may pick (the scratch is laid out for it).
+int plan_g_max(int nchains, int N, int split) {
   int L, G;
   linear_tc_plan(nchains, N, split, 0, &L, &G);
   if (split <= 0) {
     int g_min;
     plan_range(nchains, (N + 127) / 128, &g_min, &G);
   }
-  const size_t flags = (size_t)nchains * G * kFlagStride * sizeof(unsigned int);
-  return flags + (size_t)nchains * G * ((size_t)128 * d + d) * sizeof(float);
+  return G;
+}
+}  // namespace
+
+size_t linear_tc_flag_bytes(int nchains, int N, int split) {
+  return (size_t)nchains * plan_g_max(nchains, N, split) * kFlagStride * sizeof(unsigned int);
+}
+
+size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
+  const int G = plan_g_max(nchains, N, split);
+  return linear_tc_flag_bytes(nchains, N, split) + (size_t)nchains * G * ((size_t)128 * d + d) * sizeof(float);
 }
 
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
@@ -1154,11 +1165,8 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   p.zero_init = zero_init ? 1 : 0;
   p.status = &ws->status;
   uint8_t* scratch = reinterpret_cast<uint8_t*>(ws) + sizeof(WsHeader);
-  const size_t flag_bytes = (size_t)p.nchains * p.G * kFlagStride * sizeof(unsigned int);
-  p.flags = reinterpret_cast<unsigned int*>(scratch);
-  p.prefix = reinterpret_cast<float*>(scratch + flag_bytes);
-  e = cudaMemsetAsync(p.flags, 0, flag_bytes, stream);
-  if (e != cudaSuccess) return e;
+  p.flags = reinterpret_cast<unsigned int*>(scratch);  // zeroed by the caller
+  p.prefix = reinterpret_cast<float*>(scratch + linear_tc_flag_bytes(p.nchains, N, split));
   dim3 grid(p.nitems < sms ? p.nitems : sms);
   if (d == 64) {
     auto kern = linear_tc_kernel<64>;

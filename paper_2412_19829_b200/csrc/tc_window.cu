@@ -3,15 +3,17 @@
 // One CTA = one tile of 128 query rows of one (batch, head).  The keys a tile can see,
 // [i0 - w + 1, i0 + 127], are walked in 128-key tiles aligned to the query grid:
 //   S = Q K^T      tcgen05.mma, A and B from shared memory (K-major), S (128x128 fp32) in TMEM
-//   P = softmax    one thread per query row reads its S row from TMEM, masks (causal edge on
-//                  the diagonal tile, window edge on the leftmost ones), exponentiates against a
-//                  running reference maximum and writes P as bf16 back over S in TMEM
+//   P = softmax    two threads per query row (64 key columns each) read the S row from TMEM, mask
+//                  (causal edge on the diagonal tile, window edge on the leftmost ones), agree on
+//                  the row maximum through shared memory, exponentiate against a running
+//                  reference maximum and write P as bf16 back over S in TMEM
 //   O += P V       tcgen05.mma with A = P from TMEM, B = V from shared memory (MN-major)
 // O stays in TMEM across key tiles; it is rescaled only when a row's maximum moves by more than
 // 2^8 (lazy rescaling), which with bounded logits is rare.  Final rows are divided by the softmax
 // denominator, packed to bf16 and written with a TMA store.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = softmax/epilogue.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = softmax/epilogue (two
+// warps per TMEM lane quarter, one per half of the key columns / of the output columns).
 // TMEM use is 256 columns and shared memory under 113 KB so that two CTAs share an SM: while one
 // is in its softmax the other owns the tensor core.
 #include "common.cuh"
@@ -22,7 +24,7 @@ namespace {
 
 using namespace sm100;
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
@@ -60,6 +62,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint8_t* sV = sm + WinSmem<D>::kV;
   __shared__ __align__(8) uint64_t q_full, k_full, k_empty, v_full, v_empty, s_full, p_full, pv_done;
   __shared__ uint32_t tmem_base_s;
+  __shared__ float mx_s[2][2][128];  // [tile parity][column half][row]: half-row maxima
+  __shared__ float l_s[2][128];      // [column half][row]: half-row sums at the end
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int qt = blockIdx.x, h = p.h_begin + blockIdx.y, b = blockIdx.z;
@@ -74,7 +78,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&v_full, 1);
     mbar_init(&v_empty, 1);
     mbar_init(&s_full, 1);
-    mbar_init(&p_full, 128);
+    mbar_init(&p_full, 256);
     mbar_init(&pv_done, 1);
     mbar_fence_init();
     tma_prefetch_desc(&mq);
@@ -130,8 +134,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         tc_fence_after_sync();
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {
-          umma_ts(tO, tS + ks * 8, umma_smem_desc(smem_u32(sV) + ks * 2048, 16384, 1024), idesc_pv,
-                  (it > 0) || (ks > 0));
+          umma_ts(tO, tS + (ks >> 2) * 64 + (ks & 3) * 8, umma_smem_desc(smem_u32(sV) + ks * 2048, 16384, 1024),
+                  idesc_pv, (it > 0) || (ks > 0));
         }
         umma_commit(&v_empty);
         umma_commit(&pv_done);
@@ -139,44 +143,44 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue
-    const int quarter = warp & 3;  // TMEM lane quarter this warp may touch
+    const int quarter = warp & 3;    // TMEM lane quarter this warp may touch
+    const int hh = (warp - 2) >> 2;  // half of the key columns (softmax) / of the output columns (epilogue)
     const int r = quarter * 32 + lane;
     const int i = i0 + r;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
-    float m_ref = -INFINITY;  // reference maximum the stored O and l are relative to
-    float l = 0.f;
+    const int c0 = hh * 64, c1 = hh * 64 + 63;  // this thread's key columns within a tile
+    float m_ref = -INFINITY;  // reference maximum the stored O and l are relative to (same in both halves)
+    float l = 0.f;            // sum over this thread's columns
     bool ok = true;
     for (int it = 0; it < n_tiles; ++it) {
       const int j0 = (t_first + it) * 128;
       if (!mbar_wait(&s_full, it & 1, p.status, 30)) { ok = false; break; }
       tc_fence_after_sync();
-      // valid key columns of this row in this tile: [lo, hi]; of this warp's 32 rows: between
-      // [lo_w, hi_w + 31] (all rows see at least) and [lo_w + 31, hi_w] ... classified per 32-column
-      // block so that fully masked blocks cost nothing and fully visible ones need no per-element test
-      int lo = i - p.w + 1 - j0;
-      int hi = i - j0;
+      // valid key columns of this row in this tile: [lo, hi]; over the warp's 32 rows lo and hi move
+      // by 31, so the 64-column half is classified per warp: nothing visible (costs nothing), all
+      // visible to every row (no per-element test), or mixed
+      const int lo = i - p.w + 1 - j0;
+      const int hi = i - j0;
       const int lo_first = (i0 + quarter * 32) - p.w + 1 - j0;  // lo of the warp's first row (last row: +31)
       const int hi_first = (i0 + quarter * 32) - j0;            // hi of the warp's first row (last row: +31)
-      // Two sweeps over the row (maximum, then exponentials), 64 columns per TMEM round trip: the
-      // scores stay in TMEM between the sweeps, so only 64 of them are live in registers at a time.
+      const bool none = (c1 < lo_first || c0 > hi_first + 31);
+      const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);
+      // Two sweeps over the half row (maximum, then exponentials): the scores stay in TMEM between
+      // the sweeps, so that few registers are live across the exchange of the maxima.
       float mx[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-  #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const int c0 = hh * 64, c1 = hh * 64 + 63;
-        if (c1 < lo_first || c0 > hi_first + 31) continue;  // masked for every row of the warp
+      if (!none) {
         uint32_t sa[32], sb[32];
         tmem_ld32(tS + lane_off + c0, sa);
         tmem_ld32(tS + lane_off + c0 + 32, sb);
         tmem_wait_ld();
-        const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);  // visible to every row of the warp
         if (inside) {
-  #pragma unroll
+#pragma unroll
           for (int j = 0; j < 32; ++j) {
             mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(sa[j]));
             mx[(j + 2) & 3] = fmaxf(mx[(j + 2) & 3], __uint_as_float(sb[j]));
           }
         } else {
-  #pragma unroll
+#pragma unroll
           for (int j = 0; j < 32; ++j) {
             const int col = c0 + j;
             if (col >= lo && col <= hi) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(sa[j]));
@@ -184,8 +188,13 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           }
         }
       }
-      const float mt = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])) * p.scale_log2;  // scale > 0
-      // lazy rescale of what has been accumulated so far
+      // the row maximum over both halves: exchange through shared memory with the partner warp
+      // (same lane quarter, other half); double buffered by tile parity, one barrier per tile
+      const float mloc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+      mx_s[it & 1][hh][r] = mloc;
+      asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
+      const float mt = fmaxf(mloc, mx_s[it & 1][hh ^ 1][r]) * p.scale_log2;  // scale > 0
+      // lazy rescale of what has been accumulated so far (both halves take the same decision)
       float alpha = 1.f;
       bool need = false;
       if (mt > m_ref + kRescaleThreshold) {  // also true for the first finite maximum
@@ -198,84 +207,93 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (__any_sync(0xffffffffu, need)) {
           if (!mbar_wait(&pv_done, (it - 1) & 1, p.status, 31)) { ok = false; break; }
           tc_fence_after_sync();
-  #pragma unroll
+          // this warp's half of the output columns, a few at a time (the scores stay live in
+          // registers around this rare path)
+#pragma unroll 1
           for (int c = 0; c < D / 32; ++c) {
-            uint32_t oreg[32];
-            tmem_ld32(tO + lane_off + c * 32, oreg);
+            uint32_t oreg[16];
+            tmem_ld16(tO + lane_off + hh * (D / 2) + c * 16, oreg);
             tmem_wait_ld();
-  #pragma unroll
-            for (int j = 0; j < 32; ++j) oreg[j] = __float_as_uint(__uint_as_float(oreg[j]) * alpha);
-            tmem_st32(tO + lane_off + c * 32, oreg);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) oreg[j] = __float_as_uint(__uint_as_float(oreg[j]) * alpha);
+            tmem_st16(tO + lane_off + hh * (D / 2) + c * 16, oreg);
           }
           tmem_wait_st();
         }
       }
-      // p = 2^(s * scale_log2 - m_ref), bf16, back over S: the 64 scores of half hh become 32 packed
-      // columns at [32 hh, 32 hh + 32), inside columns this thread has already consumed
+      // p = 2^(s * scale_log2 - m_ref), bf16, back over S: this thread's 64 scores become 32 packed
+      // columns at [64 hh, 64 hh + 32), inside columns it has itself consumed
       const float neg_mref = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
-  #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        const int c0 = hh * 64, c1 = hh * 64 + 63;
-        uint32_t pk[32];
-        if (c1 < lo_first || c0 > hi_first + 31) {
-  #pragma unroll
-          for (int j = 0; j < 32; ++j) pk[j] = 0u;
-        } else {
-          uint32_t sa[32], sb[32];
-          tmem_ld32(tS + lane_off + c0, sa);
-          tmem_ld32(tS + lane_off + c0 + 32, sb);
-          tmem_wait_ld();
-          const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);
-          if (inside) {  // the common case, kept free of any masking arithmetic
-  #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              const float p0 = ex2_approx(fmaf(__uint_as_float(sa[2 * j]), p.scale_log2, neg_mref));
-              const float p1 = ex2_approx(fmaf(__uint_as_float(sa[2 * j + 1]), p.scale_log2, neg_mref));
-              const float p2 = ex2_approx(fmaf(__uint_as_float(sb[2 * j]), p.scale_log2, neg_mref));
-              const float p3 = ex2_approx(fmaf(__uint_as_float(sb[2 * j + 1]), p.scale_log2, neg_mref));
-              ls[j & 3] += (p0 + p1) + (p2 + p3);
-              pk[j] = pack_bf16(p0, p1);
-              pk[16 + j] = pack_bf16(p2, p3);
-            }
-          } else {
-  #pragma unroll
-            for (int j = 0; j < 16; ++j) {
-              float a0 = fmaf(__uint_as_float(sa[2 * j]), p.scale_log2, neg_mref);
-              float a1 = fmaf(__uint_as_float(sa[2 * j + 1]), p.scale_log2, neg_mref);
-              float b0 = fmaf(__uint_as_float(sb[2 * j]), p.scale_log2, neg_mref);
-              float b1 = fmaf(__uint_as_float(sb[2 * j + 1]), p.scale_log2, neg_mref);
-              const int col = c0 + 2 * j;
-              if (col < lo || col > hi) a0 = -INFINITY;
-              if (col + 1 < lo || col + 1 > hi) a1 = -INFINITY;
-              if (col + 32 < lo || col + 32 > hi) b0 = -INFINITY;
-              if (col + 33 < lo || col + 33 > hi) b1 = -INFINITY;
-              const float p0 = ex2_approx(a0), p1 = ex2_approx(a1), p2 = ex2_approx(b0), p3 = ex2_approx(b1);
-              ls[j & 3] += (p0 + p1) + (p2 + p3);
-              pk[j] = pack_bf16(p0, p1);
-              pk[16 + j] = pack_bf16(p2, p3);
-            }
-          }
-        }
-        tmem_st32(tS + lane_off + hh * 32, pk);
+      uint32_t sa[32], sb[32];
+      if (!none) {
+        tmem_ld32(tS + lane_off + c0, sa);
+        tmem_ld32(tS + lane_off + c0 + 32, sb);
+        tmem_wait_ld();
       }
-      const float lsum = (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      l += lsum;
+      // packed in place: pair j of sa / sb goes to word j of the same array once it has been read
+      if (none) {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) sa[j] = sb[j] = 0u;
+      } else if (inside) {  // the common case, kept free of any masking arithmetic
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          const float p0 = ex2_approx(fmaf(__uint_as_float(sa[2 * j]), p.scale_log2, neg_mref));
+          const float p1 = ex2_approx(fmaf(__uint_as_float(sa[2 * j + 1]), p.scale_log2, neg_mref));
+          const float p2 = ex2_approx(fmaf(__uint_as_float(sb[2 * j]), p.scale_log2, neg_mref));
+          const float p3 = ex2_approx(fmaf(__uint_as_float(sb[2 * j + 1]), p.scale_log2, neg_mref));
+          ls[j & 3] += (p0 + p1) + (p2 + p3);
+          sa[j] = pack_bf16(p0, p1);
+          sb[j] = pack_bf16(p2, p3);
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          float a0 = fmaf(__uint_as_float(sa[2 * j]), p.scale_log2, neg_mref);
+          float a1 = fmaf(__uint_as_float(sa[2 * j + 1]), p.scale_log2, neg_mref);
+          float b0 = fmaf(__uint_as_float(sb[2 * j]), p.scale_log2, neg_mref);
+          float b1 = fmaf(__uint_as_float(sb[2 * j + 1]), p.scale_log2, neg_mref);
+          const int col = c0 + 2 * j;
+          if (col < lo || col > hi) a0 = -INFINITY;
+          if (col + 1 < lo || col + 1 > hi) a1 = -INFINITY;
+          if (col + 32 < lo || col + 32 > hi) b0 = -INFINITY;
+          if (col + 33 < lo || col + 33 > hi) b1 = -INFINITY;
+          const float p0 = ex2_approx(a0), p1 = ex2_approx(a1), p2 = ex2_approx(b0), p3 = ex2_approx(b1);
+          ls[j & 3] += (p0 + p1) + (p2 + p3);
+          sa[j] = pack_bf16(p0, p1);
+          sb[j] = pack_bf16(p2, p3);
+        }
+      }
+      {
+        uint32_t pa[16], pb[16];
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+          pa[j] = sa[j];
+          pb[j] = sb[j];
+        }
+        tmem_st16(tS + lane_off + c0, pa);
+        tmem_st16(tS + lane_off + c0 + 16, pb);
+      }
+      l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       tmem_wait_st();
       tc_fence_before_sync();
       mbar_arrive(&p_full);
     }
-    // epilogue: O / l -> bf16 -> shared (swizzled, Q's buffer is free by now) -> TMA store
+    // epilogue: O / l -> bf16 -> shared (swizzled, Q's buffer is free by now) -> TMA store; this
+    // warp takes its half of the output columns
+    l_s[hh][r] = l;
+    asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
     if (ok) ok = mbar_wait(&pv_done, (n_tiles - 1) & 1, p.status, 32);
     tc_fence_after_sync();
     if (ok) {
-      const float inv = 1.f / l;
+      const float inv = 1.f / (l_s[0][r] + l_s[1][r]);
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
+      for (int c = 0; c < D / 64; ++c) {
+        const int col0 = hh * (D / 2) + c * 32;  // first of 32 output columns
         uint32_t oreg[32];
-        tmem_ld32(tO + lane_off + c * 32, oreg);
+        tmem_ld32(tO + lane_off + col0, oreg);
         tmem_wait_ld();
-        uint8_t* box = sQ + (c >> 1) * 16384;
+        uint8_t* box = sQ + (col0 >> 6) * 16384;
 #pragma unroll
         for (int g = 0; g < 4; ++g) {  // 4 chunks of 8 columns
           uint4 val;
@@ -283,13 +301,12 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           val.y = pack_bf16(__uint_as_float(oreg[8 * g + 2]) * inv, __uint_as_float(oreg[8 * g + 3]) * inv);
           val.z = pack_bf16(__uint_as_float(oreg[8 * g + 4]) * inv, __uint_as_float(oreg[8 * g + 5]) * inv);
           val.w = pack_bf16(__uint_as_float(oreg[8 * g + 6]) * inv, __uint_as_float(oreg[8 * g + 7]) * inv);
-          const uint32_t col = (c & 1) * 32 + g * 8;
-          *reinterpret_cast<uint4*>(box + swz128_offset(r, col)) = val;
+          *reinterpret_cast<uint4*>(box + swz128_offset(r, (col0 & 63) + g * 8)) = val;
         }
       }
       fence_proxy_async_smem();
     }
-    asm volatile("bar.sync 1, 128;" ::: "memory");
+    asm volatile("bar.sync 1, 256;" ::: "memory");
     if (ok && warp == 2 && elect_one()) {
       for (int c = 0; c < D / 64; ++c) tma_store_4d(&mo, sQ + c * 16384, c * 64, i0, h, b);
       tma_store_commit();
