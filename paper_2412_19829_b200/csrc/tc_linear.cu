@@ -967,6 +967,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       uint32_t n_kphi[2] = {0, 0}, n_os[2] = {0, 0};
       bool ok = true;
       const uint64_t pol_keep = l2_policy_evict_last();  // parked phi(K) tiles are read back by pass C
+      const uint64_t pol_out = l2_policy_evict_first();  // nobody reads O again: leave L2 to the tiles that come back
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
         // ---- pass A: park phi(K) tiles in the output rows of their chunk
@@ -994,7 +995,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (!mbar_wait(&bar.o_staged[sv], n_os[sv] & 1, p.status, 500)) { ok = false; break; }
           ++n_os[sv];
           for (int x = 0; x < D / 64; ++x)
-            tma_store_4d(&mo, sV + sv * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b);
+            tma_store_4d_hint(&mo, sV + sv * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b,
+                              pol_out);
           tma_store_commit();
           tma_store_wait_read<0>();
           mbar_arrive(&bar.v_free[sv]);  // the staging buffer may take the V tile two uses later

@@ -308,7 +308,8 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (ok && warp == 2 && elect_one()) {
-      for (int c = 0; c < D / 64; ++c) tma_store_4d(&mo, sQ + c * 16384, c * 64, i0, h, b);
+      const uint64_t pol_out = l2_policy_evict_first();  // nobody reads O again
+      for (int c = 0; c < D / 64; ++c) tma_store_4d_hint(&mo, sQ + c * 16384, c * 64, i0, h, b, pol_out);
       tma_store_commit();
       tma_store_wait_read<0>();
     }
