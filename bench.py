@@ -36,6 +36,8 @@ WORKLOADS = {
     "long32k": dict(B=1, H=32, N=32768, d=128, w=512, seed=2),
     "gpt2s": dict(B=8, H=12, N=2048, d=64, w=128, seed=1),
     "prefill4k": dict(B=64, H=16, N=4096, d=64, w=256, seed=3),
+    # token-by-token decoding after a 4096-token prefill: a step = `steps` decode steps of the batch
+    "decode256": dict(B=64, H=16, N=4096, d=64, w=256, seed=3, decode_steps=256),
 }
 
 
@@ -130,10 +132,50 @@ def oracle_sample_rate(c, sample_tokens):
     return c["B"] * n / dt, dt, n, oracle.num_threads()
 
 
+def oracle_decode_rate(c, steps):
+    """Times `steps` oracle decode steps of the batch on a state whose ring is full; tokens/s."""
+    import torch
+
+    import oracle
+    from paper_2412_19829_b200 import synth
+
+    B, H, d, w = c["B"], c["H"], c["d"], c["w"]
+    st = oracle.DecodeState(B, H, d, w, oracle.default_h_sparse(H))
+    st.t = c["N"]  # the ring counts as full; zero contents cost the same arithmetic as any other
+    tq, tk, tv = [t.to(torch.float64).numpy() for t in synth.decode_tokens(steps, B, H, d, "bf16", c["seed"])]
+    t0 = time.perf_counter()
+    for t in range(steps):
+        oracle.decode_step(tq[t], tk[t], tv[t], st)
+    dt = time.perf_counter() - t0
+    return B * steps / dt, dt, steps, oracle.num_threads()
+
+
 def run_reference(args, c, rank):
     if rank != 0:
         return
     import oracle  # noqa: F401  (CPU oracle: the reference arm of this benchmark)
+
+    if "decode_steps" in c:
+        n_steps = 16
+        for _ in range(args.warmup):
+            oracle_decode_rate(c, n_steps)
+        times = [oracle_decode_rate(c, n_steps)[1] for _ in range(args.steps)]
+        mean = sum(times) / len(times)
+        value = c["B"] * n_steps / mean
+        cores = oracle.num_threads()
+        line = {
+            "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, **{k: c[k] for k in ("B", "H", "d", "w")},
+                       "h_sparse": oracle.default_h_sparse(c["H"]), "decode_steps_per_step": n_steps},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{n_steps} decode steps of the batch on a full ring per step, fp64"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0,
+        }
+        print(json.dumps(line), flush=True)
+        return
 
     for _ in range(args.warmup):
         oracle_sample_rate(c, REFERENCE_STEP_TOKENS)
@@ -305,6 +347,134 @@ def run_ours(args, c, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_decode(args, c, rank, world, local_rank):
+    """Decode workload: prefill once (untimed), then time runs of `decode_steps` gformer_decode_step
+    calls, once replayed from a CUDA graph captured over all of them and once launched one by one."""
+    import torch
+
+    from paper_2412_19829_b200 import binding as gf
+    from paper_2412_19829_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    B, H, N, d, w, T = c["B"], c["H"], c["N"], c["d"], c["w"], c["decode_steps"]
+    h0 = gf.default_h_sparse(H)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", c["seed"] + 1000 * rank)
+    tq, tk, tv = synth.decode_tokens(T, B, H, d, "bf16", c["seed"] + 1000 * rank)
+    htok = [t.pin_memory() for t in (tq, tk, tv)]
+    dtok = [t.cuda() for t in htok]
+    dout = torch.empty_like(dtok[0])
+    hout = torch.empty_like(htok[0]).pin_memory()
+    st = gf.DecodeState(B, H, d, w, h0)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        gf.hybrid_attn(q.cuda(), k.cuda(), v.cuda(), w, h_sparse=h0, state_out=st, ws=ws, stream=stream)
+    stream.synchronize()
+    if ws.last_device_status(stream) != gf.GF_OK:
+        raise SystemExit("device-side wait timed out during the prefill")
+
+    def run_eager():
+        st.t = N  # every run decodes the same positions N .. N + T - 1
+        for t in range(T):
+            gf.decode_step(dtok[0][t], dtok[1][t], dtok[2][t], st, out=dout[t], stream=stream)
+
+    run_eager()
+    stream.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        run_eager()
+
+    def run_graph():
+        with torch.cuda.stream(stream):
+            graph.replay()
+
+    def run_e2e():
+        with torch.cuda.stream(stream):
+            for dst, src in zip(dtok, htok):
+                dst.copy_(src, non_blocking=True)
+            graph.replay()
+            hout.copy_(dout, non_blocking=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(steps):
+            fn()
+        e1.record(stream)
+        stream.synchronize()
+        barrier()
+        return e0.elapsed_time(e1)
+
+    for _ in range(max(args.warmup, 3)):
+        run_graph()
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
+    n0 = gf.launch_count()
+    total_ms = timed(run_graph, args.steps)
+    clocks = sampler.stop() if sampler else None
+    launches = gf.launch_count() - n0  # the graph replays the captured launches: count them below
+    eager_ms = timed(run_eager, args.steps)
+    run_e2e()
+    e2e_ms = timed(run_e2e, args.steps)
+    if dist is not None:
+        t = torch.tensor([total_ms, e2e_ms, eager_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms, e2e_ms, eager_ms = t.tolist()
+    if rank == 0:
+        tokens = world * B * T * args.steps
+        peak, which = measured_peaks()
+        # per decode step: the ring's valid slots read once (K and V), S read and written, z and the
+        # token's q, k, v, o
+        ring = 2 * B * h0 * min(N, w) * d * 2
+        state = 2 * B * (H - h0) * d * d * 4 + 2 * B * (H - h0) * d * 4
+        step_bytes = ring + state + 4 * B * H * d * 2
+        us_step = total_ms * 1e3 / (args.steps * T)
+        achieved = step_bytes / (us_step * 1e-6) / 1e9
+        line = {
+            "metric": METRIC, "value": tokens / (total_ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "B": B, "H": H, "d": d, "w": w, "h_sparse": h0, "prefill": N,
+                       "decode_steps_per_step": T, "global_batch": world * B,
+                       "parallelism": "replicas only (one batch per GPU, no collective)",
+                       "l2": "state and ring (26 MB) stay in L2 between decode steps: an L2-resident number",
+                       "launch": "one CUDA graph replay per step (all decode steps captured once)"},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None, "peak_source": which + " copy bandwidth",
+                         "algorithmic_bytes": step_bytes, "kernel": "decode_step_kernel, one launch per decode step",
+                         "us_per_decode_step_graph": us_step,
+                         "us_per_decode_step_eager": eager_ms * 1e3 / (args.steps * T)},
+            "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
+                    "h2d_bytes_per_step": 3 * T * B * H * d * 2, "d2h_bytes_per_step": T * B * H * d * 2},
+            "gpu_launches": args.steps * T if launches == 0 else launches,
+            "clocks": clocks,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            rate, dt, n, cores = oracle_decode_rate(c, 64)
+            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                    "sample": f"{n} decode steps of the batch on a full ring, {dt:.1f} s of fp64 CPU work"}
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
 def algorithmic_flops(c, h0):
     """Flops of the method itself: 4 d per (query, key) pair in the window, 4 d^2 per linear token."""
     B, H, N, d, w = c["B"], c["H"], c["N"], c["d"], c["w"]
@@ -328,6 +498,8 @@ def main():
     c = WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, c, rank)
+    elif "decode_steps" in c:
+        run_decode(args, c, rank, world, local_rank)
     else:
         run_ours(args, c, rank, world, local_rank)
 

@@ -281,6 +281,39 @@ def test_decode_state_copy_resumes_identically():
         assert torch.equal(a, b)
 
 
+def test_decode_steps_replayed_from_a_cuda_graph():
+    # the launch configuration bench.py times for the decode workload: all steps captured once in a
+    # CUDA graph, replayed; the replay must reproduce the step-by-step result bit for bit
+    B, H, d, w, h0, N0, steps = 2, 4, 64, 32, 1, 48, 12
+    q, k, v = synth.qkv(B, H, N0 + steps, d, "bf16", seed=53, gain=1.0)
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0)
+    qd, kd, vd = dev(q, k, v)
+    toks = [[x[:, :, t].contiguous() for t in range(N0, N0 + steps)] for x in (qd, kd, vd)]
+    st = gf.DecodeState(B, H, d, w, h0)
+    gf.hybrid_attn(qd[:, :, :N0].contiguous(), kd[:, :, :N0].contiguous(), vd[:, :, :N0].contiguous(), w,
+                   h_sparse=h0, state_out=st)
+    saved = {n: getattr(st, n).clone() for n in ("k_cache", "v_cache", "S", "z")}
+    eager = torch.stack([gf.decode_step(toks[0][s], toks[1][s], toks[2][s], st) for s in range(steps)])
+    assert_parity(f64(eager.permute(1, 2, 0, 3)), ref[:, :, N0:], "bf16", "eager decode")
+    for n, t in saved.items():
+        getattr(st, n).copy_(t)
+    st.t = N0
+    out = torch.empty_like(eager)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        for s in range(steps):
+            gf.decode_step(toks[0][s], toks[1][s], toks[2][s], st, out=out[s], stream=stream)
+    for _ in range(2):  # the capture itself runs nothing; each replay restarts from the saved state
+        for n, t in saved.items():
+            getattr(st, n).copy_(t)
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+
+
 def test_config4_prefill_and_decode_sampled_batch():
     c = synth.CONFIGS["decode"]
     B, H, N, d, w, steps = c["B"], c["H"], c["N"], c["d"], c["w"], 64  # 64 of the 256 steps checked
