@@ -87,6 +87,7 @@ struct LinItem {
   bool last_seg, need_dS;
 };
 
+
 __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
   LinItem it;
   it.g = item / p.nchains;
@@ -110,10 +111,16 @@ struct LinBarriers {
 };
 
 // Bounded poll of a monotonic counter in shared memory.
+__device__ __forceinline__ bool wait_epoch_slow(const int* counter, int target, unsigned int* status,
+                                                unsigned int where);
 __device__ __forceinline__ bool wait_epoch(const int* counter, int target, unsigned int* status,
                                            unsigned int where) {
+  if (*reinterpret_cast<const volatile int*>(counter) >= target) { __threadfence_block(); return true; }
+  return wait_epoch_slow(counter, target, status, where);
+}
+__device__ __forceinline__ bool wait_epoch_slow(const int* counter, int target, unsigned int* status,
+                                                unsigned int where) {
   const volatile int* c = counter;
-  if (*c >= target) { __threadfence_block(); return true; }
   const long long t0 = clock64();
   while (*c < target) {
     if (clock64() - t0 > 4000000000LL) {
@@ -674,7 +681,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (tid == 64) PROF(2, nq, 2);
         tc_fence_after_sync();
         const bool write_final = it.last_seg && (j == it.nC - 1) && p.S_io != nullptr;
-#pragma unroll
+#pragma unroll(D == 128 ? 1 : 2)
         for (int cc = 0; cc < D / 32; ++cc) {
           uint32_t v[32];
           tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
@@ -714,7 +721,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         tc_fence_after_sync();
         const float inv = 1.f / (den_s[sq][0][r] + den_s[sq][1][r]);
         uint8_t* stage = sV + sv * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
-#pragma unroll
+#pragma unroll(D == 128 ? 1 : 2)
         for (int cc = 0; cc < D / 32; ++cc) {
           uint32_t v[32];
           tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
