@@ -637,7 +637,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         } else if (p.S_io != nullptr && !p.zero_init) {
           Sin = p.S_io + (sidx * D + r) * D;  // caller's row-major state
         }
-#pragma unroll
+#pragma unroll(D == 128 ? 1 : 2)
         for (int cc = 0; cc < D / 32; ++cc) {
           uint32_t v[32];
 #pragma unroll
@@ -855,7 +855,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
           if (tt == 0) PROF(2, nq, 0);
           tc_fence_after_sync();
-  #pragma unroll
+#pragma unroll 1
           for (int e = 0; e < 2; ++e) {
             // 32-column block cc: all kept left of the diagonal block, all dropped right of it,
             // triangular on it (warp-uniform choice)
