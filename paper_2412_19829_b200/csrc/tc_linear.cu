@@ -280,13 +280,30 @@ __device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane1
   fence_proxy_async_smem();
 }
 
-// Column sums of transform_k_rows reduced over the 16 lanes that share a column chunk.
-__device__ __forceinline__ void reduce_column_sums(float (&cs)[8]) {
+// Column sums of transform_k_rows reduced over the 16 lanes that share a column chunk, as a
+// reduce-scatter (8 shuffles instead of 32): every step halves the columns a lane still carries.
+// Returns the sum of column `*col` (0..7 within the chunk: bits 3, 2, 1 of lane16; the two lanes
+// of a pair end with the same value).
+__device__ __forceinline__ float reduce_column_sums(const float (&cs)[8], int lane16, int* col) {
+  const bool b3 = lane16 & 8, b2 = lane16 & 4, b1 = lane16 & 2;
+  float a[4], b[2];
 #pragma unroll
-  for (int e = 0; e < 8; ++e) {
-#pragma unroll
-    for (int off = 8; off > 0; off >>= 1) cs[e] += __shfl_xor_sync(0xffffffffu, cs[e], off);
+  for (int e = 0; e < 4; ++e) {
+    const float send = b3 ? cs[e] : cs[e + 4];
+    const float keep = b3 ? cs[e + 4] : cs[e];
+    a[e] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
   }
+#pragma unroll
+  for (int e = 0; e < 2; ++e) {
+    const float send = b2 ? a[e] : a[e + 2];
+    const float keep = b2 ? a[e + 2] : a[e];
+    b[e] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+  }
+  const float send = b1 ? b[0] : b[1];
+  float c = (b1 ? b[1] : b[0]) + __shfl_xor_sync(0xffffffffu, send, 2);
+  c += __shfl_xor_sync(0xffffffffu, c, 1);
+  *col = (b3 ? 4 : 0) + (b2 ? 2 : 0) + (b1 ? 1 : 0);
+  return c;
 }
 
 // Critical path of the segment hand-over, run by the 16 phi warps (4 per TMEM lane quarter, each
@@ -371,7 +388,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   __shared__ __align__(16) float zcum[2][kMaxL + 1][D];
   __shared__ __align__(16) float zin[2][D];
   __shared__ float den_s[2][2][128];  // [chunk parity][column half][row]: partial denominators, K group -> row group
-  __shared__ float zpart[2][2][D]; // [tile parity][row half][column]: column sums of one K tile
+  __shared__ float zpart[kMaxL][2][D];  // [tile of the segment][row half][column]: column sums of one K tile
   __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
   __shared__ int zin_epoch;        // items whose zin is in place (monotonic)
   __shared__ int prev_epoch;       // items whose predecessor state has been seen in global memory (monotonic)
@@ -790,26 +807,31 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);  // the tile may go to the tensor core and be parked
         if (tid == 14 * 32) PROF(3, na, 5);
+        // the column sums are left per tile; nothing here waits for the other half of the tile
         if (ok && tt < 2 * D) {
-          reduce_column_sums(cs);
-          if ((tt & 15) == 0) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) zpart[j & 1][kgrp ? 0 : 1][cc * 8 + e] = cs[e];
-          }
-        }
-        if (named_bar_or(4, 512, !ok)) { ok = false; break; }  // both halves of the tile are done
-        if (kgrp) {
-          if (tt < D) zcum[ip][j + 1][tt] = zcum[ip][j][tt] + (zpart[j & 1][0][tt] + zpart[j & 1][1][tt]);
-          if (named_bar_or(3, 256, false)) { ok = false; break; }
-          ++na;
-          if (tt == 0) {
-            __threadfence_block();
-            *reinterpret_cast<volatile int*>(&ka_epoch) = na;
-          }
+          int col;
+          const float sum = reduce_column_sums(cs, tt & 15, &col);
+          if ((tt & 1) == 0) zpart[j][kgrp ? 0 : 1][cc * 8 + col] = sum;
         }
         ++nk;
       }
-      if (!ok) break;
+      // both halves of every tile are done: running column sums over the segment's chunks
+      if (named_bar_or(4, 512, !ok)) break;
+      if (kgrp) {
+        if (tt < D) {
+          float run = 0.f;
+          for (int j = 0; j < it.nC; ++j) {
+            run += zpart[j][0][tt] + zpart[j][1][tt];
+            zcum[ip][j + 1][tt] = run;
+          }
+        }
+        if (named_bar_or(3, 256, false)) break;
+        na += it.nC;
+        if (tt == 0) {
+          __threadfence_block();
+          *reinterpret_cast<volatile int*>(&ka_epoch) = na;
+        }
+      }
       nk += it.nC;  // the K ring also carries the pass-C tiles
       // ---- hand-over of S: the two groups publish the inclusive state (column quarters 0, 1 / 2, 3)
       if (it.need_dS) {
