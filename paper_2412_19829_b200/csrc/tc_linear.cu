@@ -58,7 +58,10 @@ struct LinCfg {
   static constexpr int kV = 3 * kTile;       // 2 stages
   static constexpr int kSb = 5 * kTile;      // bf16 copy of S, [D rows][D cols] in 64-column boxes
   static constexpr int kSbBytes = D * D * 2;
-  static constexpr int kBytes = 5 * kTile + kSbBytes + 1024;
+  // Pass A runs its K tiles through three slots: the two K slots and, third, the Sb buffer, which
+  // is idle in that pass (at D = 64 Sb is smaller than a tile, so the third slot gets its own room)
+  static constexpr int kKA2 = (D == 128) ? kSb : kSb + kSbBytes;
+  static constexpr int kBytes = 5 * kTile + kSbBytes + (D == 128 ? 0 : kTile) + 1024;
   static constexpr int kBoxBytes = 16384;    // one 128-row x 64-column box
   static constexpr int kSbBox = D * 128;     // one D-row x 64-column box of Sb
   // TMEM columns
@@ -104,9 +107,11 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
 
 struct LinBarriers {
   uint64_t q_full;
-  uint64_t k_full[2], ka_full[2], v_full[2], k_free[2], v_free[2];  // ka_full: K tiles of pass A, k_full: of pass C
-  uint64_t qphi_full[2], kphi_full[2], qphi_free[2];
-  uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done;
+  uint64_t ka_full[3], kphi_full[3], ka_free[3];  // K tiles of pass A (slot = tile count % 3)
+  uint64_t k_full[2], k_free[2];                  // K tiles of pass C (slot = chunk count & 1)
+  uint64_t v_full[2], v_free[2];                  // V tiles of both passes (slot = tile count & 1)
+  uint64_t qphi_full[2], qphi_free[2];
+  uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done, sb_idle, sb_parked;
   uint64_t pm_full, den_full[2], s_loaded, sb_full, o_free, o_staged[2];
 };
 
@@ -202,9 +207,11 @@ __device__ __forceinline__ bool prof_wait_flag(const unsigned int* f, unsigned i
   wait_account(where, t0);
   return ok;
 }
+#ifdef GF_PROFILE_WAITS  // the accounting itself costs time: only when asked for
 #define mbar_wait prof_mbar_wait
 #define wait_epoch prof_wait_epoch
 #define wait_flag prof_wait_flag
+#endif
 #define PROF(role, c, ev) prof_stamp(role, c, ev)
 #define PROF2(cond, ev) do { if (cond) prof2_stamp(ev); } while (0)
 #define PROF3(n, ev) prof3_stamp(n, ev)
@@ -399,16 +406,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 
   if (tid == 0) {
     mbar_init(&bar.q_full, 1);
+    for (int s = 0; s < 3; ++s) {
+      mbar_init(&bar.ka_full[s], 1);
+      mbar_init(&bar.kphi_full[s], 16);
+      mbar_init(&bar.ka_free[s], 2);  // the MMA issuer and the store warp
+    }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar.k_full[s], 1);
-      mbar_init(&bar.ka_full[s], 1);
       mbar_init(&bar.v_full[s], 1);
-      mbar_init(&bar.k_free[s], 2);
+      mbar_init(&bar.k_free[s], 1);
       mbar_init(&bar.v_free[s], 1);
       mbar_init(&bar.qphi_full[s], 8);
-      mbar_init(&bar.kphi_full[s], 16);
       mbar_init(&bar.qphi_free[s], 1);
     }
+    mbar_init(&bar.sb_idle, 1);
+    mbar_init(&bar.sb_parked, 1);
     mbar_init(&bar.p_full, 1);
     mbar_init(&bar.s_full, 1);
     mbar_init(&bar.o_full, 1);
@@ -443,17 +455,28 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   tc_fence_after_sync();
   const uint32_t tmem = tmem_base_s;
 
-  // Every role walks the same item list and keeps its own running counters: nk / nv = K / V tiles
-  // that went through the two-stage rings so far (stage = count & 1, phase = count >> 1), nq =
-  // pass-C chunks so far, na = pass-A tiles so far.
+  // Every role walks the same item list and keeps the same running counters: ta = K tiles of pass
+  // A so far (slot = ta % 3, phase = ta / 3), nq = pass-C chunks so far (K slot = nq & 1, phase =
+  // nq >> 1), nv = V tiles of both passes so far (slot = nv & 1, phase = nv >> 1).
+  auto a_kslot = [&](uint32_t slot) -> uint8_t* { return slot < 2 ? sK + slot * C::kTile : sm + C::kKA2; };
 
   if (warp == 0) {
     // ================================================================ TMA producer
     if (elect_one()) {
-      // a waiter may only use a parity wait on a barrier whose every phase it observes, so the K
-      // tiles of the two passes complete on different barriers (phi(K) group / MMA issuer)
-      uint32_t nk = 0, nv = 0, nq = 0, n_items = 0;
+      // A waiter may only use a parity wait on a barrier whose every phase it observes, so the K
+      // tiles of the two passes complete (and are released) on barriers of their own.  A buffer that
+      // serves both passes is only reloaded once its uses of either kind have drained: per barrier,
+      // uses issued so far against phases already observed.
+      uint32_t ta = 0, nv = 0, nq = 0, n_items = 0;
+      uint32_t iss_a[3] = {0, 0, 0}, obs_a[3] = {0, 0, 0}, iss_c[2] = {0, 0}, obs_c[2] = {0, 0}, obs_sbi = 0;
       bool ok = true;
+      auto drain = [&](uint64_t* b, uint32_t& obs, uint32_t issued, unsigned int where) -> bool {
+        while (obs < issued) {
+          if (!mbar_wait(b, obs & 1, p.status, where)) return false;
+          ++obs;
+        }
+        return true;
+      };
       // K, Q and the second read of V are streamed once; the first read of V (and the parked phi(K)
       // tiles) come back within the same item and should stay in L2 until then
       const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
@@ -464,16 +487,32 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           PROF3(n_items, pass);
           for (int j = 0; j < it.nC; ++j) {
             const int n0 = (it.c_begin + j) * 128;
-            const int sk = nk & 1;
-            if (nk >= 2 && !mbar_wait(&bar.k_free[sk], ((nk >> 1) + 1) & 1, p.status, 101)) { ok = false; break; }
-            uint64_t* kbar = (pass == 0) ? &bar.ka_full[sk] : &bar.k_full[sk];
-            if (pass == 0) PROF(0, nk - nq, 1);
-            mbar_arrive_expect_tx(kbar, C::kTile);
-            for (int x = 0; x < D / 64; ++x)  // pass C reads back the phi(K) tile parked in the output rows
-              tma_load_4d_hint(sK + sk * C::kTile + x * C::kBoxBytes, pass == 0 ? &mk : &mo, kbar, x * 64, n0, it.h, it.b,
-                               pol_stream);
-            ++nk;
-            if (pass == 1) ++nq;
+            if (pass == 0) {
+              const uint32_t sa = ta % 3;
+              // the slot's earlier pass-A uses, and what shares the buffer in pass C: a K slot, or
+              // (third slot) the Sb operand, idle once the previous item's last readout is done
+              ok = drain(&bar.ka_free[sa], obs_a[sa], iss_a[sa], 101) &&
+                   (sa < 2 ? drain(&bar.k_free[sa], obs_c[sa], iss_c[sa], 104)
+                           : drain(&bar.sb_idle, obs_sbi, n_items, 105));
+              if (!ok) break;
+              PROF(0, ta, 1);
+              mbar_arrive_expect_tx(&bar.ka_full[sa], C::kTile);
+              for (int x = 0; x < D / 64; ++x)
+                tma_load_4d_hint(a_kslot(sa) + x * C::kBoxBytes, &mk, &bar.ka_full[sa], x * 64, n0, it.h, it.b,
+                                 pol_stream);
+              ++iss_a[sa];
+              ++ta;
+            } else {
+              const uint32_t sc = nq & 1;
+              ok = drain(&bar.k_free[sc], obs_c[sc], iss_c[sc], 104) && drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101);
+              if (!ok) break;
+              mbar_arrive_expect_tx(&bar.k_full[sc], C::kTile);
+              for (int x = 0; x < D / 64; ++x)  // the phi(K) tile parked in the output rows
+                tma_load_4d_hint(sK + sc * C::kTile + x * C::kBoxBytes, &mo, &bar.k_full[sc], x * 64, n0, it.h, it.b,
+                                 pol_stream);
+              ++iss_c[sc];
+              ++nq;
+            }
             if (pass == 1 || it.need_dS) {
               const int sv = nv & 1;
               if (nv >= 2 && !mbar_wait(&bar.v_free[sv], ((nv >> 1) + 1) & 1, p.status, 102)) { ok = false; break; }
@@ -495,8 +534,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       constexpr uint32_t id_s = umma_idesc_bf16(128, D, true, true);      // S += Kc^T V
       constexpr uint32_t id_o = umma_idesc_bf16(128, D, false, true);     // O  = Qc Sb,  O += Pm V
       constexpr uint32_t kLboA = (D == 128) ? C::kBoxBytes : 0;           // D=64: rows 64..127 of S mirror 0..63
-      uint32_t nk = 0, nv = 0, nq = 0, n_sl = 0, n_sb = 0, n_of = 0, n_pm = 0;
-      uint32_t n_kphi[2] = {0, 0}, n_kc[2] = {0, 0};
+      uint32_t ta = 0, nv = 0, nq = 0, n_sl = 0, n_sb = 0, n_of = 0, n_pm = 0;
       bool ok = true, first_item = true;
       [[maybe_unused]] uint32_t n_items = 0;
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x, ++n_items) {
@@ -511,41 +549,39 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         first_item = false;
         // ---- pass A: dS = sum Kc^T V over the segment, from zero (only if somebody needs it)
         for (int j = 0; j < it.nC; ++j) {
-          const int sk = nk & 1;
-          if (!mbar_wait(&bar.kphi_full[sk], n_kphi[sk] & 1, p.status, 220)) { ok = false; break; }
-          ++n_kphi[sk];
-          PROF(1, nk - nq, 4);
+          const uint32_t sa = ta % 3;
+          if (!mbar_wait(&bar.kphi_full[sa], (ta / 3) & 1, p.status, 220)) { ok = false; break; }
+          PROF(1, ta, 4);
           if (it.need_dS) {
             const int sv = nv & 1;
-            const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
+            const uint32_t kbase = smem_u32(a_kslot(sa)), vbase = smem_u32(sV) + sv * C::kTile;
             if (!mbar_wait(&bar.v_full[sv], (nv >> 1) & 1, p.status, 221)) { ok = false; break; }
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
               umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
                       umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, (j > 0) || (ks > 0));
-            PROF(1, nk - nq, 5);
-            umma_commit(&bar.k_free[sk]);  // second arrival: the store warp, once the tile is parked
+            PROF(1, ta, 5);
+            umma_commit(&bar.ka_free[sa]);  // second arrival: the store warp, once the tile is parked
             umma_commit(&bar.v_free[sv]);
             ++nv;
           } else {
-            mbar_arrive(&bar.k_free[sk]);
+            mbar_arrive(&bar.ka_free[sa]);
           }
-          ++nk;
+          ++ta;
         }
         if (!ok) break;
         if (it.need_dS) umma_commit(&bar.a_done);
         // ---- pass C
         for (int j = 0; j < it.nC; ++j) {
-          const int sk = nk & 1, sv = nv & 1, sq = nq & 1;
-          const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
+          const int sv = nv & 1, sq = nq & 1;  // sq: slot of the K ring of this pass and of phi(Q)
+          const uint32_t kbase = smem_u32(sK) + sq * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
           const uint32_t tq = tmem + C::tQ + sq * (D / 2);
           if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 200) ||
-              !mbar_wait(&bar.k_full[sk], n_kc[sk] & 1, p.status, 201)) {
+              !mbar_wait(&bar.k_full[sq], (nq >> 1) & 1, p.status, 201)) {
             ok = false;
             break;
           }
-          ++n_kc[sk];
           PROF(1, nq, 0);
           if (j == 0) PROF3(n_items, 4);
           tc_fence_after_sync();
@@ -567,8 +603,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
                     umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, true);
           umma_commit(&bar.s_full);
-          umma_commit(&bar.k_free[sk]);
-          mbar_arrive(&bar.k_free[sk]);  // nothing else holds the tile in this pass
+          umma_commit(&bar.k_free[sq]);
           if (!mbar_wait(&bar.sb_full, n_sb & 1, p.status, 204)) { ok = false; break; }
           ++n_sb;
           if (nq >= 1) {
@@ -583,6 +618,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                     ks > 0);
           umma_commit(&bar.mma2_done);
           umma_commit(&bar.qphi_free[sq]);
+          if (j == it.nC - 1) umma_commit(&bar.sb_idle);  // Sb may now take a K tile of the next pass A
           if (!mbar_wait(&bar.pm_full, n_pm & 1, p.status, 206)) { ok = false; break; }
           ++n_pm;
           PROF(1, nq, 3);
@@ -593,7 +629,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                     umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
                     id_o, true);
           umma_commit(&bar.o_full);
-          ++nk;
           ++nv;
           ++nq;
         }
@@ -645,6 +680,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         tc_fence_after_sync();
         nv += it.nC;
       }
+      // Sb held K tiles in pass A: they have been parked (and, above, consumed by the tensor core)
+      ok = mbar_wait(&bar.sb_parked, n_items & 1, p.status, 314) && ok;
       {
         const float* Sin = nullptr;
         long long sin_stride = 1;  // float4 units between consecutive column groups of one row
@@ -697,13 +734,17 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         }
         if (tid == 64) PROF(2, nq, 2);
         tc_fence_after_sync();
-        const bool write_final = it.last_seg && (j == it.nC - 1) && p.S_io != nullptr;
+        // after the item's last chunk nobody reads Sb again (it may already hold a K tile of the
+        // next item's pass A), and only a chain's last segment still wants the state itself
+        const bool last_chunk = (j == it.nC - 1);
+        const bool write_final = it.last_seg && last_chunk && p.S_io != nullptr;
 #pragma unroll(D == 128 ? 1 : 2)
         for (int cc = 0; cc < D / 32; ++cc) {
+          if (last_chunk && !write_final) break;
           uint32_t v[32];
           tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
           tmem_wait_ld();
-          if (s_row) {
+          if (s_row && !last_chunk) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
               uint4 val;
@@ -713,14 +754,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
               *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
             }
-            if (write_final) {
-              float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
+          }
+          if (s_row && write_final) {
+            float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
 #pragma unroll
-              for (int jj = 0; jj < 32; jj += 4)
-                *reinterpret_cast<float4*>(dst + jj) =
-                    make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
-                                __uint_as_float(v[jj + 3]));
-            }
+            for (int jj = 0; jj < 32; jj += 4)
+              *reinterpret_cast<float4*>(dst + jj) =
+                  make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
+                              __uint_as_float(v[jj + 3]));
           }
         }
         tc_fence_before_sync();
@@ -776,8 +817,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per Q-group thread
-    uint32_t nq = 0, nk = 0, n_a = 0, n_items = 0;
-    uint32_t n_ka[2] = {0, 0};
+    uint32_t nq = 0, ta = 0, n_a = 0, n_items = 0;
     int na = 0;
     bool ok = true;
     if (tid == 6 * 32 && (int)blockIdx.x < p.nitems) {
@@ -795,26 +835,29 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       // ---- pass A: the K group takes rows 0..63 (by sixteens) of every K tile, the Q group rows
       //      64..127; the K group also keeps the cumulative column sums
       for (int j = 0; j < it.nC; ++j) {
-        const int sk = nk & 1;
-        ok = ok && mbar_wait(&bar.ka_full[sk], n_ka[sk] & 1, p.status, 410);
-        ++n_ka[sk];
-        if (tid == 14 * 32) PROF(3, na, 4);
+        const uint32_t sk = ta % 3;
+        ok = ok && mbar_wait(&bar.ka_full[sk], (ta / 3) & 1, p.status, 410);
+        if (tid == 14 * 32) PROF(3, ta, 4);
+
         const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
         float cs[8];
         if (ok && tt < 2 * D)
-          transform_k_rows(sK + sk * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
+          transform_k_rows(a_kslot(sk) + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
+
                            p.N - (it.c_begin + j) * 128, cs);
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);  // the tile may go to the tensor core and be parked
-        if (tid == 14 * 32) PROF(3, na, 5);
+        if (tid == 14 * 32) PROF(3, ta, 5);
+
         // the column sums are left per tile; nothing here waits for the other half of the tile
         if (ok && tt < 2 * D) {
           int col;
           const float sum = reduce_column_sums(cs, tt & 15, &col);
           if ((tt & 1) == 0) zpart[j][kgrp ? 0 : 1][cc * 8 + col] = sum;
         }
-        ++nk;
+        ++ta;
       }
+
       // both halves of every tile are done: running column sums over the segment's chunks
       if (named_bar_or(4, 512, !ok)) break;
       if (kgrp) {
@@ -832,7 +875,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           *reinterpret_cast<volatile int*>(&ka_epoch) = na;
         }
       }
-      nk += it.nC;  // the K ring also carries the pass-C tiles
+
       // ---- hand-over of S: the two groups publish the inclusive state (column quarters 0, 1 / 2, 3)
       if (it.need_dS) {
         ok = publish_inclusive<D>(p, it, bar, tmem, warp, lane, n_a & 1, &prev_epoch, (int)n_items);
@@ -991,9 +1034,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   } else if (warp == 22) {
     // ================================================================ TMA store warp
     if (elect_one()) {
-      uint32_t nk = 0, nv = 0, nq = 0;
+      uint32_t ta = 0, nv = 0;
       [[maybe_unused]] uint32_t n_items = 0;
-      uint32_t n_kphi[2] = {0, 0}, n_os[2] = {0, 0};
+      uint32_t n_os[2] = {0, 0};
       bool ok = true;
       const uint64_t pol_keep = l2_policy_evict_last();  // parked phi(K) tiles are read back by pass C
       const uint64_t pol_out = l2_policy_evict_first();  // nobody reads O again: leave L2 to the tiles that come back
@@ -1001,22 +1044,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         const LinItem it = decode_item(p, item);
         // ---- pass A: park phi(K) tiles in the output rows of their chunk
         for (int j = 0; j < it.nC; ++j) {
-          const int sk = nk & 1;
-          if (!mbar_wait(&bar.kphi_full[sk], n_kphi[sk] & 1, p.status, 520)) { ok = false; break; }
-          ++n_kphi[sk];
+          const uint32_t sk = ta % 3;
+          if (!mbar_wait(&bar.kphi_full[sk], (ta / 3) & 1, p.status, 520)) { ok = false; break; }
           for (int x = 0; x < D / 64; ++x)
-            tma_store_4d_hint(&mo, sK + sk * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b,
+            tma_store_4d_hint(&mo, a_kslot(sk) + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b,
                               pol_keep);
           tma_store_commit();
           tma_store_wait_read<0>();
-          PROF(0, nk - nq, 3);
-          mbar_arrive(&bar.k_free[sk]);
-          ++nk;
+          PROF(0, ta, 3);
+          mbar_arrive(&bar.ka_free[sk]);
+          ++ta;
         }
         if (!ok) break;
         tma_store_wait_all<0>();  // parked tiles are in memory before pass C asks for them
         mbar_arrive(&bar.park_done);
-        nk += it.nC;
+        mbar_arrive(&bar.sb_parked);  // ... and Sb, the third slot of the pass, has been read out
         if (it.need_dS) nv += it.nC;
         // ---- pass C: O tiles
         for (int j = 0; j < it.nC; ++j) {
@@ -1030,7 +1072,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           tma_store_wait_read<0>();
           mbar_arrive(&bar.v_free[sv]);  // the staging buffer may take the V tile two uses later
           ++nv;
-          ++nq;
         }
         PROF3(n_items, 5);
         ++n_items;
