@@ -151,7 +151,7 @@ __device__ __forceinline__ bool wait_flag(const unsigned int* flag, unsigned int
       if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
       return false;
     }
-    __nanosleep(100);
+    __nanosleep(20);
   }
 }
 
