@@ -65,17 +65,65 @@ def algorithmic_bytes(c):
 
 
 class ClockSampler:
+    """SM clock and throttle reasons sampled every 2 ms through NVML from a thread of this process,
+    between start() and stop(): the samples lie inside the timed region, and the GPU is never idle
+    waiting for a sampler to come up (an idle GPU changes its clocks).  Falls back to an
+    `nvidia-smi -lms 100` child process when the NVML binding is missing."""
+
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    REASON_BITS = {"sw_power_cap": 0x4, "hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20,
+                   "hw_thermal_slowdown": 0x40}
 
     def __init__(self, gpu_index):
         self.gpu_index = gpu_index
-        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.samples = []
+        self.thread = None
+        self.stop_flag = False
+        self.nvml = None
+        self.handle = None
+        self.file = None
         self.proc = None
+        try:
+            import pynvml
+
+            pynvml.nvmlInit()
+            # CUDA_VISIBLE_DEVICES may renumber the devices: go through the PCI bus id
+            import torch
+
+            bus = torch.cuda.get_device_properties(gpu_index).pci_bus_id if hasattr(
+                torch.cuda.get_device_properties(gpu_index), "pci_bus_id") else None
+            self.handle = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+            if bus is not None:
+                for i in range(pynvml.nvmlDeviceGetCount()):
+                    h = pynvml.nvmlDeviceGetHandleByIndex(i)
+                    if pynvml.nvmlDeviceGetPciInfo(h).bus == bus:
+                        self.handle = h
+                        break
+            self.nvml = pynvml
+        except Exception:
+            self.nvml = None
+
+    def _loop(self):
+        nv, h = self.nvml, self.handle
+        while not self.stop_flag:
+            try:
+                self.samples.append((nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM),
+                                     nv.nvmlDeviceGetCurrentClocksEventReasons(h)))
+            except Exception:
+                break
+            time.sleep(0.002)
 
     def start(self):
+        if self.nvml is not None:
+            import threading
+
+            self.thread = threading.Thread(target=self._loop, daemon=True)
+            self.thread.start()
+            return
         try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
                  "-i", str(self.gpu_index)], stdout=self.file, stderr=subprocess.DEVNULL)
@@ -84,6 +132,23 @@ class ClockSampler:
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.nvml is not None:
+            self.stop_flag = True
+            if self.thread is not None:
+                self.thread.join(timeout=2)
+            if self.samples:
+                sm = sorted(c for c, _ in self.samples)
+                bits = 0
+                for _, r in self.samples:
+                    bits |= int(r)
+                try:
+                    smax = self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM)
+                except Exception:
+                    smax = None
+                out.update(sm_mhz=float(sm[len(sm) // 2]), sm_max_mhz=float(smax) if smax else None,
+                           reasons=sorted(n for n, b in self.REASON_BITS.items() if bits & b),
+                           samples=len(sm), source="NVML every 2 ms, warm-up and timed region")
+            return out
         if self.proc is None:
             return out
         self.proc.terminate()  # the exact child started above
@@ -111,7 +176,8 @@ class ClockSampler:
         os.unlink(self.file.name)
         if sm:
             sm.sort()
-            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm),
+                       source="nvidia-smi -lms 100")
         return out
 
 
@@ -256,16 +322,16 @@ def run_ours(args, c, rank, world, local_rank):
         per = [evs[i].elapsed_time(evs[i + 1]) for i in range(steps)]
         return total_ms, per
 
+    # clocks are sampled from the first warm-up step to the end of the timed region: the GPU is
+    # under the benchmark's own load for all of it
+    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+    if sampler:
+        sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
     stream.synchronize()
     if ws.last_device_status(stream) != gf.GF_OK:
         raise SystemExit("device-side wait timed out during warm-up")
-
-    sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
-    if sampler:
-        sampler.start()
-        time.sleep(0.3)
     n0 = gf.launch_count()
     total_ms, per = timed(step, args.steps)
     launches = gf.launch_count() - n0
@@ -419,12 +485,11 @@ def run_decode(args, c, rank, world, local_rank):
         barrier()
         return e0.elapsed_time(e1)
 
-    for _ in range(max(args.warmup, 3)):
-        run_graph()
     sampler = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
     if sampler:
         sampler.start()
-        time.sleep(0.3)
+    for _ in range(max(args.warmup, 3)):
+        run_graph()
     n0 = gf.launch_count()
     total_ms = timed(run_graph, args.steps)
     clocks = sampler.stop() if sampler else None
