@@ -585,7 +585,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           PROF(1, nq, 0);
           if (j == 0) PROF3(n_items, 4);
           tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 2
           for (int ks = 0; ks < D / 16; ++ks)
             umma_ts(tmem + C::tP, tq + ks * 8,
                     umma_smem_desc(kbase + (ks >> 2) * C::kBoxBytes + (ks & 3) * 32, 16, 1024), id_p, ks > 0);
@@ -598,7 +598,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           ++n_sl;
           PROF(1, nq, 1);
           tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 2
           for (int ks = 0; ks < 8; ++ks)
             umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
                     umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, true);
@@ -612,7 +612,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           }
           PROF(1, nq, 2);
           tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 2
           for (int ks = 0; ks < D / 16; ++ks)
             umma_ts(tmem + C::tO, tq + ks * 8, umma_smem_desc(smem_u32(sSb) + ks * 2048, C::kSbBox, 1024), id_o,
                     ks > 0);
@@ -623,7 +623,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           ++n_pm;
           PROF(1, nq, 3);
           tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 2
           for (int ks = 0; ks < 8; ++ks)
             umma_ts(tmem + C::tO, tmem + C::tP + (ks >> 2) * 64 + (ks & 3) * 8,
                     umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
