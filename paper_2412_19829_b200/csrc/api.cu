@@ -277,6 +277,11 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
     if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
   }
   cudaStream_t wstream = both ? f->side : stream;
+  // Both kernels become runnable at the fork.  CTAs of the persistent linear kernel wait for one
+  // another and want every SM from the start, while a windowed-heads CTA that got onto an SM first
+  // keeps it for many tiles: hold the side stream back for a few microseconds, until the linear
+  // kernel's CTAs have been placed.
+  if (lin_first && cuda_status(gf::launch_delay(8000, wstream)) != GF_OK) return GF_ERR_CUDA;
   int rc2 = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, wstream);
   if (rc2 == GF_OK && state_out && h_sparse > 0)
     rc2 = cuda_status(gf::launch_export_ring(k, v, state_out->k_cache, state_out->v_cache, B, N, d, w, dtype,

@@ -56,6 +56,10 @@ cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void
                                void* v_cache, float* S, float* z, long long t, int B, int H, int d, int w,
                                int h_sparse, float scale, int dtype, cudaStream_t stream);
 
+// One tiny CTA that returns after about `ns` nanoseconds: holds back the work queued behind it
+// in its stream without occupying an SM's shared memory or tensor memory.
+cudaError_t launch_delay(unsigned int ns, cudaStream_t stream);
+
 // ---- tensor-core (tcgen05 / TMEM / TMA) path: bf16 storage, d in {64,128}.
 bool tc_window_supported(int N, int d, int w, int dtype);
 bool tc_linear_supported(int N, int d, int dtype);

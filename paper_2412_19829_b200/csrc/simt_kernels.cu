@@ -472,6 +472,24 @@ cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void
   return cudaGetLastError();
 }
 
+namespace {
+__global__ void delay_kernel(unsigned int ns) {
+  unsigned long long t0, t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  for (int i = 0; i < 100000; ++i) {  // bounded whatever the timer does
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    if (t - t0 >= ns) break;
+    __nanosleep(200);
+  }
+}
+}  // namespace
+
+cudaError_t launch_delay(unsigned int ns, cudaStream_t stream) {
+  delay_kernel<<<1, 32, 0, stream>>>(ns);
+  note_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
                                void* v_cache, float* S, float* z, long long t, int B, int H, int d, int w,
                                int h_sparse, float scale, int dtype, cudaStream_t stream) {
