@@ -28,9 +28,11 @@ def dev(*ts):
 def _reset_tuning():
     gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 0)
     gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0)
+    gf.set_tuning(gf.GF_TUNE_LINEAR_CTAS, 0)
     yield
     gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 0)
     gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0)
+    gf.set_tuning(gf.GF_TUNE_LINEAR_CTAS, 0)
 
 
 # ------------------------------------------------------------------ config 1: tiny fp32 hybrid
@@ -194,6 +196,46 @@ def test_run_to_run_determinism():
     a = gf.hybrid_attn(q, k, v, c["w"])
     b = gf.hybrid_attn(q, k, v, c["w"])
     assert torch.equal(a, b)
+
+
+# ------------------------------------------------------------------ persistent-kernel scheduling
+@pytest.mark.parametrize("d", [64, 128])
+def test_many_items_per_cta_ragged_tail(d):
+    # more work items than CTAs in both kernels (several items / query tiles per CTA, segments of
+    # unequal length, three-slot ring wrapping across items) and a sequence that ends mid-chunk;
+    # full size on the GPU, oracle on sampled heads (every head is an independent unit)
+    B, H, N, w = 2, 96, 2900, 300
+    h0 = gf.default_h_sparse(H)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=61, gain=1.0)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    o = gf.hybrid_attn(*dev(q, k, v), w, ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    assert torch.isfinite(o.float()).all()
+    wh = [0, h0 - 1]
+    assert_parity(f64(o[:, wh]), oracle.window_attn(f64(q[:, wh]), f64(k[:, wh]), f64(v[:, wh]), w), "bf16",
+                  "window heads")
+    lh = [h0, H // 2, H - 1]
+    assert_parity(f64(o[:, lh]), oracle.causal_linear_attn(f64(q[:, lh]), f64(k[:, lh]), f64(v[:, lh])), "bf16",
+                  "linear heads")
+
+
+@pytest.mark.parametrize("ctas", [1, 37, 100])
+def test_linear_cta_limit_gives_the_same_result(ctas):
+    # the segment plan follows the number of CTAs the persistent kernel is given; any count must
+    # reproduce the oracle (and, segment boundaries aside, the unrestricted call)
+    B, H, N, d, w = 1, 40, 4096, 128, 256
+    h0 = gf.default_h_sparse(H)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=67, gain=1.0)
+    qd, kd, vd = dev(q, k, v)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    full = gf.hybrid_attn(qd, kd, vd, w, ws=ws).cpu()
+    gf.set_tuning(gf.GF_TUNE_LINEAR_CTAS, ctas)
+    o = gf.hybrid_attn(qd, kd, vd, w, ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    assert torch.equal(o[:, :h0], full[:, :h0])  # the windowed heads do not depend on the plan
+    lh = [h0, H - 1]
+    ref = oracle.causal_linear_attn(f64(q[:, lh]), f64(k[:, lh]), f64(v[:, lh]))
+    assert_parity(f64(o[:, lh]), ref, "bf16", f"linear heads with {ctas} CTAs")
 
 
 # ------------------------------------------------------------------ config 2 (full tensors)
