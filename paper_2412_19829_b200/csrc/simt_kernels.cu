@@ -269,8 +269,9 @@ __device__ __forceinline__ float block_reduce(float x, bool is_max, float* scrat
   return scratch[32];
 }
 
+// Seven CTAs per SM: one CTA per (batch, head) then fits a batch of 64 x 16 heads in a single wave.
 template <typename T, int D>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 7)
 decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                    T* __restrict__ o, T* __restrict__ kc, T* __restrict__ vc, float* __restrict__ S,
                    float* __restrict__ z, long long t, int H, int w, int h_sparse, float scale) {
@@ -297,20 +298,26 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
       vcb[(long long)cur * D + tid] = v[io + tid];
     }
     __syncthreads();
-    // scores: one thread per slot; slot `cur` is read from the step input (same values).
+    // scores: D/4 threads per slot (a warp reads whole cache lines of the ring), partial dot
+    // products reduced over the group by shuffles; slot `cur` is read from the step input (same
+    // values).  D/4 is 16 or 32, so a group never straddles a warp.
     float mloc = -INFINITY;
-    for (int s = tid; s < nvalid; s += 256) {
-      const T* kr = (s == cur) ? (k + io) : (kcb + (long long)s * D);
+    const float4 qq = *reinterpret_cast<const float4*>(&qs[4 * c4]);
+    for (int s0 = 0; s0 < nvalid; s0 += G) {  // uniform trip count: the shuffles below are warp-wide
+      const int s = s0 + grp;
       float acc = 0.f;
-#pragma unroll
-      for (int c = 0; c < D4; ++c) {
-        const float4 kk = Vec4<T>::load(kr + 4 * c);
-        const float4 qq = *reinterpret_cast<const float4*>(&qs[4 * c]);
-        acc += qq.x * kk.x + qq.y * kk.y + qq.z * kk.z + qq.w * kk.w;
+      if (s < nvalid) {
+        const T* kr = (s == cur) ? (k + io) : (kcb + (long long)s * D);
+        const float4 kk = Vec4<T>::load(kr + 4 * c4);
+        acc = qq.x * kk.x + qq.y * kk.y + qq.z * kk.z + qq.w * kk.w;
       }
-      acc *= scale;
-      dyn[s] = acc;
-      mloc = fmaxf(mloc, acc);
+#pragma unroll
+      for (int off = D4 / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+      if (s < nvalid && c4 == 0) {
+        acc *= scale;
+        dyn[s] = acc;
+        mloc = fmaxf(mloc, acc);
+      }
     }
     const float mx = block_reduce(mloc, true, scratch);
     float lloc = 0.f;
