@@ -41,6 +41,30 @@ WORKLOADS = {
 }
 
 
+# ---- the multi-GPU contract ("replicas only"): every rank runs its own batch of the same shape on
+# its own GPU, nothing is exchanged on the data path; the job's time is the slowest rank's and its
+# throughput counts every rank's tokens.
+def replica_seed(c, rank):
+    """Seed of rank `rank`'s synthetic inputs (different data, same shapes)."""
+    return c["seed"] + 1000 * rank
+
+
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(world, units_per_rank_per_step, steps, slowest_ms):
+    """Whole-job units per second: all ranks' units over the slowest rank's time."""
+    return world * units_per_rank_per_step * steps / (slowest_ms * 1e-3)
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -283,7 +307,7 @@ def run_ours(args, c, rank, world, local_rank):
     h0 = gf.default_h_sparse(c["H"])
     B, H, N, d, w = c["B"], c["H"], c["N"], c["d"], c["w"]
 
-    q, k, v = synth.qkv(B, H, N, d, "bf16", c["seed"] + 1000 * rank)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", replica_seed(c, rank))
     hq, hk, hv = [t.pin_memory() for t in (q, k, v)]
     ho = torch.empty_like(hq).pin_memory()
     dq, dk, dv = [t.cuda() for t in (hq, hk, hv)]
@@ -360,15 +384,11 @@ def run_ours(args, c, rank, world, local_rank):
             kern[name] = {"ms_per_launch": ms / args.steps, "heads": heads,
                           "algorithmic_bytes": 4 * B * heads * N * d * 2}
 
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = t.tolist()
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, "cuda")
 
     if rank == 0:
-        tokens = world * B * N * args.steps
-        value = tokens / (total_ms * 1e-3)
-        e2e_value = tokens / (e2e_ms * 1e-3)
+        value = job_throughput(world, B * N, args.steps, total_ms)
+        e2e_value = job_throughput(world, B * N, args.steps, e2e_ms)
         peak, which = measured_peaks()
         abytes = algorithmic_bytes(c)
         mean_launch_s = (sum(per) / len(per)) * 1e-3
@@ -431,8 +451,8 @@ def run_decode(args, c, rank, world, local_rank):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     B, H, N, d, w, T = c["B"], c["H"], c["N"], c["d"], c["w"], c["decode_steps"]
     h0 = gf.default_h_sparse(H)
-    q, k, v = synth.qkv(B, H, N, d, "bf16", c["seed"] + 1000 * rank)
-    tq, tk, tv = synth.decode_tokens(T, B, H, d, "bf16", c["seed"] + 1000 * rank)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", replica_seed(c, rank))
+    tq, tk, tv = synth.decode_tokens(T, B, H, d, "bf16", replica_seed(c, rank))
     htok = [t.pin_memory() for t in (tq, tk, tv)]
     dtok = [t.cuda() for t in htok]
     dout = torch.empty_like(dtok[0])
@@ -497,10 +517,7 @@ def run_decode(args, c, rank, world, local_rank):
     eager_ms = timed(run_eager, args.steps)
     run_e2e()
     e2e_ms = timed(run_e2e, args.steps)
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms, eager_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms, eager_ms = t.tolist()
+    total_ms, e2e_ms, eager_ms = max_over_ranks([total_ms, e2e_ms, eager_ms], dist, "cuda")
     if rank == 0:
         tokens = world * B * T * args.steps
         peak, which = measured_peaks()
