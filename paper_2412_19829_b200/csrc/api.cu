@@ -251,7 +251,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   int lin_ctas = 0;
   if (both && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
     int L = 0, G = 0, dev = 0, sms = 0;
-    gf::linear_tc_plan(B * h_lin, N, g_linear_split, 0, &L, &G);
+    gf::linear_tc_plan(B * h_lin, N, d, g_linear_split, 0, &L, &G);
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return GF_ERR_CUDA;
     if ((long long)B * h_lin * G >= sms) {

@@ -69,7 +69,7 @@ cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* 
 // Segmentation used by the tensor-core linear kernel (split: 0 = automatic, else chunks per segment;
 // ctas: CTAs the kernel will run with, 0 = one per SM of a B200) and the scratch it needs beyond
 // the workspace header (sized for the largest segment count the plan may pick for any ctas).
-void linear_tc_plan(int nchains, int N, int split, int ctas, int* chunks_per_segment, int* segments_per_chain);
+void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* chunks_per_segment, int* segments_per_chain);
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split);
 // Bytes at the start of that scratch (right after the workspace header) that must be zero when the
 // kernel starts: the hand-over flags.  The caller clears them (together with the header).

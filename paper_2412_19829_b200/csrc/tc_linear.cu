@@ -36,6 +36,9 @@
 //                buffer (pass C)
 //   warp 23      polls the previous segment's flag and raises this segment's flag
 // TMEM (D=128): P 128 | O 128 | S 128 | phi(Q) 2 x 64 columns = 512.
+// When there are at least as many chains as CTAs no chain is cut (kDirect): an item is a whole
+// chain, there is no pass A, no parking and no hand-over; the phi warps transform each K tile in
+// place one chunk ahead of the chunk pipeline and keep the running column sums as they go.
 // Every wait is bounded; on expiry the kernel records a status word and drains.
 #include "common.cuh"
 #include "sm100.cuh"
@@ -113,6 +116,7 @@ struct LinBarriers {
   uint64_t qphi_full[2], qphi_free[2];
   uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done, sb_idle, sb_parked;
   uint64_t pm_full, den_full[2], s_loaded, sb_full, o_free, o_staged[2];
+  uint64_t kd_phi[2];  // kDirect: a K tile of the chunk pipeline is transformed and its column sums are posted
 };
 
 // Bounded poll of a monotonic counter in shared memory.
@@ -377,7 +381,7 @@ __device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinI
   return ok;
 }
 
-template <int D>
+template <int D, bool kDirect>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                  const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
@@ -396,6 +400,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   __shared__ __align__(16) float zin[2][D];
   __shared__ float den_s[2][2][128];  // [chunk parity][column half][row]: partial denominators, K group -> row group
   __shared__ float zpart[kMaxL][2][D];  // [tile of the segment][row half][column]: column sums of one K tile
+  __shared__ __align__(16) float zrun[2][D];  // kDirect: column sums of phi(K) over the chunks before chunk j, at [j & 1]
   __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
   __shared__ int zin_epoch;        // items whose zin is in place (monotonic)
   __shared__ int prev_epoch;       // items whose predecessor state has been seen in global memory (monotonic)
@@ -421,6 +426,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     }
     mbar_init(&bar.sb_idle, 1);
     mbar_init(&bar.sb_parked, 1);
+    mbar_init(&bar.kd_phi[0], 16);
+    mbar_init(&bar.kd_phi[1], 16);
     mbar_init(&bar.p_full, 1);
     mbar_init(&bar.s_full, 1);
     mbar_init(&bar.o_full, 1);
@@ -482,8 +489,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       const uint64_t pol_stream = l2_policy_evict_first(), pol_keep = l2_policy_evict_last();
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
-        for (int pass = 0; pass < 2 && ok; ++pass) {
-          if (pass == 1 && !mbar_wait(&bar.park_done, n_items & 1, p.status, 103)) { ok = false; break; }
+        for (int pass = kDirect ? 1 : 0; pass < 2 && ok; ++pass) {
+          if (!kDirect && pass == 1 && !mbar_wait(&bar.park_done, n_items & 1, p.status, 103)) { ok = false; break; }
           PROF3(n_items, pass);
           for (int j = 0; j < it.nC; ++j) {
             const int n0 = (it.c_begin + j) * 128;
@@ -507,9 +514,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               ok = drain(&bar.k_free[sc], obs_c[sc], iss_c[sc], 104) && drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101);
               if (!ok) break;
               mbar_arrive_expect_tx(&bar.k_full[sc], C::kTile);
-              for (int x = 0; x < D / 64; ++x)  // the phi(K) tile parked in the output rows
-                tma_load_4d_hint(sK + sc * C::kTile + x * C::kBoxBytes, &mo, &bar.k_full[sc], x * 64, n0, it.h, it.b,
-                                 pol_stream);
+              for (int x = 0; x < D / 64; ++x)  // the phi(K) tile parked in the output rows (kDirect: raw K)
+                tma_load_4d_hint(sK + sc * C::kTile + x * C::kBoxBytes, kDirect ? &mk : &mo, &bar.k_full[sc], x * 64, n0,
+                                 it.h, it.b, pol_stream);
               ++iss_c[sc];
               ++nq;
             }
@@ -548,7 +555,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         }
         first_item = false;
         // ---- pass A: dS = sum Kc^T V over the segment, from zero (only if somebody needs it)
-        for (int j = 0; j < it.nC; ++j) {
+        for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
           const uint32_t sa = ta % 3;
           if (!mbar_wait(&bar.kphi_full[sa], (ta / 3) & 1, p.status, 220)) { ok = false; break; }
           PROF(1, ta, 4);
@@ -577,8 +584,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           const int sv = nv & 1, sq = nq & 1;  // sq: slot of the K ring of this pass and of phi(Q)
           const uint32_t kbase = smem_u32(sK) + sq * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
           const uint32_t tq = tmem + C::tQ + sq * (D / 2);
+          // the chunk's phi(K) tile: read back from the park, or (kDirect) transformed in place
           if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 200) ||
-              !mbar_wait(&bar.k_full[sq], (nq >> 1) & 1, p.status, 201)) {
+              !mbar_wait(kDirect ? &bar.kd_phi[sq] : &bar.k_full[sq], (nq >> 1) & 1, p.status, 201)) {
             ok = false;
             break;
           }
@@ -649,7 +657,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       const int ip = n_items & 1;
       const long long slot = (long long)it.chain * p.G + it.g;
       // ---- hand-over of z: previous segment's inclusive z in, this segment's inclusive z out
-      na += it.nC;
+      if (!kDirect) na += it.nC;
       ok = wait_epoch(&ka_epoch, na, p.status, 311);
       ok = ok && wait_epoch(&prev_epoch, (int)n_items + 1, p.status, 312);
       if (named_bar_or(1, 128, !ok)) break;
@@ -658,7 +666,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (it.g > 0) z0 = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
         else if (p.z_io != nullptr && !p.zero_init) z0 = p.z_io[sidx * D + r];
         if (it.need_dS) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, z0 + zcum[ip][it.nC][r]);
-        if (it.last_seg && p.z_io != nullptr) p.z_io[sidx * D + r] = z0 + zcum[ip][it.nC][r];
+        if (!kDirect && it.last_seg && p.z_io != nullptr) p.z_io[sidx * D + r] = z0 + zcum[ip][it.nC][r];
         zin[ip][r] = z0;
       }
       if (it.need_dS) {
@@ -681,7 +689,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         nv += it.nC;
       }
       // Sb held K tiles in pass A: they have been parked (and, above, consumed by the tensor core)
-      ok = mbar_wait(&bar.sb_parked, n_items & 1, p.status, 314) && ok;
+      if (!kDirect) ok = mbar_wait(&bar.sb_parked, n_items & 1, p.status, 314) && ok;
       {
         const float* Sin = nullptr;
         long long sin_stride = 1;  // float4 units between consecutive column groups of one row
@@ -831,10 +839,32 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
       const int ip = n_items & 1;
-      if (kgrp && tt < D) zcum[ip][0][tt] = 0.f;
+      if (kgrp && tt < D) {
+        zcum[ip][0][tt] = 0.f;
+        if (kDirect) zrun[0][tt] = 0.f;
+      }
+      // kDirect: phi on this group's half of the K tile of chunk jrow (running index idx) of the
+      // chunk pipeline, in place; its column sums are posted before the tile is released, so
+      // whoever has seen the tile complete may read them.
+      auto transform_direct = [&](uint32_t idx, int jrow) {
+        const uint32_t sl = idx & 1;
+        ok = ok && mbar_wait(&bar.k_full[sl], (idx >> 1) & 1, p.status, 430);
+        const int cc = tt >> 4;
+        if (ok && tt < 2 * D) {
+          float cs[8];
+          transform_k_rows(sK + sl * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
+                           p.N - (it.c_begin + jrow) * 128, cs);
+          int col;
+          const float sum = reduce_column_sums(cs, tt & 15, &col);
+          if ((tt & 1) == 0) zpart[jrow & (kMaxL - 1)][kgrp ? 0 : 1][cc * 8 + col] = sum;
+        }
+        __syncwarp();
+        if (ok && lane == 0) mbar_arrive(&bar.kd_phi[sl]);
+      };
+      if (kDirect) transform_direct(nq, 0);
       // ---- pass A: the K group takes rows 0..63 (by sixteens) of every K tile, the Q group rows
       //      64..127; the K group also keeps the cumulative column sums
-      for (int j = 0; j < it.nC; ++j) {
+      for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
         const uint32_t sk = ta % 3;
         ok = ok && mbar_wait(&bar.ka_full[sk], (ta / 3) & 1, p.status, 410);
         if (tid == 14 * 32) PROF(3, ta, 4);
@@ -859,8 +889,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       }
 
       // both halves of every tile are done: running column sums over the segment's chunks
-      if (named_bar_or(4, 512, !ok)) break;
-      if (kgrp) {
+      if (!kDirect && named_bar_or(4, 512, !ok)) break;
+      if (!kDirect && kgrp) {
         if (tt < D) {
           float run = 0.f;
           for (int j = 0; j < it.nC; ++j) {
@@ -890,6 +920,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           const int sq = nq & 1;
           if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
           tc_fence_after_sync();
+          if (kDirect && tt == 0) PROF(3, nq, 4);
           // phi(q_i) . z_{c-1} over this warp's half of the head dimension, from the phi(Q) operand in
           // TMEM (the rounded values the tensor core sees); z before chunk j = zin + zcum[j]
           float part;
@@ -902,7 +933,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               tmem_ld16(tmem + C::tQ + sq * (D / 2) + lane_off + colh * W + pc * 16, qw);
               tmem_wait_ld();
               const float* za = zin[ip] + colh * (D / 2) + pc * 32;
-              const float* zb = zcum[ip][j] + colh * (D / 2) + pc * 32;
+              const float* zb = (kDirect ? zrun[j & 1] : zcum[ip][j]) + colh * (D / 2) + pc * 32;
+
 #pragma unroll
               for (int w = 0; w < 16; w += 2) {
                 const float4 a = *reinterpret_cast<const float4*>(za + 2 * w);
@@ -915,8 +947,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             }
             part = d0 + d1;
           }
+          // kDirect: this group's half of the next chunk's K tile, while the tensor core forms P
+          if (kDirect && tt == 0) PROF(3, nq, 5);
+          if (kDirect && j + 1 < it.nC) transform_direct(nq + 1, j + 1);
+          if (kDirect && tt == 0) PROF(3, nq, 6);
 
-          if (!mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
+          if (!ok || !mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
           if (tt == 0) PROF(2, nq, 0);
           tc_fence_after_sync();
 #pragma unroll 1
@@ -951,9 +987,19 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           tc_fence_before_sync();
           mbar_arrive(&bar.pm_full);
           if (tt == 0) PROF(2, nq, 1);
+          if (kDirect) {
+            // both halves of this chunk's tile have posted their column sums: z before the next chunk
+            ok = mbar_wait(&bar.kd_phi[sq], (nq >> 1) & 1, p.status, 431);
+            if (ok && tt < D)
+              zrun[(j + 1) & 1][tt] = zrun[j & 1][tt] + zpart[j & (kMaxL - 1)][0][tt] + zpart[j & (kMaxL - 1)][1][tt];
+            if (named_bar_or(3, 256, !ok)) { ok = false; break; }
+            if (tt == 0) PROF(3, nq, 7);
+          }
           ++nq;
         }
         if (!ok) break;
+        if (kDirect && tt < D && p.z_io != nullptr)
+          p.z_io[((long long)it.b * p.h_count + it.hl) * D + tt] = zin[ip][tt] + zrun[it.nC & 1][tt];
       } else {
         ok = !__any_sync(0xffffffffu, !ok);
         if (!ok) break;
@@ -1024,6 +1070,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             }
           }
           if (tid == 192) PROF(3, nq, 2);
+          if (kDirect && ok && j + 1 < it.nC) transform_direct(nq + 1, j + 1);
           ok = !__any_sync(0xffffffffu, !ok);
           ++nq;
         }
@@ -1042,7 +1089,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const LinItem it = decode_item(p, item);
         // ---- pass A: park phi(K) tiles in the output rows of their chunk
-        for (int j = 0; j < it.nC; ++j) {
+        for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
           const uint32_t sk = ta % 3;
           if (!mbar_wait(&bar.kphi_full[sk], (ta / 3) & 1, p.status, 520)) { ok = false; break; }
           for (int x = 0; x < D / 64; ++x)
@@ -1141,6 +1188,9 @@ bool tc_linear_supported(int N, int d, int dtype) {
 // hand-over, about 0.7 chunk).  The plan must not depend on the device that is current when the
 // workspace size is asked for, so without a CTA count it assumes the 148 SMs of a B200.
 namespace {
+// cost of a chunk of an uncut chain, in two-pass chunks (measured: with d = 64 the one pass is
+// bound by the same mask and conversion work per chunk as the second of two, so it gains nothing)
+constexpr double direct_chunk_cost(int d) { return d == 128 ? 0.72 : 1.05; }
 // Range of segment counts the automatic plan chooses from.
 void plan_range(int nchains, int nch, int* g_min_out, int* g_max_out) {
   const int g_min = (nch + kMaxL - 1) / kMaxL;
@@ -1157,7 +1207,7 @@ void plan_range(int nchains, int nch, int* g_min_out, int* g_max_out) {
 }
 }  // namespace
 
-void linear_tc_plan(int nchains, int N, int split, int ctas, int* L_out, int* G_out) {
+void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, int* G_out) {
   const int nch = (N + 127) / 128;
   int G;
   if (split > 0) {
@@ -1177,6 +1227,11 @@ void linear_tc_plan(int nchains, int N, int split, int ctas, int* L_out, int* G_
         G = g;
       }
     }
+    // An uncut chain needs neither the first pass nor a hand-over (the kernel transforms K inside
+    // the chunk pipeline): a chunk then costs direct_chunk_cost(d) of a two-pass one.  With many
+    // chains that is the cheaper plan even though a CTA then walks a whole chain.
+    const long long rounds1 = ((long long)nchains + kPlanSMs - 1) / kPlanSMs;
+    if ((double)rounds1 * nch * direct_chunk_cost(d) <= best) G = 1;
   }
   if (G < 1) G = 1;
   *G_out = G;
@@ -1187,7 +1242,7 @@ namespace {
 // Largest segment count the plan may pick (the scratch is laid out for it).
 int plan_g_max(int nchains, int N, int split) {
   int L, G;
-  linear_tc_plan(nchains, N, split, 0, &L, &G);
+  linear_tc_plan(nchains, N, 128, split, 0, &L, &G);
   if (split <= 0) {
     int g_min;
     plan_range(nchains, (N + 127) / 128, &g_min, &G);
@@ -1227,7 +1282,7 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   // (max_ctas > 0 leaves SMs to a kernel running beside this one.)
   if (max_ctas > 0 && max_ctas < sms) sms = max_ctas;
   int L_max = 0;
-  linear_tc_plan(p.nchains, N, split, sms, &L_max, &p.G);
+  linear_tc_plan(p.nchains, N, d, split, sms, &L_max, &p.G);
   p.seg_base = p.nch / p.G;
   p.seg_rem = p.nch % p.G;
   p.nitems = p.nchains * p.G;
@@ -1239,17 +1294,21 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   p.flags = reinterpret_cast<unsigned int*>(scratch);  // zeroed by the caller
   p.prefix = reinterpret_cast<float*>(scratch + linear_tc_flag_bytes(p.nchains, N, split));
   dim3 grid(p.nitems < sms ? p.nitems : sms);
-  if (d == 64) {
-    auto kern = linear_tc_kernel<64>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, LinCfg<64>::kBytes);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, LinCfg<64>::kBytes, stream>>>(mq, mk, mv, mo, p);
-  } else {
-    auto kern = linear_tc_kernel<128>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, LinCfg<128>::kBytes);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, LinCfg<128>::kBytes, stream>>>(mq, mk, mv, mo, p);
-  }
+  // automatic plan, chains left whole: the one-pass form of the kernel (a segment length asked
+  // for by the caller always takes the two-pass form, also when it covers the whole chain)
+  const bool direct = split <= 0 && p.G == 1;
+  auto launch = [&](auto kern, size_t smem) -> cudaError_t {
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    kern<<<grid, kThreads, smem, stream>>>(mq, mk, mv, mo, p);
+    return cudaSuccess;
+  };
+  if (d == 64)
+    e = direct ? launch(linear_tc_kernel<64, true>, LinCfg<64>::kBytes) : launch(linear_tc_kernel<64, false>, LinCfg<64>::kBytes);
+  else
+    e = direct ? launch(linear_tc_kernel<128, true>, LinCfg<128>::kBytes)
+               : launch(linear_tc_kernel<128, false>, LinCfg<128>::kBytes);
+  if (e != cudaSuccess) return e;
   note_launch();
   return cudaGetLastError();
 }
