@@ -5,8 +5,12 @@
 //   P   = Qc Kc^T                       (MMA1)   masked to j <= i           -> Pm (bf16)
 //   S_c = S_{c-1} + Kc^T V_c            (MMA4)   fp32 master copy lives in TMEM for the whole chain
 //   O   = Qc Sb_{c-1}  (+)  Pm V_c      (MMA2, MMA3)  Sb = bf16 copy of S in shared memory
-//   den = rowsum(Pm) + Qc z_{c-1},  z_c = z_{c-1} + colsum(Kc)      (fp32, CUDA cores)
+//   den = rowsum(Pm) + Qc z_{c-1},  z_c = z_{c-1} + colsum(Kc)
 //   out = O / den
+// The denominators ride on the same tensor-core products as one extra column: z is the column
+// "V = 1" of the state (MMA4 with a constant B tile whose row 0 is all ones gives colsum(Kc) in
+// fp32), Qc z_{c-1} is the readout of that column (MMA2 against z split in two bf16 terms, hi +
+// lo, so that it carries 16 bits), and rowsum(Pm) comes from MMA3 with the ones tile again.
 // A (batch, head) chain is cut into segments of L chunks; a work item is one segment.  CTAs are
 // persistent and take items round-robin in an order in which a segment's predecessor always has
 // a smaller index, so the CTA that owns it is already running.  For an item the CTA
@@ -23,22 +27,20 @@
 //   warp 0       TMA producer (raw Q, K, V tiles; K and V double buffered)
 //   warp 1       MMA issuer
 //   warps 2-5    "row group" (one thread per row): loads the state before the segment; pass C:
-//                converts S to bf16 for the next chunk's readout, divides O by the denominator
-//                and stages it for the store
+//                converts S (and z) to bf16 for the next chunk's readout, divides O by the
+//                denominator and stages it for the store; hands z over between segments
 //   warps 6-13   "Q group": pass C: applies phi to Q; the result goes to TMEM as the A operand of
-//                MMA1/MMA2, together with the per-row dot product with z_{c-1};
-//                pass A: transforms half of every K tile
+//                MMA1/MMA2; pass A: transforms half of every K tile
 //   warps 14-21  "K group": pass A: applies phi to the other half of every K tile (in place in
-//                shared memory) and keeps the cumulative column sums; pass C: masks/packs P in
-//                TMEM (two warps per TMEM lane quarter, half of the key columns each) and forms
-//                the row sums for the denominators
+//                shared memory); pass C: masks/packs P in TMEM (two warps per TMEM lane quarter,
+//                half of the key columns each)
 //   warp 22      TMA stores: parks phi(K) tiles (pass A), stores O tiles staged in the dead V
 //                buffer (pass C)
 //   warp 23      polls the previous segment's flag and raises this segment's flag
-// TMEM (D=128): P 128 | O 128 | S 128 | phi(Q) 2 x 64 columns = 512.
+// TMEM (D=128): P 128 | O 128 | S 128 | phi(Q) 64 | denominators 16 | z 16 columns = 480.
 // When there are at least as many chains as CTAs no chain is cut (kDirect): an item is a whole
 // chain, there is no pass A, no parking and no hand-over; the phi warps transform each K tile in
-// place one chunk ahead of the chunk pipeline and keep the running column sums as they go.
+// place one chunk ahead of the chunk pipeline.
 // Every wait is bounded; on expiry the kernel records a status word and drains.
 #include "common.cuh"
 #include "sm100.cuh"
@@ -49,26 +51,42 @@ namespace {
 using namespace sm100;
 
 constexpr int kThreads = 768;  // 24 warps, 80 registers each
-constexpr int kMaxL = 8;       // chunks per segment (bounded by the per-segment z history kept in shared memory)
+constexpr int kMaxL = 8;       // chunks per segment of a cut chain
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kFlagStride = 32;  // one flag per 128-byte line
 
 template <int D>
 struct LinCfg {
   static constexpr int kTile = 128 * D * 2;  // one 128 x D bf16 tile
-  static constexpr int kQ = 0;               // raw Q landing buffer
-  static constexpr int kK = kTile;           // 2 stages
-  static constexpr int kV = 3 * kTile;       // 2 stages
-  static constexpr int kSb = 5 * kTile;      // bf16 copy of S, [D rows][D cols] in 64-column boxes
+  static constexpr int kBoxBytes = 16384;    // one 128-row x 64-column box (what one TMA copy moves)
+  static constexpr int kSbBox = D * 128;     // one D-row x 64-column box of Sb
   static constexpr int kSbBytes = D * D * 2;
+  // The denominators ride along as 16 extra output columns (N = D + 16) of MMA2, MMA3 and MMA4,
+  // whose B operands are rows of 64-column boxes a fixed distance (the descriptor's leading
+  // byte offset) apart: V | ones and Sb | Zb.  The constant ones box (column 0 = 1) serves both
+  // V slots, so it must lie one box distance past the last box of either: with B = kBoxBytes,
+  //   D = 128:  V0a Q0 V1a V0b V1b Q1 ONES   (V0: distance 3B, V1: 2B; the Q boxes fill the holes)
+  //   D = 64:   V0 V1 ONES                   (V0: distance 2B, V1: 1B)
+  static constexpr int kV0 = 0;
+  static constexpr int kV1 = (D == 128) ? 2 * kBoxBytes : kBoxBytes;
+  static constexpr int kVLbo0 = (D == 128) ? 3 * kBoxBytes : 2 * kBoxBytes;
+  static constexpr int kVLbo1 = (D == 128) ? 2 * kBoxBytes : kBoxBytes;
+  static constexpr int kOnes = (D == 128) ? 6 * kBoxBytes : 2 * kBoxBytes;
+  static constexpr int kQ = (D == 128) ? kBoxBytes : 3 * kBoxBytes;  // raw Q landing buffer
+  static constexpr int kQStride = 4 * kBoxBytes;                     // between its boxes (D = 128)
+  static constexpr int kK = (D == 128) ? 7 * kBoxBytes : 4 * kBoxBytes;  // 2 stages, contiguous
+  static constexpr int kSb = kK + 2 * kTile;  // bf16 copy of S, [D rows][D cols] in 64-column boxes
+  static constexpr int kZb = kSb + kSbBytes;  // one more such box: column 0 = hi(z), column 1 = lo(z)
   // Pass A runs its K tiles through three slots: the two K slots and, third, the Sb buffer, which
   // is idle in that pass (at D = 64 Sb is smaller than a tile, so the third slot gets its own room)
-  static constexpr int kKA2 = (D == 128) ? kSb : kSb + kSbBytes;
-  static constexpr int kBytes = 5 * kTile + kSbBytes + (D == 128 ? 0 : kTile) + 1024;
-  static constexpr int kBoxBytes = 16384;    // one 128-row x 64-column box
-  static constexpr int kSbBox = D * 128;     // one D-row x 64-column box of Sb
+  static constexpr int kKA2 = (D == 128) ? kSb : kZb + kSbBox;
+  static constexpr int kBytes = ((D == 128) ? kZb + kSbBox : kKA2 + kTile) + 1024;
   // TMEM columns
-  static constexpr uint32_t tP = 0, tO = 128, tS = 128 + D, tQ = 128 + 2 * D;  // tQ: 2 x D/2
+  static constexpr int kQSlots = (D == 128) ? 1 : 2;  // phi(Q) operands in flight
+  static constexpr int kNExt = D + 16;                // S and O with the denominator columns
+  static constexpr uint32_t tP = 0, tO = 128, tS = 128 + kNExt, tQ = 128 + 2 * kNExt;  // tQ: kQSlots x D/2
+  static constexpr uint32_t tOz = tO + D;  // [0] = Qc hi(z) + rowsum(Pm), [1] = Qc lo(z)
+  static constexpr uint32_t tSz = tS + D;  // [0] = z (row = feature), the others stay zero
   static constexpr uint32_t kTmemCols = 512;
   // One published state: S then z.  S is stored [column/4][128 rows][4] so that the threads of a
   // warp (one row each, the TMEM lane order) touch consecutive 16-byte pieces.
@@ -115,8 +133,8 @@ struct LinBarriers {
   uint64_t v_full[2], v_free[2];                  // V tiles of both passes (slot = tile count & 1)
   uint64_t qphi_full[2], qphi_free[2];
   uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done, sb_idle, sb_parked;
-  uint64_t pm_full, den_full[2], s_loaded, sb_full, o_free, o_staged[2];
-  uint64_t kd_phi[2];  // kDirect: a K tile of the chunk pipeline is transformed and its column sums are posted
+  uint64_t pm_full, s_loaded, sb_full, s_final, o_free, o_staged[2];
+  uint64_t kd_phi[2];  // kDirect: a K tile of the chunk pipeline has been transformed in place
 };
 
 // Bounded poll of a monotonic counter in shared memory.
@@ -254,16 +272,10 @@ __device__ __forceinline__ uint32_t phi_bf16x2(uint32_t w) {
   const __nv_bfloat162 f = __hadd2(__hmax2(x, zero), *reinterpret_cast<const __nv_bfloat162*>(&e));
   return *reinterpret_cast<const uint32_t*>(&f);
 }
-__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// phi on rows {lane16 + 16 k8 : k8 in [k8_begin, k8_begin + 4)} x one 16-byte column chunk of a K
-// tile, in place, plus this thread's share of the column sums of those rows (to be reduced over
-// the 16 lanes that share the column chunk).  Rows at or past n_valid become 0.
-__device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane16, int k8_begin, int n_valid,
-                                                 float (&cs)[8]) {
-#pragma unroll
-  for (int e = 0; e < 8; ++e) cs[e] = 0.f;
+// phi on 64 rows (four groups of 16 from k8_begin on) x one 16-byte column chunk of a K tile, in
+// place in shared memory (128B swizzle); rows past the end of the sequence become zero.
+__device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane16, int k8_begin, int n_valid) {
   uint4 rawv[4];
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
@@ -274,14 +286,10 @@ __device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane1
   for (int k = 0; k < 4; ++k) {
     const int row = lane16 + 16 * (k8_begin + k);
     const uint32_t keep = (row < n_valid) ? 0xffffffffu : 0u;
-    uint32_t w4[4] = {rawv[k].x, rawv[k].y, rawv[k].z, rawv[k].w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      w4[e] = phi_bf16x2(w4[e]) & keep;
-      cs[2 * e] += bf16_lo(w4[e]);
-      cs[2 * e + 1] += bf16_hi(w4[e]);
-    }
-    rawv[k] = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+    rawv[k].x = phi_bf16x2(rawv[k].x) & keep;
+    rawv[k].y = phi_bf16x2(rawv[k].y) & keep;
+    rawv[k].z = phi_bf16x2(rawv[k].z) & keep;
+    rawv[k].w = phi_bf16x2(rawv[k].w) & keep;
   }
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
@@ -289,32 +297,6 @@ __device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane1
     *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k];
   }
   fence_proxy_async_smem();
-}
-
-// Column sums of transform_k_rows reduced over the 16 lanes that share a column chunk, as a
-// reduce-scatter (8 shuffles instead of 32): every step halves the columns a lane still carries.
-// Returns the sum of column `*col` (0..7 within the chunk: bits 3, 2, 1 of lane16; the two lanes
-// of a pair end with the same value).
-__device__ __forceinline__ float reduce_column_sums(const float (&cs)[8], int lane16, int* col) {
-  const bool b3 = lane16 & 8, b2 = lane16 & 4, b1 = lane16 & 2;
-  float a[4], b[2];
-#pragma unroll
-  for (int e = 0; e < 4; ++e) {
-    const float send = b3 ? cs[e] : cs[e + 4];
-    const float keep = b3 ? cs[e + 4] : cs[e];
-    a[e] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-  }
-#pragma unroll
-  for (int e = 0; e < 2; ++e) {
-    const float send = b2 ? a[e] : a[e + 2];
-    const float keep = b2 ? a[e + 2] : a[e];
-    b[e] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-  }
-  const float send = b1 ? b[0] : b[1];
-  float c = (b1 ? b[1] : b[0]) + __shfl_xor_sync(0xffffffffu, send, 2);
-  c += __shfl_xor_sync(0xffffffffu, c, 1);
-  *col = (b3 ? 4 : 0) + (b2 ? 2 : 0) + (b1 ? 1 : 0);
-  return c;
 }
 
 // Critical path of the segment hand-over, run by the 16 phi warps (4 per TMEM lane quarter, each
@@ -389,20 +371,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   using C = LinCfg<D>;
   extern __shared__ uint8_t raw_smem[];
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw_smem) + 1023) & ~(uintptr_t)1023);
-  uint8_t* sQ = sm + C::kQ;
   uint8_t* sK = sm + C::kK;
-  uint8_t* sV = sm + C::kV;
+  // box x of V slot sv (also the staging buffer of the O tile), of the Q landing buffer
+  auto v_box = [&](int sv, int x) -> uint8_t* { return sm + (sv ? C::kV1 + x * C::kVLbo1 : C::kV0 + x * C::kVLbo0); };
+  auto q_box = [&](int x) -> uint8_t* { return sm + C::kQ + x * C::kQStride; };
   uint8_t* sSb = sm + C::kSb;
   __shared__ __align__(8) LinBarriers bar;
-  // per item parity: zcum[j] = column sums of phi(K) over the first j chunks of the segment,
-  // zin = z before the segment
-  __shared__ __align__(16) float zcum[2][kMaxL + 1][D];
-  __shared__ __align__(16) float zin[2][D];
-  __shared__ float den_s[2][2][128];  // [chunk parity][column half][row]: partial denominators, K group -> row group
-  __shared__ float zpart[kMaxL][2][D];  // [tile of the segment][row half][column]: column sums of one K tile
-  __shared__ __align__(16) float zrun[2][D];  // kDirect: column sums of phi(K) over the chunks before chunk j, at [j & 1]
-  __shared__ int ka_epoch;         // pass-A tiles whose phi(K) and column sums are complete (monotonic)
-  __shared__ int zin_epoch;        // items whose zin is in place (monotonic)
+  uint8_t* sOnes = sm + C::kOnes;
+  uint8_t* sZb = sm + C::kZb;
   __shared__ int prev_epoch;       // items whose predecessor state has been seen in global memory (monotonic)
   __shared__ int q_copied;         // Q-group warps that have copied their part of a Q tile out of the landing buffer (monotonic)
   __shared__ uint32_t tmem_base_s;
@@ -436,15 +412,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.pub_done, 20);  // 16 phi warps + 4 P-group warps
     mbar_init(&bar.park_done, 1);
     mbar_init(&bar.pm_full, 256);
-    mbar_init(&bar.den_full[0], 256);
-    mbar_init(&bar.den_full[1], 256);
-    mbar_init(&bar.s_loaded, 128);
-    mbar_init(&bar.sb_full, 128);
+    mbar_init(&bar.s_loaded, 256);
+    mbar_init(&bar.sb_full, 256);
+    mbar_init(&bar.s_final, 256);
     mbar_init(&bar.o_free, 128);
     mbar_init(&bar.o_staged[0], 128);
     mbar_init(&bar.o_staged[1], 128);
-    ka_epoch = 0;
-    zin_epoch = 0;
     prev_epoch = 0;
     q_copied = 0;
     mbar_fence_init();
@@ -456,6 +429,15 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   if (warp == 1) {
     tmem_alloc(&tmem_base_s, C::kTmemCols);
     tmem_relinquish();
+  } else if (warp >= 2) {
+    // constant ones box: column 0 of every key row is 1 (128B swizzle: the row's first 16-byte
+    // chunk sits at position row & 7), all else 0; z operand cleared
+    for (int i = tid - 64; i < C::kBoxBytes / 4; i += kThreads - 64) {
+      const int row = i >> 5, w = i & 31;
+      reinterpret_cast<uint32_t*>(sOnes)[i] = (w == ((row & 7) << 2)) ? 0x00003F80u : 0u;
+    }
+    for (int i = tid - 64; i < C::kSbBox / 4; i += kThreads - 64) reinterpret_cast<uint32_t*>(sZb)[i] = 0u;
+    fence_proxy_async_smem();
   }
   tc_fence_before_sync();
   __syncthreads();
@@ -525,7 +507,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               if (nv >= 2 && !mbar_wait(&bar.v_free[sv], ((nv >> 1) + 1) & 1, p.status, 102)) { ok = false; break; }
               mbar_arrive_expect_tx(&bar.v_full[sv], C::kTile);
               for (int x = 0; x < D / 64; ++x)
-                tma_load_4d_hint(sV + sv * C::kTile + x * C::kBoxBytes, &mv, &bar.v_full[sv], x * 64, n0, it.h, it.b,
+                tma_load_4d_hint(v_box(sv, x), &mv, &bar.v_full[sv], x * 64, n0, it.h, it.b,
                                  pass == 0 ? pol_keep : pol_stream);
               ++nv;
             }
@@ -538,9 +520,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     // ================================================================ MMA issuer
     if (elect_one()) {
       constexpr uint32_t id_p = umma_idesc_bf16(128, 128, false, false);  // P  = Qc Kc^T
-      constexpr uint32_t id_s = umma_idesc_bf16(128, D, true, true);      // S += Kc^T V
-      constexpr uint32_t id_o = umma_idesc_bf16(128, D, false, true);     // O  = Qc Sb,  O += Pm V
+      constexpr uint32_t id_s = umma_idesc_bf16(128, C::kNExt, true, true);   // [S | z] += Kc^T [V | 1]
+      constexpr uint32_t id_o = umma_idesc_bf16(128, C::kNExt, false, true);  // [O | den] = Qc [Sb | Zb], += Pm [V | 1]
       constexpr uint32_t kLboA = (D == 128) ? C::kBoxBytes : 0;           // D=64: rows 64..127 of S mirror 0..63
+      constexpr int QS = C::kQSlots;
       uint32_t ta = 0, nv = 0, nq = 0, n_sl = 0, n_sb = 0, n_of = 0, n_pm = 0;
       bool ok = true, first_item = true;
       [[maybe_unused]] uint32_t n_items = 0;
@@ -561,13 +544,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           PROF(1, ta, 4);
           if (it.need_dS) {
             const int sv = nv & 1;
-            const uint32_t kbase = smem_u32(a_kslot(sa)), vbase = smem_u32(sV) + sv * C::kTile;
+            const uint32_t kbase = smem_u32(a_kslot(sa)), vbase = smem_u32(v_box(sv, 0));
+            const uint32_t vlbo = sv ? C::kVLbo1 : C::kVLbo0;
             if (!mbar_wait(&bar.v_full[sv], (nv >> 1) & 1, p.status, 221)) { ok = false; break; }
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
               umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
-                      umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, (j > 0) || (ks > 0));
+                      umma_smem_desc(vbase + ks * 2048, vlbo, 1024), id_s, (j > 0) || (ks > 0));
             PROF(1, ta, 5);
             umma_commit(&bar.ka_free[sa]);  // second arrival: the store warp, once the tile is parked
             umma_commit(&bar.v_free[sv]);
@@ -581,12 +565,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (it.need_dS) umma_commit(&bar.a_done);
         // ---- pass C
         for (int j = 0; j < it.nC; ++j) {
-          const int sv = nv & 1, sq = nq & 1;  // sq: slot of the K ring of this pass and of phi(Q)
-          const uint32_t kbase = smem_u32(sK) + sq * C::kTile, vbase = smem_u32(sV) + sv * C::kTile;
+          const int sv = nv & 1, sk = nq & 1, sq = nq % QS;  // slots of the V ring, of this pass's K ring, of phi(Q)
+          const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(v_box(sv, 0));
+          const uint32_t vlbo = sv ? C::kVLbo1 : C::kVLbo0;
           const uint32_t tq = tmem + C::tQ + sq * (D / 2);
           // the chunk's phi(K) tile: read back from the park, or (kDirect) transformed in place
-          if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 200) ||
-              !mbar_wait(kDirect ? &bar.kd_phi[sq] : &bar.k_full[sq], (nq >> 1) & 1, p.status, 201)) {
+          if (!mbar_wait(&bar.qphi_full[sq], (nq / QS) & 1, p.status, 200) ||
+              !mbar_wait(kDirect ? &bar.kd_phi[sk] : &bar.k_full[sk], (nq >> 1) & 1, p.status, 201)) {
             ok = false;
             break;
           }
@@ -598,6 +583,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             umma_ts(tmem + C::tP, tq + ks * 8,
                     umma_smem_desc(kbase + (ks >> 2) * C::kBoxBytes + (ks & 3) * 32, 16, 1024), id_p, ks > 0);
           umma_commit(&bar.p_full);
+          PROF(1, nq, 6);
           if (!mbar_wait(&bar.v_full[sv], (nv >> 1) & 1, p.status, 202) ||
               !mbar_wait(&bar.s_loaded, n_sl & 1, p.status, 203)) {
             ok = false;
@@ -609,9 +595,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 #pragma unroll 2
           for (int ks = 0; ks < 8; ++ks)
             umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
-                    umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024), id_s, true);
+                    umma_smem_desc(vbase + ks * 2048, vlbo, 1024), id_s, true);
           umma_commit(&bar.s_full);
-          umma_commit(&bar.k_free[sq]);
+          umma_commit(&bar.k_free[sk]);
           if (!mbar_wait(&bar.sb_full, n_sb & 1, p.status, 204)) { ok = false; break; }
           ++n_sb;
           if (nq >= 1) {
@@ -634,9 +620,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 #pragma unroll 2
           for (int ks = 0; ks < 8; ++ks)
             umma_ts(tmem + C::tO, tmem + C::tP + (ks >> 2) * 64 + (ks & 3) * 8,
-                    umma_smem_desc(vbase + ks * 2048, C::kBoxBytes, 1024),
+                    umma_smem_desc(vbase + ks * 2048, vlbo, 1024),
                     id_o, true);
           umma_commit(&bar.o_full);
+          PROF(1, nq, 7);
           ++nv;
           ++nq;
         }
@@ -648,37 +635,36 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const int r = quarter * 32 + lane;
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     const bool s_row = r < D;  // rows of S are feature indices a < D
+    // this feature's row of the z operand: columns 0 and 1 = hi(z), lo(z) (16 bits between them)
+    uint32_t* zb_word = reinterpret_cast<uint32_t*>(sZb + swz128_offset(r, 0));
+    auto put_z = [&](float z) {
+      const float hi = __bfloat162float(__float2bfloat16_rn(z));
+      *zb_word = pack_bf16(hi, z - hi);
+    };
     uint32_t nv = 0, nq = 0, n_a = 0, n_items = 0;
-    int na = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < p.nitems; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
       const long long sidx = (long long)it.b * p.h_count + it.hl;
-      const int ip = n_items & 1;
       const long long slot = (long long)it.chain * p.G + it.g;
-      // ---- hand-over of z: previous segment's inclusive z in, this segment's inclusive z out
-      if (!kDirect) na += it.nC;
-      ok = wait_epoch(&ka_epoch, na, p.status, 311);
+      // ---- hand-over of z (column 0 of tSz, one feature per thread): this segment's own sum is
+      //      there after pass A; previous segment's inclusive z in, this segment's inclusive z out
+      if (it.need_dS) ok = mbar_wait(&bar.a_done, n_a & 1, p.status, 311);
       ok = ok && wait_epoch(&prev_epoch, (int)n_items + 1, p.status, 312);
       if (named_bar_or(1, 128, !ok)) break;
+      float z0 = 0.f;
       if (s_row) {
-        float z0 = 0.f;
         if (it.g > 0) z0 = __ldcg(p.prefix + (slot - 1) * C::kStateFloats + C::kStateZ + r);
         else if (p.z_io != nullptr && !p.zero_init) z0 = p.z_io[sidx * D + r];
-        if (it.need_dS) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, z0 + zcum[ip][it.nC][r]);
-        if (!kDirect && it.last_seg && p.z_io != nullptr) p.z_io[sidx * D + r] = z0 + zcum[ip][it.nC][r];
-        zin[ip][r] = z0;
       }
       if (it.need_dS) {
+        tc_fence_after_sync();
+        const float dz = __uint_as_float(tmem_ld1(tmem + C::tSz + lane_off));
+        tmem_wait_ld();
+        if (s_row) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, z0 + dz);
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar.pub_done);
         PROF2(tid == 64 && n_items == 0, 5);
-      }
-      if (named_bar_or(1, 128, false)) break;
-      if (tid == 64) {
-        __threadfence_block();
-        *reinterpret_cast<volatile int*>(&zin_epoch) = (int)n_items + 1;
-        PROF2(n_items == 0, 6);
       }
       // ---- hand-over of S: the 16 phi warps publish the inclusive state (they read dS from TMEM:
       //      do not overwrite it before they are done); this group loads the state before the segment
@@ -690,6 +676,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       }
       // Sb held K tiles in pass A: they have been parked (and, above, consumed by the tensor core)
       if (!kDirect) ok = mbar_wait(&bar.sb_parked, n_items & 1, p.status, 314) && ok;
+      // the K group has read the previous item's last state out of TMEM
+      if (n_items > 0) ok = mbar_wait(&bar.s_final, (n_items - 1) & 1, p.status, 315) && ok;
+      tc_fence_after_sync();
       {
         const float* Sin = nullptr;
         long long sin_stride = 1;  // float4 units between consecutive column groups of one row
@@ -713,6 +702,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             v[jj + 3] = __float_as_uint(in.w);
           }
           tmem_st32(tmem + C::tS + lane_off + cc * 32, v);
+          if (cc == 0) {
+            uint32_t zc[16];
+#pragma unroll
+            for (int jj = 1; jj < 16; ++jj) zc[jj] = 0u;
+            zc[0] = __float_as_uint(z0);
+            tmem_st16(tmem + C::tSz + lane_off, zc);
+            if (s_row) put_z(z0);
+          }
           if (s_row) {
 #pragma unroll
             for (int g = 0; g < 4; ++g) {
@@ -728,65 +725,23 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         tmem_wait_st();
         fence_proxy_async_smem();
         tc_fence_before_sync();
-        mbar_arrive(&bar.s_loaded);
-        mbar_arrive(&bar.sb_full);
+        mbar_arrive_cnt(&bar.s_loaded, 2);  // these barriers count the K group's 256 threads
+        mbar_arrive_cnt(&bar.sb_full, 2);
       }
       // ---- pass C
       for (int j = 0; j < it.nC; ++j) {
-        const int sv = nv & 1, sq = nq & 1;
-        // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
-        //      bf16 copy, stream the new one into shared memory for the next chunk
-        if (!mbar_wait(&bar.s_full, nq & 1, p.status, 302) || !mbar_wait(&bar.mma2_done, nq & 1, p.status, 303)) {
-          ok = false;
-          break;
-        }
-        if (tid == 64) PROF(2, nq, 2);
-        tc_fence_after_sync();
-        // after the item's last chunk nobody reads Sb again (it may already hold a K tile of the
-        // next item's pass A), and only a chain's last segment still wants the state itself
-        const bool last_chunk = (j == it.nC - 1);
-        const bool write_final = it.last_seg && last_chunk && p.S_io != nullptr;
-#pragma unroll(D == 128 ? 1 : 2)
-        for (int cc = 0; cc < D / 32; ++cc) {
-          if (last_chunk && !write_final) break;
-          uint32_t v[32];
-          tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
-          tmem_wait_ld();
-          if (s_row && !last_chunk) {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              uint4 val;
-              val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
-              val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
-              val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
-              val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
-              *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
-            }
-          }
-          if (s_row && write_final) {
-            float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
-#pragma unroll
-            for (int jj = 0; jj < 32; jj += 4)
-              *reinterpret_cast<float4*>(dst + jj) =
-                  make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
-                              __uint_as_float(v[jj + 3]));
-          }
-        }
-        tc_fence_before_sync();
-        mbar_arrive(&bar.s_loaded);
-        fence_proxy_async_smem();
-        mbar_arrive(&bar.sb_full);
-        if (tid == 64) PROF(2, nq, 5);
+        const int sv = nv & 1;
         // ---- O: divide by the denominator, bf16, stage for the TMA store
-        if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304) ||
-            !mbar_wait(&bar.den_full[sq], (nq >> 1) & 1, p.status, 305)) {
+        if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304)) {
           ok = false;
           break;
         }
         if (tid == 64) PROF(2, nq, 6);
         tc_fence_after_sync();
-        const float inv = 1.f / (den_s[sq][0][r] + den_s[sq][1][r]);
-        uint8_t* stage = sV + sv * C::kTile;  // V_c is dead once MMA3 of this chunk has completed
+        uint32_t den_hi, den_lo;
+        tmem_ld2(tmem + C::tOz + lane_off, den_hi, den_lo);
+        tmem_wait_ld();
+        const float inv = 1.f / (__uint_as_float(den_hi) + __uint_as_float(den_lo));
 #pragma unroll(D == 128 ? 1 : 2)
         for (int cc = 0; cc < D / 32; ++cc) {
           uint32_t v[32];
@@ -799,7 +754,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
             val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
             val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4*>(stage + (cc >> 1) * C::kBoxBytes + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+            *reinterpret_cast<uint4*>(v_box(sv, cc >> 1) + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
           }
         }
         tc_fence_before_sync();
@@ -826,84 +781,43 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     const uint32_t lane_off = (uint32_t)(quarter * 32) << 16;
     constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per Q-group thread
     uint32_t nq = 0, ta = 0, n_a = 0, n_items = 0;
-    int na = 0;
     bool ok = true;
     if (tid == 6 * 32 && (int)blockIdx.x < p.nitems) {
       // the very first Q tile; every later one is requested by the warp that frees the landing buffer
       const LinItem first = decode_item(p, blockIdx.x);
       mbar_arrive_expect_tx(&bar.q_full, C::kTile);
       for (int x = 0; x < D / 64; ++x)
-        tma_load_4d_hint(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, first.c_begin * 128, first.h, first.b,
+        tma_load_4d_hint(q_box(x), &mq, &bar.q_full, x * 64, first.c_begin * 128, first.h, first.b,
                          l2_policy_evict_first());
     }
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
-      const int ip = n_items & 1;
-      if (kgrp && tt < D) {
-        zcum[ip][0][tt] = 0.f;
-        if (kDirect) zrun[0][tt] = 0.f;
-      }
-      // kDirect: phi on this group's half of the K tile of chunk jrow (running index idx) of the
-      // chunk pipeline, in place; its column sums are posted before the tile is released, so
-      // whoever has seen the tile complete may read them.
+      // kDirect: phi on this group's half of the K tile with running index idx (chunk jrow of the
+      // item) of the chunk pipeline, in place
       auto transform_direct = [&](uint32_t idx, int jrow) {
         const uint32_t sl = idx & 1;
         ok = ok && mbar_wait(&bar.k_full[sl], (idx >> 1) & 1, p.status, 430);
         const int cc = tt >> 4;
-        if (ok && tt < 2 * D) {
-          float cs[8];
+        if (ok && tt < 2 * D)
           transform_k_rows(sK + sl * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
-                           p.N - (it.c_begin + jrow) * 128, cs);
-          int col;
-          const float sum = reduce_column_sums(cs, tt & 15, &col);
-          if ((tt & 1) == 0) zpart[jrow & (kMaxL - 1)][kgrp ? 0 : 1][cc * 8 + col] = sum;
-        }
+                           p.N - (it.c_begin + jrow) * 128);
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kd_phi[sl]);
       };
       if (kDirect) transform_direct(nq, 0);
-      // ---- pass A: the K group takes rows 0..63 (by sixteens) of every K tile, the Q group rows
-      //      64..127; the K group also keeps the cumulative column sums
+      // ---- pass A: the K group takes rows 0..63 (by sixteens) of every K tile, the Q group rows 64..127
       for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
         const uint32_t sk = ta % 3;
         ok = ok && mbar_wait(&bar.ka_full[sk], (ta / 3) & 1, p.status, 410);
         if (tid == 14 * 32) PROF(3, ta, 4);
-
         const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
-        float cs[8];
         if (ok && tt < 2 * D)
           transform_k_rows(a_kslot(sk) + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
-
-                           p.N - (it.c_begin + j) * 128, cs);
+                           p.N - (it.c_begin + j) * 128);
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);  // the tile may go to the tensor core and be parked
         if (tid == 14 * 32) PROF(3, ta, 5);
-
-        // the column sums are left per tile; nothing here waits for the other half of the tile
-        if (ok && tt < 2 * D) {
-          int col;
-          const float sum = reduce_column_sums(cs, tt & 15, &col);
-          if ((tt & 1) == 0) zpart[j][kgrp ? 0 : 1][cc * 8 + col] = sum;
-        }
         ++ta;
-      }
-
-      // both halves of every tile are done: running column sums over the segment's chunks
-      if (!kDirect && named_bar_or(4, 512, !ok)) break;
-      if (!kDirect && kgrp) {
-        if (tt < D) {
-          float run = 0.f;
-          for (int j = 0; j < it.nC; ++j) {
-            run += zpart[j][0][tt] + zpart[j][1][tt];
-            zcum[ip][j + 1][tt] = run;
-          }
-        }
-        if (named_bar_or(3, 256, false)) break;
-        na += it.nC;
-        if (tt == 0) {
-          __threadfence_block();
-          *reinterpret_cast<volatile int*>(&ka_epoch) = na;
-        }
       }
 
       // ---- hand-over of S: the two groups publish the inclusive state (column quarters 0, 1 / 2, 3)
@@ -912,46 +826,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         ++n_a;
       }
       if (kgrp) {
-        ok = ok && wait_epoch(&zin_epoch, (int)n_items + 1, p.status, 415);
-        if (named_bar_or(3, 256, !ok)) break;
-        // ---- pass C: causal mask inside the chunk, bf16 back into TMEM, partial denominators.
+        ok = !__any_sync(0xffffffffu, !ok);
+        if (!ok) break;
+        // ---- pass C: causal mask inside the chunk, bf16 back into TMEM.
         //      This warp owns rows [32 q, 32 q + 32) x key columns [64 colh, 64 colh + 64).
         for (int j = 0; j < it.nC; ++j) {
-          const int sq = nq & 1;
-          if (!mbar_wait(&bar.qphi_full[sq], (nq >> 1) & 1, p.status, 300)) { ok = false; break; }
-          tc_fence_after_sync();
-          if (kDirect && tt == 0) PROF(3, nq, 4);
-          // phi(q_i) . z_{c-1} over this warp's half of the head dimension, from the phi(Q) operand in
-          // TMEM (the rounded values the tensor core sees); z before chunk j = zin + zcum[j]
-          float part;
-          {
-            constexpr int W = D / 4;  // packed words per half row, 16 at a time (rolled: small hot code)
-            float d0 = 0.f, d1 = 0.f;
-#pragma unroll 1
-            for (int pc = 0; pc < W / 16; ++pc) {
-              uint32_t qw[16];
-              tmem_ld16(tmem + C::tQ + sq * (D / 2) + lane_off + colh * W + pc * 16, qw);
-              tmem_wait_ld();
-              const float* za = zin[ip] + colh * (D / 2) + pc * 32;
-              const float* zb = (kDirect ? zrun[j & 1] : zcum[ip][j]) + colh * (D / 2) + pc * 32;
-
-#pragma unroll
-              for (int w = 0; w < 16; w += 2) {
-                const float4 a = *reinterpret_cast<const float4*>(za + 2 * w);
-                const float4 b = *reinterpret_cast<const float4*>(zb + 2 * w);
-                d0 = fmaf(bf16_lo(qw[w]), a.x + b.x, d0);
-                d1 = fmaf(bf16_hi(qw[w]), a.y + b.y, d1);
-                d0 = fmaf(bf16_lo(qw[w + 1]), a.z + b.z, d0);
-                d1 = fmaf(bf16_hi(qw[w + 1]), a.w + b.w, d1);
-              }
-            }
-            part = d0 + d1;
-          }
           // kDirect: this group's half of the next chunk's K tile, while the tensor core forms P
-          if (kDirect && tt == 0) PROF(3, nq, 5);
           if (kDirect && j + 1 < it.nC) transform_direct(nq + 1, j + 1);
-          if (kDirect && tt == 0) PROF(3, nq, 6);
-
           if (!ok || !mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
           if (tt == 0) PROF(2, nq, 0);
           tc_fence_after_sync();
@@ -973,7 +854,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               for (int jj = 0; jj < 16; ++jj) {
                 const float p0 = (!diag || 2 * jj <= lane) ? __uint_as_float(v[2 * jj]) : 0.f;
                 const float p1 = (!diag || 2 * jj + 1 <= lane) ? __uint_as_float(v[2 * jj + 1]) : 0.f;
-                part += p0 + p1;
                 pk[jj] = pack_bf16(p0, p1);
               }
             }
@@ -981,30 +861,81 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             // so the two warps of a lane quarter never touch each other's unread input
             tmem_st16(tmem + C::tP + lane_off + colh * 64 + e * 16, pk);
           }
-          den_s[sq][colh][r] = part;
-          mbar_arrive(&bar.den_full[sq]);
           tmem_wait_st();
           tc_fence_before_sync();
           mbar_arrive(&bar.pm_full);
           if (tt == 0) PROF(2, nq, 1);
-          if (kDirect) {
-            // both halves of this chunk's tile have posted their column sums: z before the next chunk
-            ok = mbar_wait(&bar.kd_phi[sq], (nq >> 1) & 1, p.status, 431);
-            if (ok && tt < D)
-              zrun[(j + 1) & 1][tt] = zrun[j & 1][tt] + zpart[j & (kMaxL - 1)][0][tt] + zpart[j & (kMaxL - 1)][1][tt];
-            if (named_bar_or(3, 256, !ok)) { ok = false; break; }
-            if (tt == 0) PROF(3, nq, 7);
+          // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
+          //      bf16 copy, stream the new one (and z) into shared memory for the next chunk.
+          //      This warp: rows [32 q, 32 q + 32) x columns [colh D/2, colh D/2 + D/2).
+          if (!mbar_wait(&bar.s_full, nq & 1, p.status, 302) || !mbar_wait(&bar.mma2_done, nq & 1, p.status, 303)) {
+            ok = false;
+            break;
+          }
+          if (tt == 0) PROF(2, nq, 2);
+          tc_fence_after_sync();
+          {
+            // after the item's last chunk nobody reads Sb again (it may already hold a K tile of the
+            // next item's pass A), and only a chain's last segment still wants the state itself
+            const bool s_row = r < D;  // rows of S are feature indices a < D
+            const long long sidx = (long long)it.b * p.h_count + it.hl;
+            const bool last_chunk = (j == it.nC - 1);
+            const bool write_final = it.last_seg && last_chunk && p.S_io != nullptr;
+            if (colh == 0 && (!last_chunk || (it.last_seg && p.z_io != nullptr))) {
+              const float z = __uint_as_float(tmem_ld1(tmem + C::tSz + lane_off));
+              tmem_wait_ld();
+              if (s_row) {
+                if (!last_chunk) {
+                  const float hi = __bfloat162float(__float2bfloat16_rn(z));  // columns 0, 1 = hi(z), lo(z)
+                  *reinterpret_cast<uint32_t*>(sZb + swz128_offset(r, 0)) = pack_bf16(hi, z - hi);
+                } else {
+                  p.z_io[sidx * D + r] = z;
+                }
+              }
+            }
+#pragma unroll 1
+            for (int e = 0; e < D / 64; ++e) {
+              if (last_chunk && !write_final) break;
+              const int cc = colh * (D / 64) + e;  // 32-column block
+              uint32_t v[32];
+              tmem_ld32(tmem + C::tS + lane_off + cc * 32, v);
+              tmem_wait_ld();
+              if (s_row && !last_chunk) {
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {
+                  uint4 val;
+                  val.x = pack_bf16(__uint_as_float(v[8 * g + 0]), __uint_as_float(v[8 * g + 1]));
+                  val.y = pack_bf16(__uint_as_float(v[8 * g + 2]), __uint_as_float(v[8 * g + 3]));
+                  val.z = pack_bf16(__uint_as_float(v[8 * g + 4]), __uint_as_float(v[8 * g + 5]));
+                  val.w = pack_bf16(__uint_as_float(v[8 * g + 6]), __uint_as_float(v[8 * g + 7]));
+                  *reinterpret_cast<uint4*>(sSb + (cc >> 1) * C::kSbBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+                }
+              }
+              if (s_row && write_final) {
+                float* dst = p.S_io + (sidx * D + r) * D + cc * 32;
+#pragma unroll
+                for (int jj = 0; jj < 32; jj += 4)
+                  *reinterpret_cast<float4*>(dst + jj) =
+                      make_float4(__uint_as_float(v[jj]), __uint_as_float(v[jj + 1]), __uint_as_float(v[jj + 2]),
+                                  __uint_as_float(v[jj + 3]));
+              }
+            }
+            tc_fence_before_sync();
+            mbar_arrive(&bar.s_loaded);
+            fence_proxy_async_smem();
+            mbar_arrive(&bar.sb_full);
+            if (last_chunk) mbar_arrive(&bar.s_final);
+            if (tt == 0) PROF(2, nq, 5);
           }
           ++nq;
         }
         if (!ok) break;
-        if (kDirect && tt < D && p.z_io != nullptr)
-          p.z_io[((long long)it.b * p.h_count + it.hl) * D + tt] = zin[ip][tt] + zrun[it.nC & 1][tt];
       } else {
         ok = !__any_sync(0xffffffffu, !ok);
         if (!ok) break;
         for (int j = 0; j < it.nC && ok; ++j) {
-          const int sq = nq & 1;
+          constexpr int QS = C::kQSlots;
+          const int sq = nq % QS;
           ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
           if (tid == 192) PROF(3, nq, 0);
           if (ok) {
@@ -1017,7 +948,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
               const int box = gl >> 3, cin = gl & 7;
               const uint4 rawv =
-                  *reinterpret_cast<const uint4*>(sQ + box * C::kBoxBytes + r * 128 + ((cin ^ (r & 7)) << 4));
+                  *reinterpret_cast<const uint4*>(q_box(box) + r * 128 + ((cin ^ (r & 7)) << 4));
               pk[g * 4 + 0] = rawv.x;
               pk[g * 4 + 1] = rawv.y;
               pk[g * 4 + 2] = rawv.z;
@@ -1042,18 +973,15 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                   fence_proxy_async_smem();
                   mbar_arrive_expect_tx(&bar.q_full, C::kTile);
                   for (int x = 0; x < D / 64; ++x)
-                    tma_load_4d_hint(sQ + x * C::kBoxBytes, &mq, &bar.q_full, x * 64, n_chunk * 128, nx.h, nx.b,
+                    tma_load_4d_hint(q_box(x), &mq, &bar.q_full, x * 64, n_chunk * 128, nx.h, nx.b,
                                      l2_policy_evict_first());
                 }
               }
             }
 #pragma unroll
             for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
-            if (nq >= 2) {
-              const uint32_t par = ((nq >> 1) + 1) & 1;
-              ok = mbar_wait(&bar.qphi_free[sq], par, p.status, 401) &&  // MMA1/MMA2 of two chunks ago are done with it
-                   mbar_wait(&bar.den_full[sq], par, p.status, 402);     // ... and so is the K group's dot product
-            }
+            if (nq >= QS)  // MMA1/MMA2 of the slot's previous chunk are done with it
+              ok = mbar_wait(&bar.qphi_free[sq], ((nq / QS) + 1) & 1, p.status, 401);
             if (tid == 192) PROF(3, nq, 1);
             tc_fence_after_sync();
             if (ok) {
@@ -1112,7 +1040,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (!mbar_wait(&bar.o_staged[sv], n_os[sv] & 1, p.status, 500)) { ok = false; break; }
           ++n_os[sv];
           for (int x = 0; x < D / 64; ++x)
-            tma_store_4d_hint(&mo, sV + sv * C::kTile + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b,
+            tma_store_4d_hint(&mo, v_box(sv, x), x * 64, (it.c_begin + j) * 128, it.h, it.b,
                               pol_out);
           tma_store_commit();
           tma_store_wait_read<0>();
