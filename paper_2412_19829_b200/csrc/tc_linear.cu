@@ -51,7 +51,7 @@ namespace {
 using namespace sm100;
 
 constexpr int kThreads = 768;  // 24 warps, 80 registers each
-constexpr int kMaxL = 8;       // chunks per segment of a cut chain
+constexpr int kMaxL = 32;      // most chunks per segment of a cut chain
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr int kFlagStride = 32;  // one flag per 128-byte line
 
@@ -133,7 +133,7 @@ struct LinBarriers {
   uint64_t v_full[2], v_free[2];                  // V tiles of both passes (slot = tile count & 1)
   uint64_t qphi_full[2], qphi_free[2];
   uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done, sb_idle, sb_parked;
-  uint64_t pm_full, s_loaded, sb_full, s_final, o_free, o_staged[2];
+  uint64_t pm_full, s_loaded, sb_full, s_final, o_free, o_staged[2][2];  // o_staged[V slot][box]
   uint64_t kd_phi[2];  // kDirect: a K tile of the chunk pipeline has been transformed in place
 };
 
@@ -416,8 +416,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.sb_full, 256);
     mbar_init(&bar.s_final, 256);
     mbar_init(&bar.o_free, 128);
-    mbar_init(&bar.o_staged[0], 128);
-    mbar_init(&bar.o_staged[1], 128);
+    for (int i = 0; i < 4; ++i) mbar_init(&bar.o_staged[i >> 1][i & 1], 128);
     prev_epoch = 0;
     q_copied = 0;
     mbar_fence_init();
@@ -738,15 +737,15 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         }
         if (tid == 64) PROF(2, nq, 6);
         tc_fence_after_sync();
+        // One 64-column box at a time (the store warp ships a box as soon as it is staged); the
+        // next 32 columns are on their way out of TMEM while the last ones are scaled and packed.
         uint32_t den_hi, den_lo;
+        uint32_t va[32], vb[32];
         tmem_ld2(tmem + C::tOz + lane_off, den_hi, den_lo);
+        tmem_ld32(tmem + C::tO + lane_off, va);
         tmem_wait_ld();
         const float inv = 1.f / (__uint_as_float(den_hi) + __uint_as_float(den_lo));
-#pragma unroll(D == 128 ? 1 : 2)
-        for (int cc = 0; cc < D / 32; ++cc) {
-          uint32_t v[32];
-          tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
-          tmem_wait_ld();
+        auto stage32 = [&](const uint32_t (&v)[32], int x, int c32) {
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             uint4 val;
@@ -754,13 +753,25 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
             val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
             val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4*>(v_box(sv, cc >> 1) + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+            *reinterpret_cast<uint4*>(v_box(sv, x) + swz128_offset(r, c32 + g * 8)) = val;
           }
+        };
+#pragma unroll
+        for (int x = 0; x < D / 64; ++x) {
+          tmem_ld32(tmem + C::tO + lane_off + (2 * x + 1) * 32, vb);
+          stage32(va, x, 0);
+          tmem_wait_ld();
+          if (x + 1 < D / 64) {
+            tmem_ld32(tmem + C::tO + lane_off + (2 * x + 2) * 32, va);
+          } else {
+            tc_fence_before_sync();
+            mbar_arrive(&bar.o_free);  // all of O (and the denominators) has left TMEM
+          }
+          stage32(vb, x, 32);
+          fence_proxy_async_smem();
+          mbar_arrive(&bar.o_staged[sv][x]);
+          if (x + 1 < D / 64) tmem_wait_ld();
         }
-        tc_fence_before_sync();
-        mbar_arrive(&bar.o_free);
-        fence_proxy_async_smem();
-        mbar_arrive(&bar.o_staged[sv]);
         if (tid == 64) PROF(2, nq, 7);
         ++nv;
         ++nq;
@@ -1037,11 +1048,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         // ---- pass C: O tiles
         for (int j = 0; j < it.nC; ++j) {
           const int sv = nv & 1;
-          if (!mbar_wait(&bar.o_staged[sv], n_os[sv] & 1, p.status, 500)) { ok = false; break; }
+          for (int x = 0; x < D / 64 && ok; ++x) {
+            ok = mbar_wait(&bar.o_staged[sv][x], n_os[sv] & 1, p.status, 500);
+            if (ok) tma_store_4d_hint(&mo, v_box(sv, x), x * 64, (it.c_begin + j) * 128, it.h, it.b, pol_out);
+          }
+          if (!ok) break;
           ++n_os[sv];
-          for (int x = 0; x < D / 64; ++x)
-            tma_store_4d_hint(&mo, v_box(sv, x), x * 64, (it.c_begin + j) * 128, it.h, it.b,
-                              pol_out);
           tma_store_commit();
           tma_store_wait_read<0>();
           mbar_arrive(&bar.v_free[sv]);  // the staging buffer may take the V tile two uses later
@@ -1111,25 +1123,33 @@ bool tc_linear_supported(int N, int d, int dtype) {
 
 // Segmentation of the chains: G segments per chain, their lengths differing by one chunk at most
 // (the longest has *L_out chunks).  CTAs take items round-robin, so the kernel lasts about
-// ceil(items / CTAs) rounds of one item each: among the segment counts that keep segments between
-// 4 and kMaxL chunks, take the one with the least rounds x (chunks per item + the fixed cost of a
-// hand-over, about 0.7 chunk).  The plan must not depend on the device that is current when the
-// workspace size is asked for, so without a CTA count it assumes the 148 SMs of a B200.
+// ceil(items / CTAs) rounds of one item each, an item costing its chunks plus the fixed cost h of a
+// hand-over (about one chunk); but a chain is also a serial pipeline - first pass of a segment,
+// one hand-over link per segment (about 0.65 chunk each), second pass - which bounds the time
+// from below when there are few chains.  Among the segment counts allowed, take the one with the
+// least max(rounds x (L + h), L + 0.65 G).  Segments are at least 4 chunks long and short
+// enough for what the CTAs running at one time park (phi(K) and V of their segments) to stay in
+// L2.  The plan must not depend on the device that is current when the workspace size is asked
+// for, so without a CTA count it assumes the 148 SMs of a B200.
 namespace {
-// cost of a chunk of an uncut chain, in two-pass chunks (measured: with d = 64 the one pass is
-// bound by the same mask and conversion work per chunk as the second of two, so it gains nothing)
+constexpr int kPlanL8 = 8;  // segment length the scratch is sized for when chains are many
+// cost of a chunk of an uncut chain, in two-pass chunks
 constexpr double direct_chunk_cost(int d) { return d == 128 ? 0.72 : 1.05; }
+// fixed cost of an item (hand-over, pipeline refill) in chunks: a chunk is cheaper at d = 64, the hand-over hardly
+constexpr double handover_cost(int d) { return d == 128 ? 1.1 : 1.6; }
 // Range of segment counts the automatic plan chooses from.
 void plan_range(int nchains, int nch, int* g_min_out, int* g_max_out) {
-  const int g_min = (nch + kMaxL - 1) / kMaxL;
+  const int g_min8 = (nch + kPlanL8 - 1) / kPlanL8;
   int g_max = (nch + 3) / 4;
-  // long chains in numbers: stay within a quarter more segments than the minimum (the scratch
-  // grows with the segment count); few chains: as many segments as it takes to fill the GPU
-  int cap = (5 * g_min + 3) / 4;
+  // long chains in numbers: stay within a quarter more segments than 8-chunk segments give (the
+  // scratch grows with the segment count); few chains: as many segments as it takes to fill the GPU
+  int cap = (5 * g_min8 + 3) / 4;
   const int fill = (296 + nchains - 1) / nchains;
   if (cap < fill) cap = fill;
   if (g_max > cap) g_max = cap;
-  if (g_max < g_min) g_max = g_min;
+  if (g_max < g_min8) g_max = g_min8;
+  int g_min = (nch + kMaxL - 1) / kMaxL;
+  if (g_min < 1) g_min = 1;
   *g_min_out = g_min;
   *g_max_out = g_max;
 }
@@ -1145,11 +1165,17 @@ void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, 
     const int kPlanSMs = ctas > 0 ? ctas : 148;
     int g_min, g_max;
     plan_range(nchains, nch, &g_min, &g_max);
-    G = g_min;
+    G = 1;
     double best = 1e300;
-    for (int g = g_min; g <= g_max; ++g) {
-      const long long rounds = ((long long)nchains * g + kPlanSMs - 1) / kPlanSMs;
-      const double cost = (double)rounds * ((double)nch / g + 0.7);
+    for (int g = g_min > 2 ? g_min : 2; g <= g_max; ++g) {
+      const long long items = (long long)nchains * g;
+      const long long rounds = (items + kPlanSMs - 1) / kPlanSMs;
+      const double L = (double)nch / g;
+      // what the running CTAs park at one time: about 80 MB of the 126 MB of L2
+      const double l_cap = 80e6 / ((double)(items < kPlanSMs ? items : kPlanSMs) * 4.0 * 128.0 * d);
+      if (L > (l_cap < 4.0 ? 4.0 : l_cap) && g < g_max) continue;
+      const double by_rounds = (double)rounds * (L + handover_cost(d)), by_chain = L + 0.65 * g;
+      const double cost = by_rounds > by_chain ? by_rounds : by_chain;
       if (cost < best * (1.0 - 1e-9)) {
         best = cost;
         G = g;
