@@ -737,15 +737,15 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         }
         if (tid == 64) PROF(2, nq, 6);
         tc_fence_after_sync();
-        // One 64-column box at a time (the store warp ships a box as soon as it is staged); the
-        // next 32 columns are on their way out of TMEM while the last ones are scaled and packed.
         uint32_t den_hi, den_lo;
-        uint32_t va[32], vb[32];
         tmem_ld2(tmem + C::tOz + lane_off, den_hi, den_lo);
-        tmem_ld32(tmem + C::tO + lane_off, va);
         tmem_wait_ld();
         const float inv = 1.f / (__uint_as_float(den_hi) + __uint_as_float(den_lo));
-        auto stage32 = [&](const uint32_t (&v)[32], int x, int c32) {
+#pragma unroll 1
+        for (int cc = 0; cc < D / 32; ++cc) {
+          uint32_t v[32];
+          tmem_ld32(tmem + C::tO + lane_off + cc * 32, v);
+          tmem_wait_ld();
 #pragma unroll
           for (int g = 0; g < 4; ++g) {
             uint4 val;
@@ -753,24 +753,16 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
             val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
             val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4*>(v_box(sv, x) + swz128_offset(r, c32 + g * 8)) = val;
+            *reinterpret_cast<uint4*>(v_box(sv, cc >> 1) + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
           }
-        };
-#pragma unroll
-        for (int x = 0; x < D / 64; ++x) {
-          tmem_ld32(tmem + C::tO + lane_off + (2 * x + 1) * 32, vb);
-          stage32(va, x, 0);
-          tmem_wait_ld();
-          if (x + 1 < D / 64) {
-            tmem_ld32(tmem + C::tO + lane_off + (2 * x + 2) * 32, va);
-          } else {
+          if (cc == D / 32 - 1) {
             tc_fence_before_sync();
-            mbar_arrive(&bar.o_free);  // all of O (and the denominators) has left TMEM
+            mbar_arrive(&bar.o_free);
           }
-          stage32(vb, x, 32);
-          fence_proxy_async_smem();
-          mbar_arrive(&bar.o_staged[sv][x]);
-          if (x + 1 < D / 64) tmem_wait_ld();
+          if (cc & 1) {
+            fence_proxy_async_smem();
+            mbar_arrive(&bar.o_staged[sv][cc >> 1]);
+          }
         }
         if (tid == 64) PROF(2, nq, 7);
         ++nv;
