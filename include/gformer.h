@@ -80,6 +80,15 @@ int gformer_default_h_sparse(int H);
  * concurrent calls into the library. */
 int gformer_set_tuning(int key, int value);
 
+/* How the tensor-core linear-attention kernel would cut `chains` (batch, head) sequences of N
+ * tokens (bf16, d in {64, 128}) when it runs on `ctas` CTAs (0: one per SM of a B200): the
+ * number of sequence segments per chain and the chunks (of 128 tokens) of the longest one.  One
+ * segment with GF_TUNE_LINEAR_SPLIT on auto means the one-pass form of the kernel; more mean the
+ * two-pass form with a state hand-over between segments (the chunked regrouping of Algorithm 1
+ * is exact either way).  Host arithmetic only; honours GF_TUNE_LINEAR_SPLIT.  Returns GF_OK, or
+ * GF_ERR_INVALID_ARG / GF_ERR_UNSUPPORTED without touching the outputs. */
+int gformer_linear_plan(int chains, int N, int d, int ctas, int* segments, int* chunks_per_segment);
+
 /* Number of kernels the library has launched in this process so far (all entry points,
  * all streams).  For accounting in benchmarks. */
 unsigned long long gformer_launch_count(void);

@@ -53,6 +53,8 @@ def lib() -> ctypes.CDLL:
         L.gformer_default_h_sparse.argtypes = [i]
         L.gformer_set_tuning.restype = i
         L.gformer_set_tuning.argtypes = [i, i]
+        L.gformer_linear_plan.restype = i
+        L.gformer_linear_plan.argtypes = [i, i, i, i, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
         L.gformer_workspace_bytes.restype = sz
         L.gformer_workspace_bytes.argtypes = [i] * 7
         L.gformer_last_device_status.restype = i
@@ -93,6 +95,15 @@ def set_tuning(key: int, value: int) -> None:
     rc = lib().gformer_set_tuning(int(key), int(value))
     if rc != GF_OK:
         raise GformerError(rc, "gformer_set_tuning")
+
+
+def linear_plan(chains: int, N: int, d: int, ctas: int = 0):
+    """(segments per chain, chunks of the longest segment) the linear kernel would use."""
+    g, l = ctypes.c_int(0), ctypes.c_int(0)
+    rc = lib().gformer_linear_plan(int(chains), int(N), int(d), int(ctas), ctypes.byref(g), ctypes.byref(l))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_linear_plan")
+    return g.value, l.value
 
 
 def workspace_bytes(B, H, N, d, w, h_sparse, dtype) -> int:

@@ -162,6 +162,13 @@ int gformer_set_tuning(int key, int value) {
   }
 }
 
+int gformer_linear_plan(int chains, int N, int d, int ctas, int* segments, int* chunks_per_segment) {
+  if (chains < 1 || N < 1 || ctas < 0 || segments == nullptr || chunks_per_segment == nullptr) return GF_ERR_INVALID_ARG;
+  if (!gf::tc_linear_supported(N, d, GF_BF16)) return GF_ERR_UNSUPPORTED;
+  gf::linear_tc_plan(chains, N, d, g_linear_split, ctas, chunks_per_segment, segments);
+  return GF_OK;
+}
+
 size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, int dtype) {
   (void)w;
   size_t bytes = sizeof(WsHeader);

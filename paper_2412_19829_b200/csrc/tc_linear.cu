@@ -1126,7 +1126,7 @@ bool tc_linear_supported(int N, int d, int dtype) {
 namespace {
 constexpr int kPlanL8 = 8;  // segment length the scratch is sized for when chains are many
 // cost of a chunk of an uncut chain, in two-pass chunks
-constexpr double direct_chunk_cost(int d) { return d == 128 ? 0.72 : 1.05; }
+constexpr double direct_chunk_cost(int d) { return d == 128 ? 0.8 : 0.93; }
 // fixed cost of an item (hand-over, pipeline refill) in chunks: a chunk is cheaper at d = 64, the hand-over hardly
 constexpr double handover_cost(int d) { return d == 128 ? 1.1 : 1.6; }
 // Range of segment counts the automatic plan chooses from.

@@ -73,6 +73,60 @@ def test_workspace_covers_every_plan():
     assert auto >= fixed
 
 
+def _state_scratch(chains, segments, d):
+    # per segment: one 128-byte flag line and one published state (S: 128 x d floats, z: d floats)
+    return 256 + chains * segments * (128 + (128 * d + d) * 4)
+
+
+def test_linear_plan_covers_the_chain_and_fits_the_workspace():
+    for chains in (1, 2, 13, 26, 104, 148, 200, 832):
+        for N in (1, 100, 128, 129, 1000, 4096, 32768, 65536, 262144):
+            for d in (64, 128):
+                ws = gf.workspace_bytes(1, chains, N, d, 1, 0, gf.GF_BF16)
+                for ctas in (0, 1, 37, 148):
+                    G, L = gf.linear_plan(chains, N, d, ctas)
+                    nch = -(-N // 128)
+                    assert 1 <= G <= nch
+                    assert L == -(-nch // G)  # balanced segments: the longest has ceil(nch / G) chunks
+                    if G > 1:
+                        assert 3 < nch / G <= 32
+                        assert ws >= _state_scratch(chains, G, d), (chains, N, d, ctas, G)
+
+
+def test_linear_plan_named_cases():
+    # the long-sequence workload: segments of at most 8 chunks (what 148 CTAs can park in L2 at d = 128)
+    G, L = gf.linear_plan(26, 32768, 128)
+    assert 32 <= G <= 40 and L <= 8
+    # one long chain is a serial pipeline of hand-over links: few, long segments
+    G, L = gf.linear_plan(1, 32768, 128)
+    assert 12 <= L <= 32
+    # enough whole chains for every CTA at d = 128, or chains too short to cut: the one-pass form
+    assert gf.linear_plan(832, 4096, 128)[0] == 1
+    assert gf.linear_plan(148, 8192, 128)[0] == 1
+    assert gf.linear_plan(10, 512, 64)[0] == 1
+    assert gf.linear_plan(832, 4096, 64)[0] == 1
+    # fewer chains than CTAs, long: cut, in segments of at most 16 chunks at d = 64 (16 KB tiles)
+    G, L = gf.linear_plan(104, 16384, 64)
+    assert G > 1 and L <= 16
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 8)
+    try:
+        assert gf.linear_plan(26, 32768, 128) == (32, 8)
+        assert gf.linear_plan(3, 1000, 64) == (1, 8)
+    finally:
+        gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0)
+
+
+def test_linear_plan_argument_errors():
+    L = gf.lib()
+    g, l = ctypes.c_int(-7), ctypes.c_int(-7)
+    assert L.gformer_linear_plan(0, 128, 64, 0, ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_linear_plan(1, 0, 64, 0, ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_linear_plan(1, 128, 64, -1, ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_linear_plan(1, 128, 96, 0, ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_UNSUPPORTED
+    assert L.gformer_linear_plan(1, 128, 64, 0, None, ctypes.byref(l)) == gf.GF_ERR_INVALID_ARG
+    assert (g.value, l.value) == (-7, -7)
+
+
 FAKE = 0x10000  # a 16-byte-aligned non-null address; validation fails before it is ever used
 
 

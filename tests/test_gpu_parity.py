@@ -219,6 +219,49 @@ def test_many_items_per_cta_ragged_tail(d):
                   "linear heads")
 
 
+@pytest.mark.parametrize("split,d", [(16, 128), (32, 128), (32, 64)])
+def test_linear_long_segments(split, d):
+    # segments of up to 32 chunks in the two-pass form (their length is bounded by what stays in
+    # L2, not by anything in the kernel), the last one ending mid-chunk, with the state written out
+    B, H, N = 1, 2, 2 * 32 * 128 - 50
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
+    assert gf.linear_plan(B * H, N, d) == (64 // split, split)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=71, gain=1.0)
+    S_ref = np.zeros((B, H, d, d)); z_ref = np.zeros((B, H, d))
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v), S_ref, z_ref)
+    S = torch.zeros(B, H, d, d, device="cuda"); z = torch.zeros(B, H, d, device="cuda")
+    ws = gf.Workspace.for_problem(B, H, N, d, 1, 0)
+    o = gf.causal_linear_attn(*dev(q, k, v), S, z, ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    assert_parity(f64(o), ref, "bf16", f"linear, segments of {split} chunks, d={d}")
+    assert errors(f64(S), S_ref)["rel_l2"] <= 1e-2
+    assert errors(f64(z), z_ref)["rel_l2"] <= 1e-2
+
+
+def test_one_pass_form_long_chains_with_state():
+    # more whole chains than CTAs at d = 128: no chain is cut, a CTA walks a whole chain in one
+    # pass (17 chunks, the last one ragged) and then another one; resumed from a saved state
+    B, H, N, d, cut = 2, 80, 2100, 128, 1000
+    assert gf.linear_plan(B * H, cut, d)[0] == 1 and gf.linear_plan(B * H, N - cut, d)[0] == 1
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=73, gain=1.0)
+    S = torch.zeros(B, H, d, d, device="cuda"); z = torch.zeros(B, H, d, device="cuda")
+    qd, kd, vd = dev(q, k, v)
+    ws = gf.Workspace.for_problem(B, H, N, d, 1, 0)
+    o1 = gf.causal_linear_attn(qd[:, :, :cut].contiguous(), kd[:, :, :cut].contiguous(),
+                               vd[:, :, :cut].contiguous(), S, z, ws=ws)
+    o2 = gf.causal_linear_attn(qd[:, :, cut:].contiguous(), kd[:, :, cut:].contiguous(),
+                               vd[:, :, cut:].contiguous(), S, z, ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    o = torch.cat([o1, o2], dim=2).cpu()
+    assert torch.isfinite(o.float()).all()
+    lh = [0, 37, H - 1]  # every (batch, head) is an independent unit: oracle on sampled heads
+    S_ref = np.zeros((B, len(lh), d, d)); z_ref = np.zeros((B, len(lh), d))
+    ref = oracle.causal_linear_attn(f64(q[:, lh]), f64(k[:, lh]), f64(v[:, lh]), S_ref, z_ref)
+    assert_parity(f64(o[:, lh]), ref, "bf16", "one-pass form, resumed")
+    assert errors(f64(S[:, lh]), S_ref)["rel_l2"] <= 1e-2
+    assert errors(f64(z[:, lh]), z_ref)["rel_l2"] <= 1e-2
+
+
 @pytest.mark.parametrize("ctas", [1, 37, 100])
 def test_linear_cta_limit_gives_the_same_result(ctas):
     # the segment plan follows the number of CTAs the persistent kernel is given; any count must
