@@ -41,6 +41,22 @@ __device__ __forceinline__ float ex2_approx(float x) {  // 2^x, flushes denormal
   return y;
 }
 
+// Developer instrumentation (compiled only with -DGF_PROFILE): time stamps of the first key tiles
+// of CTA 0, read back with gformer_debug_read_wprofile.
+#ifdef GF_PROFILE
+__device__ unsigned long long g_wprof[2][64][8];
+__device__ __forceinline__ void wprof(int role, unsigned int kt, int ev) {
+  if (blockIdx.x == 0 && kt < 64) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    g_wprof[role][kt][ev] = t;
+  }
+}
+#define WPROF(role, kt, ev) wprof(role, kt, ev)
+#else
+#define WPROF(role, kt, ev)
+#endif
+
 template <int D>
 struct WinSmem {
   static constexpr int kTile = 128 * D * 2;  // bytes of one 128 x D bf16 tile
@@ -193,6 +209,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (!mbar_wait(&q_full, nu & 1, p.status, 20)) break;
         for (int it = 0; it < x.n_tiles; ++it, ++kt) {
           if (!mbar_wait(&k_full, kt & 1, p.status, 21)) { ok = false; break; }
+          WPROF(0, kt, 0);
           tc_fence_after_sync();
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
@@ -202,9 +219,12 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           }
           umma_commit(&k_empty);
           umma_commit(&s_full);
+          WPROF(0, kt, 1);
           if (it == x.n_tiles - 1) umma_commit(&q_empty);  // the next unit's Q may land
           if (!mbar_wait(&p_full, kt & 1, p.status, 22)) { ok = false; break; }
+          WPROF(0, kt, 2);
           if (!mbar_wait(&v_full, kt & 1, p.status, 23)) { ok = false; break; }
+          WPROF(0, kt, 3);
           // the first product of a unit overwrites O: the previous unit's epilogue has read it
           if (it == 0 && nu >= 1 && !mbar_wait(&o_free, (nu - 1) & 1, p.status, 24)) { ok = false; break; }
           tc_fence_after_sync();
@@ -217,6 +237,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           // releases it once the store has read it
           if (it < x.n_tiles - 1) umma_commit(&v_empty);
           umma_commit(&pv_done);
+          WPROF(0, kt, 4);
           if (it == x.n_tiles - 1) umma_commit(&o_full);
         }
       }
@@ -240,6 +261,7 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       for (int it = 0; it < x.n_tiles; ++it, ++kt) {
         const int j0 = (x.t_first + it) * 128;
         if (!mbar_wait(&s_full, kt & 1, p.status, 30)) { ok = false; break; }
+        if (tid == 64) WPROF(1, kt, 0);
         tc_fence_after_sync();
         // valid key columns of this row in this tile: [lo, hi]; over the warp's 32 rows lo and hi move
         // by 31, so the 64-column half is classified per warp: nothing visible (costs nothing), all
@@ -277,7 +299,9 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         // (same lane quarter, other half); double buffered by tile parity, one barrier per tile
         const float mloc = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
         mx_s[kt & 1][hh][r] = mloc;
+        if (tid == 64) WPROF(1, kt, 1);
         asm volatile("bar.sync %0, 64;" ::"r"(2 + quarter) : "memory");
+        if (tid == 64) WPROF(1, kt, 2);
         const float mt = fmaxf(mloc, mx_s[kt & 1][hh ^ 1][r]) * p.scale_log2;  // scale > 0
         // lazy rescale of what has been accumulated so far (both halves take the same decision)
         float alpha = 1.f;
@@ -359,9 +383,11 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           tmem_st16(tS + lane_off + c0 + 16, pb);
         }
         l += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+        if (tid == 64) WPROF(1, kt, 3);
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(&p_full);
+        if (tid == 64) WPROF(1, kt, 4);
       }
       if (!ok) break;
       // epilogue: O / l -> bf16 -> shared (swizzled; the unit's last V tile is dead once its product
@@ -413,6 +439,12 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 }
 
 }  // namespace
+
+#ifdef GF_PROFILE
+extern "C" int gformer_debug_read_wprofile(unsigned long long* host_dst) {
+  return (int)cudaMemcpyFromSymbol(host_dst, g_wprof, sizeof(g_wprof));
+}
+#endif
 
 bool tc_window_supported(int N, int d, int w, int dtype) {
   (void)N;
