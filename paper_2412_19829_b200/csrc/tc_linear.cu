@@ -66,15 +66,15 @@ struct LinCfg {
   // byte offset) apart: V | ones and Sb | Zb.  The constant ones box (column 0 = 1) serves both
   // V slots, so it must lie one box distance past the last box of either: with B = kBoxBytes,
   //   D = 128:  V0a Q0 V1a V0b V1b Q1 ONES   (V0: distance 3B, V1: 2B; the Q boxes fill the holes)
-  //   D = 64:   V0 V1 ONES                   (V0: distance 2B, V1: 1B)
-  static constexpr int kV0 = 0;
-  static constexpr int kV1 = (D == 128) ? 2 * kBoxBytes : kBoxBytes;
-  static constexpr int kVLbo0 = (D == 128) ? 3 * kBoxBytes : 2 * kBoxBytes;
-  static constexpr int kVLbo1 = (D == 128) ? 2 * kBoxBytes : kBoxBytes;
-  static constexpr int kOnes = (D == 128) ? 6 * kBoxBytes : 2 * kBoxBytes;
-  static constexpr int kQ = (D == 128) ? kBoxBytes : 3 * kBoxBytes;  // raw Q landing buffer
+  //   D = 64:   V0 V1 V2 V3 ONES             (slot s: distance (4 - s) B; a V tile is one box, and
+  //                                           there is room for four slots)
+  static constexpr int kVSlots = (D == 128) ? 2 : 4;
+  __host__ __device__ static constexpr int v_off(int sv) { return (D == 128) ? (sv ? 2 : 0) * kBoxBytes : sv * kBoxBytes; }
+  __host__ __device__ static constexpr int v_lbo(int sv) { return (D == 128) ? (sv ? 2 : 3) * kBoxBytes : (4 - sv) * kBoxBytes; }
+  static constexpr int kOnes = (D == 128) ? 6 * kBoxBytes : 4 * kBoxBytes;
+  static constexpr int kQ = (D == 128) ? kBoxBytes : 5 * kBoxBytes;  // raw Q landing buffer
   static constexpr int kQStride = 4 * kBoxBytes;                     // between its boxes (D = 128)
-  static constexpr int kK = (D == 128) ? 7 * kBoxBytes : 4 * kBoxBytes;  // 2 stages, contiguous
+  static constexpr int kK = (D == 128) ? 7 * kBoxBytes : 6 * kBoxBytes;  // 2 stages, contiguous
   static constexpr int kSb = kK + 2 * kTile;  // bf16 copy of S, [D rows][D cols] in 64-column boxes
   static constexpr int kZb = kSb + kSbBytes;  // one more such box: column 0 = hi(z), column 1 = lo(z)
   // Pass A runs its K tiles through three slots: the two K slots and, third, the Sb buffer, which
@@ -130,10 +130,10 @@ struct LinBarriers {
   uint64_t q_full;
   uint64_t ka_full[3], kphi_full[3], ka_free[3];  // K tiles of pass A (slot = tile count % 3)
   uint64_t k_full[2], k_free[2];                  // K tiles of pass C (slot = chunk count & 1)
-  uint64_t v_full[2], v_free[2];                  // V tiles of both passes (slot = tile count & 1)
+  uint64_t v_full[4], v_free[4];                  // V tiles of both passes (slot = tile count % kVSlots)
   uint64_t qphi_full[2], qphi_free[2];
   uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done, sb_idle, sb_parked;
-  uint64_t pm_full, s_loaded, sb_full, s_final, o_free, o_staged[2][2];  // o_staged[V slot][box]
+  uint64_t pm_full, s_loaded, sb_full, s_final, o_free, o_staged[4][2];  // o_staged[V slot][box]
   uint64_t kd_phi[2];  // kDirect: a K tile of the chunk pipeline has been transformed in place
 };
 
@@ -373,7 +373,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   uint8_t* sm = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw_smem) + 1023) & ~(uintptr_t)1023);
   uint8_t* sK = sm + C::kK;
   // box x of V slot sv (also the staging buffer of the O tile), of the Q landing buffer
-  auto v_box = [&](int sv, int x) -> uint8_t* { return sm + (sv ? C::kV1 + x * C::kVLbo1 : C::kV0 + x * C::kVLbo0); };
+  auto v_box = [&](int sv, int x) -> uint8_t* { return sm + C::v_off(sv) + x * C::v_lbo(sv); };
+  constexpr int VS = C::kVSlots;
   auto q_box = [&](int x) -> uint8_t* { return sm + C::kQ + x * C::kQStride; };
   uint8_t* sSb = sm + C::kSb;
   __shared__ __align__(8) LinBarriers bar;
@@ -395,6 +396,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     for (int s = 0; s < 2; ++s) {
       mbar_init(&bar.k_full[s], 1);
       mbar_init(&bar.v_full[s], 1);
+      mbar_init(&bar.v_full[s + 2], 1);
+      mbar_init(&bar.v_free[s + 2], 1);
       mbar_init(&bar.k_free[s], 1);
       mbar_init(&bar.v_free[s], 1);
       mbar_init(&bar.qphi_full[s], 8);
@@ -416,7 +419,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.sb_full, 256);
     mbar_init(&bar.s_final, 256);
     mbar_init(&bar.o_free, 128);
-    for (int i = 0; i < 4; ++i) mbar_init(&bar.o_staged[i >> 1][i & 1], 128);
+    for (int i = 0; i < 8; ++i) mbar_init(&bar.o_staged[i >> 1][i & 1], 128);
     prev_epoch = 0;
     q_copied = 0;
     mbar_fence_init();
@@ -445,7 +448,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 
   // Every role walks the same item list and keeps the same running counters: ta = K tiles of pass
   // A so far (slot = ta % 3, phase = ta / 3), nq = pass-C chunks so far (K slot = nq & 1, phase =
-  // nq >> 1), nv = V tiles of both passes so far (slot = nv & 1, phase = nv >> 1).
+  // nq >> 1), nv = V tiles of both passes so far (slot = nv % VS, phase = nv / VS).
   auto a_kslot = [&](uint32_t slot) -> uint8_t* { return slot < 2 ? sK + slot * C::kTile : sm + C::kKA2; };
 
   if (warp == 0) {
@@ -502,8 +505,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               ++nq;
             }
             if (pass == 1 || it.need_dS) {
-              const int sv = nv & 1;
-              if (nv >= 2 && !mbar_wait(&bar.v_free[sv], ((nv >> 1) + 1) & 1, p.status, 102)) { ok = false; break; }
+              const int sv = nv % VS;
+              if (nv >= VS && !mbar_wait(&bar.v_free[sv], ((nv / VS) + 1) & 1, p.status, 102)) { ok = false; break; }
               mbar_arrive_expect_tx(&bar.v_full[sv], C::kTile);
               for (int x = 0; x < D / 64; ++x)
                 tma_load_4d_hint(v_box(sv, x), &mv, &bar.v_full[sv], x * 64, n0, it.h, it.b,
@@ -542,10 +545,10 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (!mbar_wait(&bar.kphi_full[sa], (ta / 3) & 1, p.status, 220)) { ok = false; break; }
           PROF(1, ta, 4);
           if (it.need_dS) {
-            const int sv = nv & 1;
+            const int sv = nv % VS;
             const uint32_t kbase = smem_u32(a_kslot(sa)), vbase = smem_u32(v_box(sv, 0));
-            const uint32_t vlbo = sv ? C::kVLbo1 : C::kVLbo0;
-            if (!mbar_wait(&bar.v_full[sv], (nv >> 1) & 1, p.status, 221)) { ok = false; break; }
+            const uint32_t vlbo = C::v_lbo(sv);
+            if (!mbar_wait(&bar.v_full[sv], (nv / VS) & 1, p.status, 221)) { ok = false; break; }
             tc_fence_after_sync();
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks)
@@ -564,9 +567,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (it.need_dS) umma_commit(&bar.a_done);
         // ---- pass C
         for (int j = 0; j < it.nC; ++j) {
-          const int sv = nv & 1, sk = nq & 1, sq = nq % QS;  // slots of the V ring, of this pass's K ring, of phi(Q)
+          const int sv = nv % VS, sk = nq & 1, sq = nq % QS;  // slots of the V ring, of this pass's K ring, of phi(Q)
           const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(v_box(sv, 0));
-          const uint32_t vlbo = sv ? C::kVLbo1 : C::kVLbo0;
+          const uint32_t vlbo = C::v_lbo(sv);
           const uint32_t tq = tmem + C::tQ + sq * (D / 2);
           // the chunk's phi(K) tile: read back from the park, or (kDirect) transformed in place
           if (!mbar_wait(&bar.qphi_full[sq], (nq / QS) & 1, p.status, 200) ||
@@ -583,7 +586,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                     umma_smem_desc(kbase + (ks >> 2) * C::kBoxBytes + (ks & 3) * 32, 16, 1024), id_p, ks > 0);
           umma_commit(&bar.p_full);
           PROF(1, nq, 6);
-          if (!mbar_wait(&bar.v_full[sv], (nv >> 1) & 1, p.status, 202) ||
+          if (!mbar_wait(&bar.v_full[sv], (nv / VS) & 1, p.status, 202) ||
               !mbar_wait(&bar.s_loaded, n_sl & 1, p.status, 203)) {
             ok = false;
             break;
@@ -729,7 +732,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       }
       // ---- pass C
       for (int j = 0; j < it.nC; ++j) {
-        const int sv = nv & 1;
+        const int sv = nv % VS;
         // ---- O: divide by the denominator, bf16, stage for the TMA store
         if (!mbar_wait(&bar.o_full, nq & 1, p.status, 304)) {
           ok = false;
@@ -1013,7 +1016,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     if (elect_one()) {
       uint32_t ta = 0, nv = 0;
       [[maybe_unused]] uint32_t n_items = 0;
-      uint32_t n_os[2] = {0, 0};
+      uint32_t n_os[4] = {0, 0, 0, 0};
       bool ok = true;
       const uint64_t pol_keep = l2_policy_evict_last();  // parked phi(K) tiles are read back by pass C
       const uint64_t pol_out = l2_policy_evict_first();  // nobody reads O again: leave L2 to the tiles that come back
@@ -1039,7 +1042,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (it.need_dS) nv += it.nC;
         // ---- pass C: O tiles
         for (int j = 0; j < it.nC; ++j) {
-          const int sv = nv & 1;
+          const int sv = nv % VS;
           for (int x = 0; x < D / 64 && ok; ++x) {
             ok = mbar_wait(&bar.o_staged[sv][x], n_os[sv] & 1, p.status, 500);
             if (ok) tma_store_4d_hint(&mo, v_box(sv, x), x * 64, (it.c_begin + j) * 128, it.h, it.b, pol_out);
