@@ -74,8 +74,11 @@ struct LinCfg {
   static constexpr int kOnes = (D == 128) ? 6 * kBoxBytes : 4 * kBoxBytes;
   static constexpr int kQ = (D == 128) ? kBoxBytes : 5 * kBoxBytes;  // raw Q landing buffer
   static constexpr int kQStride = 4 * kBoxBytes;                     // between its boxes (D = 128)
-  static constexpr int kK = (D == 128) ? 7 * kBoxBytes : 6 * kBoxBytes;  // 2 stages, contiguous
-  static constexpr int kSb = kK + 2 * kTile;  // bf16 copy of S, [D rows][D cols] in 64-column boxes
+  // K ring of the chunk pipeline, contiguous: two stages; four in the one-pass form at D = 64, where there is
+  // room and the pipeline runs at about one tile-load latency per chunk
+  static constexpr int kKSlotsMax = (D == 128) ? 2 : 4;
+  static constexpr int kK = (D == 128) ? 7 * kBoxBytes : 6 * kBoxBytes;
+  static constexpr int kSb = kK + kKSlotsMax * kTile;  // bf16 copy of S, [D rows][D cols] in 64-column boxes
   static constexpr int kZb = kSb + kSbBytes;  // one more such box: column 0 = hi(z), column 1 = lo(z)
   // Pass A runs its K tiles through three slots: the two K slots and, third, the Sb buffer, which
   // is idle in that pass (at D = 64 Sb is smaller than a tile, so the third slot gets its own room)
@@ -129,12 +132,12 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
 struct LinBarriers {
   uint64_t q_full;
   uint64_t ka_full[3], kphi_full[3], ka_free[3];  // K tiles of pass A (slot = tile count % 3)
-  uint64_t k_full[2], k_free[2];                  // K tiles of pass C (slot = chunk count & 1)
+  uint64_t k_full[4], k_free[4];                  // K tiles of pass C (slot = chunk count % KS)
   uint64_t v_full[4], v_free[4];                  // V tiles of both passes (slot = tile count % kVSlots)
   uint64_t qphi_full[2], qphi_free[2];
   uint64_t p_full, s_full, o_full, mma2_done, a_done, pub_done, park_done, sb_idle, sb_parked;
   uint64_t pm_full, s_loaded, sb_full, s_final, o_free, o_staged[4][2];  // o_staged[V slot][box]
-  uint64_t kd_phi[2];  // kDirect: a K tile of the chunk pipeline has been transformed in place
+  uint64_t kd_phi[4];  // kDirect: a K tile of the chunk pipeline has been transformed in place
 };
 
 // Bounded poll of a monotonic counter in shared memory.
@@ -375,6 +378,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   // box x of V slot sv (also the staging buffer of the O tile), of the Q landing buffer
   auto v_box = [&](int sv, int x) -> uint8_t* { return sm + C::v_off(sv) + x * C::v_lbo(sv); };
   constexpr int VS = C::kVSlots;
+  constexpr int KS = (kDirect && D == 64) ? 4 : 2;  // K ring of the chunk pipeline
   auto q_box = [&](int x) -> uint8_t* { return sm + C::kQ + x * C::kQStride; };
   uint8_t* sSb = sm + C::kSb;
   __shared__ __align__(8) LinBarriers bar;
@@ -405,8 +409,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     }
     mbar_init(&bar.sb_idle, 1);
     mbar_init(&bar.sb_parked, 1);
-    mbar_init(&bar.kd_phi[0], 16);
-    mbar_init(&bar.kd_phi[1], 16);
+    for (int i = 0; i < 4; ++i) mbar_init(&bar.kd_phi[i], 16);
+    for (int i = 2; i < 4; ++i) {
+      mbar_init(&bar.k_full[i], 1);
+      mbar_init(&bar.k_free[i], 1);
+    }
     mbar_init(&bar.p_full, 1);
     mbar_init(&bar.s_full, 1);
     mbar_init(&bar.o_full, 1);
@@ -447,8 +454,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   const uint32_t tmem = tmem_base_s;
 
   // Every role walks the same item list and keeps the same running counters: ta = K tiles of pass
-  // A so far (slot = ta % 3, phase = ta / 3), nq = pass-C chunks so far (K slot = nq & 1, phase =
-  // nq >> 1), nv = V tiles of both passes so far (slot = nv % VS, phase = nv / VS).
+  // A so far (slot = ta % 3, phase = ta / 3), nq = pass-C chunks so far (K slot = nq % KS, phase =
+  // nq / KS), nv = V tiles of both passes so far (slot = nv % VS, phase = nv / VS).
   auto a_kslot = [&](uint32_t slot) -> uint8_t* { return slot < 2 ? sK + slot * C::kTile : sm + C::kKA2; };
 
   if (warp == 0) {
@@ -459,7 +466,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       // serves both passes is only reloaded once its uses of either kind have drained: per barrier,
       // uses issued so far against phases already observed.
       uint32_t ta = 0, nv = 0, nq = 0, n_items = 0;
-      uint32_t iss_a[3] = {0, 0, 0}, obs_a[3] = {0, 0, 0}, iss_c[2] = {0, 0}, obs_c[2] = {0, 0}, obs_sbi = 0;
+      uint32_t iss_a[3] = {0, 0, 0}, obs_a[3] = {0, 0, 0}, iss_c[4] = {0, 0, 0, 0}, obs_c[4] = {0, 0, 0, 0}, obs_sbi = 0;
       bool ok = true;
       auto drain = [&](uint64_t* b, uint32_t& obs, uint32_t issued, unsigned int where) -> bool {
         while (obs < issued) {
@@ -494,8 +501,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               ++iss_a[sa];
               ++ta;
             } else {
-              const uint32_t sc = nq & 1;
-              ok = drain(&bar.k_free[sc], obs_c[sc], iss_c[sc], 104) && drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101);
+              const uint32_t sc = nq % KS;
+              ok = drain(&bar.k_free[sc], obs_c[sc], iss_c[sc], 104) &&
+                   (kDirect || drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101));
               if (!ok) break;
               mbar_arrive_expect_tx(&bar.k_full[sc], C::kTile);
               for (int x = 0; x < D / 64; ++x)  // the phi(K) tile parked in the output rows (kDirect: raw K)
@@ -567,13 +575,13 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (it.need_dS) umma_commit(&bar.a_done);
         // ---- pass C
         for (int j = 0; j < it.nC; ++j) {
-          const int sv = nv % VS, sk = nq & 1, sq = nq % QS;  // slots of the V ring, of this pass's K ring, of phi(Q)
+          const int sv = nv % VS, sk = nq % KS, sq = nq % QS;  // slots of the V ring, of this pass's K ring, of phi(Q)
           const uint32_t kbase = smem_u32(sK) + sk * C::kTile, vbase = smem_u32(v_box(sv, 0));
           const uint32_t vlbo = C::v_lbo(sv);
           const uint32_t tq = tmem + C::tQ + sq * (D / 2);
           // the chunk's phi(K) tile: read back from the park, or (kDirect) transformed in place
           if (!mbar_wait(&bar.qphi_full[sq], (nq / QS) & 1, p.status, 200) ||
-              !mbar_wait(kDirect ? &bar.kd_phi[sk] : &bar.k_full[sk], (nq >> 1) & 1, p.status, 201)) {
+              !mbar_wait(kDirect ? &bar.kd_phi[sk] : &bar.k_full[sk], (nq / KS) & 1, p.status, 201)) {
             ok = false;
             break;
           }
@@ -801,8 +809,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       // kDirect: phi on this group's half of the K tile with running index idx (chunk jrow of the
       // item) of the chunk pipeline, in place
       auto transform_direct = [&](uint32_t idx, int jrow) {
-        const uint32_t sl = idx & 1;
-        ok = ok && mbar_wait(&bar.k_full[sl], (idx >> 1) & 1, p.status, 430);
+        const uint32_t sl = idx % KS;
+        ok = ok && mbar_wait(&bar.k_full[sl], (idx / KS) & 1, p.status, 430);
         const int cc = tt >> 4;
         if (ok && tt < 2 * D)
           transform_k_rows(sK + sl * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
