@@ -72,12 +72,13 @@ struct LinCfg {
   __host__ __device__ static constexpr int v_off(int sv) { return (D == 128) ? (sv ? 2 : 0) * kBoxBytes : sv * kBoxBytes; }
   __host__ __device__ static constexpr int v_lbo(int sv) { return (D == 128) ? (sv ? 2 : 3) * kBoxBytes : (4 - sv) * kBoxBytes; }
   static constexpr int kOnes = (D == 128) ? 6 * kBoxBytes : 4 * kBoxBytes;
-  static constexpr int kQ = (D == 128) ? kBoxBytes : 5 * kBoxBytes;  // raw Q landing buffer
-  static constexpr int kQStride = 4 * kBoxBytes;                     // between its boxes (D = 128)
+  static constexpr int kQ = (D == 128) ? kBoxBytes : 5 * kBoxBytes;  // raw Q landing buffer(s)
+  static constexpr int kQStride = 4 * kBoxBytes;                     // between a tile's boxes (D = 128)
+  static constexpr int kQLand = (D == 128) ? 1 : 2;                  // landing buffers (D = 64: one box each)
   // K ring of the chunk pipeline, contiguous: two stages; four in the one-pass form at D = 64, where there is
   // room and the pipeline runs at about one tile-load latency per chunk
   static constexpr int kKSlotsMax = (D == 128) ? 2 : 4;
-  static constexpr int kK = (D == 128) ? 7 * kBoxBytes : 6 * kBoxBytes;
+  static constexpr int kK = (D == 128) ? 7 * kBoxBytes : 7 * kBoxBytes;
   static constexpr int kSb = kK + kKSlotsMax * kTile;  // bf16 copy of S, [D rows][D cols] in 64-column boxes
   static constexpr int kZb = kSb + kSbBytes;  // one more such box: column 0 = hi(z), column 1 = lo(z)
   // Pass A runs its K tiles through three slots: the two K slots and, third, the Sb buffer, which
@@ -130,7 +131,7 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
 }
 
 struct LinBarriers {
-  uint64_t q_full;
+  uint64_t q_full[2];  // raw Q tiles (landing buffer = chunk count % kQLand)
   uint64_t ka_full[3], kphi_full[3], ka_free[3];  // K tiles of pass A (slot = tile count % 3)
   uint64_t k_full[4], k_free[4];                  // K tiles of pass C (slot = chunk count % KS)
   uint64_t v_full[4], v_free[4];                  // V tiles of both passes (slot = tile count % kVSlots)
@@ -379,19 +380,21 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   auto v_box = [&](int sv, int x) -> uint8_t* { return sm + C::v_off(sv) + x * C::v_lbo(sv); };
   constexpr int VS = C::kVSlots;
   constexpr int KS = (kDirect && D == 64) ? 4 : 2;  // K ring of the chunk pipeline
-  auto q_box = [&](int x) -> uint8_t* { return sm + C::kQ + x * C::kQStride; };
+  auto q_box = [&](int slot, int x) -> uint8_t* { return sm + C::kQ + slot * C::kTile + x * C::kQStride; };
+  constexpr int QL = C::kQLand;
   uint8_t* sSb = sm + C::kSb;
   __shared__ __align__(8) LinBarriers bar;
   uint8_t* sOnes = sm + C::kOnes;
   uint8_t* sZb = sm + C::kZb;
   __shared__ int prev_epoch;       // items whose predecessor state has been seen in global memory (monotonic)
-  __shared__ int q_copied;         // Q-group warps that have copied their part of a Q tile out of the landing buffer (monotonic)
+  __shared__ int q_copied[2];      // per landing buffer: Q-group warps that have copied their part of a tile out (monotonic)
   __shared__ uint32_t tmem_base_s;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
-    mbar_init(&bar.q_full, 1);
+    mbar_init(&bar.q_full[0], 1);
+    mbar_init(&bar.q_full[1], 1);
     for (int s = 0; s < 3; ++s) {
       mbar_init(&bar.ka_full[s], 1);
       mbar_init(&bar.kphi_full[s], 16);
@@ -428,7 +431,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     mbar_init(&bar.o_free, 128);
     for (int i = 0; i < 8; ++i) mbar_init(&bar.o_staged[i >> 1][i & 1], 128);
     prev_epoch = 0;
-    q_copied = 0;
+    q_copied[0] = q_copied[1] = 0;
     mbar_fence_init();
     tma_prefetch_desc(&mq);
     tma_prefetch_desc(&mk);
@@ -796,13 +799,30 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     constexpr int kChunksPerHalf = D / 16;  // 16-byte chunks of one row handled per Q-group thread
     uint32_t nq = 0, ta = 0, n_a = 0, n_items = 0;
     bool ok = true;
-    if (tid == 6 * 32 && (int)blockIdx.x < p.nitems) {
-      // the very first Q tile; every later one is requested by the warp that frees the landing buffer
-      const LinItem first = decode_item(p, blockIdx.x);
-      mbar_arrive_expect_tx(&bar.q_full, C::kTile);
+    // Raw Q tiles are requested by the Q group itself: the first QL tiles of this CTA's work here,
+    // every later one by the warp that frees a landing buffer.  `step` moves (item, chunk of the
+    // item) to the CTA's next chunk; false when there is none.
+    auto step = [&](int& w_item, int& w_j, LinItem& w_it) -> bool {
+      if (++w_j < w_it.nC) return true;
+      w_item += gridDim.x;
+      if (w_item >= p.nitems) return false;
+      w_it = decode_item(p, w_item);
+      w_j = 0;
+      return true;
+    };
+    auto request_q = [&](int slot, const LinItem& w_it, int w_j) {
+      mbar_arrive_expect_tx(&bar.q_full[slot], C::kTile);
       for (int x = 0; x < D / 64; ++x)
-        tma_load_4d_hint(q_box(x), &mq, &bar.q_full, x * 64, first.c_begin * 128, first.h, first.b,
+        tma_load_4d_hint(q_box(slot, x), &mq, &bar.q_full[slot], x * 64, (w_it.c_begin + w_j) * 128, w_it.h, w_it.b,
                          l2_policy_evict_first());
+    };
+    if (tid == 6 * 32 && (int)blockIdx.x < p.nitems) {
+      int w_item = blockIdx.x, w_j = 0;
+      LinItem w_it = decode_item(p, w_item);
+      for (int slot = 0; slot < QL; ++slot) {
+        request_q(slot, w_it, w_j);
+        if (!step(w_item, w_j, w_it)) break;
+      }
     }
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
       const LinItem it = decode_item(p, item);
@@ -950,11 +970,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         for (int j = 0; j < it.nC && ok; ++j) {
           constexpr int QS = C::kQSlots;
           const int sq = nq % QS;
-          ok = mbar_wait(&bar.q_full, nq & 1, p.status, 400);
+          const int ql = nq % QL;  // landing buffer of this chunk's tile
+          ok = mbar_wait(&bar.q_full[ql], (nq / QL) & 1, p.status, 400);
           if (tid == 192) PROF(3, nq, 0);
           if (ok) {
             // copy the raw row half out of the landing buffer; the last warp to have done so
-            // starts the load of the next Q tile at once (the next chunk's, or the first one of
+            // starts the load of the tile that takes the buffer next (a later chunk's, or one of
             // this CTA's next item), so that it is in flight while this one is transformed
             uint32_t pk[kChunksPerHalf * 4];
 #pragma unroll
@@ -962,7 +983,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               const int gl = half * kChunksPerHalf + g;  // logical 16-byte chunk within the row (8 columns)
               const int box = gl >> 3, cin = gl & 7;
               const uint4 rawv =
-                  *reinterpret_cast<const uint4*>(q_box(box) + r * 128 + ((cin ^ (r & 7)) << 4));
+                  *reinterpret_cast<const uint4*>(q_box(ql, box) + r * 128 + ((cin ^ (r & 7)) << 4));
               pk[g * 4 + 0] = rawv.x;
               pk[g * 4 + 1] = rawv.y;
               pk[g * 4 + 2] = rawv.z;
@@ -971,24 +992,17 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             __syncwarp();
             if (lane == 0) {
               __threadfence_block();
-              const int before = atomicAdd(&q_copied, 1);
+              const int before = atomicAdd(&q_copied[ql], 1);
               if ((before & 7) == 7) {
-                int n_item = item, n_chunk = it.c_begin + j + 1;
-                LinItem nx = it;
-                if (j + 1 == it.nC) {
-                  n_item = item + gridDim.x;
-                  if (n_item < p.nitems) {
-                    nx = decode_item(p, n_item);
-                    n_chunk = nx.c_begin;
-                  }
-                }
-                if (n_item < p.nitems) {
+                // the buffer is free: it takes the tile QL chunks ahead of this one
+                int w_item = item, w_j = j;
+                LinItem w_it = it;
+                bool more = true;
+                for (int a = 0; a < QL && more; ++a) more = step(w_item, w_j, w_it);
+                if (more) {
                   __threadfence_block();
                   fence_proxy_async_smem();
-                  mbar_arrive_expect_tx(&bar.q_full, C::kTile);
-                  for (int x = 0; x < D / 64; ++x)
-                    tma_load_4d_hint(q_box(x), &mq, &bar.q_full, x * 64, n_chunk * 128, nx.h, nx.b,
-                                     l2_policy_evict_first());
+                  request_q(ql, w_it, w_j);
                 }
               }
             }
