@@ -817,11 +817,19 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                          l2_policy_evict_first());
     };
     if (tid == 6 * 32 && (int)blockIdx.x < p.nitems) {
-      int w_item = blockIdx.x, w_j = 0;
-      LinItem w_it = decode_item(p, w_item);
-      for (int slot = 0; slot < QL; ++slot) {
-        request_q(slot, w_it, w_j);
-        if (!step(w_item, w_j, w_it)) break;
+      if constexpr (QL == 1) {
+        const LinItem first = decode_item(p, blockIdx.x);
+        mbar_arrive_expect_tx(&bar.q_full[0], C::kTile);
+        for (int x = 0; x < D / 64; ++x)
+          tma_load_4d_hint(q_box(0, x), &mq, &bar.q_full[0], x * 64, first.c_begin * 128, first.h, first.b,
+                           l2_policy_evict_first());
+      } else {
+        int w_item = blockIdx.x, w_j = 0;
+        LinItem w_it = decode_item(p, w_item);
+        for (int slot = 0; slot < QL; ++slot) {
+          request_q(slot, w_it, w_j);
+          if (!step(w_item, w_j, w_it)) break;
+        }
       }
     }
     for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
@@ -993,7 +1001,27 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             if (lane == 0) {
               __threadfence_block();
               const int before = atomicAdd(&q_copied[ql], 1);
-              if ((before & 7) == 7) {
+              if constexpr (QL == 1) {
+                if ((before & 7) == 7) {  // the buffer is free: next chunk's tile, or the next item's first
+                  int n_item = item, n_chunk = it.c_begin + j + 1;
+                  LinItem nx = it;
+                  if (j + 1 == it.nC) {
+                    n_item = item + gridDim.x;
+                    if (n_item < p.nitems) {
+                      nx = decode_item(p, n_item);
+                      n_chunk = nx.c_begin;
+                    }
+                  }
+                  if (n_item < p.nitems) {
+                    __threadfence_block();
+                    fence_proxy_async_smem();
+                    mbar_arrive_expect_tx(&bar.q_full[0], C::kTile);
+                    for (int x = 0; x < D / 64; ++x)
+                      tma_load_4d_hint(q_box(0, x), &mq, &bar.q_full[0], x * 64, n_chunk * 128, nx.h, nx.b,
+                                       l2_policy_evict_first());
+                  }
+                }
+              } else if ((before & 7) == 7) {
                 // the buffer is free: it takes the tile QL chunks ahead of this one
                 int w_item = item, w_j = j;
                 LinItem w_it = it;
