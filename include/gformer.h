@@ -183,6 +183,20 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o,
 int gformer_decode_step(const void* q, const void* k, const void* v, void* o,
                         gf_decode_state* st, float scale, int phi, void* cuda_stream);
 
+/*
+ * The same step for a batch whose sequences are at different positions (continuous batching):
+ * t_seq is a device array of B token counts, 8-byte aligned, owned by the caller.  Sequence b is
+ * processed as token index t_seq[b] exactly as gformer_decode_step would process it at st->t =
+ * t_seq[b] (ring slot t_seq[b] mod w, softmax over min(t_seq[b] + 1, w) cached keys); a negative
+ * entry marks an idle slot: its state is left untouched and its output rows are zero.  After the
+ * step the non-negative entries are incremented on the device (so a captured CUDA graph of steps
+ * advances by itself); st->t is neither read nor changed.  The paper decodes whole batches in
+ * lock step (Sec. III-A); this entry point only lets the rows of one batch be at different t.
+ */
+int gformer_decode_step_ragged(const void* q, const void* k, const void* v, void* o,
+                               gf_decode_state* st, long long* t_seq, float scale, int phi,
+                               void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -303,8 +303,22 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   return GF_OK;
 }
 
+static int decode_step_impl(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
+                            long long* t_seq, float scale, int phi, void* cuda_stream);
+
 int gformer_decode_step(const void* q, const void* k, const void* v, void* o, gf_decode_state* st, float scale,
                         int phi, void* cuda_stream) {
+  return decode_step_impl(q, k, v, o, st, nullptr, scale, phi, cuda_stream);
+}
+
+int gformer_decode_step_ragged(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
+                               long long* t_seq, float scale, int phi, void* cuda_stream) {
+  if (!t_seq || (reinterpret_cast<uintptr_t>(t_seq) & 7u) != 0) return GF_ERR_INVALID_ARG;
+  return decode_step_impl(q, k, v, o, st, t_seq, scale, phi, cuda_stream);
+}
+
+static int decode_step_impl(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
+                            long long* t_seq, float scale, int phi, void* cuda_stream) {
   if (!q || !k || !v || !o || !st) return GF_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return GF_ERR_INVALID_ARG;
   if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
@@ -322,10 +336,11 @@ int gformer_decode_step(const void* q, const void* k, const void* v, void* o, gf
   const size_t bytes = (size_t)st->B * st->H * st->d * elem_size(st->dtype);
   if (overlaps(o, q, bytes) || overlaps(o, k, bytes) || overlaps(o, v, bytes)) return GF_ERR_INVALID_ARG;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)st->d);
-  cudaError_t e = gf::launch_decode_step(q, k, v, o, st->k_cache, st->v_cache, st->S, st->z, st->t, st->B, st->H,
-                                         st->d, st->w, st->h_sparse, scale, st->dtype, (cudaStream_t)cuda_stream);
+  cudaError_t e = gf::launch_decode_step(q, k, v, o, st->k_cache, st->v_cache, st->S, st->z, st->t, t_seq, st->B,
+                                         st->H, st->d, st->w, st->h_sparse, scale, st->dtype,
+                                         (cudaStream_t)cuda_stream);
   if (e != cudaSuccess) return GF_ERR_CUDA;
-  st->t += 1;
+  if (t_seq == nullptr) st->t += 1;
   return GF_OK;
 }
 

@@ -52,9 +52,11 @@ cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void
                                bool zero_init, cudaStream_t stream);
 cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void* v_cache, int B, int N, int d,
                                int w, int dtype, Strides st, int h_sparse, cudaStream_t stream);
+// t_seq == nullptr: every sequence is at position t; else sequence b is at t_seq[b] (device array,
+// negative = idle slot) and the positions are advanced on the device after the step.
 cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
-                               void* v_cache, float* S, float* z, long long t, int B, int H, int d, int w,
-                               int h_sparse, float scale, int dtype, cudaStream_t stream);
+                               void* v_cache, float* S, float* z, long long t, long long* t_seq, int B, int H,
+                               int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream);
 
 // One tiny CTA that returns after about `ns` nanoseconds: holds back the work queued behind it
 // in its stream without occupying an SM's shared memory or tensor memory.

@@ -274,7 +274,8 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256, 7)
 decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                    T* __restrict__ o, T* __restrict__ kc, T* __restrict__ vc, float* __restrict__ S,
-                   float* __restrict__ z, long long t, int H, int w, int h_sparse, float scale) {
+                   float* __restrict__ z, long long t_all, const long long* __restrict__ t_seq, int H, int w,
+                   int h_sparse, float scale) {
   constexpr int D4 = D / 4;
   constexpr int G = 256 / D4;  // thread groups along the reduced dimension
   extern __shared__ __align__(16) float dyn[];  // window heads: w scores
@@ -286,6 +287,13 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const long long io = ((long long)b * H + h) * D;
   const int c4 = tid % D4, grp = tid / D4;
+  // position of this sequence: the whole batch in lock step, or its own entry of t_seq (a negative
+  // entry marks an idle slot of the batch: state untouched, output row zero)
+  const long long t = (t_seq != nullptr) ? t_seq[b] : t_all;
+  if (t < 0) {
+    if (tid < D) o[io + tid] = from_f32<T>(0.f);
+    return;
+  }
 
   if (h < h_sparse) {
     T* kcb = kc + ((long long)b * h_sparse + h) * (long long)w * D;
@@ -386,6 +394,12 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
   }
 }
 
+// Advances the per-sequence positions after a step (idle slots stay negative).
+__global__ void advance_positions_kernel(long long* t_seq, int B) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < B && t_seq[b] >= 0) t_seq[b] += 1;
+}
+
 template <typename T>
 cudaError_t window_dispatch(const void* q, const void* k, const void* v, void* o, int B, int N, int d, int w,
                             float scale, Strides st, int h_begin, int h_count, cudaStream_t stream) {
@@ -417,8 +431,8 @@ cudaError_t linear_dispatch(const void* q, const void* k, const void* v, void* o
 
 template <typename T>
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, void* o, void* kc, void* vc, float* S,
-                            float* z, long long t, int B, int H, int d, int w, int h_sparse, float scale,
-                            cudaStream_t stream) {
+                            float* z, long long t, long long* t_seq, int B, int H, int d, int w, int h_sparse,
+                            float scale, cudaStream_t stream) {
   dim3 grid(H, B);
   const size_t dyn = (size_t)w * sizeof(float);
   if (d == 64) {
@@ -427,18 +441,22 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, void* o
       cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
       if (e != cudaSuccess) return e;
     }
-    kern<<<grid, 256, dyn, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, (T*)kc, (T*)vc, S, z, t, H,
-                                     w, h_sparse, scale);
+    kern<<<grid, 256, dyn, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, (T*)kc, (T*)vc, S, z, t, t_seq,
+                                     H, w, h_sparse, scale);
   } else {
     auto kern = decode_step_kernel<T, 128>;
     if (dyn > 40 * 1024) {
       cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn);
       if (e != cudaSuccess) return e;
     }
-    kern<<<grid, 256, dyn, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, (T*)kc, (T*)vc, S, z, t, H,
-                                     w, h_sparse, scale);
+    kern<<<grid, 256, dyn, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, (T*)kc, (T*)vc, S, z, t, t_seq,
+                                     H, w, h_sparse, scale);
   }
   note_launch();
+  if (t_seq != nullptr) {  // every CTA of the step has read its position: move them on
+    advance_positions_kernel<<<(B + 255) / 256, 256, 0, stream>>>(t_seq, B);
+    note_launch();
+  }
   return cudaGetLastError();
 }
 
@@ -498,11 +516,12 @@ cudaError_t launch_delay(unsigned int ns, cudaStream_t stream) {
 }
 
 cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
-                               void* v_cache, float* S, float* z, long long t, int B, int H, int d, int w,
-                               int h_sparse, float scale, int dtype, cudaStream_t stream) {
+                               void* v_cache, float* S, float* z, long long t, long long* t_seq, int B, int H,
+                               int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream) {
   if (dtype == GF_F32)
-    return decode_dispatch<float>(q, k, v, o, k_cache, v_cache, S, z, t, B, H, d, w, h_sparse, scale, stream);
-  return decode_dispatch<__nv_bfloat16>(q, k, v, o, k_cache, v_cache, S, z, t, B, H, d, w, h_sparse, scale,
+    return decode_dispatch<float>(q, k, v, o, k_cache, v_cache, S, z, t, t_seq, B, H, d, w, h_sparse, scale,
+                                  stream);
+  return decode_dispatch<__nv_bfloat16>(q, k, v, o, k_cache, v_cache, S, z, t, t_seq, B, H, d, w, h_sparse, scale,
                                         stream);
 }
 

@@ -182,3 +182,15 @@ def test_decode_argument_errors():
     assert L.gformer_decode_step(q, k, v, o, ctypes.byref(st), 0.0, 0, None) == gf.GF_ERR_INVALID_ARG
     assert L.gformer_decode_step(q, k, v, o, None, 0.0, 0, None) == gf.GF_ERR_INVALID_ARG
     assert st.t == 0
+
+
+def test_ragged_decode_argument_errors():
+    L = gf.lib()
+    st = gf.DecodeStateC(FAKE, FAKE + (1 << 20), FAKE + (2 << 20), FAKE + (3 << 20), 0, 2, 4, 64, 16, 1, gf.GF_BF16)
+    a = (FAKE + (4 << 20), FAKE + (5 << 20), FAKE + (6 << 20), FAKE + (7 << 20))
+    assert L.gformer_decode_step_ragged(*a, ctypes.byref(st), None, 0.0, gf.GF_PHI_ELU1, None) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_decode_step_ragged(*a, ctypes.byref(st), FAKE + (8 << 20) + 4, 0.0, gf.GF_PHI_ELU1, None) == \
+        gf.GF_ERR_INVALID_ARG
+    assert L.gformer_decode_step_ragged(a[0], a[1], a[2], 0, ctypes.byref(st), FAKE + (8 << 20), 0.0, gf.GF_PHI_ELU1,
+                                        None) == gf.GF_ERR_INVALID_ARG
+    assert st.t == 0

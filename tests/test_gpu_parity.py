@@ -399,6 +399,69 @@ def test_decode_steps_replayed_from_a_cuda_graph():
         assert torch.equal(out, eager)
 
 
+def _alias_state(big, b):
+    """A one-sequence view of slot b of a batch decode state (same device buffers)."""
+    st = gf.DecodeState(1, big.c.H, big.c.d, big.c.w, big.c.h_sparse, dtype=big.k_cache.dtype)
+    st.k_cache, st.v_cache, st.S, st.z = big.k_cache[b:b + 1], big.v_cache[b:b + 1], big.S[b:b + 1], big.z[b:b + 1]
+    st.c.k_cache, st.c.v_cache = st.k_cache.data_ptr(), st.v_cache.data_ptr()
+    st.c.S, st.c.z = st.S.data_ptr(), st.z.data_ptr()
+    return st
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_ragged_decode_matches_every_sequence_alone(dtype):
+    # continuous batching: four slots whose sequences are at different positions -- one starts
+    # from scratch, one was prefilled with 130 tokens (more than the window), one slot is idle and
+    # taken by a new sequence after ten steps, one sequence ends early and leaves its slot idle
+    B, H, d, w, h0, steps = 4, 4, 64, 48, 2, 30
+    tdt = synth.torch_dtype(dtype)
+    lens = [steps, 130 + steps, steps - 10, 12]  # total tokens of the sequence each slot ends up holding
+    seqs = [synth.qkv(1, H, n, d, dtype, seed=90 + i, gain=1.0) for i, n in enumerate(lens)]
+    refs = [oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0) for q, k, v in seqs]
+    st = gf.DecodeState(B, H, d, w, h0, dtype=tdt)
+    t_seq = torch.tensor([0, 130, -1, 0], dtype=torch.int64, device="cuda")
+    q1, k1, v1 = dev(*seqs[1])
+    o1 = gf.hybrid_attn(q1[:, :, :130].contiguous(), k1[:, :, :130].contiguous(), v1[:, :, :130].contiguous(), w,
+                        h_sparse=h0, state_out=_alias_state(st, 1))
+    assert_parity(f64(o1), refs[1][:, :, :130], kind_of(dtype), "prefill of slot 1")
+    pos = [0, 130, 0, 0]          # next token of each slot's sequence
+    got = [[], [], [], []]
+    for step in range(steps):
+        if step == 10:            # a new sequence takes the idle slot: fresh state, position 0
+            st.S[2].zero_(); st.z[2].zero_()
+            t_seq[2] = 0
+        if step == 12:            # the short sequence has ended
+            t_seq[3] = -1
+        active = [bool(x >= 0) for x in t_seq.tolist()]
+        qs = torch.zeros(B, H, d, dtype=tdt); ks = torch.zeros_like(qs); vs = torch.zeros_like(qs)
+        for b in range(B):
+            if active[b]:
+                qs[b], ks[b], vs[b] = (x[0, :, pos[b]] for x in seqs[b])
+        o = gf.decode_step_ragged(qs.cuda(), ks.cuda(), vs.cuda(), st, t_seq)
+        for b in range(B):
+            if active[b]:
+                got[b].append(o[b].cpu()); pos[b] += 1
+            else:
+                assert torch.count_nonzero(o[b]) == 0
+    assert t_seq.tolist() == [steps, 130 + steps, steps - 10, -1] and st.t == 0
+    first = [0, 130, 0, 0]
+    for b in range(B):
+        out = torch.stack(got[b], dim=1).unsqueeze(0)  # [1, H, tokens, d]
+        assert out.shape[2] == lens[b] - first[b]
+        assert_parity(f64(out), refs[b][:, :, first[b]:lens[b]], kind_of(dtype), f"ragged decode, slot {b}")
+
+
+def test_ragged_decode_equals_lock_step_when_positions_agree():
+    B, H, d, w, h0, T = 3, 4, 128, 20, 1, 25
+    q, k, v = dev(*synth.qkv(B, H, T, d, "bf16", seed=97, gain=1.0))
+    a = gf.DecodeState(B, H, d, w, h0); b = gf.DecodeState(B, H, d, w, h0)
+    t_seq = torch.zeros(B, dtype=torch.int64, device="cuda")
+    for t in range(T):
+        x = [u[:, :, t].contiguous() for u in (q, k, v)]
+        assert torch.equal(gf.decode_step(*x, a), gf.decode_step_ragged(*x, b, t_seq))
+    assert torch.equal(a.S, b.S) and torch.equal(a.k_cache, b.k_cache) and t_seq.tolist() == [T] * B
+
+
 def test_config4_prefill_and_decode_sampled_batch():
     c = synth.CONFIGS["decode"]
     B, H, N, d, w, steps = c["B"], c["H"], c["N"], c["d"], c["w"], 64  # 64 of the 256 steps checked
