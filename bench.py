@@ -515,9 +515,30 @@ def run_decode(args, c, rank, world, local_rank):
     clocks = sampler.stop() if sampler else None
     launches = gf.launch_count() - n0  # the graph replays the captured launches: count them below
     eager_ms = timed(run_eager, args.steps)
+
+    # the same steps with per-sequence positions kept on the device (they advance from replay to
+    # replay, the ring wraps): what a continuously batched server would replay
+    t_seq = torch.full((B,), N, dtype=torch.int64, device="cuda")
+
+    def run_ragged():
+        for t in range(T):
+            gf.decode_step_ragged(dtok[0][t], dtok[1][t], dtok[2][t], st, t_seq, out=dout[t], stream=stream)
+
+    run_ragged()
+    stream.synchronize()
+    rgraph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(rgraph, stream=stream):
+        run_ragged()
+
+    def run_rgraph():
+        with torch.cuda.stream(stream):
+            rgraph.replay()
+
+    run_rgraph()
+    ragged_ms = timed(run_rgraph, args.steps)
     run_e2e()
     e2e_ms = timed(run_e2e, args.steps)
-    total_ms, e2e_ms, eager_ms = max_over_ranks([total_ms, e2e_ms, eager_ms], dist, "cuda")
+    total_ms, e2e_ms, eager_ms, ragged_ms = max_over_ranks([total_ms, e2e_ms, eager_ms, ragged_ms], dist, "cuda")
     if rank == 0:
         tokens = world * B * T * args.steps
         peak, which = measured_peaks()
@@ -541,7 +562,8 @@ def run_decode(args, c, rank, world, local_rank):
                          "traffic": None, "peak_source": which + " copy bandwidth",
                          "algorithmic_bytes": step_bytes, "kernel": "decode_step_kernel, one launch per decode step",
                          "us_per_decode_step_graph": us_step,
-                         "us_per_decode_step_eager": eager_ms * 1e3 / (args.steps * T)},
+                         "us_per_decode_step_eager": eager_ms * 1e3 / (args.steps * T),
+                         "us_per_decode_step_ragged_graph": ragged_ms * 1e3 / (args.steps * T)},
             "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": UNIT,
                     "h2d_bytes_per_step": 3 * T * B * H * d * 2, "d2h_bytes_per_step": T * B * H * d * 2},
             "gpu_launches": args.steps * T if launches == 0 else launches,
