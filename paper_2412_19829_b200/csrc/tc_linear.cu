@@ -7,40 +7,41 @@
 //   O   = Qc Sb_{c-1}  (+)  Pm V_c      (MMA2, MMA3)  Sb = bf16 copy of S in shared memory
 //   den = rowsum(Pm) + Qc z_{c-1},  z_c = z_{c-1} + colsum(Kc)
 //   out = O / den
-// The denominators ride on the same tensor-core products as one extra column: z is the column
-// "V = 1" of the state (MMA4 with a constant B tile whose row 0 is all ones gives colsum(Kc) in
-// fp32), Qc z_{c-1} is the readout of that column (MMA2 against z split in two bf16 terms, hi +
-// lo, so that it carries 16 bits), and rowsum(Pm) comes from MMA3 with the ones tile again.
+// The denominators ride on the same tensor-core products as extra output columns (N = D + 16): V
+// is followed by a constant box whose column 0 is all ones, so MMA4 leaves z = sum phi(K) in
+// column D of the fp32 state and MMA3 adds rowsum(Pm) to column D of O; the bf16 copy of S is
+// followed by a box holding z split in two bf16 terms (hi + lo: 16 bits), so MMA2 leaves Qc z in
+// columns D, D + 1 of O.  The epilogue divides by the sum of those two columns.
 // A (batch, head) chain is cut into segments of L chunks; a work item is one segment.  CTAs are
 // persistent and take items round-robin in an order in which a segment's predecessor always has
 // a smaller index, so the CTA that owns it is already running.  For an item the CTA
 //   (A) applies phi to the segment's K tiles once, parks the results in the rows of the OUTPUT
 //       tensor that this segment will later overwrite (no extra scratch, and the lines are still
-//       in L2 when pass C reads them back), keeps the running column sums of phi(K) in shared
-//       memory, and accumulates the segment's own state contribution dS = sum Kc^T V (not for a
-//       chain's last segment, whose contribution nobody needs),
+//       in L2 when pass C reads them back) and accumulates the segment's own state contribution
+//       dS | dz = sum Kc^T [V | 1] (not for a chain's last segment, whose contribution nobody needs),
 //   (B) waits for the inclusive state of the previous segment in global scratch (one bounded
 //       poller per CTA), publishes its own inclusive state = previous + dS and raises its flag,
 //   (C) walks its chunks with the full pipeline starting from the previous segment's state,
 //       reading phi(K) back instead of K, so every exponential of the layer is computed once.
 // Warp roles:
-//   warp 0       TMA producer (raw Q, K, V tiles; K and V double buffered)
+//   warp 0       TMA producer (K, V tiles; rings of 2 K and 2 V slots at D = 128, 4 V slots at D = 64)
 //   warp 1       MMA issuer
-//   warps 2-5    "row group" (one thread per row): loads the state before the segment; pass C:
-//                converts S (and z) to bf16 for the next chunk's readout, divides O by the
-//                denominator and stages it for the store; hands z over between segments
-//   warps 6-13   "Q group": pass C: applies phi to Q; the result goes to TMEM as the A operand of
-//                MMA1/MMA2; pass A: transforms half of every K tile
+//   warps 2-5    "row group" (one thread per row): hands z over between segments, loads the state
+//                before the segment; pass C: divides O by the denominator and stages it for the
+//                store, one 64-column box at a time
+//   warps 6-13   "Q group": pass C: requests the raw Q tiles and applies phi to them; the result goes
+//                to TMEM as the A operand of MMA1/MMA2; pass A: transforms half of every K tile
 //   warps 14-21  "K group": pass A: applies phi to the other half of every K tile (in place in
 //                shared memory); pass C: masks/packs P in TMEM (two warps per TMEM lane quarter,
-//                half of the key columns each)
-//   warp 22      TMA stores: parks phi(K) tiles (pass A), stores O tiles staged in the dead V
+//                half of the key columns each), then converts the new S and z to bf16 for the next
+//                chunk's readout
+//   warp 22      TMA stores: parks phi(K) tiles (pass A), stores O boxes staged in the dead V
 //                buffer (pass C)
 //   warp 23      polls the previous segment's flag and raises this segment's flag
-// TMEM (D=128): P 128 | O 128 | S 128 | phi(Q) 64 | denominators 16 | z 16 columns = 480.
-// When there are at least as many chains as CTAs no chain is cut (kDirect): an item is a whole
-// chain, there is no pass A, no parking and no hand-over; the phi warps transform each K tile in
-// place one chunk ahead of the chunk pipeline.
+// TMEM (D=128): P 128 | O + denominators 144 | S + z 144 | phi(Q) 64 columns = 480.
+// When the plan leaves every chain whole (kDirect): an item is a whole chain, there is no pass A,
+// no parking and no hand-over; the phi warps transform each K tile in place one chunk ahead of
+// the chunk pipeline (four K slots at D = 64).
 // Every wait is bounded; on expiry the kernel records a status word and drains.
 #include "common.cuh"
 #include "sm100.cuh"
