@@ -188,9 +188,12 @@ int gformer_decode_step(const void* q, const void* k, const void* v, void* o,
  * t_seq is a device array of B token counts, 8-byte aligned, owned by the caller.  Sequence b is
  * processed as token index t_seq[b] exactly as gformer_decode_step would process it at st->t =
  * t_seq[b] (ring slot t_seq[b] mod w, softmax over min(t_seq[b] + 1, w) cached keys); a negative
- * entry marks an idle slot: its state is left untouched and its output rows are zero.  After the
- * step the non-negative entries are incremented on the device (so a captured CUDA graph of steps
- * advances by itself); st->t is neither read nor changed.  The paper decodes whole batches in
+ * entry marks an idle slot: its state is left untouched and its output rows are zero.  The step
+ * itself increments the non-negative entries on the device (so a captured CUDA graph of steps
+ * advances by itself); while a step is running, bits 48..62 of an entry count the heads that
+ * have read it, so positions must stay below 2^48 and H at most 4096 (GF_ERR_UNSUPPORTED), and
+ * the array must not be read or written while a step is in flight.  st->t is neither read nor
+ * changed.  The paper decodes whole batches in
  * lock step (Sec. III-A); this entry point only lets the rows of one batch be at different t.
  */
 int gformer_decode_step_ragged(const void* q, const void* k, const void* v, void* o,

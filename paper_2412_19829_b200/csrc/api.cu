@@ -314,6 +314,7 @@ int gformer_decode_step(const void* q, const void* k, const void* v, void* o, gf
 int gformer_decode_step_ragged(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
                                long long* t_seq, float scale, int phi, void* cuda_stream) {
   if (!t_seq || (reinterpret_cast<uintptr_t>(t_seq) & 7u) != 0) return GF_ERR_INVALID_ARG;
+  if (st && st->H > 4096) return GF_ERR_UNSUPPORTED;  // the arrival count of a sequence's heads has 15 bits
   return decode_step_impl(q, k, v, o, st, t_seq, scale, phi, cuda_stream);
 }
 

@@ -53,7 +53,7 @@ cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void
 cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void* v_cache, int B, int N, int d,
                                int w, int dtype, Strides st, int h_sparse, cudaStream_t stream);
 // t_seq == nullptr: every sequence is at position t; else sequence b is at t_seq[b] (device array,
-// negative = idle slot) and the positions are advanced on the device after the step.
+// negative = idle slot, otherwise below 2^48) and the kernel itself moves the positions on.
 cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
                                void* v_cache, float* S, float* z, long long t, long long* t_seq, int B, int H,
                                int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream);

@@ -274,7 +274,7 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256, 7)
 decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                    T* __restrict__ o, T* __restrict__ kc, T* __restrict__ vc, float* __restrict__ S,
-                   float* __restrict__ z, long long t_all, const long long* __restrict__ t_seq, int H, int w,
+                   float* __restrict__ z, long long t_all, long long* __restrict__ t_seq, int H, int w,
                    int h_sparse, float scale) {
   constexpr int D4 = D / 4;
   constexpr int G = 256 / D4;  // thread groups along the reduced dimension
@@ -287,9 +287,39 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const long long io = ((long long)b * H + h) * D;
   const int c4 = tid % D4, grp = tid / D4;
-  // position of this sequence: the whole batch in lock step, or its own entry of t_seq (a negative
-  // entry marks an idle slot of the batch: state untouched, output row zero)
-  const long long t = (t_seq != nullptr) ? t_seq[b] : t_all;
+  // Position of this sequence: the whole batch in lock step, or its own entry of t_seq (a negative
+  // entry marks an idle slot of the batch: state untouched, output row zero).  The sequence's H
+  // CTAs count their arrivals in bits 48..62 of the entry; the last one clears the count and moves
+  // the position on, so the step needs no second launch.
+  // (A thread that loads none of the step's inputs fetches the position, so that the two global
+  // round trips overlap.)
+  float qv = 0.f;
+  T kin = from_f32<T>(0.f), vin = from_f32<T>(0.f);
+  long long t = t_all;
+  if (t_seq != nullptr) {
+    __shared__ long long t_sh;
+    if (tid == 255) {
+      long long cur = *reinterpret_cast<const volatile long long*>(t_seq + b);
+      if (cur >= 0) {
+        unsigned long long* slot = reinterpret_cast<unsigned long long*>(t_seq + b);
+        const unsigned long long old = atomicAdd(slot, 1ull << 48);
+        cur = (long long)(old & ((1ull << 48) - 1));
+        if ((old >> 48) + 1 == (unsigned long long)H) atomicAdd(slot, 1ull - ((unsigned long long)H << 48));
+      }
+      t_sh = cur;
+    }
+    if (tid < D) {
+      qv = to_f32(q[io + tid]);
+      kin = k[io + tid];
+      vin = v[io + tid];
+    }
+    __syncthreads();
+    t = t_sh;
+  } else if (tid < D) {
+    qv = to_f32(q[io + tid]);
+    kin = k[io + tid];
+    vin = v[io + tid];
+  }
   if (t < 0) {
     if (tid < D) o[io + tid] = from_f32<T>(0.f);
     return;
@@ -301,9 +331,9 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
     const int cur = (int)(t % w);
     const int nvalid = (t + 1 < (long long)w) ? (int)(t + 1) : w;
     if (tid < D) {
-      qs[tid] = to_f32(q[io + tid]);
-      kcb[(long long)cur * D + tid] = k[io + tid];
-      vcb[(long long)cur * D + tid] = v[io + tid];
+      qs[tid] = qv;
+      kcb[(long long)cur * D + tid] = kin;
+      vcb[(long long)cur * D + tid] = vin;
     }
     __syncthreads();
     // scores: D/4 threads per slot (a warp reads whole cache lines of the ring), partial dot
@@ -359,8 +389,8 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
     float* zb = z + sidx * D;
     float denloc = 0.f;
     if (tid < D) {
-      const float qp = phi_elu1(to_f32(q[io + tid]));
-      const float kp = phi_elu1(to_f32(k[io + tid]));
+      const float qp = phi_elu1(qv);
+      const float kp = phi_elu1(to_f32(kin));
       qs[tid] = qp;
       ks[tid] = kp;
       const float zn = zb[tid] + kp;
@@ -392,12 +422,6 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
       o[io + tid] = from_f32<T>(sum / den);
     }
   }
-}
-
-// Advances the per-sequence positions after a step (idle slots stay negative).
-__global__ void advance_positions_kernel(long long* t_seq, int B) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b < B && t_seq[b] >= 0) t_seq[b] += 1;
 }
 
 template <typename T>
@@ -453,10 +477,6 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, void* o
                                      H, w, h_sparse, scale);
   }
   note_launch();
-  if (t_seq != nullptr) {  // every CTA of the step has read its position: move them on
-    advance_positions_kernel<<<(B + 255) / 256, 256, 0, stream>>>(t_seq, B);
-    note_launch();
-  }
   return cudaGetLastError();
 }
 
