@@ -262,6 +262,37 @@ def test_one_pass_form_long_chains_with_state():
     assert errors(f64(z[:, lh]), z_ref)["rel_l2"] <= 1e-2
 
 
+def _random_shapes():
+    # seeded draw of layer shapes around the edges of the plans and rings: lengths just below, at
+    # and above chunk multiples, chain counts around the CTA count, both head dimensions, windows
+    # from one token to longer than the sequence
+    rng = np.random.default_rng(20241219)
+    shapes = []
+    for i in range(14):
+        d = int(rng.choice([64, 128]))
+        H = int(rng.integers(1, 7))
+        B = int(rng.choice([1, 2, 3, 30, 75])) if i % 3 == 0 else int(rng.integers(1, 4))
+        N = int(rng.choice([1, 127, 128, 129, 255, 511, 640, 1025, 1500, 2049, 3000]))
+        if B * H > 40:
+            N = min(N, 640)
+        w = int(rng.choice([1, 2, 63, 64, 65, 128, 200, 513, 4000]))
+        h0 = int(rng.integers(0, H + 1))
+        shapes.append((B, H, N, d, w, h0))
+    return shapes
+
+
+@pytest.mark.parametrize("B,H,N,d,w,h0", _random_shapes())
+def test_random_layer_shapes(B, H, N, d, w, h0):
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=1000 + N + 7 * B + H, gain=1.0)
+    qd, kd, vd = dev(q, k, v)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    o = gf.hybrid_attn(qd, kd, vd, w, h_sparse=h0, ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    bs = sorted({0, B - 1})  # every (batch, head) is an independent unit: oracle on the outer batch rows
+    ref = oracle.hybrid_attn(f64(q[bs]), f64(k[bs]), f64(v[bs]), w, h_sparse=h0)
+    assert_parity(f64(o[bs]), ref, "bf16", f"B={B} H={H} N={N} d={d} w={w} h0={h0}")
+
+
 @pytest.mark.parametrize("ctas", [1, 37, 100])
 def test_linear_cta_limit_gives_the_same_result(ctas):
     # the segment plan follows the number of CTAs the persistent kernel is given; any count must
