@@ -105,6 +105,28 @@ def causal_linear_attn(q, k, v, S=None, z=None):
     return o
 
 
+def hybrid_attn_self(q, k, v, w: int, h_sparse: int | None = None, scale: float | None = None):
+    """The bidirectional ("self") layer: heads [0, h_sparse) see the keys with |i - j| < w,
+    the others run global linear attention phi(Q)(phi(K)^T V) with row normalisation."""
+    q, k, v = _f64(q), _f64(k), _f64(v)
+    B, H, N, d = q.shape
+    h0 = default_h_sparse(H) if h_sparse is None else int(h_sparse)
+    assert 0 <= h0 <= H
+    s = default_scale(d) if scale is None else float(scale)
+    o = np.empty_like(q)
+    _load().gfo_hybrid_attn_self(_p(q), _p(k), _p(v), _p(o), ctypes.c_long(B), ctypes.c_long(H), ctypes.c_long(N),
+                                 ctypes.c_int(d), ctypes.c_long(w), ctypes.c_long(h0), ctypes.c_double(s))
+    return o
+
+
+def window_attn_self(q, k, v, w: int, scale: float | None = None):
+    return hybrid_attn_self(q, k, v, w, h_sparse=np.asarray(q).shape[1], scale=scale)
+
+
+def linear_attn_self(q, k, v):
+    return hybrid_attn_self(q, k, v, 1, h_sparse=0)
+
+
 class DecodeState:
     """Ring-buffer KV cache of the windowed heads plus (S, z) of the linear heads."""
 

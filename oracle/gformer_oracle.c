@@ -24,6 +24,14 @@
  *                 windowed, the rest linear; every head writes its own slot of O.
  *   decode        Algorithm 1 advanced one token at a time plus the window rule on a
  *                 ring buffer of w cached keys/values (token j lives in slot j mod w).
+ *   "self" layer  (the bidirectional variant of Sec. II-A used for ViT, Sec. IV-D/E; next in
+ *                 line for the CUDA library, no kernel yet)  window head: Eq. 1 without the
+ *                 causal mask, over a two-sided window.  The paper does not print the
+ *                 two-sided rule; reading taken: token i sees the keys j with |i - j| < w
+ *                 (itself, the w-1 tokens before and the w-1 after), truncated at both
+ *                 ends -- the causal window mirrored.  Linear head: the unmasked form of
+ *                 Sec. II-B, phi(Q) (phi(K)^T V), every row normalised like Algorithm 1
+ *                 does, by phi(Q_i) . sum_j phi(K_j) over all j.
  *
  * No blocking, no fusion, no reordering: loops are in the paper's order.
  * OpenMP is used only across independent (batch, head) pairs.
@@ -102,6 +110,80 @@ static void linear_head(const double* q, const double* k, const double* v, doubl
       for (int a = 0; a < d; ++a) num += qp[a] * S[a * d + c];
       o[i * d + c] = num / den;
     }
+  }
+}
+
+/* One two-sided windowed head ("self" variant): keys j with |i - j| < w. */
+static void window_head_sym(const double* q, const double* k, const double* v, double* o,
+                            long N, int d, long w, double scale, double* e /* >= min(2w-1,N) */) {
+  for (long i = 0; i < N; ++i) {
+    long lo = i - w + 1, hi = i + w - 1;
+    if (lo < 0) lo = 0;
+    if (hi > N - 1) hi = N - 1;
+    double m = -INFINITY;
+    for (long j = lo; j <= hi; ++j) {
+      double s = 0.0;
+      for (int c = 0; c < d; ++c) s += q[i * d + c] * k[j * d + c];
+      s *= scale;
+      e[j - lo] = s;
+      if (s > m) m = s;
+    }
+    double l = 0.0;
+    for (long j = lo; j <= hi; ++j) {
+      e[j - lo] = exp(e[j - lo] - m);
+      l += e[j - lo];
+    }
+    for (int c = 0; c < d; ++c) {
+      double acc = 0.0;
+      for (long j = lo; j <= hi; ++j) acc += e[j - lo] * v[j * d + c];
+      o[i * d + c] = acc / l;
+    }
+  }
+}
+
+/* One global (unmasked) linear head, Sec. II-B: S = sum_j phi(K_j) (x) V_j and z = sum_j
+ * phi(K_j) over the whole sequence first, then H_i = phi(Q_i)^T S / (phi(Q_i) . z). */
+static void linear_head_global(const double* q, const double* k, const double* v, double* o,
+                               long N, int d, double* S, double* z, double* qp) {
+  memset(S, 0, sizeof(double) * (size_t)d * (size_t)d);
+  memset(z, 0, sizeof(double) * (size_t)d);
+  for (long j = 0; j < N; ++j)
+    for (int a = 0; a < d; ++a) {
+      double kp = gfo_phi(k[j * d + a]);
+      for (int c = 0; c < d; ++c) S[a * d + c] += kp * v[j * d + c];
+      z[a] += kp;
+    }
+  for (long i = 0; i < N; ++i) {
+    double den = 0.0;
+    for (int a = 0; a < d; ++a) {
+      qp[a] = gfo_phi(q[i * d + a]);
+      den += qp[a] * z[a];
+    }
+    for (int c = 0; c < d; ++c) {
+      double num = 0.0;
+      for (int a = 0; a < d; ++a) num += qp[a] * S[a * d + c];
+      o[i * d + c] = num / den;
+    }
+  }
+}
+
+/* The "self" hybrid layer: heads [0, h_sparse) two-sided windowed, heads [h_sparse, H) global
+ * linear (Sec. III-A routing, unchanged). */
+void gfo_hybrid_attn_self(const double* q, const double* k, const double* v, double* o,
+                          long B, long H, long N, int d, long w, long h_sparse, double scale) {
+  long span = 2 * w - 1 < N ? 2 * w - 1 : N;
+#pragma omp parallel
+  {
+    double* e = (double*)malloc(sizeof(double) * (size_t)(span > 0 ? span : 1));
+    double* S = (double*)malloc(sizeof(double) * ((size_t)d * (size_t)d + 2 * (size_t)d));
+#pragma omp for schedule(dynamic, 1)
+    for (long bh = 0; bh < B * H; ++bh) {
+      size_t off = (size_t)bh * (size_t)N * (size_t)d;
+      if (bh % H < h_sparse) window_head_sym(q + off, k + off, v + off, o + off, N, d, w, scale, e);
+      else linear_head_global(q + off, k + off, v + off, o + off, N, d, S, S + (size_t)d * d, S + (size_t)d * d + d);
+    }
+    free(e);
+    free(S);
   }
 }
 

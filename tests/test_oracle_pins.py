@@ -315,3 +315,68 @@ def test_prefill_export_then_decode_equals_one_long_sequence(N0, w):
     for t in range(N0, N):
         o = oracle.decode_step(q[:, :, t], k[:, :, t], v[:, :, t], st)
         np.testing.assert_allclose(o, ref[:, :, t], rtol=1e-11, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------- "self" (bidirectional) layer
+# The next row of the scope table has its oracle first; these pins are what fixes it.
+def test_self_window_covering_the_sequence_is_library_softmax_attention():
+    q, k, v = rnd((2, 2, 37, 16), 501), rnd((2, 2, 37, 16), 502), rnd((2, 2, 37, 16), 503)
+    for w in (37, 38, 500):  # |i - j| < w holds for every pair: plain Eq. 1, no mask
+        got = oracle.window_attn_self(q, k, v, w)
+        ref = torch.nn.functional.scaled_dot_product_attention(
+            torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v)).numpy()
+        np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-12)
+
+
+@pytest.mark.parametrize("N,w", [(1, 1), (9, 1), (9, 2), (23, 5), (40, 17), (40, 39)])
+def test_self_window_equals_library_attention_with_an_explicit_band_mask(N, w):
+    q, k, v = rnd((1, 3, N, 8), 510 + N), rnd((1, 3, N, 8), 511 + N), rnd((1, 3, N, 8), 512 + N)
+    i = torch.arange(N)[:, None]
+    j = torch.arange(N)[None, :]
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q), torch.from_numpy(k), torch.from_numpy(v), attn_mask=(i - j).abs() < w).numpy()
+    np.testing.assert_allclose(oracle.window_attn_self(q, k, v, w), ref, rtol=1e-11, atol=1e-12)
+
+
+def test_self_window_mirror_symmetry_and_relation_to_the_causal_window():
+    q, k, v = rnd((1, 2, 50, 8), 520), rnd((1, 2, 50, 8), 521), rnd((1, 2, 50, 8), 522)
+    w = 7
+    fwd = oracle.window_attn_self(q, k, v, w)
+    rev = oracle.window_attn_self(q[:, :, ::-1], k[:, :, ::-1], v[:, :, ::-1], w)
+    np.testing.assert_allclose(rev[:, :, ::-1], fwd, rtol=1e-12, atol=1e-13)  # the rule has no direction
+    # the last row has nothing to its right: it is the causal window's last row
+    np.testing.assert_allclose(fwd[:, :, -1], oracle.window_attn(q, k, v, w)[:, :, -1], rtol=1e-12, atol=1e-13)
+    # w = 1: every token sees only itself
+    np.testing.assert_allclose(oracle.window_attn_self(q, k, v, 1), v, rtol=0, atol=1e-15)
+    # a needle w - 1 to the right is seen, one at distance w is not
+    qn = np.zeros((1, 1, 30, 4)); kn = np.zeros((1, 1, 30, 4)); vn = np.zeros((1, 1, 30, 4))
+    qn[0, 0, 10, 0] = 30.0; kn[0, 0, 16, 0] = 30.0; vn[0, 0, 16, :] = 1.0
+    assert oracle.window_attn_self(qn, kn, vn, 7, scale=1.0)[0, 0, 10, 0] > 0.99
+    assert oracle.window_attn_self(qn, kn, vn, 6, scale=1.0)[0, 0, 10, 0] == 0.0
+
+
+def test_self_linear_equals_the_quadratic_unmasked_form_and_the_causal_last_row():
+    q, k, v = rnd((2, 2, 33, 8), 530), rnd((2, 2, 33, 8), 531), rnd((2, 2, 33, 8), 532)
+    got = oracle.linear_attn_self(q, k, v)
+    # (phi(Q) phi(K)^T) V with rows normalised: the N x N attention matrix written out
+    A = np.einsum("bhia,bhja->bhij", np_phi(q), np_phi(k))
+    ref = np.einsum("bhij,bhjc->bhic", A / A.sum(axis=-1, keepdims=True), v)
+    np.testing.assert_allclose(got, ref, rtol=1e-11, atol=1e-12)
+    # the last token of Algorithm 1 has seen every key: same row
+    np.testing.assert_allclose(got[:, :, -1], oracle.causal_linear_attn(q, k, v)[:, :, -1], rtol=1e-11, atol=1e-12)
+    # the keys form a set: permuting (k_j, v_j) pairs changes nothing; permuting queries permutes rows
+    perm = np.random.default_rng(5).permutation(33)
+    np.testing.assert_allclose(oracle.linear_attn_self(q, k[:, :, perm], v[:, :, perm]), got, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(oracle.linear_attn_self(q[:, :, perm], k, v), got[:, :, perm], rtol=1e-11, atol=1e-12)
+    # rows are convex combinations of the values (phi > 0): constant values come back, outputs stay in range
+    np.testing.assert_allclose(oracle.linear_attn_self(q, k, np.full_like(v, 2.5)), 2.5, rtol=1e-12)
+    assert (got <= v.max(axis=2, keepdims=True) + 1e-12).all() and (got >= v.min(axis=2, keepdims=True) - 1e-12).all()
+
+
+def test_self_hybrid_routes_heads_like_the_causal_layer():
+    q, k, v = rnd((2, 5, 21, 8), 540), rnd((2, 5, 21, 8), 541), rnd((2, 5, 21, 8), 542)
+    o = oracle.hybrid_attn_self(q, k, v, 4, h_sparse=2)
+    np.testing.assert_array_equal(o[:, :2], oracle.window_attn_self(q[:, :2], k[:, :2], v[:, :2], 4))
+    np.testing.assert_array_equal(o[:, 2:], oracle.linear_attn_self(q[:, 2:], k[:, 2:], v[:, 2:]))
+    assert oracle.hybrid_attn_self(q, k, v, 4).shape == q.shape  # default split: max(1, round(3 H / 16)) = 1
+    np.testing.assert_array_equal(oracle.hybrid_attn_self(q, k, v, 4)[:, 1:], oracle.linear_attn_self(q[:, 1:], k[:, 1:], v[:, 1:]))
