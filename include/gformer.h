@@ -113,6 +113,18 @@ int gformer_window_attn(const void* q, const void* k, const void* v, void* o,
                         int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * The windowed heads of the bidirectional ("self") layer (Sec. II-A: tokens attend to the
+ * left and to the right, as in ViT): Eq. 1 without the causal mask over a two-sided window,
+ *   j in [max(0, i-w+1), min(N-1, i+w-1)]   (the causal window mirrored: |i - j| < w;
+ * the paper prints no two-sided rule, this is the reading taken).  Same arguments, layouts
+ * and errors as gformer_window_attn.  The linear heads of that layer (global linear
+ * attention) have no kernel yet.
+ */
+int gformer_window_attn_self(const void* q, const void* k, const void* v, void* o,
+                        int B, int H, int N, int d, int w, float scale,
+                        int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Causal linear attention on all H heads (Algorithm 1, readout after the updates of
  * step i; phi applied to raw q and k, no logit scale):
  *   S_i = S_{i-1} + phi(k_i) v_i^T,  z_i = z_{i-1} + phi(k_i),

@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
         L.gformer_last_device_status.argtypes = [vp, vp]
         L.gformer_window_attn.restype = i
         L.gformer_window_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp, sz, vp]
+        L.gformer_window_attn_self.restype = i
+        L.gformer_window_attn_self.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp, sz, vp]
         L.gformer_causal_linear_attn.restype = i
         L.gformer_causal_linear_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, vp, i, i, vp, sz, vp]
         L.gformer_noalloc_scratch_bytes.restype = sz
@@ -187,6 +189,20 @@ def window_attn(q, k, v, w: int, scale: float = 0.0, layout: int = GF_BHND, out=
                                    float(scale), dt, layout, W.ptr, W.nbytes, _stream_ptr(stream))
     if rc != GF_OK:
         raise GformerError(rc, "gformer_window_attn")
+    return o
+
+
+def window_attn_self(q, k, v, w: int, scale: float = 0.0, layout: int = GF_BHND, out=None, ws=None, stream=None):
+    """gformer_window_attn_self: softmax attention over the keys with |i - j| < w (no causal mask)."""
+    _check_qkv(q, k, v)
+    B, H, N, d = _dims(q, layout)
+    o = torch.empty_like(q) if out is None else out
+    dt = _dtype_code(q)
+    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, H, dt))
+    rc = lib().gformer_window_attn_self(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, int(w),
+                                        float(scale), dt, layout, W.ptr, W.nbytes, _stream_ptr(stream))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_window_attn_self")
     return o
 
 

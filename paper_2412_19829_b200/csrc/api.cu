@@ -86,13 +86,14 @@ int cuda_status(cudaError_t e) { return e == cudaSuccess ? GF_OK : GF_ERR_CUDA; 
 // Window heads [h_begin, h_begin+h_count) on `stream`.
 int run_window(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
                float scale, int dtype, int layout, int h_begin, int h_count, WsHeader* ws,
-               cudaStream_t stream) {
+               cudaStream_t stream, bool two_sided = false) {
   if (h_count <= 0) return GF_OK;
-  const int w_eff = w > N ? N : w;  // keys before token 0 do not exist
+  const int w_eff = w > N ? N : w;  // keys before token 0 (or after the last one) do not exist
+  const int fwd = two_sided ? w_eff - 1 : 0;
   if (!g_force_simt && gf::tc_window_supported(N, d, w_eff, dtype))
     return cuda_status(
-        gf::launch_window_tc(q, k, v, o, B, H, N, d, w_eff, scale, layout, h_begin, h_count, ws, stream));
-  return cuda_status(gf::launch_window_simt(q, k, v, o, B, N, d, w_eff, scale, dtype,
+        gf::launch_window_tc(q, k, v, o, B, H, N, d, w_eff, fwd, scale, layout, h_begin, h_count, ws, stream));
+  return cuda_status(gf::launch_window_simt(q, k, v, o, B, N, d, w_eff, fwd, scale, dtype,
                                             gf::make_strides(layout, H, N, d), h_begin, h_count, stream));
 }
 
@@ -202,6 +203,21 @@ int gformer_window_attn(const void* q, const void* k, const void* v, void* o, in
   rc = clear_ws(ws, stream);
   if (rc != GF_OK) return rc;
   return run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream);
+}
+
+int gformer_window_attn_self(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                             int w, float scale, int dtype, int layout, void* ws, size_t ws_bytes,
+                             void* cuda_stream) {
+  int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
+  if (rc != GF_OK) return rc;
+  if (w < 1) return GF_ERR_INVALID_ARG;
+  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, H, dtype));
+  if (rc != GF_OK) return rc;
+  if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  rc = clear_ws(ws, stream);
+  if (rc != GF_OK) return rc;
+  return run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream, true);
 }
 
 int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,

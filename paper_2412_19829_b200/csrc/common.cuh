@@ -43,8 +43,9 @@ void note_launch(int n = 1);
 
 // ---- SIMT (CUDA-core, fp32 arithmetic) path: any w, d in {64,128}, f32 or bf16 storage.
 // Heads [h_begin, h_begin + h_count) of the [B, H, N, d] tensors are processed.
+// fwd: keys after the query it may see: 0 = the causal window, w - 1 = the two-sided window |i - j| < w.
 cudaError_t launch_window_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
-                               int w, float scale, int dtype, Strides st, int h_begin, int h_count,
+                               int w, int fwd, float scale, int dtype, Strides st, int h_begin, int h_count,
                                cudaStream_t stream);
 // S_io/z_io: [B, h_count, d, d] / [B, h_count, d] or null.  zero_init: ignore their contents on entry.
 cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
@@ -66,7 +67,7 @@ cudaError_t launch_delay(unsigned int ns, cudaStream_t stream);
 bool tc_window_supported(int N, int d, int w, int dtype);
 bool tc_linear_supported(int N, int d, int dtype);
 cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
-                             int w, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
+                             int w, int fwd, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
                              cudaStream_t stream);
 // Segmentation used by the tensor-core linear kernel (split: 0 = automatic, else chunks per segment;
 // ctas: CTAs the kernel will run with, 0 = one per SM of a B200) and the scratch it needs beyond

@@ -40,7 +40,8 @@ template <> struct Vec4<__nv_bfloat16> {
 template <typename T, int D>
 __global__ void __launch_bounds__(128)
 window_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
-                   T* __restrict__ o, int N, int w, float scale, Strides st, int h_begin) {
+                   T* __restrict__ o, int N, int w, int fwd, float scale, Strides st, int h_begin) {
+  // fwd: keys after the query that it may see (0: the causal window; w - 1: the two-sided one)
   constexpr int CH = D / 16;  // float4 chunks per thread
   __shared__ __align__(16) float Ks[32][D];
   __shared__ __align__(16) float Vs[32][D];
@@ -62,7 +63,7 @@ window_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
 
   int jlo = i0 - w + 1;
   if (jlo < 0) jlo = 0;
-  int jhi = i0 + 31;
+  int jhi = i0 + 31 + fwd;
   if (jhi > N - 1) jhi = N - 1;
 
   for (int j0 = jlo; j0 <= jhi; j0 += 32) {
@@ -90,7 +91,7 @@ window_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
       }
       s += __shfl_xor_sync(0xffffffffu, s, 1);
       s += __shfl_xor_sync(0xffffffffu, s, 2);
-      const bool valid = (i < N) && (j <= i) && (j > i - w);
+      const bool valid = (i < N) && (j <= i + fwd) && (j > i - w) && (j < N);
       if (valid) {
         s *= scale;
         const float m_new = fmaxf(m, s);
@@ -426,13 +427,13 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
 
 template <typename T>
 cudaError_t window_dispatch(const void* q, const void* k, const void* v, void* o, int B, int N, int d, int w,
-                            float scale, Strides st, int h_begin, int h_count, cudaStream_t stream) {
+                            int fwd, float scale, Strides st, int h_begin, int h_count, cudaStream_t stream) {
   dim3 grid((N + 31) / 32, h_count, B);
   if (d == 64)
-    window_simt_kernel<T, 64><<<grid, 128, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, w,
+    window_simt_kernel<T, 64><<<grid, 128, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, w, fwd,
                                                         scale, st, h_begin);
   else
-    window_simt_kernel<T, 128><<<grid, 128, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, w,
+    window_simt_kernel<T, 128><<<grid, 128, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, w, fwd,
                                                          scale, st, h_begin);
   note_launch();
   return cudaGetLastError();
@@ -483,11 +484,12 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, void* o
 }  // namespace
 
 cudaError_t launch_window_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d, int w,
-                               float scale, int dtype, Strides st, int h_begin, int h_count,
+                               int fwd, float scale, int dtype, Strides st, int h_begin, int h_count,
                                cudaStream_t stream) {
   if (h_count <= 0 || B <= 0) return cudaSuccess;
-  if (dtype == GF_F32) return window_dispatch<float>(q, k, v, o, B, N, d, w, scale, st, h_begin, h_count, stream);
-  return window_dispatch<__nv_bfloat16>(q, k, v, o, B, N, d, w, scale, st, h_begin, h_count, stream);
+  if (dtype == GF_F32)
+    return window_dispatch<float>(q, k, v, o, B, N, d, w, fwd, scale, st, h_begin, h_count, stream);
+  return window_dispatch<__nv_bfloat16>(q, k, v, o, B, N, d, w, fwd, scale, st, h_begin, h_count, stream);
 }
 
 cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,

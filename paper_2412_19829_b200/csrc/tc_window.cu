@@ -68,6 +68,7 @@ struct WinSmem {
 
 struct WinParams {
   int N, w, tiles_back;  // tiles_back = number of key tiles before the diagonal one
+  int fwd, tiles_fwd;    // keys after the query it may see (0: causal; w - 1: two-sided) and the tiles they span
   float scale_log2;
   int h_begin, h_count, nqt, total;  // work units: (batch, head, query tile), query tile fastest
   unsigned int* status;
@@ -91,7 +92,7 @@ __device__ __forceinline__ bool win_wait_epoch(const int* counter, int target, u
   return true;
 }
 
-template <int D>
+template <int D, bool kTwoSided>
 __global__ void __launch_bounds__(kThreads, 2)
 window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                  const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
@@ -156,7 +157,9 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
     x.b = bh / p.h_count;
     x.i0 = x.qt * 128;
     x.t_first = (x.qt - p.tiles_back) > 0 ? (x.qt - p.tiles_back) : 0;
-    x.n_tiles = x.qt - x.t_first + 1;
+    // kTwoSided: the tiles after the diagonal one that the window reaches, up to the sequence end
+    const int t_last = !kTwoSided ? x.qt : ((x.qt + p.tiles_fwd) < p.nqt ? (x.qt + p.tiles_fwd) : p.nqt - 1);
+    x.n_tiles = t_last - x.t_first + 1;
     return x;
   };
   auto unit_at = [&](uint32_t n) -> int {
@@ -267,10 +270,13 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         // by 31, so the 64-column half is classified per warp: nothing visible (costs nothing), all
         // visible to every row (no per-element test), or mixed
         const int lo = i - p.w + 1 - j0;
-        const int hi = i - j0;
-        const int lo_first = (i0 + quarter * 32) - p.w + 1 - j0;  // lo of the warp's first row (last row: +31)
-        const int hi_first = (i0 + quarter * 32) - j0;            // hi of the warp's first row (last row: +31)
-        const bool none = (c1 < lo_first || c0 > hi_first + 31);
+        const int i_first = i0 + quarter * 32;  // the warp's first row
+        // (two-sided window: the query also sees p.fwd keys after it, and keys past the end do not exist)
+        const int hi = kTwoSided ? min(i + p.fwd, p.N - 1) - j0 : i - j0;
+        const int lo_first = i_first - p.w + 1 - j0;  // lo of the warp's first row (last row: +31)
+        const int hi_first = kTwoSided ? min(i_first + p.fwd, p.N - 1) - j0 : i_first - j0;  // hi of its first row
+        const int hi_last = kTwoSided ? min(i_first + 31 + p.fwd, p.N - 1) - j0 : hi_first + 31;  // ... of its last row
+        const bool none = (c1 < lo_first || c0 > hi_last);
         const bool inside = (c0 >= lo_first + 31) && (c1 <= hi_first);
         // Two sweeps over the half row (maximum, then exponentials): the scores stay in TMEM between
         // the sweeps, so that few registers are live across the exchange of the maxima.
@@ -453,7 +459,7 @@ bool tc_window_supported(int N, int d, int w, int dtype) {
 }
 
 cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
-                             int w, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
+                             int w, int fwd, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
                              cudaStream_t stream) {
   if (h_count <= 0) return cudaSuccess;
   CUtensorMap mq, mk, mv, mo;
@@ -464,6 +470,8 @@ cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* 
   p.N = N;
   p.w = w;
   p.tiles_back = (w - 1 + 127) / 128;
+  p.fwd = fwd;
+  p.tiles_fwd = (fwd + 127) / 128;
   p.scale_log2 = scale * kLog2e;
   p.h_begin = h_begin;
   p.h_count = h_count;
@@ -480,17 +488,19 @@ cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* 
   // persistent CTAs, two per SM; they never wait for one another, so it does not matter how many
   // of them are resident at a time
   dim3 grid((unsigned)(total < 2LL * sms ? total : 2LL * sms));
-  if (d == 64) {
-    auto kern = window_tc_kernel<64>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, WinSmem<64>::kBytes);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, WinSmem<64>::kBytes, stream>>>(mq, mk, mv, mo, p);
-  } else {
-    auto kern = window_tc_kernel<128>;
-    e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, WinSmem<128>::kBytes);
-    if (e != cudaSuccess) return e;
-    kern<<<grid, kThreads, WinSmem<128>::kBytes, stream>>>(mq, mk, mv, mo, p);
-  }
+  auto launch = [&](auto kern, int smem) -> cudaError_t {
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err != cudaSuccess) return err;
+    kern<<<grid, kThreads, smem, stream>>>(mq, mk, mv, mo, p);
+    return cudaSuccess;
+  };
+  if (d == 64)
+    e = fwd > 0 ? launch(window_tc_kernel<64, true>, WinSmem<64>::kBytes)
+                : launch(window_tc_kernel<64, false>, WinSmem<64>::kBytes);
+  else
+    e = fwd > 0 ? launch(window_tc_kernel<128, true>, WinSmem<128>::kBytes)
+                : launch(window_tc_kernel<128, false>, WinSmem<128>::kBytes);
+  if (e != cudaSuccess) return e;
   note_launch();
   return cudaGetLastError();
 }

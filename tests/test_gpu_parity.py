@@ -81,6 +81,36 @@ def test_window_tensor_core(N, w, d, gain):
     assert_parity(f64(o), ref, "bf16", f"window tc N={N} w={w} d={d}")
 
 
+@pytest.mark.parametrize("dtype,force_simt", [("f32", 0), ("bf16", 1), ("bf16", 0)])
+@pytest.mark.parametrize("N,w,d", [(1, 1, 64), (100, 1, 64), (128, 128, 128), (129, 2, 64), (300, 64, 128), (777, 129, 64),
+                                   (1000, 128, 128), (1030, 300, 128), (640, 5000, 64), (2100, 513, 128)])
+def test_window_self_two_sided(dtype, force_simt, N, w, d):
+    # the windowed heads of the bidirectional layer: keys with |i - j| < w, ragged ends on both sides
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, force_simt)
+    q, k, v = synth.qkv(2, 2, N, d, dtype, seed=300 + N + w, gain=1.0)
+    ref = oracle.window_attn_self(f64(q), f64(k), f64(v), w)
+    ws = gf.Workspace.for_problem(2, 2, N, d, w, 2)
+    o = gf.window_attn_self(*dev(q, k, v), w, ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    kind = "f32" if dtype == "f32" else "bf16"
+    assert_parity(f64(o), ref, kind, f"two-sided window N={N} w={w} d={d} {dtype} simt={force_simt}")
+
+
+def test_window_self_needles_at_both_window_edges_tensor_core():
+    N, d, w = 700, 64, 130
+    q = torch.zeros(1, 1, N, d); k = torch.zeros(1, 1, N, d); v = torch.zeros(1, 1, N, d)
+    i = 300
+    q[0, 0, i, 0] = 8.0
+    for j, val in ((i - w + 1, 1.0), (i + w - 1, 2.0), (i - w, 64.0), (i + w, 128.0)):  # two inside, two just outside
+        k[0, 0, j, 0] = 8.0
+        v[0, 0, j, :] = val
+    qb, kb, vb = (t.to(torch.bfloat16) for t in (q, k, v))
+    ref = oracle.window_attn_self(f64(qb), f64(kb), f64(vb), w, scale=1.0)
+    o = gf.window_attn_self(*dev(qb, kb, vb), w, scale=1.0)
+    assert_parity(f64(o), ref, "bf16", "needles at the two-sided window's edges")
+    assert 1.4 < float(o[0, 0, i, 0]) < 1.6  # both inside needles, neither outside one
+
+
 def test_window_needle_at_window_edges_tensor_core():
     # A key with a dominant logit: every row whose window holds it must return its value row,
     # rows one past the window must not see it.
