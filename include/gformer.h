@@ -117,8 +117,7 @@ int gformer_window_attn(const void* q, const void* k, const void* v, void* o,
  * left and to the right, as in ViT): Eq. 1 without the causal mask over a two-sided window,
  *   j in [max(0, i-w+1), min(N-1, i+w-1)]   (the causal window mirrored: |i - j| < w;
  * the paper prints no two-sided rule, this is the reading taken).  Same arguments, layouts
- * and errors as gformer_window_attn.  The linear heads of that layer (global linear
- * attention) have no kernel yet.
+ * and errors as gformer_window_attn.
  */
 int gformer_window_attn_self(const void* q, const void* k, const void* v, void* o,
                         int B, int H, int N, int d, int w, float scale,
@@ -184,6 +183,19 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o,
                         int phi, int chunk, int dtype, int layout,
                         gf_decode_state* state_out,
                         void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * The bidirectional ("self") layer (Sec. II-A / III-A: the same head split, no causal mask):
+ * heads [0, h_sparse) as gformer_window_attn_self, heads [h_sparse, H) global linear attention,
+ *   S = sum_j phi(k_j) v_j^T,  z = sum_j phi(k_j)  over all j,   o_i = phi(q_i)^T S / (phi(q_i) . z)
+ * (Sec. II-B, rows normalised as in Algorithm 1).  The linear heads need bf16 storage and d in
+ * {64, 128} (GF_ERR_UNSUPPORTED otherwise, also under GF_TUNE_FORCE_SIMT); h_sparse = H runs the
+ * windowed heads alone with any supported dtype.  Workspace: gformer_workspace_bytes.
+ */
+int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* o,
+                             int B, int H, int N, int d, int w, int h_sparse, float scale,
+                             int phi, int dtype, int layout,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * One autoregressive step for token index st->t: q, k, v, o are [B, H, d].  Windowed

@@ -63,6 +63,8 @@ def lib() -> ctypes.CDLL:
         L.gformer_window_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp, sz, vp]
         L.gformer_window_attn_self.restype = i
         L.gformer_window_attn_self.argtypes = [vp, vp, vp, vp, i, i, i, i, i, f, i, i, vp, sz, vp]
+        L.gformer_hybrid_attn_self.restype = i
+        L.gformer_hybrid_attn_self.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, f, i, i, i, vp, sz, vp]
         L.gformer_causal_linear_attn.restype = i
         L.gformer_causal_linear_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, vp, i, i, vp, sz, vp]
         L.gformer_noalloc_scratch_bytes.restype = sz
@@ -203,6 +205,22 @@ def window_attn_self(q, k, v, w: int, scale: float = 0.0, layout: int = GF_BHND,
                                         float(scale), dt, layout, W.ptr, W.nbytes, _stream_ptr(stream))
     if rc != GF_OK:
         raise GformerError(rc, "gformer_window_attn_self")
+    return o
+
+
+def hybrid_attn_self(q, k, v, w: int, h_sparse: int = -1, scale: float = 0.0, layout: int = GF_BHND, out=None,
+                     ws=None, stream=None):
+    """gformer_hybrid_attn_self: the bidirectional layer (two-sided windowed heads, global linear heads)."""
+    _check_qkv(q, k, v)
+    B, H, N, d = _dims(q, layout)
+    o = torch.empty_like(q) if out is None else out
+    dt = _dtype_code(q)
+    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, h_sparse, dt))
+    rc = lib().gformer_hybrid_attn_self(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, int(w),
+                                        int(h_sparse), float(scale), GF_PHI_ELU1, dt, layout, W.ptr, W.nbytes,
+                                        _stream_ptr(stream))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_hybrid_attn_self")
     return o
 
 

@@ -177,8 +177,12 @@ size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, 
   if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
   if (h_sparse > H) h_sparse = H;
   const int h_lin = H - h_sparse;
-  if (h_lin > 0 && !g_force_simt && gf::tc_linear_supported(N, d, dtype))
-    bytes += gf::linear_tc_workspace_bytes(B * h_lin, N, d, g_linear_split);
+  if (h_lin > 0 && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
+    // the causal kernel's hand-over scratch, or the bidirectional layer's segment sums: whichever is larger
+    const size_t causal = gf::linear_tc_workspace_bytes(B * h_lin, N, d, g_linear_split);
+    const size_t self = gf::linear_self_workspace_bytes(B * h_lin, N, d);
+    bytes += causal > self ? causal : self;
+  }
   return bytes;
 }
 
@@ -218,6 +222,29 @@ int gformer_window_attn_self(const void* q, const void* k, const void* v, void* 
   rc = clear_ws(ws, stream);
   if (rc != GF_OK) return rc;
   return run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream, true);
+}
+
+int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                             int w, int h_sparse, float scale, int phi, int dtype, int layout, void* ws,
+                             size_t ws_bytes, void* cuda_stream) {
+  int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
+  if (rc != GF_OK) return rc;
+  if (w < 1) return GF_ERR_INVALID_ARG;
+  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
+  if (h_sparse > H) return GF_ERR_INVALID_ARG;
+  // the global linear heads exist as tensor-core kernels only (bf16 storage, d in {64, 128})
+  if (h_sparse < H && (g_force_simt || !gf::tc_linear_supported(N, d, dtype))) return GF_ERR_UNSUPPORTED;
+  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, h_sparse, dtype));
+  if (rc != GF_OK) return rc;
+  if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
+  cudaStream_t stream = (cudaStream_t)cuda_stream;
+  rc = clear_ws(ws, stream);
+  if (rc != GF_OK) return rc;
+  rc = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, stream, true);
+  if (rc != GF_OK) return rc;
+  return cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
+                                               sizeof(WsHeader), stream));
 }
 
 int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,

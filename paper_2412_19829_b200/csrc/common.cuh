@@ -69,6 +69,12 @@ bool tc_linear_supported(int N, int d, int dtype);
 cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int w, int fwd, float scale, int layout, int h_begin, int h_count, WsHeader* ws,
                              cudaStream_t stream);
+// Global (unmasked) linear attention of the bidirectional layer, heads [h_begin, h_begin + h_count):
+// three launches (segment sums, totals, readout); its scratch starts scratch_offset bytes into ws.
+size_t linear_self_workspace_bytes(int nchains, int N, int d);
+cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                                  int layout, int h_begin, int h_count, WsHeader* ws, size_t scratch_offset,
+                                  cudaStream_t stream);
 // Segmentation used by the tensor-core linear kernel (split: 0 = automatic, else chunks per segment;
 // ctas: CTAs the kernel will run with, 0 = one per SM of a B200) and the scratch it needs beyond
 // the workspace header (sized for the largest segment count the plan may pick for any ctas).

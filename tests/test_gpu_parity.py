@@ -96,6 +96,32 @@ def test_window_self_two_sided(dtype, force_simt, N, w, d):
     assert_parity(f64(o), ref, kind, f"two-sided window N={N} w={w} d={d} {dtype} simt={force_simt}")
 
 
+@pytest.mark.parametrize("B,H,N,d,w,h0", [(1, 2, 128, 128, 16, 0), (2, 3, 300, 64, 40, 1), (1, 4, 1000, 128, 128, 2),
+                                            (2, 2, 129, 64, 1, 0), (1, 3, 2500, 64, 300, 1), (3, 5, 640, 128, 64, 5),
+                                            (1, 2, 5000, 128, 200, 0), (40, 4, 260, 64, 33, 1), (1, 1, 1, 64, 1, 0)])
+def test_self_layer_against_the_oracle(B, H, N, d, w, h0):
+    # the bidirectional layer: two-sided windowed heads, global linear heads (segment sums, totals, readout)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=700 + N + H, gain=1.0)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    o = gf.hybrid_attn_self(*dev(q, k, v), w, h_sparse=h0, ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    bs = sorted({0, B - 1})
+    ref = oracle.hybrid_attn_self(f64(q[bs]), f64(k[bs]), f64(v[bs]), w, h_sparse=h0)
+    assert_parity(f64(o[bs]), ref, "bf16", f"self layer B={B} H={H} N={N} d={d} w={w} h0={h0}")
+
+
+def test_self_layer_is_deterministic_and_merges_by_head():
+    B, H, N, d, w, h0 = 2, 4, 1500, 128, 100, 1
+    q, k, v = dev(*synth.qkv(B, H, N, d, "bf16", seed=777, gain=1.0))
+    a = gf.hybrid_attn_self(q, k, v, w, h_sparse=h0)
+    b = gf.hybrid_attn_self(q, k, v, w, h_sparse=h0)
+    assert torch.equal(a, b)  # segment sums are added in a fixed order
+    assert torch.equal(a[:, :h0], gf.window_attn_self(q[:, :h0].contiguous(), k[:, :h0].contiguous(),
+                                                      v[:, :h0].contiguous(), w))
+    lin = gf.hybrid_attn_self(q[:, h0:].contiguous(), k[:, h0:].contiguous(), v[:, h0:].contiguous(), w, h_sparse=0)
+    assert torch.equal(a[:, h0:], lin)
+
+
 def test_window_self_needles_at_both_window_edges_tensor_core():
     N, d, w = 700, 64, 130
     q = torch.zeros(1, 1, N, d); k = torch.zeros(1, 1, N, d); v = torch.zeros(1, 1, N, d)
