@@ -36,6 +36,8 @@ WORKLOADS = {
     "long32k": dict(B=1, H=32, N=32768, d=128, w=512, seed=2),
     "gpt2s": dict(B=8, H=12, N=2048, d=64, w=128, seed=1),
     "prefill4k": dict(B=64, H=16, N=4096, d=64, w=256, seed=3),
+    # the bidirectional ("self") layer on the long-sequence shape: two-sided windowed heads, global linear heads
+    "self32k": dict(B=1, H=32, N=32768, d=128, w=512, seed=2, self_layer=True),
     # token-by-token decoding after a 4096-token prefill: a step = `steps` decode steps of the batch
     "decode256": dict(B=64, H=16, N=4096, d=64, w=256, seed=3, decode_steps=256),
 }
@@ -217,7 +219,7 @@ def oracle_sample_rate(c, sample_tokens):
     a = [t.to(torch.float64).numpy() for t in (q, k, v)]
     h0 = oracle.default_h_sparse(c["H"])
     t0 = time.perf_counter()
-    oracle.hybrid_attn(a[0], a[1], a[2], c["w"], h_sparse=h0)
+    (oracle.hybrid_attn_self if c.get("self_layer") else oracle.hybrid_attn)(a[0], a[1], a[2], c["w"], h_sparse=h0)
     dt = time.perf_counter() - t0
     return c["B"] * n / dt, dt, n, oracle.num_threads()
 
@@ -321,8 +323,11 @@ def run_ours(args, c, rank, world, local_rank):
             dist.barrier()
         torch.cuda.synchronize()
 
+    self_layer = bool(c.get("self_layer"))
+    layer = gf.hybrid_attn_self if self_layer else gf.hybrid_attn
+
     def step():
-        gf.hybrid_attn(dq, dk, dv, w, h_sparse=h0, out=do, ws=ws, stream=stream)
+        layer(dq, dk, dv, w, h_sparse=h0, out=do, ws=ws, stream=stream)
 
     def step_e2e():
         with torch.cuda.stream(stream):
@@ -375,9 +380,15 @@ def run_ours(args, c, rank, world, local_rank):
         lq, lk, lv, lo_ = dq[:, h0:], dk[:, h0:], dv[:, h0:], do[:, h0:]
         wq, wk, wv, wo_ = dq[:, :h0], dk[:, :h0], dv[:, :h0], do[:, :h0]
         ws_l = gf.Workspace.for_problem(B, H - h0, N, d, 1, 0)
-        lin = lambda: gf.causal_linear_attn(lq, lk, lv, out=lo_, ws=ws_l, stream=stream)
-        win = lambda: gf.window_attn(wq, wk, wv, w, out=wo_, ws=ws, stream=stream)
-        for name, fn, heads in (("linear_tc_kernel", lin, H - h0), ("window_tc_kernel", win, h0)):
+        if self_layer:
+            lin = lambda: gf.hybrid_attn_self(lq, lk, lv, w, h_sparse=0, out=lo_, ws=ws_l, stream=stream)
+            win = lambda: gf.window_attn_self(wq, wk, wv, w, out=wo_, ws=ws, stream=stream)
+            names = ("linear_self kernels (reduce, sum, readout)", "window_tc_kernel (two-sided)")
+        else:
+            lin = lambda: gf.causal_linear_attn(lq, lk, lv, out=lo_, ws=ws_l, stream=stream)
+            win = lambda: gf.window_attn(wq, wk, wv, w, out=wo_, ws=ws, stream=stream)
+            names = ("linear_tc_kernel", "window_tc_kernel")
+        for name, fn, heads in ((names[0], lin, H - h0), (names[1], win, h0)):
             for _ in range(3):
                 fn()
             ms, _ = timed(fn, args.steps)
@@ -584,6 +595,8 @@ def algorithmic_flops(c, h0):
     B, H, N, d, w = c["B"], c["H"], c["N"], c["d"], c["w"]
     we = min(w, N)
     pairs = N * we - we * (we - 1) // 2
+    if c.get("self_layer"):  # |i - j| < w: the causal band and its mirror share the diagonal
+        pairs = 2 * pairs - N
     return B * (h0 * 4 * d * pairs + (H - h0) * 4 * N * d * d)
 
 

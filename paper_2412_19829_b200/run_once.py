@@ -1,6 +1,8 @@
 """Runs one entry point twice on random bf16 inputs (a small driver for profilers).
 
-    python -m paper_2412_19829_b200.run_once {linear|window|hybrid} B H N d w
+    python -m paper_2412_19829_b200.run_once {linear|window|hybrid|self} B H N d w
+
+(`self`: the bidirectional layer with all heads linear, i.e. its three linear-attention kernels.)
 """
 import sys
 
@@ -20,6 +22,8 @@ def main(argv):
             gf.causal_linear_attn(q, k, v, out=o)
         elif kind == "window":
             gf.window_attn(q, k, v, w, out=o)
+        elif kind == "self":
+            gf.hybrid_attn_self(q, k, v, w, h_sparse=0, out=o)
         else:
             gf.hybrid_attn(q, k, v, w, out=o)
     torch.cuda.synchronize()
