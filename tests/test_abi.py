@@ -194,3 +194,30 @@ def test_ragged_decode_argument_errors():
     assert L.gformer_decode_step_ragged(a[0], a[1], a[2], 0, ctypes.byref(st), FAKE + (8 << 20), 0.0, gf.GF_PHI_ELU1,
                                         None) == gf.GF_ERR_INVALID_ARG
     assert st.t == 0
+
+
+def test_self_layer_argument_errors():
+    L = gf.lib()
+    a = dict(q=FAKE, k=FAKE + (1 << 30), v=FAKE + (2 << 30), o=FAKE + (3 << 30), B=1, H=4, N=256, d=64, w=32,
+             h_sparse=1, scale=0.0, phi=gf.GF_PHI_ELU1, dtype=gf.GF_BF16, layout=gf.GF_BHND, ws=FAKE + (4 << 30),
+             ws_bytes=1 << 30)
+    order = ("q", "k", "v", "o", "B", "H", "N", "d", "w", "h_sparse", "scale", "phi", "dtype", "layout", "ws", "ws_bytes")
+
+    def call(**kw):
+        b = dict(a, **kw)
+        return L.gformer_hybrid_attn_self(*[b[n] for n in order], None)
+
+    assert call(q=0) == gf.GF_ERR_INVALID_ARG
+    assert call(w=0) == gf.GF_ERR_INVALID_ARG
+    assert call(h_sparse=5) == gf.GF_ERR_INVALID_ARG
+    assert call(d=96) == gf.GF_ERR_UNSUPPORTED
+    assert call(phi=1) == gf.GF_ERR_UNSUPPORTED
+    assert call(dtype=gf.GF_F32) == gf.GF_ERR_UNSUPPORTED      # the global linear heads are bf16 tensor-core kernels only
+    assert call(ws_bytes=8) == gf.GF_ERR_WORKSPACE
+    assert call(ws=0) == gf.GF_ERR_WORKSPACE
+    # the bidirectional layer's segment sums fit the workspace the size query reports
+    for chains, N, d in ((1, 128, 64), (26, 32768, 128), (832, 4096, 64), (3, 100000, 128)):
+        ws = gf.workspace_bytes(1, chains, N, d, 1, 0, gf.GF_BF16)
+        nch = -(-N // 128)
+        G = max(1, min(-(-296 // chains), (nch + 3) // 4))
+        assert ws >= 256 + chains * (G + 1) * (d * d + d) * 4
