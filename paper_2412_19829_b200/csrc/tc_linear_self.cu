@@ -524,13 +524,26 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
   if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
-// Segments per chain: enough items for two rounds of the SMs, segments of at least four chunks.
+// Segments per chain.  CTAs take items (segments) round-robin, so a launch lasts ceil(items / CTAs)
+// rounds of one item each: among the segment counts that keep segments at least four chunks long
+// (and the scratch within 64 slots per chain), take the one with the least rounds x (chunks of the
+// longest segment + about one chunk of fixed cost per item).  The plan must not depend on the
+// device that is current when the workspace size is asked for: it assumes the 148 SMs of a B200.
 int self_segments(int nchains, int nch) {
-  int G = (296 + nchains - 1) / nchains;
-  const int g_max = (nch + 3) / 4;
-  if (G > g_max) G = g_max;
-  if (G < 1) G = 1;
-  return G;
+  constexpr int kPlanSMs = 148;
+  int g_max = (nch + 3) / 4;
+  if (g_max > 64) g_max = 64;
+  int best_g = 1;
+  long long best = -1;
+  for (int g = 1; g <= g_max; ++g) {
+    const long long rounds = ((long long)nchains * g + kPlanSMs - 1) / kPlanSMs;
+    const long long cost = rounds * ((nch + g - 1) / g + 1);
+    if (best < 0 || cost < best) {
+      best = cost;
+      best_g = g;
+    }
+  }
+  return best_g;
 }
 
 }  // namespace
