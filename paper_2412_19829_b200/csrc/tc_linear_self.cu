@@ -288,8 +288,8 @@ struct OutCfg {
   static constexpr int kQ = 0;            // two raw Q tiles
   static constexpr int kSb = 2 * kTile;   // bf16 totals [D rows][D columns] in 64-column boxes ...
   static constexpr int kZb = kSb + D * D * 2;  // ... followed by one more box: columns 0, 1 = hi(z), lo(z)
-  static constexpr int kStage = kZb + kSbBox;  // output tile staged for the TMA store
-  static constexpr int kBytes = kStage + kTile + 1024;
+  static constexpr int kStage = kZb + kSbBox;  // two output tiles staged for the TMA store
+  static constexpr int kBytes = kStage + 2 * kTile + 1024;
   static constexpr int kAcc = D + 16;
   static constexpr uint32_t tQ = 0, tO = D;  // phi(Q): 2 x D/2 columns; O | den: 2 x (D + 16)
   static constexpr int kThreads = 15 * 32;
@@ -307,7 +307,7 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
   uint8_t* sZb = sm + C::kZb;
   uint8_t* sStage = sm + C::kStage;
   __shared__ __align__(8) uint64_t q_full[2], q_free[2], qphi_full[2], tq_free[2], o_full[2], o_free[2], sb_ready,
-      o_staged, stage_free;
+      o_staged[2], stage_free[2];
   __shared__ uint32_t tmem_base_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
@@ -321,8 +321,10 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
       mbar_init(&o_free[i], 128);
     }
     mbar_init(&sb_ready, 128);
-    mbar_init(&o_staged, 128);
-    mbar_init(&stage_free, 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&o_staged[i], 128);
+      mbar_init(&stage_free[i], 1);
+    }
     mbar_fence_init();
     tma_prefetch_desc(&mq);
     tma_prefetch_desc(&mo);
@@ -420,7 +422,7 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
       for (int j = 0; j < it.nC; ++j, ++nq) {
         const uint32_t s = nq & 1;
         if (!mbar_wait(&o_full[s], (nq >> 1) & 1, p.status, 820) ||
-            (nq >= 1 && !mbar_wait(&stage_free, (nq + 1) & 1, p.status, 821))) {
+            (nq >= 2 && !mbar_wait(&stage_free[s], ((nq >> 1) + 1) & 1, p.status, 821))) {
           ok = false;
           break;
         }
@@ -442,13 +444,13 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
             val.y = pack_bf16(__uint_as_float(v[8 * g + 2]) * inv, __uint_as_float(v[8 * g + 3]) * inv);
             val.z = pack_bf16(__uint_as_float(v[8 * g + 4]) * inv, __uint_as_float(v[8 * g + 5]) * inv);
             val.w = pack_bf16(__uint_as_float(v[8 * g + 6]) * inv, __uint_as_float(v[8 * g + 7]) * inv);
-            *reinterpret_cast<uint4*>(sStage + (cc >> 1) * kBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
+            *reinterpret_cast<uint4*>(sStage + s * C::kTile + (cc >> 1) * kBox + swz128_offset(r, (cc & 1) * 32 + g * 8)) = val;
           }
         }
         tc_fence_before_sync();
         mbar_arrive(&o_free[s]);
         fence_proxy_async_smem();
-        mbar_arrive(&o_staged);
+        mbar_arrive(&o_staged[s]);
       }
     }
   } else if (warp < 14) {
@@ -508,12 +510,16 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
       for (int item = blockIdx.x; item < p.nitems && ok; item += gridDim.x) {
         const SelfItem it = self_item(p, item);
         for (int j = 0; j < it.nC; ++j, ++nq) {
-          if (!mbar_wait(&o_staged, nq & 1, p.status, 840)) { ok = false; break; }
+          const uint32_t s = nq & 1;
+          if (!mbar_wait(&o_staged[s], (nq >> 1) & 1, p.status, 840)) { ok = false; break; }
           for (int x = 0; x < D / 64; ++x)
-            tma_store_4d_hint(&mo, sStage + x * kBox, x * 64, (it.c_begin + j) * 128, it.h, it.b, pol);
+            tma_store_4d_hint(&mo, sStage + s * C::kTile + x * kBox, x * 64, (it.c_begin + j) * 128, it.h, it.b, pol);
           tma_store_commit();
-          tma_store_wait_read<0>();
-          mbar_arrive(&stage_free);
+          // the other buffer's store (the previous chunk's) has read its tile: hand that buffer back
+          if (nq >= 1) {
+            tma_store_wait_read<1>();
+            mbar_arrive(&stage_free[s ^ 1]);
+          }
         }
       }
       tma_store_wait_all<0>();
