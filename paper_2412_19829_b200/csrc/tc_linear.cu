@@ -380,7 +380,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   // box x of V slot sv (also the staging buffer of the O tile), of the Q landing buffer
   auto v_box = [&](int sv, int x) -> uint8_t* { return sm + C::v_off(sv) + x * C::v_lbo(sv); };
   constexpr int VS = C::kVSlots;
-  constexpr int KS = (kDirect && D == 64) ? 4 : 2;  // K ring of the chunk pipeline
+  constexpr int KS = (D == 64) ? 4 : 2;  // K ring of the chunk pipeline (its slots 0, 1 also serve pass A)
   auto q_box = [&](int slot, int x) -> uint8_t* { return sm + C::kQ + slot * C::kTile + x * C::kQStride; };
   constexpr int QL = C::kQLand;
   uint8_t* sSb = sm + C::kSb;
@@ -507,7 +507,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             } else {
               const uint32_t sc = nq % KS;
               ok = drain(&bar.k_free[sc], obs_c[sc], iss_c[sc], 104) &&
-                   (kDirect || drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101));
+                   (kDirect || sc >= 2 || drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101));
               if (!ok) break;
               mbar_arrive_expect_tx(&bar.k_full[sc], C::kTile);
               for (int x = 0; x < D / 64; ++x)  // the phi(K) tile parked in the output rows (kDirect: raw K)
