@@ -133,7 +133,7 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
 
 struct LinBarriers {
   uint64_t q_full[2];  // raw Q tiles (landing buffer = chunk count % kQLand)
-  uint64_t ka_full[3], kphi_full[3], ka_free[3];  // K tiles of pass A (slot = tile count % 3)
+  uint64_t ka_full[5], kphi_full[5], ka_free[5];  // K tiles of pass A (slot = tile count % KA)
   uint64_t k_full[4], k_free[4];                  // K tiles of pass C (slot = chunk count % KS)
   uint64_t v_full[4], v_free[4];                  // V tiles of both passes (slot = tile count % kVSlots)
   uint64_t qphi_full[2], qphi_free[2];
@@ -396,7 +396,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   if (tid == 0) {
     mbar_init(&bar.q_full[0], 1);
     mbar_init(&bar.q_full[1], 1);
-    for (int s = 0; s < 3; ++s) {
+    for (int s = 0; s < 5; ++s) {
       mbar_init(&bar.ka_full[s], 1);
       mbar_init(&bar.kphi_full[s], 16);
       mbar_init(&bar.ka_free[s], 2);  // the MMA issuer and the store warp
@@ -458,9 +458,11 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   const uint32_t tmem = tmem_base_s;
 
   // Every role walks the same item list and keeps the same running counters: ta = K tiles of pass
-  // A so far (slot = ta % 3, phase = ta / 3), nq = pass-C chunks so far (K slot = nq % KS, phase =
+  // A so far (slot = ta % KA, phase = ta / KA), nq = pass-C chunks so far (K slot = nq % KS, phase =
   // nq / KS), nv = V tiles of both passes so far (slot = nv % VS, phase = nv / VS).
-  auto a_kslot = [&](uint32_t slot) -> uint8_t* { return slot < 2 ? sK + slot * C::kTile : sm + C::kKA2; };
+  // pass A runs its K tiles through the K ring's slots and one more (KA in all)
+  constexpr int KA = KS + 1;
+  auto a_kslot = [&](uint32_t slot) -> uint8_t* { return slot < (uint32_t)KS ? sK + slot * C::kTile : sm + C::kKA2; };
 
   if (warp == 0) {
     // ================================================================ TMA producer
@@ -470,7 +472,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       // serves both passes is only reloaded once its uses of either kind have drained: per barrier,
       // uses issued so far against phases already observed.
       uint32_t ta = 0, nv = 0, nq = 0, n_items = 0;
-      uint32_t iss_a[3] = {0, 0, 0}, obs_a[3] = {0, 0, 0}, iss_c[4] = {0, 0, 0, 0}, obs_c[4] = {0, 0, 0, 0}, obs_sbi = 0;
+      uint32_t iss_a[5] = {0, 0, 0, 0, 0}, obs_a[5] = {0, 0, 0, 0, 0}, iss_c[4] = {0, 0, 0, 0}, obs_c[4] = {0, 0, 0, 0}, obs_sbi = 0;
       bool ok = true;
       auto drain = [&](uint64_t* b, uint32_t& obs, uint32_t issued, unsigned int where) -> bool {
         while (obs < issued) {
@@ -490,12 +492,18 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           for (int j = 0; j < it.nC; ++j) {
             const int n0 = (it.c_begin + j) * 128;
             if (pass == 0) {
-              const uint32_t sa = ta % 3;
+              const uint32_t sa = ta % KA;
               // the slot's earlier pass-A uses, and what shares the buffer in pass C: a K slot, or
               // (third slot) the Sb operand, idle once the previous item's last readout is done
-              ok = drain(&bar.ka_free[sa], obs_a[sa], iss_a[sa], 101) &&
-                   (sa < 2 ? drain(&bar.k_free[sa], obs_c[sa], iss_c[sa], 104)
-                           : drain(&bar.sb_idle, obs_sbi, n_items, 105));
+              // (sb_idle completes once per item whether or not the item's tiles reach this slot, so
+              // several of its phases may be outstanding: they complete in order, only the last one
+              // is waited for -- a parity wait on an older phase could block on the current one)
+              ok = drain(&bar.ka_free[sa], obs_a[sa], iss_a[sa], 101);
+              if (ok && sa < KS) ok = drain(&bar.k_free[sa], obs_c[sa], iss_c[sa], 104);
+              if (ok && sa >= KS && obs_sbi < n_items) {
+                ok = mbar_wait(&bar.sb_idle, (n_items - 1) & 1, p.status, 105);
+                obs_sbi = n_items;
+              }
               if (!ok) break;
               PROF(0, ta, 1);
               mbar_arrive_expect_tx(&bar.ka_full[sa], C::kTile);
@@ -507,7 +515,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             } else {
               const uint32_t sc = nq % KS;
               ok = drain(&bar.k_free[sc], obs_c[sc], iss_c[sc], 104) &&
-                   (kDirect || sc >= 2 || drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101));
+                   (kDirect || drain(&bar.ka_free[sc], obs_a[sc], iss_a[sc], 101));
               if (!ok) break;
               mbar_arrive_expect_tx(&bar.k_full[sc], C::kTile);
               for (int x = 0; x < D / 64; ++x)  // the phi(K) tile parked in the output rows (kDirect: raw K)
@@ -553,8 +561,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         first_item = false;
         // ---- pass A: dS = sum Kc^T V over the segment, from zero (only if somebody needs it)
         for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
-          const uint32_t sa = ta % 3;
-          if (!mbar_wait(&bar.kphi_full[sa], (ta / 3) & 1, p.status, 220)) { ok = false; break; }
+          const uint32_t sa = ta % KA;
+          if (!mbar_wait(&bar.kphi_full[sa], (ta / KA) & 1, p.status, 220)) { ok = false; break; }
           PROF(1, ta, 4);
           if (it.need_dS) {
             const int sv = nv % VS;
@@ -850,8 +858,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       if (kDirect) transform_direct(nq, 0);
       // ---- pass A: the K group takes rows 0..63 (by sixteens) of every K tile, the Q group rows 64..127
       for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
-        const uint32_t sk = ta % 3;
-        ok = ok && mbar_wait(&bar.ka_full[sk], (ta / 3) & 1, p.status, 410);
+        const uint32_t sk = ta % KA;
+        ok = ok && mbar_wait(&bar.ka_full[sk], (ta / KA) & 1, p.status, 410);
         if (tid == 14 * 32) PROF(3, ta, 4);
         const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
         if (ok && tt < 2 * D)
@@ -1075,8 +1083,8 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         const LinItem it = decode_item(p, item);
         // ---- pass A: park phi(K) tiles in the output rows of their chunk
         for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
-          const uint32_t sk = ta % 3;
-          if (!mbar_wait(&bar.kphi_full[sk], (ta / 3) & 1, p.status, 520)) { ok = false; break; }
+          const uint32_t sk = ta % KA;
+          if (!mbar_wait(&bar.kphi_full[sk], (ta / KA) & 1, p.status, 520)) { ok = false; break; }
           for (int x = 0; x < D / 64; ++x)
             tma_store_4d_hint(&mo, a_kslot(sk) + x * C::kBoxBytes, x * 64, (it.c_begin + j) * 128, it.h, it.b,
                               pol_keep);

@@ -349,6 +349,22 @@ def test_random_layer_shapes(B, H, N, d, w, h0):
     assert_parity(f64(o[bs]), ref, "bf16", f"B={B} H={H} N={N} d={d} w={w} h0={h0}")
 
 
+@pytest.mark.parametrize("d,split", [(128, 1), (128, 2), (64, 2), (64, 4)])
+def test_many_short_segments_per_cta(d, split):
+    # segments shorter than the streaming pass's slot ring, many of them per CTA: some items never
+    # reach the last slot, whose buffer-idle barrier then runs several phases ahead of the producer
+    B, H, N = 2, 100, 1024
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
+    assert gf.linear_plan(B * H, N, d) == (8 // split, split)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=83, gain=1.0)
+    ws = gf.Workspace.for_problem(B, H, N, d, 1, 0)
+    o = gf.causal_linear_attn(*dev(q, k, v), ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    lh = [0, 51, H - 1]
+    ref = oracle.causal_linear_attn(f64(q[:, lh]), f64(k[:, lh]), f64(v[:, lh]))
+    assert_parity(f64(o[:, lh]), ref, "bf16", f"segments of {split} chunks, d={d}")
+
+
 @pytest.mark.parametrize("ctas", [1, 37, 100])
 def test_linear_cta_limit_gives_the_same_result(ctas):
     # the segment plan follows the number of CTAs the persistent kernel is given; any count must
