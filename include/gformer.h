@@ -188,9 +188,9 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o,
  * The bidirectional ("self") layer (Sec. II-A / III-A: the same head split, no causal mask):
  * heads [0, h_sparse) as gformer_window_attn_self, heads [h_sparse, H) global linear attention,
  *   S = sum_j phi(k_j) v_j^T,  z = sum_j phi(k_j)  over all j,   o_i = phi(q_i)^T S / (phi(q_i) . z)
- * (Sec. II-B, rows normalised as in Algorithm 1).  The linear heads need bf16 storage and d in
- * {64, 128} (GF_ERR_UNSUPPORTED otherwise, also under GF_TUNE_FORCE_SIMT); h_sparse = H runs the
- * windowed heads alone with any supported dtype.  Workspace: gformer_workspace_bytes.
+ * (Sec. II-B, rows normalised as in Algorithm 1).  bf16 storage takes the tensor-core kernels,
+ * fp32 storage (or GF_TUNE_FORCE_SIMT) CUDA-core kernels in fp32 arithmetic, as in the causal
+ * layer.  Workspace: gformer_workspace_bytes.
  */
 int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* o,
                              int B, int H, int N, int d, int w, int h_sparse, float scale,

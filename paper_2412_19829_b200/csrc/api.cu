@@ -233,8 +233,6 @@ int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* 
   if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
   if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
   if (h_sparse > H) return GF_ERR_INVALID_ARG;
-  // the global linear heads exist as tensor-core kernels only (bf16 storage, d in {64, 128})
-  if (h_sparse < H && (g_force_simt || !gf::tc_linear_supported(N, d, dtype))) return GF_ERR_UNSUPPORTED;
   rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, h_sparse, dtype));
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
@@ -243,8 +241,13 @@ int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* 
   if (rc != GF_OK) return rc;
   rc = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, stream, true);
   if (rc != GF_OK) return rc;
-  return cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
-                                               sizeof(WsHeader), stream));
+  if (h_sparse == H) return GF_OK;
+  if (!g_force_simt && gf::tc_linear_supported(N, d, dtype))
+    return cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
+                                                 sizeof(WsHeader), stream));
+  // fp32 storage (or the CUDA-core knob): token by token, a summing sweep and a readout sweep
+  return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d), h_sparse,
+                                            H - h_sparse, nullptr, nullptr, true, stream, true));
 }
 
 int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,

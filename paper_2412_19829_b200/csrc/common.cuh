@@ -48,9 +48,10 @@ cudaError_t launch_window_simt(const void* q, const void* k, const void* v, void
                                int w, int fwd, float scale, int dtype, Strides st, int h_begin, int h_count,
                                cudaStream_t stream);
 // S_io/z_io: [B, h_count, d, d] / [B, h_count, d] or null.  zero_init: ignore their contents on entry.
+// global_sum: the unmasked linear attention of the bidirectional layer (sum over all tokens, then readout).
 cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
                                int dtype, Strides st, int h_begin, int h_count, float* S_io, float* z_io,
-                               bool zero_init, cudaStream_t stream);
+                               bool zero_init, cudaStream_t stream, bool global_sum = false);
 cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void* v_cache, int B, int N, int d,
                                int w, int dtype, Strides st, int h_sparse, cudaStream_t stream);
 // t_seq == nullptr: every sequence is at position t; else sequence b is at t_seq[b] (device array,

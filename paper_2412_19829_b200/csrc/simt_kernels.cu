@@ -125,12 +125,14 @@ window_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
 // One CTA = one head x one slice of 32 value columns.  Warp g owns features
 // a in [g*D/8, (g+1)*D/8); lane c owns value column c of the slice.  S lives in registers
 // (D/8 per thread), z is replicated per lane.  Tokens are staged 16 at a time.
+// global_sum != 0: the unmasked form of the bidirectional layer (Sec. II-B) -- a first sweep over
+// the tokens only accumulates S and z, a second one only reads them out.
 // ------------------------------------------------------------------------------------
 template <typename T, int D>
 __global__ void __launch_bounds__(256)
 linear_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                    T* __restrict__ o, int N, Strides st, int h_begin, int h_count,
-                   float* __restrict__ S_io, float* __restrict__ z_io, int zero_init) {
+                   float* __restrict__ S_io, float* __restrict__ z_io, int zero_init, int global_sum) {
   constexpr int TB = 16;
   constexpr int AR = D / 8;
   __shared__ float qs[TB][D];
@@ -159,6 +161,8 @@ linear_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
     }
   }
 
+  for (int sweep = global_sum ? 0 : 1; sweep < 2; ++sweep) {
+  const bool accumulate = !global_sum || sweep == 0, readout = !global_sum || sweep == 1;
   for (int n0 = 0; n0 < N; n0 += TB) {
     __syncthreads();
     for (int idx = tid; idx < TB * D; idx += 256) {
@@ -184,7 +188,7 @@ linear_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
       float num = 0.f, den = 0.f;
 #pragma unroll
       for (int a = 0; a < AR; ++a) {
-        const float kk = ks[tok][g * AR + a];
+        const float kk = accumulate ? ks[tok][g * AR + a] : 0.f;
         const float qq = qs[tok][g * AR + a];
         S[a] = fmaf(kk, vv, S[a]);
         zr[a] += kk;
@@ -204,8 +208,9 @@ linear_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
         num += red[tok][gg][cc];
         den += redden[tok][gg];
       }
-      if (n < N) o[base + (long long)n * st.n + slice * 32 + cc] = from_f32<T>(num / den);
+      if (n < N && readout) o[base + (long long)n * st.n + slice * 32 + cc] = from_f32<T>(num / den);
     }
+  }
   }
   if (S_io != nullptr) {
 #pragma unroll
@@ -442,14 +447,14 @@ cudaError_t window_dispatch(const void* q, const void* k, const void* v, void* o
 template <typename T>
 cudaError_t linear_dispatch(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
                             Strides st, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                            cudaStream_t stream) {
+                            bool global_sum, cudaStream_t stream) {
   dim3 grid(d / 32, h_count, B);
   if (d == 64)
-    linear_simt_kernel<T, 64><<<grid, 256, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, st,
-                                                        h_begin, h_count, S_io, z_io, zero_init ? 1 : 0);
+    linear_simt_kernel<T, 64><<<grid, 256, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, st, h_begin,
+                                                        h_count, S_io, z_io, zero_init ? 1 : 0, global_sum ? 1 : 0);
   else
-    linear_simt_kernel<T, 128><<<grid, 256, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, st,
-                                                         h_begin, h_count, S_io, z_io, zero_init ? 1 : 0);
+    linear_simt_kernel<T, 128><<<grid, 256, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, st, h_begin,
+                                                         h_count, S_io, z_io, zero_init ? 1 : 0, global_sum ? 1 : 0);
   note_launch();
   return cudaGetLastError();
 }
@@ -494,11 +499,13 @@ cudaError_t launch_window_simt(const void* q, const void* k, const void* v, void
 
 cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
                                int dtype, Strides st, int h_begin, int h_count, float* S_io, float* z_io,
-                               bool zero_init, cudaStream_t stream) {
+                               bool zero_init, cudaStream_t stream, bool global_sum) {
   if (h_count <= 0 || B <= 0) return cudaSuccess;
   if (dtype == GF_F32)
-    return linear_dispatch<float>(q, k, v, o, B, N, d, st, h_begin, h_count, S_io, z_io, zero_init, stream);
-  return linear_dispatch<__nv_bfloat16>(q, k, v, o, B, N, d, st, h_begin, h_count, S_io, z_io, zero_init, stream);
+    return linear_dispatch<float>(q, k, v, o, B, N, d, st, h_begin, h_count, S_io, z_io, zero_init, global_sum,
+                                  stream);
+  return linear_dispatch<__nv_bfloat16>(q, k, v, o, B, N, d, st, h_begin, h_count, S_io, z_io, zero_init, global_sum,
+                                        stream);
 }
 
 cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void* v_cache, int B, int N, int d,

@@ -212,7 +212,6 @@ def test_self_layer_argument_errors():
     assert call(h_sparse=5) == gf.GF_ERR_INVALID_ARG
     assert call(d=96) == gf.GF_ERR_UNSUPPORTED
     assert call(phi=1) == gf.GF_ERR_UNSUPPORTED
-    assert call(dtype=gf.GF_F32) == gf.GF_ERR_UNSUPPORTED      # the global linear heads are bf16 tensor-core kernels only
     assert call(ws_bytes=8) == gf.GF_ERR_WORKSPACE
     assert call(ws=0) == gf.GF_ERR_WORKSPACE
     # the bidirectional layer's segment sums fit the workspace the size query reports

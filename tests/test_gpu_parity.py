@@ -110,6 +110,16 @@ def test_self_layer_against_the_oracle(B, H, N, d, w, h0):
     assert_parity(f64(o[bs]), ref, "bf16", f"self layer B={B} H={H} N={N} d={d} w={w} h0={h0}")
 
 
+@pytest.mark.parametrize("dtype,force_simt", [("f32", 0), ("bf16", 1)])
+@pytest.mark.parametrize("N,d,w,h0", [(1, 64, 1, 0), (100, 64, 7, 1), (300, 128, 40, 1), (1000, 64, 128, 2)])
+def test_self_layer_cuda_core_path(dtype, force_simt, N, d, w, h0):
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, force_simt)
+    q, k, v = synth.qkv(2, 3, N, d, dtype, seed=750 + N, gain=1.0)
+    ref = oracle.hybrid_attn_self(f64(q), f64(k), f64(v), w, h_sparse=h0)
+    o = gf.hybrid_attn_self(*dev(q, k, v), w, h_sparse=h0)
+    assert_parity(f64(o), ref, "f32" if dtype == "f32" else "bf16", f"self layer, CUDA cores, N={N} d={d} {dtype}")
+
+
 def test_self_layer_is_deterministic_and_merges_by_head():
     B, H, N, d, w, h0 = 2, 4, 1500, 128, 100, 1
     q, k, v = dev(*synth.qkv(B, H, N, d, "bf16", seed=777, gain=1.0))
