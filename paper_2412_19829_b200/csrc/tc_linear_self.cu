@@ -478,6 +478,10 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
             pk[g * 4 + 3] = rawv.w;
           }
         }
+        // the buffer goes back to the TMA engine: these reads (generic proxy) must be ordered before its
+        // next write (async proxy), which a barrier arrival alone does not do
+        __threadfence_block();
+        fence_proxy_async_smem();
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&q_free[s]);  // this warp has its part of the raw tile in registers
         if (ok) {

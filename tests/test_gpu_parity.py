@@ -120,6 +120,19 @@ def test_self_layer_cuda_core_path(dtype, force_simt, N, d, w, h0):
     assert_parity(f64(o), ref, "f32" if dtype == "f32" else "bf16", f"self layer, CUDA cores, N={N} d={d} {dtype}")
 
 
+def test_self_layer_bnhd_layout_and_many_chains():
+    B, H, N, d, w, h0 = 2, 90, 600, 128, 70, 2  # 176 linear chains: more than one round of CTAs in reduce and readout
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=761, gain=1.0)
+    qn, kn, vn = [t.permute(0, 2, 1, 3).contiguous().cuda() for t in (q, k, v)]
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    o = gf.hybrid_attn_self(qn, kn, vn, w, h_sparse=h0, layout=gf.GF_BNHD, ws=ws).permute(0, 2, 1, 3).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    hs = [0, 1, 2, 47, H - 1]
+    ref = oracle.hybrid_attn_self(f64(q[:, hs]), f64(k[:, hs]), f64(v[:, hs]), w, h_sparse=2)
+    assert_parity(f64(o[:, hs]), ref, "bf16", "self layer, BNHD, 176 chains")
+    assert torch.equal(o, gf.hybrid_attn_self(*dev(q, k, v), w, h_sparse=h0).cpu())
+
+
 def test_self_layer_is_deterministic_and_merges_by_head():
     B, H, N, d, w, h0 = 2, 4, 1500, 128, 100, 1
     q, k, v = dev(*synth.qkv(B, H, N, d, "bf16", seed=777, gain=1.0))
@@ -240,6 +253,20 @@ def test_hybrid_merge_equals_pure_calls(h0):
     if h0 < H:
         ol = gf.causal_linear_attn(qd[:, h0:].contiguous(), kd[:, h0:].contiguous(), vd[:, h0:].contiguous())
         assert torch.equal(ol, o[:, h0:])
+
+
+@pytest.mark.parametrize("B,H,N,d,w,h0,split", [(2, 88, 1300, 128, 64, 8, 0), (2, 90, 900, 64, 100, 10, 0),
+                                                   (1, 40, 4096, 128, 64, 0, 4)])
+def test_both_layouts_give_the_same_bits(B, H, N, d, w, h0, split):
+    # [B, N, H, d] tensors make every tile load a gather of 128 short rows: slower loads, other
+    # interleavings of the roles, the same arithmetic -- a missing wait or fence shows up here
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=5 + N, gain=1.0)
+    qn, kn, vn = [t.permute(0, 2, 1, 3).contiguous().cuda() for t in (q, k, v)]
+    ref = gf.hybrid_attn(*dev(q, k, v), w, h_sparse=h0).cpu()
+    for _ in range(4):
+        x = gf.hybrid_attn(qn, kn, vn, w, h_sparse=h0, layout=gf.GF_BNHD).permute(0, 2, 1, 3).cpu()
+        assert torch.equal(x, ref)
 
 
 def test_negative_controls_fail_the_gates():
