@@ -1181,9 +1181,9 @@ bool tc_linear_supported(int N, int d, int dtype) {
 // hand-over (about one chunk); but a chain is also a serial pipeline - first pass of a segment,
 // one hand-over link per segment (about 0.65 chunk each), second pass - which bounds the time
 // from below when there are few chains.  Among the segment counts allowed, take the one with the
-// least max(rounds x (L + h), L + 0.65 G).  Segments are at least 4 chunks long and short
-// enough for what the CTAs running at one time park (phi(K) and V of their segments) to stay in
-// L2.  The plan must not depend on the device that is current when the workspace size is asked
+// least max(rounds x (L + h) x spill, L + 0.65 G).  Segments are between 4 and 32 chunks long;
+// spill > 1 charges segments too long for what the CTAs running at one time park (phi(K) and V of
+// their segments) to stay in L2.  The plan must not depend on the device that is current when the workspace size is asked
 // for, so without a CTA count it assumes the 148 SMs of a B200.
 namespace {
 constexpr int kPlanL8 = 8;  // segment length the scratch is sized for when chains are many
@@ -1225,10 +1225,12 @@ void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, 
       const long long items = (long long)nchains * g;
       const long long rounds = (items + kPlanSMs - 1) / kPlanSMs;
       const double L = (double)nch / g;
-      // what the running CTAs park at one time: about 80 MB of the 126 MB of L2
+      // What the running CTAs park at one time should stay in L2 (about 80 MB of its 126 MB): of a
+      // longer segment the excess comes back from DRAM, up to 40 % more time per chunk when the
+      // rounds bound the time (when the serial chain does, DRAM has slack and nothing is charged).
       const double l_cap = 80e6 / ((double)(items < kPlanSMs ? items : kPlanSMs) * 4.0 * 128.0 * d);
-      if (L > (l_cap < 4.0 ? 4.0 : l_cap) && g < g_max) continue;
-      const double by_rounds = (double)rounds * (L + handover_cost(d)), by_chain = L + 0.65 * g;
+      const double spill = L > l_cap ? 1.0 + 0.4 * (1.0 - l_cap / L) : 1.0;
+      const double by_rounds = (double)rounds * (L + handover_cost(d)) * spill, by_chain = L + 0.65 * g;
       const double cost = by_rounds > by_chain ? by_rounds : by_chain;
       if (cost < best * (1.0 - 1e-9)) {
         best = cost;

@@ -100,14 +100,18 @@ def test_linear_plan_named_cases():
     # one long chain is a serial pipeline of hand-over links: few, long segments
     G, L = gf.linear_plan(1, 32768, 128)
     assert 12 <= L <= 32
+    G, L = gf.linear_plan(1, 262144, 128)  # ... also when its parked tiles no longer fit L2
+    assert L >= 24
+    G, L = gf.linear_plan(4, 131072, 128)
+    assert L >= 20
     # enough whole chains for every CTA at d = 128, or chains too short to cut: the one-pass form
     assert gf.linear_plan(832, 4096, 128)[0] == 1
     assert gf.linear_plan(148, 8192, 128)[0] == 1
     assert gf.linear_plan(10, 512, 64)[0] == 1
     assert gf.linear_plan(832, 4096, 64)[0] == 1
-    # fewer chains than CTAs, long: cut, in segments of at most 16 chunks at d = 64 (16 KB tiles)
+    # fewer chains than CTAs, long: cut, in segments of about what stays in L2 at d = 64 (16 chunks of 16 KB tiles)
     G, L = gf.linear_plan(104, 16384, 64)
-    assert G > 1 and L <= 16
+    assert G > 1 and L <= 20
     gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 8)
     try:
         assert gf.linear_plan(26, 32768, 128) == (32, 8)
