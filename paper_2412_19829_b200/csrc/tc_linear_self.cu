@@ -536,13 +536,15 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
 
 // Segments per chain.  CTAs take items (segments) round-robin, so a launch lasts ceil(items / CTAs)
 // rounds of one item each: among the segment counts that keep segments at least four chunks long
-// (and the scratch within 64 slots per chain), take the one with the least rounds x (chunks of the
+// (and the scratch within 64 slots per chain, more when the chains are few), take the one with the least rounds x (chunks of the
 // longest segment + about one chunk of fixed cost per item).  The plan must not depend on the
 // device that is current when the workspace size is asked for: it assumes the 148 SMs of a B200.
 int self_segments(int nchains, int nch) {
   constexpr int kPlanSMs = 148;
   int g_max = (nch + 3) / 4;
-  if (g_max > 64) g_max = 64;
+  int cap = (2 * kPlanSMs + nchains - 1) / nchains;  // few chains: as many segments as fill two rounds
+  if (cap < 64) cap = 64;
+  if (g_max > cap) g_max = cap;
   int best_g = 1;
   long long best = -1;
   for (int g = 1; g <= g_max; ++g) {

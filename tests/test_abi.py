@@ -221,5 +221,4 @@ def test_self_layer_argument_errors():
     # the bidirectional layer's segment sums fit the workspace the size query reports
     for chains, N, d in ((1, 128, 64), (26, 32768, 128), (832, 4096, 64), (3, 100000, 128)):
         ws = gf.workspace_bytes(1, chains, N, d, 1, 0, gf.GF_BF16)
-        assert ws >= 256 + chains * (min(64, max(1, (-(-N // 128) + 3) // 4)) + 1) * (d * d + d) * 4 or \
-            ws >= 256 + chains * 2 * (d * d + d) * 4  # at most 64 segment slots per chain, plus the totals
+        assert ws >= 256 + chains * 2 * (d * d + d) * 4  # at least one segment slot per chain plus the totals
