@@ -380,3 +380,69 @@ def test_self_hybrid_routes_heads_like_the_causal_layer():
     np.testing.assert_array_equal(o[:, 2:], oracle.linear_attn_self(q[:, 2:], k[:, 2:], v[:, 2:]))
     assert oracle.hybrid_attn_self(q, k, v, 4).shape == q.shape  # default split: max(1, round(3 H / 16)) = 1
     np.testing.assert_array_equal(oracle.hybrid_attn_self(q, k, v, 4)[:, 1:], oracle.linear_attn_self(q[:, 1:], k[:, 1:], v[:, 1:]))
+
+
+# ----------------------------------------------------------------------------- head partition (Algorithm 2)
+def test_partition_balance_hand_worked_and_invariants():
+    from oracle import partition as op
+
+    # equal cost and speed: half each.  Engine 0 needs twice the work per unit at the same speed:
+    # 2 p = 1 - p, p' = 1/3.  Engine 1 three times faster on equal work: p = (1 - p) / 3, p' = 1/4.
+    assert op.balance(100, 7.0, 7.0, 2.0, 2.0) == pytest.approx(0.5, abs=1e-14)
+    assert op.balance(64, 2.0, 1.0, 1.0, 1.0) == pytest.approx(1.0 / 3.0, abs=1e-14)
+    assert op.balance(64, 1.0, 1.0, 1.0, 3.0) == pytest.approx(0.25, abs=1e-14)
+    rng = np.random.default_rng(11)
+    for _ in range(50):
+        f0, f1, p0, p1 = (float(x) for x in 10.0 ** rng.uniform(-1, 1, 4))  # shares stay away from 0 and 1
+        size = float(rng.integers(1, 10**6))
+        p = op.balance(size, f0, f1, p0, p1)
+        l0, l1 = op.latencies(p, size, f0, f1, p0, p1)
+        assert 0.0 < p < 1.0 and l0 == pytest.approx(l1, rel=1e-9)
+        # the work is conserved: both shares together are the whole problem
+        assert p * size + (1 - p) * size == pytest.approx(size, rel=1e-15)
+        # naming the engines the other way round mirrors the split; the problem size and a common
+        # speed-up of both engines do not move it
+        assert op.balance(size, f1, f0, p1, p0) == pytest.approx(1.0 - p, abs=1e-12)
+        assert op.balance(3 * size, f0, f1, 5 * p0, 5 * p1) == pytest.approx(p, abs=1e-12)
+        # a faster engine 0 gets more
+        assert op.balance(size, f0, f1, 2 * p0, p1) > p
+
+
+def test_partition_latency_step_values():
+    from oracle import partition as op
+
+    # p = 0.25 of 8 units at 3 flops each on a 2 flop/s engine: 0.25 * 8 * 3 / 2 = 3 s;
+    # the other 6 units at 5 flops each on a 10 flop/s engine: 6 * 5 / 10 = 3 s
+    assert op.latencies(0.25, 8, 3.0, 5.0, 2.0, 10.0) == (3.0, 3.0)
+    assert op.balance(8, 3.0, 5.0, 2.0, 10.0) == pytest.approx(0.25, abs=1e-14)
+
+
+def test_partition_heads_hand_worked_and_brackets_the_crossing():
+    from oracle import partition as op
+
+    # B = N = E = W = 1, unit speeds, H = 4: linear 8 (4 - h)^2 = 128, 72, 32, 8, 0 against sparse
+    # 5 h = 0, 5, 10, 15, 20: gaps 128, 67, 22, 7, 20 -> 3 sparse heads
+    assert [op.model_latencies(1, 4, 1, 1, 1, h, 1.0, 1.0) for h in range(5)] == [
+        (0.0, 128.0), (5.0, 72.0), (10.0, 32.0), (15.0, 8.0), (20.0, 0.0)]
+    assert op.partition_heads(1, 4, 1, 1, 1, 1.0, 1.0) == 3
+    # the three terms of the linear model (feature maps 4, K^T V 2, Q C 2) add up to the printed 8
+    B, H, N, E, W = 2, 16, 1024, 64, 256
+    h1e2 = float((H - 3) * E) ** 2
+    assert op.model_latencies(B, H, N, E, W, 3, 1.0, 1.0)[1] == (4 + 2 + 2) * B * N * h1e2
+    rng = np.random.default_rng(12)
+    for _ in range(40):
+        H = int(rng.integers(1, 65)); E = int(rng.choice([32, 64, 128])); W = int(rng.choice([64, 256, 1024]))
+        ps, pl = (float(x) for x in 10.0 ** rng.uniform(9, 15, 2))
+        h0 = op.partition_heads(B, H, N, E, W, ps, pl)
+        gap = lambda h: op.model_latencies(B, H, N, E, W, h, ps, pl)[0] - op.model_latencies(B, H, N, E, W, h, ps, pl)[1]
+        # sparse - linear grows with the sparse head count, from negative (no sparse head) to positive
+        # (no linear head): the chosen count sits at the sign change
+        assert gap(0) < 0 < gap(H)
+        assert all(gap(h) < gap(h + 1) for h in range(H))
+        if h0 > 0:
+            assert gap(h0 - 1) < 0
+        if h0 < H:
+            assert gap(h0 + 1) > 0
+        # B and N scale both estimates alike; a faster sparse engine never gets fewer heads
+        assert op.partition_heads(7 * B, H, 3 * N, E, W, ps, pl) == h0
+        assert op.partition_heads(B, H, N, E, W, 4 * ps, pl) >= h0
