@@ -89,6 +89,25 @@ int gformer_set_tuning(int key, int value);
  * GF_ERR_INVALID_ARG / GF_ERR_UNSUPPORTED without touching the outputs. */
 int gformer_linear_plan(int chains, int N, int d, int ctas, int* segments, int* chunks_per_segment);
 
+/* Algorithm 2 (Sec. III-D): the share p' in (0, 1) of a problem given to engine 0 at which the two
+ * latency estimates  p size flops_per0 / perf0  and  (1 - p) size flops_per1 / perf1  are equal
+ * (size cancels).  flops_per_i: work per unit of the part engine i runs; perf_i: that engine's
+ * measured rate in the same work unit per second -- measured seconds per head and a rate of 1 do
+ * as well.  Host arithmetic in fp64, no device work.  p_out: host pointer.  Returns GF_OK, or
+ * GF_ERR_INVALID_ARG (null pointer, a non-positive or non-finite input) without touching *p_out. */
+int gformer_partition_balance(double flops_per0, double flops_per1, double perf0, double perf1, double* p_out);
+
+/* The FLOP model of Sec. III-D for H heads of width E over B sequences of N tokens with window W:
+ * h_sparse windowed heads cost 5 B h_sparse N W / perf_sparse seconds and the H - h_sparse linear
+ * heads 8 B N ((H - h_sparse) E)^2 / perf_linear (both formulas as the section prints them;
+ * perf_* in FLOP/s).  *h_sparse_out receives the whole number of windowed heads in [0, H] for which
+ * the two estimates are closest (the smaller count on a tie); the optional latency outputs (host
+ * pointers, may be null) receive the two estimates at that count.  Host arithmetic in fp64.
+ * Returns GF_OK, or GF_ERR_INVALID_ARG (null h_sparse_out, a size below 1, a non-positive or
+ * non-finite rate) without touching the outputs. */
+int gformer_partition_heads(int B, int H, int N, int E, int W, double perf_sparse, double perf_linear,
+                            int* h_sparse_out, double* latency_sparse_out, double* latency_linear_out);
+
 /* Number of kernels the library has launched in this process so far (all entry points,
  * all streams).  For accounting in benchmarks. */
 unsigned long long gformer_launch_count(void);

@@ -7,6 +7,11 @@ file takes those steps in the algorithm's order, in fp64, and finds the meeting 
 bisection and by exhaustive search: no closed form appears here, so that the closed forms
 the library uses can be checked against it.
 
+Pinned by hand-worked splits, mirror and scale invariants and the sign change of the latency
+gap.  The section's own worked example (3 sparse heads of 16 at 4k tokens with rates of 13.37
+and 2.31 TFLOP/s) is not what its printed formulas give with those rates (13 to 16 heads for any
+window from 16 to 1024), so that example pins nothing: parity unpinned for the example.
+
 Nothing here imports the CUDA package and the CUDA package never imports this.
 """
 from __future__ import annotations

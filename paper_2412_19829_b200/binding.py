@@ -55,6 +55,11 @@ def lib() -> ctypes.CDLL:
         L.gformer_set_tuning.argtypes = [i, i]
         L.gformer_linear_plan.restype = i
         L.gformer_linear_plan.argtypes = [i, i, i, i, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(ctypes.c_int)]
+        dbl, pdbl = ctypes.c_double, ctypes.POINTER(ctypes.c_double)
+        L.gformer_partition_balance.restype = i
+        L.gformer_partition_balance.argtypes = [dbl, dbl, dbl, dbl, pdbl]
+        L.gformer_partition_heads.restype = i
+        L.gformer_partition_heads.argtypes = [i, i, i, i, i, dbl, dbl, ctypes.POINTER(ctypes.c_int), pdbl, pdbl]
         L.gformer_workspace_bytes.restype = sz
         L.gformer_workspace_bytes.argtypes = [i] * 7
         L.gformer_last_device_status.restype = i
@@ -110,6 +115,26 @@ def linear_plan(chains: int, N: int, d: int, ctas: int = 0):
     if rc != GF_OK:
         raise GformerError(rc, "gformer_linear_plan")
     return g.value, l.value
+
+
+def partition_balance(flops_per0: float, flops_per1: float, perf0: float, perf1: float) -> float:
+    """Share of the problem for engine 0 at which the two latency estimates of Algorithm 2 meet."""
+    p = ctypes.c_double(0.0)
+    rc = lib().gformer_partition_balance(float(flops_per0), float(flops_per1), float(perf0), float(perf1),
+                                         ctypes.byref(p))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_partition_balance")
+    return p.value
+
+
+def partition_heads(B: int, H: int, N: int, E: int, W: int, perf_sparse: float, perf_linear: float):
+    """(windowed heads, sparse latency, linear latency) of the FLOP model of Sec. III-D."""
+    h0, ls, ll = ctypes.c_int(0), ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = lib().gformer_partition_heads(int(B), int(H), int(N), int(E), int(W), float(perf_sparse),
+                                       float(perf_linear), ctypes.byref(h0), ctypes.byref(ls), ctypes.byref(ll))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_partition_heads")
+    return h0.value, ls.value, ll.value
 
 
 def workspace_bytes(B, H, N, d, w, h_sparse, dtype) -> int:

@@ -131,6 +131,62 @@ def test_linear_plan_argument_errors():
     assert (g.value, l.value) == (-7, -7)
 
 
+def test_partition_balance_against_the_oracle():
+    """Algorithm 2: the library's closed form against the oracle's bisection."""
+    import numpy as np
+    from oracle import partition as op
+
+    assert gf.partition_balance(2.0, 1.0, 1.0, 1.0) == pytest.approx(1.0 / 3.0, abs=1e-15)
+    rng = np.random.default_rng(21)
+    for _ in range(200):
+        f0, f1, p0, p1 = (float(x) for x in 10.0 ** rng.uniform(-2, 2, 4))
+        size = float(rng.integers(1, 10**6))
+        assert gf.partition_balance(f0, f1, p0, p1) == pytest.approx(op.balance(size, f0, f1, p0, p1), abs=1e-12)
+    # measured seconds per head as the work, unit rates: 16 heads, a windowed head 3x as slow
+    p = gf.partition_balance(3.0e-6, 1.0e-6, 1.0, 1.0)
+    assert p == pytest.approx(op.balance(16, 3.0e-6, 1.0e-6, 1.0, 1.0), abs=1e-12) and round(p * 16) == 4
+
+
+def test_partition_heads_against_the_oracle():
+    """FLOP model of Sec. III-D: the library's root-and-neighbours search against the oracle's
+    exhaustive one, both deciding in fp64."""
+    import numpy as np
+    from oracle import partition as op
+
+    assert gf.partition_heads(1, 4, 1, 1, 1, 1.0, 1.0) == (3, 15.0, 8.0)
+    rng = np.random.default_rng(22)
+    cases = [(1, 32, 32768, 128, 512, 1.0e12, 1.0e15), (8, 12, 4096, 64, 256, 3.0e12, 1.0e14), (1, 1, 1, 1, 1, 1.0, 1.0),
+             (64, 4096, 262144, 128, 4096, 1.0e9, 1.0e9), (1, 16, 2048, 64, 1, 1.0e15, 1.0), (1, 16, 2048, 64, 2048, 1.0, 1.0e15)]
+    for _ in range(300):
+        cases.append((int(rng.integers(1, 9)), int(rng.integers(1, 130)), int(rng.integers(1, 70000)),
+                      int(rng.choice([1, 32, 64, 128])), int(rng.integers(1, 5000)),
+                      float(10.0 ** rng.uniform(6, 16)), float(10.0 ** rng.uniform(6, 16))))
+    for B, H, N, E, W, ps, pl in cases:
+        h0, ls, ll = gf.partition_heads(B, H, N, E, W, ps, pl)
+        want = op.partition_heads(B, H, N, E, W, ps, pl)
+        s, l = op.model_latencies(B, H, N, E, W, h0, ps, pl)
+        assert ls == pytest.approx(s, rel=1e-14) and ll == pytest.approx(l, rel=1e-14)
+        if h0 != want:  # only where the two gaps agree to rounding may the counts differ
+            sw, lw = op.model_latencies(B, H, N, E, W, want, ps, pl)
+            assert abs(s - l) == pytest.approx(abs(sw - lw), rel=1e-12), (B, H, N, E, W, ps, pl, h0, want)
+
+
+def test_partition_argument_errors():
+    L = gf.lib()
+    p = ctypes.c_double(-7.0)
+    for bad in ((0.0, 1.0, 1.0, 1.0), (1.0, -1.0, 1.0, 1.0), (1.0, 1.0, float("inf"), 1.0), (1.0, 1.0, 1.0, float("nan"))):
+        assert L.gformer_partition_balance(*bad, ctypes.byref(p)) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_partition_balance(1.0, 1.0, 1.0, 1.0, None) == gf.GF_ERR_INVALID_ARG
+    assert p.value == -7.0
+    h0 = ctypes.c_int(-7)
+    for bad in ((0, 4, 1, 1, 1, 1.0, 1.0), (1, 0, 1, 1, 1, 1.0, 1.0), (1, 4, 0, 1, 1, 1.0, 1.0), (1, 4, 1, 0, 1, 1.0, 1.0),
+                (1, 4, 1, 1, 0, 1.0, 1.0), (1, 4, 1, 1, 1, 0.0, 1.0), (1, 4, 1, 1, 1, 1.0, float("nan"))):
+        assert L.gformer_partition_heads(*bad, ctypes.byref(h0), None, None) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_partition_heads(1, 4, 1, 1, 1, 1.0, 1.0, None, None, None) == gf.GF_ERR_INVALID_ARG
+    assert h0.value == -7
+    assert L.gformer_partition_heads(1, 4, 1, 1, 1, 1.0, 1.0, ctypes.byref(h0), None, None) == gf.GF_OK and h0.value == 3
+
+
 FAKE = 0x10000  # a 16-byte-aligned non-null address; validation fails before it is ever used
 
 

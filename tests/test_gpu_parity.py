@@ -647,3 +647,26 @@ def test_config5_sweep_point(idx):
     ref = oracle.causal_linear_attn(f64(q[b:b + 1, hl:hl + 1]), f64(k[b:b + 1, hl:hl + 1]),
                                     f64(v[b:b + 1, hl:hl + 1]))
     assert_parity(f64(o[b:b + 1, hl:hl + 1]), ref, "bf16", "sweep linear head")
+
+
+# ----------------------------------------------------------------------------- head partition (Algorithm 2)
+@pytest.mark.gpu
+def test_measured_partition_balances_the_two_head_kinds():
+    """The balance rule on measured per-head times: the split it returns is the whole number of
+    heads nearest to equal time on both sides, and the layer runs at that split."""
+    from oracle import partition as op
+    from paper_2412_19829_b200 import partition
+
+    r = partition.measure(1, 16, 8192, 64, 256, iters=3)
+    tw, tl, H = r["s_per_window_head"], r["s_per_linear_head"], r["H"]
+    assert tw > 0 and tl > 0 and 0 < r["h_sparse_balanced"] < H
+    assert r["p_balanced"] == pytest.approx(op.balance(H, tw, tl, 1.0, 1.0), abs=1e-12)
+    assert abs(r["p_balanced"] * H - r["h_sparse_balanced"]) <= 0.5 + 1e-9
+    assert r["layer_us_at_balanced"] > 0
+    fm = r["flop_model"]
+    assert 0 <= fm["h_sparse"] <= H
+    perf_s, perf_l = 5.0 * 8192 * 256 / tw, 8.0 * 8192 * float(H * 64) ** 2 / (H * tl)
+    want = op.partition_heads(1, H, 8192, 64, 256, perf_s, perf_l)
+    s, l = op.model_latencies(1, H, 8192, 64, 256, fm["h_sparse"], perf_s, perf_l)
+    sw, lw = op.model_latencies(1, H, 8192, 64, 256, want, perf_s, perf_l)
+    assert fm["h_sparse"] == want or abs(s - l) == pytest.approx(abs(sw - lw), rel=1e-9)

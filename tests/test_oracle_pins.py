@@ -446,3 +446,13 @@ def test_partition_heads_hand_worked_and_brackets_the_crossing():
         # B and N scale both estimates alike; a faster sparse engine never gets fewer heads
         assert op.partition_heads(7 * B, H, 3 * N, E, W, ps, pl) == h0
         assert op.partition_heads(B, H, N, E, W, 4 * ps, pl) >= h0
+
+
+def test_partition_printed_example_is_not_what_the_printed_model_gives():
+    """Sec. IV-C reports 3 sparse heads of 16 (4k tokens, 13.37 and 2.31 TFLOP/s).  The printed
+    formulas with those rates balance far from it whatever the window, so the example is no pin;
+    this records the fact rather than bending the model to it."""
+    from oracle import partition as op
+
+    counts = [op.partition_heads(1, 16, 4096, 64, W, 2.31e12, 13.37e12) for W in (16, 32, 64, 128, 256, 512, 1024)]
+    assert counts == [16, 16, 15, 15, 14, 14, 13]
