@@ -190,8 +190,11 @@ int gformer_causal_linear_attn_noalloc(const void* q, const void* k, const void*
 /*
  * The hybrid layer (Sec. III-A): heads [0, h_sparse) as gformer_window_attn, heads
  * [h_sparse, H) as gformer_causal_linear_attn with a zero initial state; h_sparse < 0
- * selects gformer_default_h_sparse(H).  The two groups overlap on the device when the
- * linear heads alone do not fill it; otherwise they run back to back on `cuda_stream`.
+ * selects gformer_default_h_sparse(H).  The two groups run side by side on the device (on two
+ * streams of the library's own, forked from and joined back into `cuda_stream`, so the caller
+ * sees a single-stream call that may also be captured into a CUDA graph).  Host threads may call
+ * concurrently, each with its own workspace and stream; on one device their fork .. join sections
+ * are enqueued one after the other.
  * state_out (may be NULL): if given, its B, H, d, w, h_sparse, dtype must match the call
  * and its buffers receive the decode state after the N tokens: the last min(N, w) keys
  * and values of the windowed heads in ring slots j mod w, the final S and z of the linear

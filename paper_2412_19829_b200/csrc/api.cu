@@ -26,6 +26,10 @@ struct Fork {
   cudaStream_t side = nullptr, first = nullptr;  // lowest / highest stream priority
   cudaEvent_t fork = nullptr, join = nullptr, join_first = nullptr;
   bool ready = false;
+  // held while a call enqueues its fork .. join section: the events are shared by every call on
+  // the device, and a record from another host thread between this call's record and its waits
+  // would make the side streams wait for the wrong point
+  std::mutex enqueue;
 };
 Fork g_fork[kMaxDevices];
 std::mutex g_fork_mutex;
@@ -313,6 +317,8 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   }
   Fork* f = both ? get_fork() : nullptr;
   if (both && f == nullptr) return GF_ERR_CUDA;
+  std::unique_lock<std::mutex> enqueue_guard;
+  if (both) enqueue_guard = std::unique_lock<std::mutex>(f->enqueue);
   if (both) {
     // fork: the linear heads (the long serial chains) stay on the caller's stream, the
     // windowed heads go to the side stream; join before returning control to the stream.

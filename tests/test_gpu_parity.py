@@ -649,6 +649,74 @@ def test_config5_sweep_point(idx):
     assert_parity(f64(o[b:b + 1, hl:hl + 1]), ref, "bf16", "sweep linear head")
 
 
+@pytest.mark.gpu
+def test_hybrid_layer_replayed_from_a_cuda_graph():
+    # the layer forks onto streams of its own and joins back: captured from the caller's stream it
+    # must replay with the bits of the eager call, also after the inputs changed in place
+    B, H, N, d, w, h0 = 2, 8, 1024, 64, 128, 2
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=61)
+    qd, kd, vd = dev(q, k, v)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    eager = gf.hybrid_attn(qd, kd, vd, w, h_sparse=h0, ws=ws).clone()
+    assert_parity(f64(eager), oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0), "bf16", "eager")
+    out = torch.empty_like(eager)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        gf.hybrid_attn(qd, kd, vd, w, h_sparse=h0, out=out, ws=ws, stream=stream)
+    torch.cuda.synchronize()
+    for _ in range(2):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager)
+    q2, k2, v2 = synth.qkv(B, H, N, d, "bf16", seed=62)
+    for dst, src in ((qd, q2), (kd, k2), (vd, v2)):
+        dst.copy_(src)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert ws.last_device_status() == gf.GF_OK
+    assert torch.equal(out, gf.hybrid_attn(qd, kd, vd, w, h_sparse=h0, ws=ws))
+
+
+@pytest.mark.gpu
+def test_hybrid_layer_called_from_two_host_threads():
+    # each thread has its own stream, workspace and tensors; the library's fork/join streams are
+    # shared by both, so their enqueue sections must not interleave
+    import threading
+
+    B, H, N, d, w, h0 = 1, 8, 2048, 64, 128, 3
+    jobs = []
+    for seed in (71, 72):
+        q, k, v = dev(*synth.qkv(B, H, N, d, "bf16", seed=seed))
+        ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+        want = gf.hybrid_attn(q, k, v, w, h_sparse=h0, ws=ws).clone()
+        jobs.append(dict(q=q, k=k, v=v, ws=ws, want=want, stream=torch.cuda.Stream(), bad=[]))
+    torch.cuda.synchronize()
+
+    def run(job):
+        try:
+            for it in range(40):
+                out = torch.zeros_like(job["want"])
+                with torch.cuda.stream(job["stream"]):
+                    gf.hybrid_attn(job["q"], job["k"], job["v"], w, h_sparse=h0, out=out, ws=job["ws"], stream=job["stream"])
+                job["stream"].synchronize()
+                if not torch.equal(out, job["want"]):
+                    job["bad"].append(it)
+        except Exception as e:  # noqa: BLE001 - reported by the assertion below
+            job["bad"].append(repr(e))
+
+    threads = [threading.Thread(target=run, args=(j,)) for j in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=120)
+    assert not any(t.is_alive() for t in threads)
+    for j in jobs:
+        assert j["bad"] == [] and j["ws"].last_device_status() == gf.GF_OK
+
+
 # ----------------------------------------------------------------------------- head partition (Algorithm 2)
 @pytest.mark.gpu
 def test_measured_partition_balances_the_two_head_kinds():
