@@ -243,10 +243,33 @@ int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* 
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   rc = clear_ws(ws, stream);
   if (rc != GF_OK) return rc;
+  const bool tc_linear = !g_force_simt && gf::tc_linear_supported(N, d, dtype);
+  if (h_sparse > 0 && h_sparse < H && tc_linear) {
+    // Both head groups on tensor-core kernels: the three launches of the linear heads go to the
+    // library's high-priority stream, the windowed heads to its side stream a few microseconds
+    // later; their CTAs run while the small totals kernel has the device and in the tails of the
+    // two big ones.  Forked from and joined back into the caller's stream.
+    Fork* f = get_fork();
+    if (f == nullptr) return GF_ERR_CUDA;
+    std::unique_lock<std::mutex> enqueue_guard(f->enqueue);
+    if (cudaEventRecord(f->fork, stream) != cudaSuccess) return GF_ERR_CUDA;
+    if (cudaStreamWaitEvent(f->side, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
+    if (cudaStreamWaitEvent(f->first, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
+    rc = cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
+                                               sizeof(WsHeader), f->first));
+    if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
+    if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
+    int rc2 = cuda_status(gf::launch_delay(8000, f->side));
+    if (rc2 == GF_OK)
+      rc2 = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, f->side, true);
+    if (cudaEventRecord(f->join, f->side) != cudaSuccess) return GF_ERR_CUDA;
+    if (cudaStreamWaitEvent(stream, f->join, 0) != cudaSuccess) return GF_ERR_CUDA;
+    return rc != GF_OK ? rc : rc2;
+  }
   rc = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, stream, true);
   if (rc != GF_OK) return rc;
   if (h_sparse == H) return GF_OK;
-  if (!g_force_simt && gf::tc_linear_supported(N, d, dtype))
+  if (tc_linear)
     return cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
                                                  sizeof(WsHeader), stream));
   // fp32 storage (or the CUDA-core knob): token by token, a summing sweep and a readout sweep
