@@ -212,7 +212,8 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o,
  *   S = sum_j phi(k_j) v_j^T,  z = sum_j phi(k_j)  over all j,   o_i = phi(q_i)^T S / (phi(q_i) . z)
  * (Sec. II-B, rows normalised as in Algorithm 1).  bf16 storage takes the tensor-core kernels,
  * fp32 storage (or GF_TUNE_FORCE_SIMT) CUDA-core kernels in fp32 arithmetic, as in the causal
- * layer.  Workspace: gformer_workspace_bytes.
+ * layer.  Streams, graph capture and host threads as for gformer_hybrid_attn.  Workspace:
+ * gformer_workspace_bytes.
  */
 int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* o,
                              int B, int H, int N, int d, int w, int h_sparse, float scale,

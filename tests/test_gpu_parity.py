@@ -681,6 +681,25 @@ def test_hybrid_layer_replayed_from_a_cuda_graph():
 
 
 @pytest.mark.gpu
+def test_self_layer_replayed_from_a_cuda_graph():
+    B, H, N, d, w, h0 = 1, 8, 1536, 128, 200, 3
+    qd, kd, vd = dev(*synth.qkv(B, H, N, d, "bf16", seed=63))
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    eager = gf.hybrid_attn_self(qd, kd, vd, w, h_sparse=h0, ws=ws).clone()
+    out = torch.zeros_like(eager)
+    stream = torch.cuda.Stream()
+    stream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        gf.hybrid_attn_self(qd, kd, vd, w, h_sparse=h0, out=out, ws=ws, stream=stream)
+    for _ in range(2):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, eager) and ws.last_device_status() == gf.GF_OK
+
+
+@pytest.mark.gpu
 def test_hybrid_layer_called_from_two_host_threads():
     # each thread has its own stream, workspace and tensors; the library's fork/join streams are
     # shared by both, so their enqueue sections must not interleave
