@@ -451,6 +451,23 @@ def test_config3_long_sequence_sampled_heads():
     assert_parity(f64(o[:, lh]), ref_l, "bf16", "config 3 linear heads")
 
 
+def test_self_layer_long_sequence_sampled_heads():
+    # the bidirectional layer at the size and launch configuration `bench.py --workload self32k` times
+    c = synth.CONFIGS["long32k"]
+    q, k, v = synth.qkv(c["B"], c["H"], c["N"], c["d"], "bf16", c["seed"])
+    h0 = gf.default_h_sparse(c["H"])
+    ws = gf.Workspace.for_problem(c["B"], c["H"], c["N"], c["d"], c["w"], -1)
+    o = gf.hybrid_attn_self(*dev(q, k, v), c["w"], ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    assert torch.isfinite(o.float()).all()
+    wh = [0, h0 - 1]
+    ref_w = oracle.window_attn_self(f64(q[:, wh]), f64(k[:, wh]), f64(v[:, wh]), c["w"])
+    assert_parity(f64(o[:, wh]), ref_w, "bf16", "self layer at 32K, window heads")
+    lh = [h0, c["H"] // 2, c["H"] - 1]
+    ref_l = oracle.linear_attn_self(f64(q[:, lh]), f64(k[:, lh]), f64(v[:, lh]))
+    assert_parity(f64(o[:, lh]), ref_l, "bf16", "self layer at 32K, linear heads")
+
+
 # ------------------------------------------------------------------ decode
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d,w,h0", [(64, 16, 1), (128, 40, 2), (64, 300, 3), (64, 8, 0)])
