@@ -468,6 +468,31 @@ def test_self_layer_long_sequence_sampled_heads():
     assert_parity(f64(o[:, lh]), ref_l, "bf16", "self layer at 32K, linear heads")
 
 
+def test_tensors_of_2_to_the_31_elements_sampled_chains():
+    # element offsets beyond 32 bits: B*H*N*d = 2^31 per tensor (4.3 GB each in bf16).  Inputs are drawn on the
+    # device (seeded); the oracle checks chains from both ends of the tensors, both kinds of heads, both layers.
+    B, H, N, d, w, h0 = 64, 16, 32768, 64, 256, 3
+    assert B * H * N * d == 2 ** 31
+    g = torch.Generator(device="cuda").manual_seed(4242)
+    q, k, v = [torch.randn(B, H, N, d, device="cuda", generator=g, dtype=torch.bfloat16) for _ in range(3)]
+    o = torch.empty_like(q)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    picks = [(0, 0), (B - 1, h0 - 1), (B - 1, H - 1), (B // 2, h0), (0, H - 1)]
+
+    def chain(t, b, h):
+        return f64(t[b:b + 1, h:h + 1].cpu())
+
+    for layer, win, lin, name in ((gf.hybrid_attn, oracle.window_attn, oracle.causal_linear_attn, "causal"),
+                                  (gf.hybrid_attn_self, oracle.window_attn_self, oracle.linear_attn_self, "self")):
+        o.zero_()
+        layer(q, k, v, w, h_sparse=h0, out=o, ws=ws)
+        assert ws.last_device_status() == gf.GF_OK
+        for b, h in picks:
+            qc, kc, vc = chain(q, b, h), chain(k, b, h), chain(v, b, h)
+            ref = win(qc, kc, vc, w) if h < h0 else lin(qc, kc, vc)
+            assert_parity(chain(o, b, h), ref, "bf16", f"{name} layer, 2^31 elements, chain ({b}, {h})")
+
+
 # ------------------------------------------------------------------ decode
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("d,w,h0", [(64, 16, 1), (128, 40, 2), (64, 300, 3), (64, 8, 0)])
