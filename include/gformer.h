@@ -51,7 +51,8 @@ typedef enum { GF_PHI_ELU1 = 0 } gf_phi;
 /* Process-wide knobs for tests and benchmarks (gformer_set_tuning). */
 typedef enum {
   GF_TUNE_FORCE_SIMT = 0, /* 1: never take the tensor-core kernels (default 0)              */
-  GF_TUNE_LINEAR_SPLIT = 1, /* 128-row chunks per sequence segment of a linear chain: 0 = auto   */
+  GF_TUNE_LINEAR_SPLIT = 1, /* 128-row chunks per sequence segment of a linear chain: 0 = auto,
+                               -1 = never cut a chain (the one-pass form of the kernel)          */
   GF_TUNE_LINEAR_CTAS = 2   /* gformer_hybrid_attn: CTAs of the persistent linear-attention kernel
                                when it shares the GPU with the windowed heads; 0 = auto, else an
                                upper bound in [1, 65535] (the SM count bounds it too)              */

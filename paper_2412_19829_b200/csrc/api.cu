@@ -155,7 +155,7 @@ int gformer_set_tuning(int key, int value) {
       g_force_simt = value ? 1 : 0;
       return GF_OK;
     case GF_TUNE_LINEAR_SPLIT:
-      if (value < 0 || value > 4096) return GF_ERR_INVALID_ARG;
+      if (value < -1 || value > 4096) return GF_ERR_INVALID_ARG;
       g_linear_split = value;
       return GF_OK;
     case GF_TUNE_LINEAR_CTAS:

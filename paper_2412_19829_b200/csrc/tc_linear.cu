@@ -1188,7 +1188,11 @@ bool tc_linear_supported(int N, int d, int dtype) {
 namespace {
 constexpr int kPlanL8 = 8;  // segment length the scratch is sized for when chains are many
 // cost of a chunk of an uncut chain, in two-pass chunks
-constexpr double direct_chunk_cost(int d) { return d == 128 ? 0.8 : 0.93; }
+constexpr double direct_chunk_cost(int d) { return d == 128 ? 0.8 : 0.83; }
+// ... and in a round that only part of the CTAs take part in: at d = 128 a full round of uncut chains is bound by
+// HBM (3.3 us per chunk on a B200), a thin one by the CTA's own pipeline (2.4 us); at d = 64 the CTA's pipeline
+// bounds both
+constexpr double direct_chunk_floor(int d) { return d == 128 ? 0.59 : 0.83; }
 // fixed cost of an item (hand-over, pipeline refill) in chunks: a chunk is cheaper at d = 64, the hand-over hardly
 constexpr double handover_cost(int d) { return d == 128 ? 1.1 : 1.6; }
 // Range of segment counts the automatic plan chooses from.
@@ -1215,6 +1219,8 @@ void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, 
   if (split > 0) {
     const int L = split > kMaxL ? kMaxL : split;
     G = (nch + L - 1) / L;
+  } else if (split < 0) {
+    G = 1;  // never cut: the one-pass form whatever the shape
   } else {
     const int kPlanSMs = ctas > 0 ? ctas : 148;
     int g_min, g_max;
@@ -1240,8 +1246,13 @@ void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, 
     // An uncut chain needs neither the first pass nor a hand-over (the kernel transforms K inside
     // the chunk pipeline): a chunk then costs direct_chunk_cost(d) of a two-pass one.  With many
     // chains that is the cheaper plan even though a CTA then walks a whole chain.
-    const long long rounds1 = ((long long)nchains + kPlanSMs - 1) / kPlanSMs;
-    if ((double)rounds1 * nch * direct_chunk_cost(d) <= best) G = 1;
+    const int full = nchains / kPlanSMs, rest = nchains % kPlanSMs;
+    double last = 0.0;  // the round of the chains left over after the full rounds
+    if (rest > 0) {
+      last = direct_chunk_cost(d) * rest / kPlanSMs;
+      if (last < direct_chunk_floor(d)) last = direct_chunk_floor(d);
+    }
+    if ((double)nch * (full * direct_chunk_cost(d) + last) <= best) G = 1;
   }
   if (G < 1) G = 1;
   *G_out = G;

@@ -54,7 +54,10 @@ def test_workspace_bytes_nonzero():
 def test_tuning_rejects_unknown_keys():
     L = gf.lib()
     assert L.gformer_set_tuning(99, 1) == gf.GF_ERR_INVALID_ARG
-    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, -1) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, -2) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 5000) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, -1) == gf.GF_OK  # never cut a chain
+    assert gf.linear_plan(26, 32768, 128) == (1, 256)
     assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 0) == gf.GF_OK
     assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_CTAS, -1) == gf.GF_ERR_INVALID_ARG
     assert L.gformer_set_tuning(gf.GF_TUNE_LINEAR_CTAS, 70000) == gf.GF_ERR_INVALID_ARG
@@ -109,6 +112,13 @@ def test_linear_plan_named_cases():
     assert gf.linear_plan(148, 8192, 128)[0] == 1
     assert gf.linear_plan(10, 512, 64)[0] == 1
     assert gf.linear_plan(832, 4096, 64)[0] == 1
+    # chains that nearly fill one round of CTAs, or spill thinly into a second one: whole, also when long
+    # (measured on a B200: 100 chains of 32K tokens at d = 128 take 706 us whole and 841 us cut)
+    for chains in (100, 120, 190, 208, 296):
+        assert gf.linear_plan(chains, 32768, 128)[0] == 1, chains
+    assert gf.linear_plan(120, 32768, 64)[0] == 1 and gf.linear_plan(230, 32768, 64)[0] == 1
+    # ... while half a round of long chains is cut
+    assert gf.linear_plan(74, 32768, 128)[0] > 1 and gf.linear_plan(90, 32768, 64)[0] > 1
     # fewer chains than CTAs, long: cut, in segments of about what stays in L2 at d = 64 (16 chunks of 16 KB tiles)
     G, L = gf.linear_plan(104, 16384, 64)
     assert G > 1 and L <= 20
