@@ -90,6 +90,15 @@ int gformer_set_tuning(int key, int value);
  * GF_ERR_INVALID_ARG / GF_ERR_UNSUPPORTED without touching the outputs. */
 int gformer_linear_plan(int chains, int N, int d, int ctas, int* segments, int* chunks_per_segment);
 
+/* The same plan with its parts named.  With somewhat more chains than CTAs the kernel is launched
+ * twice: the first *whole_chains chains (full rounds of one chain per CTA) in the one-pass form, the
+ * leftover chains behind them in the two-pass form, cut into *segments segments of at most
+ * *chunks_per_segment chunks -- the figures gformer_linear_plan reports.  *whole_chains is 0 when
+ * every chain is cut and `chains` (with one segment) when none is.  Same arguments, status codes
+ * and behaviour on error as gformer_linear_plan; whole_chains must not be null. */
+int gformer_linear_plan_parts(int chains, int N, int d, int ctas, int* whole_chains, int* segments,
+                              int* chunks_per_segment);
+
 /* Algorithm 2 (Sec. III-D): the share p' in (0, 1) of a problem given to engine 0 at which the two
  * latency estimates  p size flops_per0 / perf0  and  (1 - p) size flops_per1 / perf1  are equal
  * (size cancels).  flops_per_i: work per unit of the part engine i runs; perf_i: that engine's

@@ -60,6 +60,9 @@ def lib() -> ctypes.CDLL:
         L.gformer_partition_balance.argtypes = [dbl, dbl, dbl, dbl, pdbl]
         L.gformer_partition_heads.restype = i
         L.gformer_partition_heads.argtypes = [i, i, i, i, i, dbl, dbl, ctypes.POINTER(ctypes.c_int), pdbl, pdbl]
+        pint = ctypes.POINTER(ctypes.c_int)
+        L.gformer_linear_plan_parts.restype = i
+        L.gformer_linear_plan_parts.argtypes = [i, i, i, i, pint, pint, pint]
         L.gformer_workspace_bytes.restype = sz
         L.gformer_workspace_bytes.argtypes = [i] * 7
         L.gformer_last_device_status.restype = i
@@ -115,6 +118,16 @@ def linear_plan(chains: int, N: int, d: int, ctas: int = 0):
     if rc != GF_OK:
         raise GformerError(rc, "gformer_linear_plan")
     return g.value, l.value
+
+
+def linear_plan_parts(chains: int, N: int, d: int, ctas: int = 0):
+    """(chains left whole, segments per cut chain, chunks of the longest segment)."""
+    wh, g, l = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    rc = lib().gformer_linear_plan_parts(int(chains), int(N), int(d), int(ctas), ctypes.byref(wh), ctypes.byref(g),
+                                         ctypes.byref(l))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_linear_plan_parts")
+    return wh.value, g.value, l.value
 
 
 def partition_balance(flops_per0: float, flops_per1: float, perf0: float, perf1: float) -> float:

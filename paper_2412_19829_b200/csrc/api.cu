@@ -174,6 +174,15 @@ int gformer_linear_plan(int chains, int N, int d, int ctas, int* segments, int* 
   return GF_OK;
 }
 
+int gformer_linear_plan_parts(int chains, int N, int d, int ctas, int* whole_chains, int* segments,
+                              int* chunks_per_segment) {
+  if (chains < 1 || N < 1 || ctas < 0 || whole_chains == nullptr || segments == nullptr || chunks_per_segment == nullptr)
+    return GF_ERR_INVALID_ARG;
+  if (!gf::tc_linear_supported(N, d, GF_BF16)) return GF_ERR_UNSUPPORTED;
+  gf::linear_tc_plan_parts(chains, N, d, g_linear_split, ctas, whole_chains, chunks_per_segment, segments);
+  return GF_OK;
+}
+
 size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, int dtype) {
   (void)w;
   size_t bytes = sizeof(WsHeader);
@@ -330,8 +339,9 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   const bool both = h_sparse > 0 && h_lin > 0;
   int lin_ctas = 0;
   if (both && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
-    int L = 0, G = 0, dev = 0, sms = 0;
-    gf::linear_tc_plan(B * h_lin, N, d, g_linear_split, 0, &L, &G);
+    int L = 0, G = 0, whole = 0, dev = 0, sms = 0;
+    gf::linear_tc_plan_parts(B * h_lin, N, d, g_linear_split, 0, &whole, &L, &G);
+    if (whole > 0) G = 1;  // items of the first launch: the chains left whole
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return GF_ERR_CUDA;
     if ((long long)B * h_lin * G >= sms) {

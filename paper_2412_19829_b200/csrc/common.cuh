@@ -80,6 +80,11 @@ cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, v
 // ctas: CTAs the kernel will run with, 0 = one per SM of a B200) and the scratch it needs beyond
 // the workspace header (sized for the largest segment count the plan may pick for any ctas).
 void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* chunks_per_segment, int* segments_per_chain);
+// The same plan with its two parts named: the first *whole_chains chains are left whole, the others cut
+// (with somewhat more chains than CTAs the full rounds go whole and the leftover chains are cut, in a
+// second launch); *whole_chains = nchains and one segment per chain when nothing is cut.
+void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* whole_chains, int* chunks_per_segment,
+                          int* segments_per_chain);
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split);
 // Bytes at the start of that scratch (right after the workspace header) that must be zero when the
 // kernel starts: the hand-over flags.  The caller clears them (together with the header).

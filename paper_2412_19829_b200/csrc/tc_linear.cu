@@ -100,7 +100,8 @@ struct LinCfg {
 };
 
 struct LinParams {
-  int N, nch, h_begin, h_count, nchains;
+  int N, nch, h_begin, h_count, nchains;  // nchains: chains of this launch, the first being chain0 of the call
+  int chain0;
   int G, nitems;         // segments per chain, nchains * G
   int seg_base, seg_rem; // the first seg_rem segments of a chain have seg_base + 1 chunks, the others seg_base
   float* S_io;           // [B, h_count, D, D] or null
@@ -121,8 +122,9 @@ __device__ __forceinline__ LinItem decode_item(const LinParams& p, int item) {
   LinItem it;
   it.g = item / p.nchains;
   it.chain = item - it.g * p.nchains;
-  it.b = it.chain / p.h_count;
-  it.hl = it.chain - it.b * p.h_count;
+  const int call_chain = p.chain0 + it.chain;
+  it.b = call_chain / p.h_count;
+  it.hl = call_chain - it.b * p.h_count;
   it.h = p.h_begin + it.hl;
   it.c_begin = it.g * p.seg_base + (it.g < p.seg_rem ? it.g : p.seg_rem);
   it.nC = p.seg_base + (it.g < p.seg_rem ? 1 : 0);
@@ -1213,19 +1215,13 @@ void plan_range(int nchains, int nch, int* g_min_out, int* g_max_out) {
 }
 }  // namespace
 
-void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, int* G_out) {
-  const int nch = (N + 127) / 128;
-  int G;
-  if (split > 0) {
-    const int L = split > kMaxL ? kMaxL : split;
-    G = (nch + L - 1) / L;
-  } else if (split < 0) {
-    G = 1;  // never cut: the one-pass form whatever the shape
-  } else {
-    const int kPlanSMs = ctas > 0 ? ctas : 148;
+namespace {
+// Best two-pass plan for nchains chains of nch chunks: its cost in two-pass chunks (1e300 and
+// *G_out = 1 when the chains are too short to cut).
+double best_cut(int nchains, int nch, int d, int kPlanSMs, int* G_out) {
     int g_min, g_max;
     plan_range(nchains, nch, &g_min, &g_max);
-    G = 1;
+    int G = 1;
     double best = 1e300;
     for (int g = g_min > 2 ? g_min : 2; g <= g_max; ++g) {
       const long long items = (long long)nchains * g;
@@ -1243,24 +1239,67 @@ void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, 
         G = g;
       }
     }
-    // An uncut chain needs neither the first pass nor a hand-over (the kernel transforms K inside
-    // the chunk pipeline): a chunk then costs direct_chunk_cost(d) of a two-pass one.  With many
-    // chains that is the cheaper plan even though a CTA then walks a whole chain.
+    *G_out = G;
+    return best;
+}
+
+// Fixed cost, in two-pass chunks, of running the leftover chains as a launch of their own (the gap
+// between the launches, the second kernel's start-up and its uneven end: about 15 us).
+constexpr double kSecondLaunchCost = 6.0;
+}  // namespace
+
+// `*whole_out` leading chains are left whole (the one-pass form), the others are cut into *G_out
+// segments (the two-pass form; *G_out = 1 and *whole_out = nchains when no chain is cut).
+// An uncut chain needs neither the first pass nor a hand-over (the kernel transforms K inside the
+// chunk pipeline): a chunk then costs direct_chunk_cost(d) of a two-pass one, so with many chains
+// that is the cheaper plan even though a CTA then walks a whole chain.  With somewhat more chains
+// than CTAs the full rounds go whole and only the leftover chains are cut, in a second launch.
+void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* whole_out, int* L_out, int* G_out) {
+  const int nch = (N + 127) / 128;
+  int G, whole = 0;
+  if (split > 0) {
+    const int L = split > kMaxL ? kMaxL : split;
+    G = (nch + L - 1) / L;
+  } else if (split < 0) {
+    G = 1;  // never cut: the one-pass form whatever the shape
+    whole = nchains;
+  } else {
+    const int kPlanSMs = ctas > 0 ? ctas : 148;
+    double best = best_cut(nchains, nch, d, kPlanSMs, &G);
     const int full = nchains / kPlanSMs, rest = nchains % kPlanSMs;
     double last = 0.0;  // the round of the chains left over after the full rounds
     if (rest > 0) {
       last = direct_chunk_cost(d) * rest / kPlanSMs;
       if (last < direct_chunk_floor(d)) last = direct_chunk_floor(d);
     }
-    if ((double)nch * (full * direct_chunk_cost(d) + last) <= best) G = 1;
+    const double full_cost = (double)nch * full * direct_chunk_cost(d);
+    if (full_cost + (double)nch * last <= best) {
+      best = full_cost + (double)nch * last;
+      G = 1;
+      whole = nchains;
+    }
+    if (full > 0 && rest > 0) {
+      int g_rest = 1;
+      const double mixed = full_cost + kSecondLaunchCost + best_cut(rest, nch, d, kPlanSMs, &g_rest);
+      if (g_rest > 1 && mixed < best) {
+        G = g_rest;
+        whole = full * kPlanSMs;
+      }
+    }
   }
   if (G < 1) G = 1;
+  *whole_out = whole;
   *G_out = G;
   *L_out = (nch + G - 1) / G;
 }
 
+void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, int* G_out) {
+  int whole;
+  linear_tc_plan_parts(nchains, N, d, split, ctas, &whole, L_out, G_out);
+}
+
 namespace {
-// Largest segment count the plan may pick (the scratch is laid out for it).
+// Largest segment count the plan may pick for nchains chains (the scratch is laid out for it).
 int plan_g_max(int nchains, int N, int split) {
   int L, G;
   linear_tc_plan(nchains, N, 128, split, 0, &L, &G);
@@ -1270,15 +1309,29 @@ int plan_g_max(int nchains, int N, int split) {
   }
   return G;
 }
+
+// Largest number of hand-over slots (chains x segments) a launch of a call on nchains chains may
+// use, whatever the CTA count: all chains cut, or the r < nchains chains left over after the full
+// rounds (plan_range gives those at most min(ceil(nch / 4), max(the cap for many chains,
+// ceil(296 / r))) segments, and r x that stays below the bound taken here).
+long long plan_slots_max(int nchains, int N, int split) {
+  long long m = (long long)nchains * plan_g_max(nchains, N, split);
+  if (split == 0 && nchains > 1) {
+    const long long nch4 = ((N + 127) / 128 + 3) / 4, r = nchains - 1;
+    const long long rest = r * nch4 < 296 + r ? r * nch4 : 296 + r;
+    if (m < rest) m = rest;
+  }
+  return m;
+}
 }  // namespace
 
 size_t linear_tc_flag_bytes(int nchains, int N, int split) {
-  return (size_t)nchains * plan_g_max(nchains, N, split) * kFlagStride * sizeof(unsigned int);
+  return (size_t)plan_slots_max(nchains, N, split) * kFlagStride * sizeof(unsigned int);
 }
 
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
-  const int G = plan_g_max(nchains, N, split);
-  return linear_tc_flag_bytes(nchains, N, split) + (size_t)nchains * G * ((size_t)128 * d + d) * sizeof(float);
+  return linear_tc_flag_bytes(nchains, N, split) +
+         (size_t)plan_slots_max(nchains, N, split) * ((size_t)128 * d + d) * sizeof(float);
 }
 
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
@@ -1294,7 +1347,7 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   p.nch = (N + 127) / 128;
   p.h_begin = h_begin;
   p.h_count = h_count;
-  p.nchains = B * h_count;
+  const int nchains = B * h_count;
   int dev = 0, sms = 0;
   cudaError_t e;
   if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
@@ -1302,36 +1355,43 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   // One CTA per SM at most: every CTA must be resident for the segment hand-over to make progress.
   // (max_ctas > 0 leaves SMs to a kernel running beside this one.)
   if (max_ctas > 0 && max_ctas < sms) sms = max_ctas;
-  int L_max = 0;
-  linear_tc_plan(p.nchains, N, d, split, sms, &L_max, &p.G);
-  p.seg_base = p.nch / p.G;
-  p.seg_rem = p.nch % p.G;
-  p.nitems = p.nchains * p.G;
+  int L_max = 0, whole = 0, G = 1;
+  linear_tc_plan_parts(nchains, N, d, split, sms, &whole, &L_max, &G);
   p.S_io = S_io;
   p.z_io = z_io;
   p.zero_init = zero_init ? 1 : 0;
   p.status = &ws->status;
   uint8_t* scratch = reinterpret_cast<uint8_t*>(ws) + sizeof(WsHeader);
   p.flags = reinterpret_cast<unsigned int*>(scratch);  // zeroed by the caller
-  p.prefix = reinterpret_cast<float*>(scratch + linear_tc_flag_bytes(p.nchains, N, split));
-  dim3 grid(p.nitems < sms ? p.nitems : sms);
-  // automatic plan, chains left whole: the one-pass form of the kernel (a segment length asked
-  // for by the caller always takes the two-pass form, also when it covers the whole chain)
-  const bool direct = split <= 0 && p.G == 1;
+  p.prefix = reinterpret_cast<float*>(scratch + linear_tc_flag_bytes(nchains, N, split));
   auto launch = [&](auto kern, size_t smem) -> cudaError_t {
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
+    dim3 grid(p.nitems < sms ? p.nitems : sms);
     kern<<<grid, kThreads, smem, stream>>>(mq, mk, mv, mo, p);
-    return cudaSuccess;
+    note_launch();
+    return cudaGetLastError();
   };
-  if (d == 64)
-    e = direct ? launch(linear_tc_kernel<64, true>, LinCfg<64>::kBytes) : launch(linear_tc_kernel<64, false>, LinCfg<64>::kBytes);
-  else
-    e = direct ? launch(linear_tc_kernel<128, true>, LinCfg<128>::kBytes)
-               : launch(linear_tc_kernel<128, false>, LinCfg<128>::kBytes);
-  if (e != cudaSuccess) return e;
-  note_launch();
-  return cudaGetLastError();
+  // Chains [chain0, chain0 + count) of the call in one launch: whole (the one-pass form of the kernel) or cut
+  // into g segments (the two-pass form).  The one-pass form neither reads nor writes the hand-over scratch.
+  auto run = [&](int chain0, int count, int g, bool direct) -> cudaError_t {
+    p.chain0 = chain0;
+    p.nchains = count;
+    p.G = g;
+    p.seg_base = p.nch / g;
+    p.seg_rem = p.nch % g;
+    p.nitems = count * g;
+    if (d == 64)
+      return direct ? launch(linear_tc_kernel<64, true>, LinCfg<64>::kBytes)
+                    : launch(linear_tc_kernel<64, false>, LinCfg<64>::kBytes);
+    return direct ? launch(linear_tc_kernel<128, true>, LinCfg<128>::kBytes)
+                  : launch(linear_tc_kernel<128, false>, LinCfg<128>::kBytes);
+  };
+  // `whole` leading chains uncut (automatic plan only: a segment length asked for by the caller always takes
+  // the two-pass form, also when it covers the whole chain), the others cut into G segments behind them
+  if (whole > 0 && (e = run(0, whole, 1, true)) != cudaSuccess) return e;
+  if (whole < nchains && (e = run(whole, nchains - whole, G, false)) != cudaSuccess) return e;
+  return cudaSuccess;
 }
 
 }  // namespace gf

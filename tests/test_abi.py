@@ -91,9 +91,15 @@ def test_linear_plan_covers_the_chain_and_fits_the_workspace():
                     nch = -(-N // 128)
                     assert 1 <= G <= nch
                     assert L == -(-nch // G)  # balanced segments: the longest has ceil(nch / G) chunks
+                    whole, G2, L2 = gf.linear_plan_parts(chains, N, d, ctas)
+                    assert (G2, L2) == (G, L) and 0 <= whole <= chains
                     if G > 1:
                         assert 3 < nch / G <= 32
-                        assert ws >= _state_scratch(chains, G, d), (chains, N, d, ctas, G)
+                        # the first `whole` chains are not cut and need no scratch
+                        assert whole % (ctas or 148) == 0
+                        assert ws >= _state_scratch(chains - whole, G, d), (chains, N, d, ctas, G)
+                    else:
+                        assert whole in (0, chains)
 
 
 def test_linear_plan_named_cases():
@@ -114,9 +120,20 @@ def test_linear_plan_named_cases():
     assert gf.linear_plan(832, 4096, 64)[0] == 1
     # chains that nearly fill one round of CTAs, or spill thinly into a second one: whole, also when long
     # (measured on a B200: 100 chains of 32K tokens at d = 128 take 706 us whole and 841 us cut)
-    for chains in (100, 120, 190, 208, 296):
-        assert gf.linear_plan(chains, 32768, 128)[0] == 1, chains
-    assert gf.linear_plan(120, 32768, 64)[0] == 1 and gf.linear_plan(230, 32768, 64)[0] == 1
+    for chains in (100, 120, 230, 296):
+        assert gf.linear_plan_parts(chains, 32768, 128) == (chains, 1, 256), chains
+    assert gf.linear_plan(120, 32768, 64)[0] == 1 and gf.linear_plan(296, 32768, 64)[0] == 1
+    # somewhat more chains than CTAs, long: the full rounds whole, the leftover chains cut in a launch of their own
+    # (measured: 150 chains of 32K tokens at d = 128 take 946 us this way, 1271 us all cut, 1453 us all whole)
+    for chains, d in ((150, 128), (156, 128), (208, 128), (300, 128), (150, 64), (230, 64), (832, 64)):
+        whole, G, L = gf.linear_plan_parts(chains, 32768, d)
+        assert whole == chains // 148 * 148 and G > 1 and 4 <= L <= 32, (chains, d)
+        assert gf.linear_plan(chains, 32768, d) == (G, L)
+        w37 = gf.linear_plan_parts(chains, 32768, d, 37)[0]
+        assert w37 % 37 == 0 or w37 == chains
+    # ... but not when the second launch would cost what it saves (the 4K prefill: 832 short chains)
+    assert gf.linear_plan_parts(832, 4096, 64) == (832, 1, 32)
+    assert gf.linear_plan_parts(26, 32768, 128)[0] == 0
     # ... while half a round of long chains is cut
     assert gf.linear_plan(74, 32768, 128)[0] > 1 and gf.linear_plan(90, 32768, 64)[0] > 1
     # fewer chains than CTAs, long: cut, in segments of about what stays in L2 at d = 64 (16 chunks of 16 KB tiles)
@@ -139,6 +156,13 @@ def test_linear_plan_argument_errors():
     assert L.gformer_linear_plan(1, 128, 96, 0, ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_UNSUPPORTED
     assert L.gformer_linear_plan(1, 128, 64, 0, None, ctypes.byref(l)) == gf.GF_ERR_INVALID_ARG
     assert (g.value, l.value) == (-7, -7)
+    wh = ctypes.c_int(-7)
+    assert L.gformer_linear_plan_parts(0, 128, 64, 0, ctypes.byref(wh), ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_linear_plan_parts(1, 128, 96, 0, ctypes.byref(wh), ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_UNSUPPORTED
+    assert L.gformer_linear_plan_parts(1, 128, 64, 0, None, ctypes.byref(g), ctypes.byref(l)) == gf.GF_ERR_INVALID_ARG
+    assert (wh.value, g.value, l.value) == (-7, -7, -7)
+    assert L.gformer_linear_plan_parts(1, 128, 64, 0, ctypes.byref(wh), ctypes.byref(g), ctypes.byref(l)) == gf.GF_OK
+    assert (wh.value, g.value, l.value) == (1, 1, 1)
 
 
 def test_partition_balance_against_the_oracle():

@@ -220,6 +220,64 @@ def test_linear_tensor_core(N, d, gain):
     assert_parity(f64(o), ref, "bf16", f"linear tc N={N} d={d}")
 
 
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("bnhd", [False, True])
+def test_whole_and_cut_chains_in_one_call(d, bnhd):
+    # 156 chains on 148 CTAs: the plan leaves the first 148 whole and cuts the other 8 in a second launch.
+    # Chains on both sides of that border against the oracle, with an initial state and the final state.
+    B, H, N = 2, 78, 4096
+    whole, G, L = gf.linear_plan_parts(B * H, N, d)
+    assert whole == 148 and G > 1
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=910 + d, gain=1.0)
+    rng = np.random.default_rng(911)
+    S0 = np.abs(rng.standard_normal((B, H, d, d))) * 0.5
+    z0 = np.abs(rng.standard_normal((B, H, d))) * 8.0 + 4.0
+    S = torch.tensor(S0, dtype=torch.float32, device="cuda")
+    z = torch.tensor(z0, dtype=torch.float32, device="cuda")
+    S0, z0 = f64(S), f64(z)  # what the kernel starts from, after rounding to fp32
+    ws = gf.Workspace.for_problem(B, H, N, d)
+    if bnhd:
+        qn, kn, vn = [t.permute(0, 2, 1, 3).contiguous().cuda() for t in (q, k, v)]
+        o = gf.causal_linear_attn(qn, kn, vn, S, z, layout=gf.GF_BNHD, ws=ws).permute(0, 2, 1, 3).cpu()
+    else:
+        o = gf.causal_linear_attn(*dev(q, k, v), S, z, ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    assert torch.isfinite(o.float()).all()
+    for b, h in ((0, 0), (1, 68), (1, 69), (1, 70), (1, 71), (1, 77)):  # chains 0, 146, 147 | 148, 149, 155
+        Sr, zr = S0[b:b + 1, h:h + 1].copy(), z0[b:b + 1, h:h + 1].copy()
+        ref = oracle.causal_linear_attn(f64(q[b:b + 1, h:h + 1]), f64(k[b:b + 1, h:h + 1]), f64(v[b:b + 1, h:h + 1]), Sr, zr)
+        assert_parity(f64(o[b:b + 1, h:h + 1]), ref, "bf16", f"chain ({b}, {h}) d={d} bnhd={bnhd}")
+        assert errors(f64(S[b:b + 1, h:h + 1].cpu()), Sr)["rel_l2"] <= 1e-2
+        assert errors(f64(z[b:b + 1, h:h + 1].cpu()), zr)["rel_l2"] <= 1e-2
+    # the plan is a matter of speed only: cutting every chain, or none, gives the same values within rounding
+    for split in (8, -1):
+        gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
+        S2 = torch.tensor(S0, dtype=torch.float32, device="cuda"); z2 = torch.tensor(z0, dtype=torch.float32, device="cuda")
+        o2 = gf.causal_linear_attn(*dev(q, k, v), S2, z2).cpu()
+        assert errors(f64(o2), f64(o))["max_abs"] <= 2e-2
+        assert errors(f64(S2), f64(S))["rel_l2"] <= 1e-3
+
+
+def test_hybrid_with_whole_and_cut_linear_chains_and_state_export():
+    # the layer with 160 linear chains (148 whole + 12 cut) beside windowed heads, exporting the decode state
+    B, H, N, d, w, h0 = 2, 83, 2048, 64, 100, 3
+    assert gf.linear_plan_parts(B * (H - h0), N, d)[0] == 148 and gf.linear_plan_parts(B * (H - h0), N, d)[1] > 1
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=920, gain=1.0)
+    st = gf.DecodeState(B, H, d, w, h0)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    o = gf.hybrid_attn(*dev(q, k, v), w, h_sparse=h0, state_out=st, ws=ws).cpu()
+    assert ws.last_device_status() == gf.GF_OK
+    ref_w = oracle.window_attn(f64(q[:, [0, 2]]), f64(k[:, [0, 2]]), f64(v[:, [0, 2]]), w)
+    assert_parity(f64(o[:, [0, 2]]), ref_w, "bf16", "window heads beside whole and cut chains")
+    lin = [3, 40, 70, 71, 76, 77, 78, H - 1]  # batch 1: linear chains 80 + (h - 3), so 147 | 148 are heads 70 | 71
+    Sr = np.zeros((B, len(lin), d, d)); zr = np.zeros((B, len(lin), d))
+    ref_l = oracle.causal_linear_attn(f64(q[:, lin]), f64(k[:, lin]), f64(v[:, lin]), Sr, zr)
+    assert_parity(f64(o[:, lin]), ref_l, "bf16", "linear heads, whole and cut")
+    idx = [h - h0 for h in lin]
+    assert errors(f64(st.S[:, idx].cpu()), Sr)["rel_l2"] <= 1e-2
+    assert errors(f64(st.z[:, idx].cpu()), zr)["rel_l2"] <= 1e-2
+
+
 @pytest.mark.parametrize("split", [1, 2, 4])
 def test_linear_tensor_core_split_invariance(split):
     gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
