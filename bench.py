@@ -329,6 +329,45 @@ def run_ours(args, c, rank, world, local_rank):
     def step():
         layer(dq, dk, dv, w, h_sparse=h0, out=do, ws=ws, stream=stream)
 
+    # End to end, the way a caller would stream batches through the layer: two sets of device
+    # buffers, the host-to-device copy of step i+1 and the device-to-host copy of step i-1 run on
+    # streams of their own beside the layer call of step i (the link is full duplex and the copy
+    # engines are separate from the SMs).  Every step still copies its own Q, K, V in from pinned
+    # memory and its own output back; the timed region runs from the first copy to the last one.
+    def timed_e2e_pipelined(steps):
+        sets = [(dq, dk, dv, do), tuple(torch.empty_like(t) for t in (dq, dk, dv, do))]
+        hos = [ho, torch.empty_like(ho).pin_memory()]
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        ev_in = [torch.cuda.Event() for _ in range(steps)]
+        ev_done = [torch.cuda.Event() for _ in range(steps)]
+        ev_out = [torch.cuda.Event() for _ in range(steps)]
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        t0.record(s_in)
+        for i in range(steps):
+            q_, k_, v_, o_ = sets[i % 2]
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_done[i - 2])  # the layer call that last read this input set
+                q_.copy_(hq, non_blocking=True)
+                k_.copy_(hk, non_blocking=True)
+                v_.copy_(hv, non_blocking=True)
+                ev_in[i].record(s_in)
+            stream.wait_event(ev_in[i])
+            if i >= 2:
+                stream.wait_event(ev_out[i - 2])  # the copy that last read this output buffer
+            layer(q_, k_, v_, w, h_sparse=h0, out=o_, ws=ws, stream=stream)
+            ev_done[i].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[i])
+                hos[i % 2].copy_(o_, non_blocking=True)
+                ev_out[i].record(s_out)
+        t1.record(s_out)
+        s_out.synchronize()
+        stream.synchronize()
+        barrier()
+        return t0.elapsed_time(t1)
+
     def step_e2e():
         with torch.cuda.stream(stream):
             dq.copy_(hq, non_blocking=True)
@@ -371,7 +410,8 @@ def run_ours(args, c, rank, world, local_rank):
 
     for _ in range(2):
         step_e2e()
-    e2e_ms, _ = timed(step_e2e, args.steps)
+    stream.synchronize()
+    e2e_ms = timed_e2e_pipelined(args.steps)
 
     # The two kernels of a step, each timed alone over the same number of launches (B = 1 makes the
     # head slices contiguous): the dominant one carries the roofline entry.
@@ -428,7 +468,9 @@ def run_ours(args, c, rank, world, local_rank):
                          "step": {"achieved": step_gbs, "frac": step_gbs / peak, "algorithmic_bytes": abytes,
                                   "tflops_algorithmic": algorithmic_flops(c, h0) / mean_launch_s / 1e12}},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * tensor_bytes,
-                    "d2h_bytes_per_step": tensor_bytes},
+                    "d2h_bytes_per_step": tensor_bytes,
+                    "how": "two buffer sets: the copies of neighbouring steps run on their own streams beside "
+                           "the layer call; timed from the first copy in to the last copy out"},
             "gpu_launches": launches,
             "clocks": clocks,
             "step_ms_min": min(per), "step_ms_max": max(per),
