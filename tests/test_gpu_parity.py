@@ -460,7 +460,7 @@ def test_many_short_segments_per_cta(d, split):
     assert_parity(f64(o[:, lh]), ref, "bf16", f"segments of {split} chunks, d={d}")
 
 
-@pytest.mark.parametrize("ctas", [1, 37, 100])
+@pytest.mark.parametrize("ctas", [1, 10, 25, 37, 100])  # 10, 25: rounds of whole chains, then the leftover chains cut
 def test_linear_cta_limit_gives_the_same_result(ctas):
     # the segment plan follows the number of CTAs the persistent kernel is given; any count must
     # reproduce the oracle (and, segment boundaries aside, the unrestricted call)
@@ -474,7 +474,7 @@ def test_linear_cta_limit_gives_the_same_result(ctas):
     o = gf.hybrid_attn(qd, kd, vd, w, ws=ws).cpu()
     assert ws.last_device_status() == gf.GF_OK
     assert torch.equal(o[:, :h0], full[:, :h0])  # the windowed heads do not depend on the plan
-    lh = [h0, H - 1]
+    lh = [h0, h0 + 24, h0 + 25, H - 3, H - 2, H - 1]
     ref = oracle.causal_linear_attn(f64(q[:, lh]), f64(k[:, lh]), f64(v[:, lh]))
     assert_parity(f64(o[:, lh]), ref, "bf16", f"linear heads with {ctas} CTAs")
 
