@@ -103,11 +103,11 @@ int run_window(const void* q, const void* k, const void* v, void* o, int B, int 
 
 int run_linear(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
                int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init, int max_ctas,
-               WsHeader* ws, cudaStream_t stream) {
+               WsHeader* ws, cudaStream_t stream, bool shared = false) {
   if (h_count <= 0) return GF_OK;
   if (!g_force_simt && gf::tc_linear_supported(N, d, dtype))
     return cuda_status(gf::launch_linear_tc(q, k, v, o, B, H, N, d, layout, h_begin, h_count, S_io, z_io,
-                                            zero_init, g_linear_split, max_ctas, ws, stream));
+                                            zero_init, g_linear_split, max_ctas, ws, stream, shared));
   return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d),
                                             h_begin, h_count, S_io, z_io, zero_init, stream));
 }
@@ -340,7 +340,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   int lin_ctas = 0;
   if (both && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
     int L = 0, G = 0, whole = 0, dev = 0, sms = 0;
-    gf::linear_tc_plan_parts(B * h_lin, N, d, g_linear_split, 0, &whole, &L, &G);
+    gf::linear_tc_plan_parts(B * h_lin, N, d, g_linear_split, 0, &whole, &L, &G, true);
     if (whole > 0) G = 1;  // items of the first launch: the chains left whole
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return GF_ERR_CUDA;
@@ -363,7 +363,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   const bool lin_first = both && lin_ctas > 0;
   if (lin_first && cudaStreamWaitEvent(f->first, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
   rc = run_linear(q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, lin_ctas,
-                  (WsHeader*)ws, lin_first ? f->first : stream);
+                  (WsHeader*)ws, lin_first ? f->first : stream, both);
   if (lin_first) {
     if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;

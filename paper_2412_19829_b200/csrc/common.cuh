@@ -83,15 +83,16 @@ void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* chunks_
 // The same plan with its two parts named: the first *whole_chains chains are left whole, the others cut
 // (with somewhat more chains than CTAs the full rounds go whole and the leftover chains are cut, in a
 // second launch); *whole_chains = nchains and one segment per chain when nothing is cut.
+// shared: other kernels run beside this one and fill the SMs a thin round of whole chains leaves idle.
 void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* whole_chains, int* chunks_per_segment,
-                          int* segments_per_chain);
+                          int* segments_per_chain, bool shared = false);
 size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split);
 // Bytes at the start of that scratch (right after the workspace header) that must be zero when the
 // kernel starts: the hand-over flags.  The caller clears them (together with the header).
 size_t linear_tc_flag_bytes(int nchains, int N, int split);
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream);
+                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared = false);
 
 // ---- device helpers
 __device__ __forceinline__ float to_f32(float x) { return x; }

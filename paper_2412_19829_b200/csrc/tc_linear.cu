@@ -1254,7 +1254,8 @@ constexpr double kSecondLaunchCost = 6.0;
 // chunk pipeline): a chunk then costs direct_chunk_cost(d) of a two-pass one, so with many chains
 // that is the cheaper plan even though a CTA then walks a whole chain.  With somewhat more chains
 // than CTAs the full rounds go whole and only the leftover chains are cut, in a second launch.
-void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* whole_out, int* L_out, int* G_out) {
+void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* whole_out, int* L_out, int* G_out,
+                          bool shared) {
   const int nch = (N + 127) / 128;
   int G, whole = 0;
   if (split > 0) {
@@ -1273,12 +1274,19 @@ void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* w
       if (last < direct_chunk_floor(d)) last = direct_chunk_floor(d);
     }
     const double full_cost = (double)nch * full * direct_chunk_cost(d);
+    // With a round or more of chains and other kernels to fill the idle SMs of a thin last round, cutting every
+    // chain only adds SM-time (measured in the hybrid layer at d = 64: 17-22 % slower than whole chains).
+    if (shared && full > 0) best = 1e300;
     if (full_cost + (double)nch * last <= best) {
       best = full_cost + (double)nch * last;
       G = 1;
       whole = nchains;
     }
-    if (full > 0 && rest > 0) {
+    // When other kernels share the GPU (the windowed heads of the hybrid layer), their CTAs fill the SMs
+    // that a thin last round of whole chains leaves idle, and cutting the leftover chains only pays when
+    // they are few (measured with 3 of 16 heads windowed: a gain up to 13 % for 8 to 21 leftover
+    // chains on 148 CTAs, a loss of 3 to 11 % from 34 on).
+    if (full > 0 && rest > 0 && (!shared || 6 * rest <= kPlanSMs)) {
       int g_rest = 1;
       const double mixed = full_cost + kSecondLaunchCost + best_cut(rest, nch, d, kPlanSMs, &g_rest);
       if (g_rest > 1 && mixed < best) {
@@ -1295,7 +1303,7 @@ void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* w
 
 void linear_tc_plan(int nchains, int N, int d, int split, int ctas, int* L_out, int* G_out) {
   int whole;
-  linear_tc_plan_parts(nchains, N, d, split, ctas, &whole, L_out, G_out);
+  linear_tc_plan_parts(nchains, N, d, split, ctas, &whole, L_out, G_out, false);
 }
 
 namespace {
@@ -1336,7 +1344,7 @@ size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
 
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream) {
+                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared) {
   if (h_count <= 0) return cudaSuccess;
   CUtensorMap mq, mk, mv, mo;
   if (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128) ||
@@ -1356,7 +1364,7 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   // (max_ctas > 0 leaves SMs to a kernel running beside this one.)
   if (max_ctas > 0 && max_ctas < sms) sms = max_ctas;
   int L_max = 0, whole = 0, G = 1;
-  linear_tc_plan_parts(nchains, N, d, split, sms, &whole, &L_max, &G);
+  linear_tc_plan_parts(nchains, N, d, split, sms, &whole, &L_max, &G, shared);
   p.S_io = S_io;
   p.z_io = z_io;
   p.zero_init = zero_init ? 1 : 0;
