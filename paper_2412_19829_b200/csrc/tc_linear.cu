@@ -1276,7 +1276,9 @@ void linear_tc_plan_parts(int nchains, int N, int d, int split, int ctas, int* w
     const double full_cost = (double)nch * full * direct_chunk_cost(d);
     // With a round or more of chains and other kernels to fill the idle SMs of a thin last round, cutting every
     // chain only adds SM-time (measured in the hybrid layer at d = 64: 17-22 % slower than whole chains).
-    if (shared && full > 0) best = 1e300;
+    // The same holds from half a round of chains on (measured at d = 64 with 78 to 104 chains: whole chains
+    // 3-23 % faster than cut ones beside the windowed heads; with 65 chains the cut plan still wins).
+    if (shared && (full > 0 || 2 * nchains >= kPlanSMs)) best = 1e300;
     if (full_cost + (double)nch * last <= best) {
       best = full_cost + (double)nch * last;
       G = 1;
