@@ -221,11 +221,12 @@ def test_linear_tensor_core(N, d, gain):
 
 
 @pytest.mark.parametrize("d", [64, 128])
-@pytest.mark.parametrize("bnhd", [False, True])
-def test_whole_and_cut_chains_in_one_call(d, bnhd):
+@pytest.mark.parametrize("bnhd,N", [(False, 4096), (True, 4096), (False, 4001)])
+def test_whole_and_cut_chains_in_one_call(d, bnhd, N):
     # 156 chains on 148 CTAs: the plan leaves the first 148 whole and cuts the other 8 in a second launch.
-    # Chains on both sides of that border against the oracle, with an initial state and the final state.
-    B, H, N = 2, 78, 4096
+    # Chains on both sides of that border against the oracle, with an initial state and the final state
+    # (N = 4001: a ragged last chunk in both forms).
+    B, H = 2, 78
     whole, G, L = gf.linear_plan_parts(B * H, N, d)
     assert whole == 148 and G > 1
     q, k, v = synth.qkv(B, H, N, d, "bf16", seed=910 + d, gain=1.0)
