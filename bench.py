@@ -11,6 +11,10 @@ the data path); rank 0 prints one JSON line.
 
 --impl reference times the fp64 CPU oracle on the host cores, on a bounded sample of the
 same workload (the first tokens of every head); it is a deliberately slow reference.
+
+Other workloads (--workload): gpt2s, prefill4k, self32k (the bidirectional layer), decode256,
+sweep5 (the 32 points of the fixed-65536-token sweep, one JSON line).  --kernel-only linear|window
+runs only that head group's kernel a few times (a small driver for profilers).
 """
 from __future__ import annotations
 
@@ -29,7 +33,7 @@ if ROOT not in sys.path:
 METRIC = "hybrid_attention_tokens_per_s"
 UNIT = "tokens/s"
 # oracle samples: the first tokens of every head of the workload
-CPU_BASELINE_TOKENS = 32768  # cpu_baseline leg: about 10 s of fp64 work on 8 cores at d=128
+CPU_BASELINE_TOKENS = 32768  # cpu_baseline leg: a few seconds of fp64 work at d=128 (3 s on 16 cores)
 REFERENCE_STEP_TOKENS = 4096  # --impl reference: about 1 s per step
 
 WORKLOADS = {
@@ -40,7 +44,10 @@ WORKLOADS = {
     "self32k": dict(B=1, H=32, N=32768, d=128, w=512, seed=2, self_layer=True),
     # token-by-token decoding after a 4096-token prefill: a step = `steps` decode steps of the batch
     "decode256": dict(B=64, H=16, N=4096, d=64, w=256, seed=3, decode_steps=256),
+    # the 32 points of the sweep at 65 536 tokens per launch (N, d, w vary; H = 16): one JSON line
+    "sweep5": dict(sweep=True, H=16, seed=4),
 }
+NOMINAL_HBM_GBS = 8000.0  # the figure the target is phrased against; fractions of it are printed beside the measured ones
 
 
 # ---- the multi-GPU contract ("replicas only"): every rank runs its own batch of the same shape on
@@ -83,6 +90,22 @@ def recorded_traffic(workload):
         with open(p) as f:
             return json.load(f).get(workload)
     return None
+
+
+def l2_bytes(device_index):
+    """Size of the L2 cache of the device (126 MB on a B200)."""
+    import torch
+
+    return int(torch.cuda.get_device_properties(device_index).L2_cache_size)
+
+
+def rotation_sets(set_bytes, l2):
+    """How many independent (Q, K, V, O) buffer sets a timed loop rotates through so that its traffic
+    is real HBM traffic: one when a set alone exceeds the L2, else at least four and at least twice
+    the L2 in total."""
+    if set_bytes > l2:
+        return 1
+    return max(4, -(-2 * l2 // set_bytes))
 
 
 def algorithmic_bytes(c):
@@ -326,8 +349,37 @@ def run_ours(args, c, rank, world, local_rank):
     self_layer = bool(c.get("self_layer"))
     layer = gf.hybrid_attn_self if self_layer else gf.hybrid_attn
 
+    # Inputs that fit the L2 are rotated over several buffer sets, so that every step reads its
+    # inputs from HBM; the L2-resident figure (one set, back to back) is reported beside it.
+    l2 = l2_bytes(local_rank)
+    set_bytes = 4 * B * H * N * d * 2
+    n_sets = rotation_sets(set_bytes, l2)
+    sets = [(dq, dk, dv, do)] + [tuple(t.clone() for t in (dq, dk, dv, do)) for _ in range(n_sets - 1)]
+    turn = [0]
+
     def step():
+        q_, k_, v_, o_ = sets[turn[0] % n_sets]
+        turn[0] += 1
+        layer(q_, k_, v_, w, h_sparse=h0, out=o_, ws=ws, stream=stream)
+
+    def step_resident():
         layer(dq, dk, dv, w, h_sparse=h0, out=do, ws=ws, stream=stream)
+
+    if args.kernel_only:  # a small driver for profilers: that head group's kernel alone, a few launches
+        if args.kernel_only == "linear":
+            lq, lk, lv, lo_ = [t[:, h0:].contiguous() for t in (dq, dk, dv, do)]
+            ws_l = gf.Workspace.for_problem(B, H - h0, N, d, 1, 0)
+            run = (lambda: gf.hybrid_attn_self(lq, lk, lv, w, h_sparse=0, out=lo_, ws=ws_l, stream=stream)) if self_layer \
+                else (lambda: gf.causal_linear_attn(lq, lk, lv, out=lo_, ws=ws_l, stream=stream))
+        else:
+            wq, wk, wv, wo_ = [t[:, :h0].contiguous() for t in (dq, dk, dv, do)]
+            run = (lambda: gf.window_attn_self(wq, wk, wv, w, out=wo_, ws=ws, stream=stream)) if self_layer \
+                else (lambda: gf.window_attn(wq, wk, wv, w, out=wo_, ws=ws, stream=stream))
+        for _ in range(max(args.warmup, 1) + args.steps):
+            run()
+        stream.synchronize()
+        print(json.dumps({"kernel_only": args.kernel_only, "workload": args.workload, "launches": max(args.warmup, 1) + args.steps}))
+        return
 
     # End to end, the way a caller would stream batches through the layer: two sets of device
     # buffers, the host-to-device copy of step i+1 and the device-to-host copy of step i-1 run on
@@ -408,6 +460,29 @@ def run_ours(args, c, rank, world, local_rank):
     if ws.last_device_status(stream) != gf.GF_OK:
         raise SystemExit("device-side wait timed out during the timed region")
 
+    # Sustained figure: at least a second of back-to-back steps with the clocks sampled throughout
+    # (a 1 kW part settles below its boost clock under a long load; time x clock tells the two apart).
+    sustained = None
+    if not args.no_sustained:  # every rank runs it (the timing helper holds a barrier); rank 0 samples the clocks
+        n_long = max(args.steps, int(1.2e3 / max(total_ms / args.steps, 1e-3)))
+        s2 = ClockSampler(torch.cuda.current_device()) if rank == 0 else None
+        if s2:
+            s2.start()
+        long_ms, _ = timed(step, n_long)
+        (long_ms,) = max_over_ranks([long_ms], dist, "cuda")
+        if s2:
+            ck = s2.stop()
+            sustained = {"steps": n_long, "seconds": long_ms * 1e-3, "ms_per_step": long_ms / n_long,
+                         "sm_mhz_median": ck.get("sm_mhz"), "reasons": ck.get("reasons"),
+                         "clock_samples": ck.get("samples"),
+                         "ms_x_mhz": (long_ms / n_long) * ck["sm_mhz"] if ck.get("sm_mhz") else None}
+    resident = None
+    if n_sets > 1:
+        for _ in range(3):
+            step_resident()
+        r_ms, _ = timed(step_resident, args.steps)
+        resident = {"ms_per_step": r_ms / args.steps, "note": "one buffer set back to back: inputs stay in L2"}
+
     for _ in range(2):
         step_e2e()
     stream.synchronize()
@@ -460,12 +535,17 @@ def run_ours(args, c, rank, world, local_rank):
             "config": {"workload": args.workload, "B": B, "H": H, "N": N, "d": d, "w": w, "h_sparse": h0,
                        "global_batch": world * B, "seq_len": N,
                        "parallelism": "replicas only (one batch element per GPU, no collective)",
-                       "l2": "inputs larger than L2 (Q+K+V = %.0f MB per step)" % (3 * tensor_bytes / 1e6)},
+                       "l2": ("inputs larger than L2 (Q+K+V+O = %.0f MB per step, L2 %.0f MB)" % (set_bytes / 1e6, l2 / 1e6))
+                       if n_sets == 1 else
+                       ("inputs fit the L2 (%.0f MB of %.0f MB): steps rotate over %d buffer sets so that they read HBM; "
+                        "the L2-resident figure is in l2_resident" % (set_bytes / 1e6, l2 / 1e6, n_sets))},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "traffic": recorded_traffic(args.workload),
+                         "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                         "traffic": recorded_traffic(args.workload),
                          "peak_source": which + " copy bandwidth", "algorithmic_bytes": dom_bytes,
                          "kernel": dom_desc, "kernels": kern,
-                         "step": {"achieved": step_gbs, "frac": step_gbs / peak, "algorithmic_bytes": abytes,
+                         "step": {"achieved": step_gbs, "frac": step_gbs / peak,
+                                  "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS, "algorithmic_bytes": abytes,
                                   "tflops_algorithmic": algorithmic_flops(c, h0) / mean_launch_s / 1e12}},
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 3 * tensor_bytes,
                     "d2h_bytes_per_step": tensor_bytes,
@@ -475,6 +555,12 @@ def run_ours(args, c, rank, world, local_rank):
             "clocks": clocks,
             "step_ms_min": min(per), "step_ms_max": max(per),
         }
+        if sustained:
+            sustained["frac"] = abytes / (sustained["ms_per_step"] * 1e-3) / 1e9 / peak
+            line["sustained"] = sustained
+        if resident:
+            resident["frac"] = abytes / (resident["ms_per_step"] * 1e-3) / 1e9 / peak
+            line["l2_resident"] = resident
         if world == 1 and not args.no_cpu_baseline:
             rate, dt, n, cores = oracle_sample_rate(c, CPU_BASELINE_TOKENS)
             line["cpu_baseline"] = {
@@ -632,6 +718,77 @@ def run_decode(args, c, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_sweep(args, c, rank, world, local_rank):
+    """The 32 points of the sweep (65 536 tokens per launch, H = 16, default head split): per point the
+    median launch time of `steps` launches and the fraction of the HBM roofline for the layer's
+    algorithmic bytes; one JSON line.  Points whose tensors fit the L2 rotate over several buffer sets."""
+    import statistics
+
+    import torch
+
+    from paper_2412_19829_b200 import binding as gf
+    from paper_2412_19829_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if rank != 0:  # every point is one GPU's work: the other ranks of a multi-rank launch have nothing to do
+        return
+    stream = torch.cuda.Stream()
+    peak, which = measured_peaks()
+    l2 = l2_bytes(local_rank)
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    points, total_ms, total_tokens, launches0 = [], 0.0, 0, gf.launch_count()
+    for pt in synth.sweep_points():
+        B, H, N, d, w = pt["B"], pt["H"], pt["N"], pt["d"], pt["w"]
+        h0 = gf.default_h_sparse(H)
+        g = torch.Generator(device="cuda").manual_seed(replica_seed(pt, rank))
+        set_bytes = 4 * B * H * N * d * 2
+        n_sets = rotation_sets(set_bytes, l2)
+        sets = []
+        for _ in range(n_sets):
+            q, k, v = [torch.randn(B, H, N, d, device="cuda", generator=g).mul_(d ** -0.5).to(torch.bfloat16)
+                       for _ in range(3)]
+            sets.append((q, k, v, torch.empty_like(q)))
+        ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+        evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        for i in range(max(args.warmup, 3)):
+            q, k, v, o = sets[i % n_sets]
+            gf.hybrid_attn(q, k, v, w, h_sparse=h0, out=o, ws=ws, stream=stream)
+        stream.synchronize()
+        evs[0].record(stream)
+        for i in range(args.steps):
+            q, k, v, o = sets[i % n_sets]
+            gf.hybrid_attn(q, k, v, w, h_sparse=h0, out=o, ws=ws, stream=stream)
+            evs[i + 1].record(stream)
+        stream.synchronize()
+        if ws.last_device_status(stream) != gf.GF_OK:
+            raise SystemExit("device-side wait timed out")
+        ms = statistics.median(evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps))
+        points.append({"N": N, "B": B, "d": d, "w": w, "h_sparse": h0, "ms": ms, "buffer_sets": n_sets,
+                       "frac": set_bytes / (ms * 1e-3) / 1e9 / peak})
+        total_ms += ms
+        total_tokens += B * N
+        del sets
+    clocks = sampler.stop()
+    fracs = sorted(p_["frac"] for p_ in points)
+    line = {
+        "metric": METRIC, "value": total_tokens / (total_ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": total_ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic (seeded, generated on the device: timing only)",
+        "config": {"workload": "sweep5", "points": len(points), "tokens_per_launch": 65536, "H": 16,
+                   "step": "one launch of each of the 32 points (median launch times summed)",
+                   "l2": "points that fit the L2 (%.0f MB) rotate over several buffer sets" % (l2 / 1e6)},
+        "roofline": {"bound": "hbm", "peak": peak, "unit": "GB/s", "peak_source": which + " copy bandwidth",
+                     "frac": fracs[len(fracs) // 2], "frac_worst": fracs[0], "frac_best": fracs[-1],
+                     "achieved": fracs[len(fracs) // 2] * peak, "traffic": None,
+                     "kernel": "whole layer per point (both kernels); frac is the median over the points"},
+        "points": points, "gpu_launches": gf.launch_count() - launches0, "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def algorithmic_flops(c, h0):
     """Flops of the method itself: 4 d per (query, key) pair in the window, 4 d^2 per linear token."""
     B, H, N, d, w = c["B"], c["H"], c["N"], c["d"], c["w"]
@@ -650,12 +807,22 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="long32k", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the one-second sustained run")
+    ap.add_argument("--kernel-only", choices=["linear", "window"], default=None,
+                    help="run only that head group's kernel (no timing): a driver for profilers")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     c = WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if c.get("sweep"):
+        if args.impl == "reference":
+            if rank == 0:
+                print(json.dumps({"impl": "reference", "unavailable": "the sweep workload has no reference arm: "
+                                  "time the oracle on a single shape with --workload long32k/gpt2s/prefill4k"}))
+            return
+        run_sweep(args, c, rank, world, local_rank)
+    elif args.impl == "reference":
         run_reference(args, c, rank)
     elif "decode_steps" in c:
         run_decode(args, c, rank, world, local_rank)
