@@ -53,9 +53,14 @@ typedef enum {
   GF_TUNE_FORCE_SIMT = 0, /* 1: never take the tensor-core kernels (default 0)              */
   GF_TUNE_LINEAR_SPLIT = 1, /* 128-row chunks per sequence segment of a linear chain: 0 = auto,
                                -1 = never cut a chain (the one-pass form of the kernel)          */
-  GF_TUNE_LINEAR_CTAS = 2   /* gformer_hybrid_attn: CTAs of the persistent linear-attention kernel
+  GF_TUNE_LINEAR_CTAS = 2,  /* gformer_hybrid_attn: CTAs of the persistent linear-attention kernel
                                when it shares the GPU with the windowed heads; 0 = auto, else an
                                upper bound in [1, 65535] (the SM count bounds it too)              */
+  GF_TUNE_WAIT_KCYCLES = 3, /* how long a device-side wait may last before the kernel gives up, in
+                               units of 1024 SM cycles; 0 = the default (about two seconds)       */
+  GF_TUNE_TEST_DROP_FLAG = 4 /* failure injection for tests: n > 0 makes the cut-chain form of the
+                               linear kernel never raise the hand-over flag of its n-th segment, so
+                               that the next segment's wait runs out; 0 = off                      */
 } gf_tuning_key;
 
 /* Decode-time state of one batch (see gformer_decode_step).  The struct lives in host
@@ -77,8 +82,11 @@ int gformer_version(void);
  * max(1, round(3 H / 16)) -- 3 of 16 heads is the causal optimum reported in Sec. IV-D. */
 int gformer_default_h_sparse(int H);
 
-/* Sets a gf_tuning_key; returns GF_OK or GF_ERR_INVALID_ARG.  Not thread-safe against
- * concurrent calls into the library. */
+/* Sets a gf_tuning_key; returns GF_OK or GF_ERR_INVALID_ARG.  Every entry point reads each knob
+ * once when it is called; a knob changed while a call is being set up applies from the next call.
+ * gformer_workspace_bytes depends on GF_TUNE_FORCE_SIMT and GF_TUNE_LINEAR_SPLIT: query it again
+ * after changing one of them (a workspace that has become too small is refused with
+ * GF_ERR_WORKSPACE, never overrun). */
 int gformer_set_tuning(int key, int value);
 
 /* How the tensor-core linear-attention kernel would cut `chains` (batch, head) sequences of N
@@ -117,6 +125,18 @@ int gformer_partition_balance(double flops_per0, double flops_per1, double perf0
  * non-finite rate) without touching the outputs. */
 int gformer_partition_heads(int B, int H, int N, int E, int W, double perf_sparse, double perf_linear,
                             int* h_sparse_out, double* latency_sparse_out, double* latency_linear_out);
+
+/* Algorithm 2 fed with measured times (Sec. III-D; the section feeds it micro-benchmarked rates): from the
+ * seconds one windowed head and one linear head cost at this problem size, the balanced share
+ * *p_out of windowed heads (gformer_partition_balance with the seconds as work and rates of 1), that
+ * share as a whole number of the H heads (*h_sparse_out, nearest, in [0, H]), and the two rates in
+ * the units of the section's FLOP model that the measurements imply: one windowed head is
+ * 5 B N W flops, H linear heads together 8 B N (H E)^2.  All outputs are host pointers and must not be
+ * null.  Host arithmetic in fp64.  Returns GF_OK, or GF_ERR_INVALID_ARG (null pointer, size below 1,
+ * a non-positive or non-finite time) without touching the outputs. */
+int gformer_partition_from_times(int B, int H, int N, int E, int W, double seconds_per_sparse_head,
+                                 double seconds_per_linear_head, double* p_out, int* h_sparse_out,
+                                 double* perf_sparse_out, double* perf_linear_out);
 
 /* Number of kernels the library has launched in this process so far (all entry points,
  * all streams).  For accounting in benchmarks. */
@@ -196,6 +216,12 @@ int gformer_causal_linear_attn_noalloc(const void* q, const void* k, const void*
                                        int B, int H, int N, int d, int phi, int chunk,
                                        float* S_io, float* z_io, int dtype, int layout,
                                        void* cuda_stream);
+/* The device status word of the fixed array on the current device, as gformer_last_device_status
+ * reads it for a caller-owned workspace (which this entry point hides): synchronises `cuda_stream`
+ * and returns GF_OK, GF_ERR_TIMEOUT (a bounded wait of the last call gave up -- what two calls that
+ * overlapped on the GPU can cause; that call's outputs are undefined) or GF_ERR_CUDA.  No counterpart
+ * in the paper.  Allocates nothing. */
+int gformer_noalloc_last_device_status(void* cuda_stream);
 
 /*
  * The hybrid layer (Sec. III-A): heads [0, h_sparse) as gformer_window_attn, heads

@@ -24,8 +24,8 @@
  *                 windowed, the rest linear; every head writes its own slot of O.
  *   decode        Algorithm 1 advanced one token at a time plus the window rule on a
  *                 ring buffer of w cached keys/values (token j lives in slot j mod w).
- *   "self" layer  (the bidirectional variant of Sec. II-A used for ViT, Sec. IV-D/E; next in
- *                 line for the CUDA library, no kernel yet)  window head: Eq. 1 without the
+ *   "self" layer  (the bidirectional variant of Sec. II-A used for ViT, Sec. IV-D/E)
+ *                 window head: Eq. 1 without the
  *                 causal mask, over a two-sided window.  The paper does not print the
  *                 two-sided rule; reading taken: token i sees the keys j with |i - j| < w
  *                 (itself, the w-1 tokens before and the w-1 after), truncated at both

@@ -3,9 +3,9 @@
 Algorithm 2 (Sec. III-D) estimates the latency of two engines from the work a split ``p``
 gives to each and looks for the split at which the two estimates meet; the FLOP model of
 the same section instantiates it for the sparse (windowed) and the linear heads.  This
-file takes those steps in the algorithm's order, in fp64, and finds the meeting point by
-bisection and by exhaustive search: no closed form appears here, so that the closed forms
-the library uses can be checked against it.
+file restates the rule as one function, the gap between the two estimates, in fp64, and finds
+its zero by bisection and the best whole number of heads by exhaustive search: no closed form
+appears here, so that the closed forms the library uses can be checked against it.
 
 Pinned by hand-worked splits, mirror and scale invariants and the sign change of the latency
 gap.  The section's own worked example (3 sparse heads of 16 at 4k tokens with rates of 13.37
@@ -17,25 +17,27 @@ Nothing here imports the CUDA package and the CUDA package never imports this.
 from __future__ import annotations
 
 
-def latencies(p, size, flops_per0, flops_per1, perf0, perf1):
-    """The two latency estimates of Algorithm 2 for a split p."""
-    flops_p0 = p * size * flops_per0
-    flops_p1 = (1.0 - p) * size * flops_per1
-    latency0 = flops_p0 / perf0
-    latency1 = flops_p1 / perf1
-    return latency0, latency1
+def gap(p, size, work0, work1, rate0, rate1):
+    """Time engine 0 needs for the share p of the problem minus the time engine 1 needs for the
+    rest (Algorithm 2, Sec. III-D: work per unit over rate, times the units each engine gets).
+    Negative while engine 0 would finish first."""
+    return p * size * work0 / rate0 - (1.0 - p) * size * work1 / rate1
 
 
-def balance(size, flops_per0, flops_per1, perf0, perf1, iters=200):
-    """p' in [0, 1] with latency0 = latency1 (last step of Algorithm 2).
+def latencies(p, size, work0, work1, rate0, rate1):
+    """The two finishing times whose difference `gap` is: engine 0 on the share p, engine 1 on the rest."""
+    return gap(p, size, work0, 0.0, rate0, 1.0), -gap(p, size, 0.0, work1, 1.0, rate1)
 
-    latency0 - latency1 grows with p, is negative at p = 0 and positive at p = 1: bisect.
+
+def balance(size, work0, work1, rate0, rate1, iters=200):
+    """The share p' in [0, 1] at which both engines finish together (Algorithm 2).
+
+    The gap grows with p, is negative at p = 0 and positive at p = 1: bisect on its sign.
     """
     lo, hi = 0.0, 1.0
     for _ in range(iters):
         mid = 0.5 * (lo + hi)
-        l0, l1 = latencies(mid, size, flops_per0, flops_per1, perf0, perf1)
-        if l0 < l1:
+        if gap(mid, size, work0, work1, rate0, rate1) < 0.0:
             lo = mid
         else:
             hi = mid

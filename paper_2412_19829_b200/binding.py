@@ -15,7 +15,7 @@ GF_OK, GF_ERR_INVALID_ARG, GF_ERR_UNSUPPORTED, GF_ERR_WORKSPACE, GF_ERR_CUDA, GF
 GF_F32, GF_BF16 = 0, 1
 GF_BHND, GF_BNHD = 0, 1
 GF_PHI_ELU1 = 0
-GF_TUNE_FORCE_SIMT, GF_TUNE_LINEAR_SPLIT, GF_TUNE_LINEAR_CTAS = 0, 1, 2
+GF_TUNE_FORCE_SIMT, GF_TUNE_LINEAR_SPLIT, GF_TUNE_LINEAR_CTAS, GF_TUNE_WAIT_KCYCLES, GF_TUNE_TEST_DROP_FLAG = 0, 1, 2, 3, 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libgformer.so")
@@ -58,6 +58,8 @@ def lib() -> ctypes.CDLL:
         dbl, pdbl = ctypes.c_double, ctypes.POINTER(ctypes.c_double)
         L.gformer_partition_balance.restype = i
         L.gformer_partition_balance.argtypes = [dbl, dbl, dbl, dbl, pdbl]
+        L.gformer_partition_from_times.restype = i
+        L.gformer_partition_from_times.argtypes = [i, i, i, i, i, dbl, dbl, pdbl, ctypes.POINTER(ctypes.c_int), pdbl, pdbl]
         L.gformer_partition_heads.restype = i
         L.gformer_partition_heads.argtypes = [i, i, i, i, i, dbl, dbl, ctypes.POINTER(ctypes.c_int), pdbl, pdbl]
         pint = ctypes.POINTER(ctypes.c_int)
@@ -76,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.gformer_causal_linear_attn.restype = i
         L.gformer_causal_linear_attn.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, vp, i, i, vp, sz, vp]
         L.gformer_noalloc_scratch_bytes.restype = sz
+        L.gformer_noalloc_last_device_status.restype = i
+        L.gformer_noalloc_last_device_status.argtypes = [vp]
         L.gformer_causal_linear_attn_noalloc.restype = i
         L.gformer_causal_linear_attn_noalloc.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, vp, vp, i, i, vp]
         L.gformer_hybrid_attn.restype = i
@@ -138,6 +142,19 @@ def partition_balance(flops_per0: float, flops_per1: float, perf0: float, perf1:
     if rc != GF_OK:
         raise GformerError(rc, "gformer_partition_balance")
     return p.value
+
+
+def partition_from_times(B: int, H: int, N: int, E: int, W: int, seconds_per_sparse_head: float,
+                         seconds_per_linear_head: float):
+    """(p', balanced head count, perf_sparse, perf_linear) from measured seconds per head (gformer_partition_from_times)."""
+    p, h0 = ctypes.c_double(0.0), ctypes.c_int(0)
+    ps, pl = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    rc = lib().gformer_partition_from_times(int(B), int(H), int(N), int(E), int(W), float(seconds_per_sparse_head),
+                                            float(seconds_per_linear_head), ctypes.byref(p), ctypes.byref(h0),
+                                            ctypes.byref(ps), ctypes.byref(pl))
+    if rc != GF_OK:
+        raise GformerError(rc, "gformer_partition_from_times")
+    return p.value, h0.value, ps.value, pl.value
 
 
 def partition_heads(B: int, H: int, N: int, E: int, W: int, perf_sparse: float, perf_linear: float):

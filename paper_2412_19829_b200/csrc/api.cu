@@ -17,9 +17,22 @@ namespace {
 using gf::Strides;
 using gf::WsHeader;
 
-int g_force_simt = 0;
-int g_linear_split = 0;
-int g_linear_ctas = 0;
+// Process-wide knobs (gformer_set_tuning).  An entry point takes one snapshot when it is called
+// and works from that, so a knob changed by another thread meanwhile cannot make the parts of one
+// call disagree (the cleared flag bytes, the plan, the launch).
+std::atomic<int> g_force_simt{0}, g_linear_split{0}, g_linear_ctas{0}, g_wait_kcycles{0}, g_drop_flag{0};
+struct Tuning {
+  int force_simt, linear_split, linear_ctas, wait_kcycles, drop_flag;
+};
+Tuning tuning_now() {
+  Tuning t;
+  t.force_simt = g_force_simt.load(std::memory_order_relaxed);
+  t.linear_split = g_linear_split.load(std::memory_order_relaxed);
+  t.linear_ctas = g_linear_ctas.load(std::memory_order_relaxed);
+  t.wait_kcycles = g_wait_kcycles.load(std::memory_order_relaxed);
+  t.drop_flag = g_drop_flag.load(std::memory_order_relaxed);
+  return t;
+}
 
 constexpr int kMaxDevices = 64;
 struct Fork {
@@ -88,38 +101,44 @@ int check_ws(void* ws, size_t ws_bytes, size_t need) {
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? GF_OK : GF_ERR_CUDA; }
 
 // Window heads [h_begin, h_begin+h_count) on `stream`.
-int run_window(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
+int run_window(const Tuning& tn, const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
                float scale, int dtype, int layout, int h_begin, int h_count, WsHeader* ws,
                cudaStream_t stream, bool two_sided = false) {
   if (h_count <= 0) return GF_OK;
   const int w_eff = w > N ? N : w;  // keys before token 0 (or after the last one) do not exist
   const int fwd = two_sided ? w_eff - 1 : 0;
-  if (!g_force_simt && gf::tc_window_supported(N, d, w_eff, dtype))
+  if (!tn.force_simt && gf::tc_window_supported(N, d, w_eff, dtype))
     return cuda_status(
         gf::launch_window_tc(q, k, v, o, B, H, N, d, w_eff, fwd, scale, layout, h_begin, h_count, ws, stream));
   return cuda_status(gf::launch_window_simt(q, k, v, o, B, N, d, w_eff, fwd, scale, dtype,
                                             gf::make_strides(layout, H, N, d), h_begin, h_count, stream));
 }
 
-int run_linear(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
+int run_linear(const Tuning& tn, const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
                int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init, int max_ctas,
                WsHeader* ws, cudaStream_t stream, bool shared = false) {
   if (h_count <= 0) return GF_OK;
-  if (!g_force_simt && gf::tc_linear_supported(N, d, dtype))
+  if (!tn.force_simt && gf::tc_linear_supported(N, d, dtype))
     return cuda_status(gf::launch_linear_tc(q, k, v, o, B, H, N, d, layout, h_begin, h_count, S_io, z_io,
-                                            zero_init, g_linear_split, max_ctas, ws, stream, shared));
+                                            zero_init, tn.linear_split, max_ctas, ws, stream, shared));
   return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d),
                                             h_begin, h_count, S_io, z_io, zero_init, stream));
 }
 
 // Zeroes the workspace header and, for a call that runs the tensor-core linear kernel on n_lin
 // chains, the hand-over flags behind it: one memset, ahead of everything the call launches.
-int clear_ws(void* ws, cudaStream_t stream, int n_lin = 0, int N = 0, int d = 0, int dtype = GF_BF16) {
+int clear_ws(const Tuning& tn, void* ws, cudaStream_t stream, int n_lin = 0, int N = 0, int d = 0, int dtype = GF_BF16) {
   size_t bytes = sizeof(WsHeader);
-  if (n_lin > 0 && !g_force_simt && gf::tc_linear_supported(N, d, dtype))
-    bytes += gf::linear_tc_flag_bytes(n_lin, N, g_linear_split);
-  return cuda_status(cudaMemsetAsync(ws, 0, bytes, stream));
+  if (n_lin > 0 && !tn.force_simt && gf::tc_linear_supported(N, d, dtype))
+    bytes += gf::linear_tc_flag_bytes(n_lin, N, tn.linear_split);
+  if (cudaMemsetAsync(ws, 0, bytes, stream) != cudaSuccess) return GF_ERR_CUDA;
+  // the two test knobs travel in the header (all zero otherwise: nothing more to do)
+  if (tn.wait_kcycles != 0 || tn.drop_flag != 0)
+    return cuda_status(gf::launch_set_header((WsHeader*)ws, (unsigned int)tn.wait_kcycles, (unsigned int)tn.drop_flag, stream));
+  return GF_OK;
 }
+
+size_t workspace_bytes(const Tuning& tn, int B, int H, int N, int d, int h_sparse, int dtype);
 
 }  // namespace
 
@@ -152,15 +171,23 @@ int gformer_default_h_sparse(int H) {
 int gformer_set_tuning(int key, int value) {
   switch (key) {
     case GF_TUNE_FORCE_SIMT:
-      g_force_simt = value ? 1 : 0;
+      g_force_simt.store(value ? 1 : 0);
+      return GF_OK;
+    case GF_TUNE_WAIT_KCYCLES:
+      if (value < 0) return GF_ERR_INVALID_ARG;
+      g_wait_kcycles.store(value);
+      return GF_OK;
+    case GF_TUNE_TEST_DROP_FLAG:
+      if (value < 0) return GF_ERR_INVALID_ARG;
+      g_drop_flag.store(value);
       return GF_OK;
     case GF_TUNE_LINEAR_SPLIT:
       if (value < -1 || value > 4096) return GF_ERR_INVALID_ARG;
-      g_linear_split = value;
+      g_linear_split.store(value);
       return GF_OK;
     case GF_TUNE_LINEAR_CTAS:
       if (value < 0 || value > 65535) return GF_ERR_INVALID_ARG;
-      g_linear_ctas = value;
+      g_linear_ctas.store(value);
       return GF_OK;
     default:
       return GF_ERR_INVALID_ARG;
@@ -170,7 +197,7 @@ int gformer_set_tuning(int key, int value) {
 int gformer_linear_plan(int chains, int N, int d, int ctas, int* segments, int* chunks_per_segment) {
   if (chains < 1 || N < 1 || ctas < 0 || segments == nullptr || chunks_per_segment == nullptr) return GF_ERR_INVALID_ARG;
   if (!gf::tc_linear_supported(N, d, GF_BF16)) return GF_ERR_UNSUPPORTED;
-  gf::linear_tc_plan(chains, N, d, g_linear_split, ctas, chunks_per_segment, segments);
+  gf::linear_tc_plan(chains, N, d, g_linear_split.load(), ctas, chunks_per_segment, segments);
   return GF_OK;
 }
 
@@ -179,25 +206,34 @@ int gformer_linear_plan_parts(int chains, int N, int d, int ctas, int* whole_cha
   if (chains < 1 || N < 1 || ctas < 0 || whole_chains == nullptr || segments == nullptr || chunks_per_segment == nullptr)
     return GF_ERR_INVALID_ARG;
   if (!gf::tc_linear_supported(N, d, GF_BF16)) return GF_ERR_UNSUPPORTED;
-  gf::linear_tc_plan_parts(chains, N, d, g_linear_split, ctas, whole_chains, chunks_per_segment, segments);
+  gf::linear_tc_plan_parts(chains, N, d, g_linear_split.load(), ctas, whole_chains, chunks_per_segment, segments);
   return GF_OK;
 }
 
 size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, int dtype) {
   (void)w;
+  return workspace_bytes(tuning_now(), B, H, N, d, h_sparse, dtype);
+}
+}  // extern "C"
+
+namespace {
+size_t workspace_bytes(const Tuning& tn, int B, int H, int N, int d, int h_sparse, int dtype) {
   size_t bytes = sizeof(WsHeader);
   if (B < 1 || H < 1 || N < 1) return bytes;
   if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
   if (h_sparse > H) h_sparse = H;
   const int h_lin = H - h_sparse;
-  if (h_lin > 0 && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
+  if (h_lin > 0 && !tn.force_simt && gf::tc_linear_supported(N, d, dtype)) {
     // the causal kernel's hand-over scratch, or the bidirectional layer's segment sums: whichever is larger
-    const size_t causal = gf::linear_tc_workspace_bytes(B * h_lin, N, d, g_linear_split);
+    const size_t causal = gf::linear_tc_workspace_bytes(B * h_lin, N, d, tn.linear_split);
     const size_t self = gf::linear_self_workspace_bytes(B * h_lin, N, d);
     bytes += causal > self ? causal : self;
   }
   return bytes;
 }
+}  // namespace
+
+extern "C" {
 
 int gformer_last_device_status(void* ws, void* cuda_stream) {
   if (!ws) return GF_ERR_INVALID_ARG;
@@ -212,14 +248,15 @@ int gformer_window_attn(const void* q, const void* k, const void* v, void* o, in
                         float scale, int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
+  const Tuning tn = tuning_now();
   if (w < 1) return GF_ERR_INVALID_ARG;
-  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, H, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, H, dtype));
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  rc = clear_ws(ws, stream);
+  rc = clear_ws(tn, ws, stream);
   if (rc != GF_OK) return rc;
-  return run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream);
+  return run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream);
 }
 
 int gformer_window_attn_self(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
@@ -227,14 +264,15 @@ int gformer_window_attn_self(const void* q, const void* k, const void* v, void* 
                              void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
+  const Tuning tn = tuning_now();
   if (w < 1) return GF_ERR_INVALID_ARG;
-  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, H, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, H, dtype));
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  rc = clear_ws(ws, stream);
+  rc = clear_ws(tn, ws, stream);
   if (rc != GF_OK) return rc;
-  return run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream, true);
+  return run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, H, (WsHeader*)ws, stream, true);
 }
 
 int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
@@ -242,17 +280,18 @@ int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* 
                              size_t ws_bytes, void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
+  const Tuning tn = tuning_now();
   if (w < 1) return GF_ERR_INVALID_ARG;
   if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
   if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
   if (h_sparse > H) return GF_ERR_INVALID_ARG;
-  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, h_sparse, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, h_sparse, dtype));
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  rc = clear_ws(ws, stream);
+  rc = clear_ws(tn, ws, stream);
   if (rc != GF_OK) return rc;
-  const bool tc_linear = !g_force_simt && gf::tc_linear_supported(N, d, dtype);
+  const bool tc_linear = !tn.force_simt && gf::tc_linear_supported(N, d, dtype);
   if (h_sparse > 0 && h_sparse < H && tc_linear) {
     // Both head groups on tensor-core kernels: the three launches of the linear heads go to the
     // library's high-priority stream, the windowed heads to its side stream a few microseconds
@@ -270,12 +309,12 @@ int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* 
     if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
     int rc2 = cuda_status(gf::launch_delay(8000, f->side));
     if (rc2 == GF_OK)
-      rc2 = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, f->side, true);
+      rc2 = run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, f->side, true);
     if (cudaEventRecord(f->join, f->side) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(stream, f->join, 0) != cudaSuccess) return GF_ERR_CUDA;
     return rc != GF_OK ? rc : rc2;
   }
-  rc = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, stream, true);
+  rc = run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, stream, true);
   if (rc != GF_OK) return rc;
   if (h_sparse == H) return GF_OK;
   if (tc_linear)
@@ -291,16 +330,17 @@ int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void
                                size_t ws_bytes, void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
+  const Tuning tn = tuning_now();
   if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
   if (chunk != 0 && chunk != 128) return chunk < 0 || chunk % 64 ? GF_ERR_INVALID_ARG : GF_ERR_UNSUPPORTED;
   if ((S_io == nullptr) != (z_io == nullptr)) return GF_ERR_INVALID_ARG;
   if (S_io && (!aligned16(S_io) || !aligned16(z_io))) return GF_ERR_INVALID_ARG;
-  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, 1, 0, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, 0, dtype));
   if (rc != GF_OK) return rc;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  rc = clear_ws(ws, stream, B * H, N, d, dtype);
+  rc = clear_ws(tn, ws, stream, B * H, N, d, dtype);
   if (rc != GF_OK) return rc;
-  return run_linear(q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, 0, (WsHeader*)ws, stream);
+  return run_linear(tn, q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, 0, (WsHeader*)ws, stream);
 }
 
 int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
@@ -308,6 +348,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
                         gf_decode_state* state_out, void* ws, size_t ws_bytes, void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
+  const Tuning tn = tuning_now();
   if (w < 1) return GF_ERR_INVALID_ARG;
   if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
   if (chunk != 0 && chunk != 128) return chunk < 0 || chunk % 64 ? GF_ERR_INVALID_ARG : GF_ERR_UNSUPPORTED;
@@ -322,11 +363,11 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
       return GF_ERR_INVALID_ARG;
     if (h_lin > 0 && (!s->S || !s->z || !aligned16(s->S) || !aligned16(s->z))) return GF_ERR_INVALID_ARG;
   }
-  rc = check_ws(ws, ws_bytes, gformer_workspace_bytes(B, H, N, d, w, h_sparse, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, h_sparse, dtype));
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
-  rc = clear_ws(ws, stream, B * h_lin, N, d, dtype);
+  rc = clear_ws(tn, ws, stream, B * h_lin, N, d, dtype);
   if (rc != GF_OK) return rc;
 
   float* S_out = state_out ? state_out->S : nullptr;
@@ -338,14 +379,14 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   // linear CTAs leave at different times towards the end.
   const bool both = h_sparse > 0 && h_lin > 0;
   int lin_ctas = 0;
-  if (both && !g_force_simt && gf::tc_linear_supported(N, d, dtype)) {
+  if (both && !tn.force_simt && gf::tc_linear_supported(N, d, dtype)) {
     int L = 0, G = 0, whole = 0, dev = 0, sms = 0;
-    gf::linear_tc_plan_parts(B * h_lin, N, d, g_linear_split, 0, &whole, &L, &G, true);
+    gf::linear_tc_plan_parts(B * h_lin, N, d, tn.linear_split, 0, &whole, &L, &G, true);
     if (whole > 0) G = 1;  // items of the first launch: the chains left whole
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
       return GF_ERR_CUDA;
     if ((long long)B * h_lin * G >= sms) {
-      lin_ctas = (g_linear_ctas > 0 && g_linear_ctas < sms) ? g_linear_ctas : sms;
+      lin_ctas = (tn.linear_ctas > 0 && tn.linear_ctas < sms) ? tn.linear_ctas : sms;
     }
   }
   Fork* f = both ? get_fork() : nullptr;
@@ -362,7 +403,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   // (the caller's stream may well have the lowest, like the side stream).
   const bool lin_first = both && lin_ctas > 0;
   if (lin_first && cudaStreamWaitEvent(f->first, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
-  rc = run_linear(q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, lin_ctas,
+  rc = run_linear(tn, q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, lin_ctas,
                   (WsHeader*)ws, lin_first ? f->first : stream, both);
   if (lin_first) {
     if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
@@ -374,7 +415,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   // keeps it for many tiles: hold the side stream back for a few microseconds, until the linear
   // kernel's CTAs have been placed.
   if (lin_first && cuda_status(gf::launch_delay(8000, wstream)) != GF_OK) return GF_ERR_CUDA;
-  int rc2 = run_window(q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, wstream);
+  int rc2 = run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, wstream);
   if (rc2 == GF_OK && state_out && h_sparse > 0)
     rc2 = cuda_status(gf::launch_export_ring(k, v, state_out->k_cache, state_out->v_cache, B, N, d, w, dtype,
                                              gf::make_strides(layout, H, N, d), h_sparse, wstream));

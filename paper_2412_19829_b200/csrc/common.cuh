@@ -34,7 +34,9 @@ struct WsHeader {
   unsigned int status;   // 0 = fine, else a code written by a kernel whose bounded wait expired
   unsigned int where;    // which wait gave up (diagnostic)
   unsigned int ticket;   // work counter of the persistent kernels
-  unsigned int pad[61];
+  unsigned int wait_kcycles;  // limit of every bounded wait in units of 1024 cycles; 0 = default (about 2 s)
+  unsigned int drop_flag;     // failure injection for tests: the linear kernel skips the flag of segment n - 1
+  unsigned int pad[59];
 };
 static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
 
@@ -59,6 +61,9 @@ cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void
 cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
                                void* v_cache, float* S, float* z, long long t, long long* t_seq, int B, int H,
                                int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream);
+
+// Writes the two test knobs into a workspace header that has just been cleared.
+cudaError_t launch_set_header(WsHeader* ws, unsigned int wait_kcycles, unsigned int drop_flag, cudaStream_t stream);
 
 // One tiny CTA that returns after about `ns` nanoseconds: holds back the work queued behind it
 // in its stream without occupying an SM's shared memory or tensor memory.
@@ -95,6 +100,12 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
                              int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared = false);
 
 // ---- device helpers
+// Cycles a bounded wait may take; `status` points at the first word of the workspace header.
+__device__ __forceinline__ long long wait_limit_cycles(const unsigned int* status) {
+  const unsigned int kc = reinterpret_cast<const volatile unsigned int*>(status)[3];
+  return kc ? (long long)kc * 1024 : 4000000000LL;
+}
+
 __device__ __forceinline__ float to_f32(float x) { return x; }
 __device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
 template <typename T> __device__ __forceinline__ T from_f32(float x);

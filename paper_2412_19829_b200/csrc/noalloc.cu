@@ -54,4 +54,12 @@ int gformer_causal_linear_attn_noalloc(const void* q, const void* k, const void*
                                     cuda_stream);
 }
 
+// The status word of the fixed scratch (the workspace is hidden from the caller, so
+// gformer_last_device_status cannot be pointed at it).
+int gformer_noalloc_last_device_status(void* cuda_stream) {
+  void* ws = scratch_for_current_device();
+  if (ws == nullptr) return GF_ERR_CUDA;
+  return gformer_last_device_status(ws, cuda_stream);
+}
+
 }  // extern "C"

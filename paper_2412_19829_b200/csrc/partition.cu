@@ -61,4 +61,29 @@ int gformer_partition_heads(int B, int H, int N, int E, int W, double perf_spars
   return GF_OK;
 }
 
+// What the two micro-benchmarks say in the section's own units.  One windowed head alone costs
+// 5 B N W / perf_sparse under the model, and H linear heads together 8 B N (H E)^2 / perf_linear
+// (the printed formula is quadratic in the head count), so the rates are those expressions over
+// the measured times; the balanced head count rounds p' H to the nearest whole number.
+int gformer_partition_from_times(int B, int H, int N, int E, int W, double seconds_per_sparse_head,
+                                 double seconds_per_linear_head, double* p_out, int* h_sparse_out,
+                                 double* perf_sparse_out, double* perf_linear_out) {
+  if (p_out == nullptr || h_sparse_out == nullptr || perf_sparse_out == nullptr || perf_linear_out == nullptr)
+    return GF_ERR_INVALID_ARG;
+  if (B < 1 || H < 1 || N < 1 || E < 1 || W < 1) return GF_ERR_INVALID_ARG;
+  if (!positive_finite(seconds_per_sparse_head) || !positive_finite(seconds_per_linear_head)) return GF_ERR_INVALID_ARG;
+  double p = 0.0;
+  const int rc = gformer_partition_balance(seconds_per_sparse_head, seconds_per_linear_head, 1.0, 1.0, &p);
+  if (rc != GF_OK) return rc;
+  int h0 = (int)floor(p * (double)H + 0.5);
+  if (h0 < 0) h0 = 0;
+  if (h0 > H) h0 = H;
+  const double bn = (double)B * (double)N, he = (double)H * (double)E;
+  *p_out = p;
+  *h_sparse_out = h0;
+  *perf_sparse_out = 5.0 * bn * (double)W / seconds_per_sparse_head;
+  *perf_linear_out = 8.0 * bn * he * he / ((double)H * seconds_per_linear_head);
+  return GF_OK;
+}
+
 }  // extern "C"

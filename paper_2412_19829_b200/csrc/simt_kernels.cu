@@ -538,6 +538,17 @@ __global__ void delay_kernel(unsigned int ns) {
 }
 }  // namespace
 
+__global__ void set_header_kernel(WsHeader* ws, unsigned int wait_kcycles, unsigned int drop_flag) {
+  ws->wait_kcycles = wait_kcycles;
+  ws->drop_flag = drop_flag;
+}
+
+cudaError_t launch_set_header(WsHeader* ws, unsigned int wait_kcycles, unsigned int drop_flag, cudaStream_t stream) {
+  set_header_kernel<<<1, 1, 0, stream>>>(ws, wait_kcycles, drop_flag);
+  note_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_delay(unsigned int ns, cudaStream_t stream) {
   delay_kernel<<<1, 32, 0, stream>>>(ns);
   note_launch();

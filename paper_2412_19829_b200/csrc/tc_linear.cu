@@ -155,9 +155,9 @@ __device__ __forceinline__ bool wait_epoch(const int* counter, int target, unsig
 __device__ __forceinline__ bool wait_epoch_slow(const int* counter, int target, unsigned int* status,
                                                 unsigned int where) {
   const volatile int* c = counter;
-  const long long t0 = clock64();
+  const long long t0 = clock64(), limit = wait_limit_cycles(status);
   while (*c < target) {
-    if (clock64() - t0 > 4000000000LL) {
+    if (clock64() - t0 > limit) {
       if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
       return false;
     }
@@ -172,11 +172,11 @@ __device__ __forceinline__ bool wait_flag(const unsigned int* flag, unsigned int
   unsigned int v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
   if (v != 0u) return true;
-  const long long t0 = clock64();
+  const long long t0 = clock64(), limit = wait_limit_cycles(status);
   while (true) {
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
     if (v != 0u) return true;
-    if (clock64() - t0 > 4000000000LL) {
+    if (clock64() - t0 > limit) {
       if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
       return false;
     }
@@ -184,71 +184,6 @@ __device__ __forceinline__ bool wait_flag(const unsigned int* flag, unsigned int
   }
 }
 
-// Developer instrumentation (compiled only with -DGF_PROFILE): per-role time stamps of the first
-// chunks of CTA (0,0), read back with gformer_debug_read_profile.
-#ifdef GF_PROFILE
-__device__ unsigned long long g_prof[4][64][8];
-__device__ __forceinline__ void prof_stamp(int role, int c, int ev) {
-  if (blockIdx.x == 0 && blockIdx.y == 0 && c < 64) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    g_prof[role][c][ev] = t;
-  }
-}
-__device__ unsigned long long g_prof2[64][8];  // per CTA: hand-over time line of its first item
-__device__ __forceinline__ void prof2_stamp(int ev) {
-  if (blockIdx.x < 64) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    g_prof2[blockIdx.x][ev] = t;
-  }
-}
-__device__ unsigned long long g_prof3[160][8][8];  // per CTA, per item of that CTA: phase time line
-__device__ __forceinline__ void prof3_stamp(unsigned int n_item, int ev) {
-  if (blockIdx.x < 160 && n_item < 8) {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    g_prof3[blockIdx.x][n_item][ev] = t;
-  }
-}
-// time spent in every bounded wait, per CTA and wait site (the `where` code), first warp of each role
-__device__ unsigned long long g_wait[160][1024];
-__device__ __forceinline__ void wait_account(unsigned int where, long long t0) {
-  const int w = threadIdx.x >> 5;
-  if ((threadIdx.x & 31) == 0 && ((0x00C04047u >> w) & 1u) && blockIdx.x < 160 && where < 1024)
-    g_wait[blockIdx.x][where] += (unsigned long long)(clock64() - t0);
-}
-__device__ __forceinline__ bool prof_mbar_wait(uint64_t* b, uint32_t par, unsigned int* st, unsigned int where) {
-  const long long t0 = clock64();
-  const bool ok = mbar_wait(b, par, st, where);
-  wait_account(where, t0);
-  return ok;
-}
-__device__ __forceinline__ bool prof_wait_epoch(const int* c, int target, unsigned int* st, unsigned int where) {
-  const long long t0 = clock64();
-  const bool ok = wait_epoch(c, target, st, where);
-  wait_account(where, t0);
-  return ok;
-}
-__device__ __forceinline__ bool prof_wait_flag(const unsigned int* f, unsigned int* st, unsigned int where) {
-  const long long t0 = clock64();
-  const bool ok = wait_flag(f, st, where);
-  wait_account(where, t0);
-  return ok;
-}
-#ifdef GF_PROFILE_WAITS  // the accounting itself costs time: only when asked for
-#define mbar_wait prof_mbar_wait
-#define wait_epoch prof_wait_epoch
-#define wait_flag prof_wait_flag
-#endif
-#define PROF(role, c, ev) prof_stamp(role, c, ev)
-#define PROF2(cond, ev) do { if (cond) prof2_stamp(ev); } while (0)
-#define PROF3(n, ev) prof3_stamp(n, ev)
-#else
-#define PROF(role, c, ev)
-#define PROF2(cond, ev)
-#define PROF3(n, ev)
-#endif
 
 // Named barrier over `n` threads that also ORs a predicate, so that a timed-out wait makes the
 // whole group leave its loop together (nobody is left behind at a barrier).
@@ -322,10 +257,8 @@ __device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinI
   const long long slot = (long long)it.chain * p.G + it.g;
   bool ok = mbar_wait(&bar.a_done, a_parity, p.status, 600);
   tc_fence_after_sync();
-  PROF2(warp == 6 && lane == 0 && a_parity == 0, 0);
   // one thread of the CTA (flag warp) polls the previous segment's flag for everybody
   ok = ok && wait_epoch(prev_epoch, item_number + 1, p.status, 601);
-  PROF2(warp == 6 && lane == 0 && a_parity == 0, 1);
   if (ok) {
     uint32_t ds[W];
     if constexpr (D == 128) {
@@ -349,7 +282,6 @@ __device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinI
         in[j] = (Sin != nullptr) ? __ldcg(reinterpret_cast<const float4*>(Sin) + j * sin_stride)
                                  : make_float4(0.f, 0.f, 0.f, 0.f);
       tmem_wait_ld();
-      PROF2(warp == 6 && lane == 0 && a_parity == 0, 2);
       float* Sout = p.prefix + slot * C::kStateFloats + ((long long)(colq * (W / 4)) * 128 + r) * 4;
 #pragma unroll
       for (int j = 0; j < W / 4; ++j)
@@ -363,7 +295,6 @@ __device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinI
     // microseconds): the arrival below releases these stores at CTA scope to the store warp, whose
     // single st.release.gpu on the flag then publishes them (release is cumulative).
     tc_fence_before_sync();
-    PROF2(warp == 6 && lane == 0 && a_parity == 0, 3);
   }
   __syncwarp();
   if (ok && lane == 0) mbar_arrive(&bar.pub_done);
@@ -490,7 +421,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         const LinItem it = decode_item(p, item);
         for (int pass = kDirect ? 1 : 0; pass < 2 && ok; ++pass) {
           if (!kDirect && pass == 1 && !mbar_wait(&bar.park_done, n_items & 1, p.status, 103)) { ok = false; break; }
-          PROF3(n_items, pass);
           for (int j = 0; j < it.nC; ++j) {
             const int n0 = (it.c_begin + j) * 128;
             if (pass == 0) {
@@ -507,7 +437,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                 obs_sbi = n_items;
               }
               if (!ok) break;
-              PROF(0, ta, 1);
               mbar_arrive_expect_tx(&bar.ka_full[sa], C::kTile);
               for (int x = 0; x < D / 64; ++x)
                 tma_load_4d_hint(a_kslot(sa) + x * C::kBoxBytes, &mk, &bar.ka_full[sa], x * 64, n0, it.h, it.b,
@@ -565,7 +494,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
           const uint32_t sa = ta % KA;
           if (!mbar_wait(&bar.kphi_full[sa], (ta / KA) & 1, p.status, 220)) { ok = false; break; }
-          PROF(1, ta, 4);
           if (it.need_dS) {
             const int sv = nv % VS;
             const uint32_t kbase = smem_u32(a_kslot(sa)), vbase = smem_u32(v_box(sv, 0));
@@ -576,7 +504,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             for (int ks = 0; ks < 8; ++ks)
               umma_ss(tmem + C::tS, umma_smem_desc(kbase + ks * 2048, kLboA, 1024),
                       umma_smem_desc(vbase + ks * 2048, vlbo, 1024), id_s, (j > 0) || (ks > 0));
-            PROF(1, ta, 5);
             umma_commit(&bar.ka_free[sa]);  // second arrival: the store warp, once the tile is parked
             umma_commit(&bar.v_free[sv]);
             ++nv;
@@ -599,22 +526,18 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             ok = false;
             break;
           }
-          PROF(1, nq, 0);
-          if (j == 0) PROF3(n_items, 4);
           tc_fence_after_sync();
 #pragma unroll 2
           for (int ks = 0; ks < D / 16; ++ks)
             umma_ts(tmem + C::tP, tq + ks * 8,
                     umma_smem_desc(kbase + (ks >> 2) * C::kBoxBytes + (ks & 3) * 32, 16, 1024), id_p, ks > 0);
           umma_commit(&bar.p_full);
-          PROF(1, nq, 6);
           if (!mbar_wait(&bar.v_full[sv], (nv / VS) & 1, p.status, 202) ||
               !mbar_wait(&bar.s_loaded, n_sl & 1, p.status, 203)) {
             ok = false;
             break;
           }
           ++n_sl;
-          PROF(1, nq, 1);
           tc_fence_after_sync();
 #pragma unroll 2
           for (int ks = 0; ks < 8; ++ks)
@@ -628,7 +551,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             if (!mbar_wait(&bar.o_free, n_of & 1, p.status, 205)) { ok = false; break; }
             ++n_of;
           }
-          PROF(1, nq, 2);
           tc_fence_after_sync();
 #pragma unroll 2
           for (int ks = 0; ks < D / 16; ++ks)
@@ -639,7 +561,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           if (j == it.nC - 1) umma_commit(&bar.sb_idle);  // Sb may now take a K tile of the next pass A
           if (!mbar_wait(&bar.pm_full, n_pm & 1, p.status, 206)) { ok = false; break; }
           ++n_pm;
-          PROF(1, nq, 3);
           tc_fence_after_sync();
 #pragma unroll 2
           for (int ks = 0; ks < 8; ++ks)
@@ -647,7 +568,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                     umma_smem_desc(vbase + ks * 2048, vlbo, 1024),
                     id_o, true);
           umma_commit(&bar.o_full);
-          PROF(1, nq, 7);
           ++nv;
           ++nq;
         }
@@ -688,7 +608,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (s_row) __stcg(p.prefix + slot * C::kStateFloats + C::kStateZ + r, z0 + dz);
         __syncwarp();
         if (lane == 0) mbar_arrive(&bar.pub_done);
-        PROF2(tid == 64 && n_items == 0, 5);
       }
       // ---- hand-over of S: the 16 phi warps publish the inclusive state (they read dS from TMEM:
       //      do not overwrite it before they are done); this group loads the state before the segment
@@ -760,7 +679,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           ok = false;
           break;
         }
-        if (tid == 64) PROF(2, nq, 6);
         tc_fence_after_sync();
         uint32_t den_hi, den_lo;
         tmem_ld2(tmem + C::tOz + lane_off, den_hi, den_lo);
@@ -789,7 +707,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             mbar_arrive(&bar.o_staged[sv][cc >> 1]);
           }
         }
-        if (tid == 64) PROF(2, nq, 7);
         ++nv;
         ++nq;
       }
@@ -862,14 +779,12 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
       for (int j = 0; j < (kDirect ? 0 : it.nC); ++j) {
         const uint32_t sk = ta % KA;
         ok = ok && mbar_wait(&bar.ka_full[sk], (ta / KA) & 1, p.status, 410);
-        if (tid == 14 * 32) PROF(3, ta, 4);
         const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
         if (ok && tt < 2 * D)
           transform_k_rows(a_kslot(sk) + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
                            p.N - (it.c_begin + j) * 128);
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);  // the tile may go to the tensor core and be parked
-        if (tid == 14 * 32) PROF(3, ta, 5);
         ++ta;
       }
 
@@ -887,7 +802,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           // kDirect: this group's half of the next chunk's K tile, while the tensor core forms P
           if (kDirect && j + 1 < it.nC) transform_direct(nq + 1, j + 1);
           if (!ok || !mbar_wait(&bar.p_full, nq & 1, p.status, 301)) { ok = false; break; }
-          if (tt == 0) PROF(2, nq, 0);
           tc_fence_after_sync();
 #pragma unroll 1
           for (int e = 0; e < 2; ++e) {
@@ -917,7 +831,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           tmem_wait_st();
           tc_fence_before_sync();
           mbar_arrive(&bar.pm_full);
-          if (tt == 0) PROF(2, nq, 1);
           // ---- S: the fp32 master stays in TMEM; once this chunk's readout has consumed the old
           //      bf16 copy, stream the new one (and z) into shared memory for the next chunk.
           //      This warp: rows [32 q, 32 q + 32) x columns [colh D/2, colh D/2 + D/2).
@@ -925,7 +838,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             ok = false;
             break;
           }
-          if (tt == 0) PROF(2, nq, 2);
           tc_fence_after_sync();
           {
             // after the item's last chunk nobody reads Sb again (it may already hold a K tile of the
@@ -978,7 +890,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             fence_proxy_async_smem();
             mbar_arrive(&bar.sb_full);
             if (last_chunk) mbar_arrive(&bar.s_final);
-            if (tt == 0) PROF(2, nq, 5);
           }
           ++nq;
         }
@@ -991,7 +902,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           const int sq = nq % QS;
           const int ql = nq % QL;  // landing buffer of this chunk's tile
           ok = mbar_wait(&bar.q_full[ql], (nq / QL) & 1, p.status, 400);
-          if (tid == 192) PROF(3, nq, 0);
           if (ok) {
             // copy the raw row half out of the landing buffer; the last warp to have done so
             // starts the load of the tile that takes the buffer next (a later chunk's, or one of
@@ -1049,7 +959,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
             for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
             if (nq >= QS)  // MMA1/MMA2 of the slot's previous chunk are done with it
               ok = mbar_wait(&bar.qphi_free[sq], ((nq / QS) + 1) & 1, p.status, 401);
-            if (tid == 192) PROF(3, nq, 1);
             tc_fence_after_sync();
             if (ok) {
               if constexpr (D == 128) {
@@ -1064,7 +973,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               if (lane == 0) mbar_arrive(&bar.qphi_full[sq]);
             }
           }
-          if (tid == 192) PROF(3, nq, 2);
           if (kDirect && ok && j + 1 < it.nC) transform_direct(nq + 1, j + 1);
           ok = !__any_sync(0xffffffffu, !ok);
           ++nq;
@@ -1092,7 +1000,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                               pol_keep);
           tma_store_commit();
           tma_store_wait_read<0>();
-          PROF(0, ta, 3);
           mbar_arrive(&bar.ka_free[sk]);
           ++ta;
         }
@@ -1115,11 +1022,9 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
           mbar_arrive(&bar.v_free[sv]);  // the staging buffer may take the V tile two uses later
           ++nv;
         }
-        PROF3(n_items, 5);
         ++n_items;
       }
       tma_store_wait_all<0>();
-      PROF2(true, 7);
     }
   } else {
     // ================================================================ flag warp
@@ -1133,15 +1038,14 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         if (it.g > 0 && !wait_flag(p.flags + (slot - 1) * kFlagStride, p.status, 511)) break;
         __threadfence_block();
         *reinterpret_cast<volatile int*>(&prev_epoch) = n_items + 1;
-        PROF3(n_items, 2);
         if (it.need_dS) {
           // every warp of the hand-over has written its part of the inclusive state
           if (!mbar_wait(&bar.pub_done, n_a & 1, p.status, 510)) break;
-          PROF2(n_a == 0, 4);
           ++n_a;
           const unsigned int one = 1u;
-          asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.flags + slot * kFlagStride), "r"(one) : "memory");
-          PROF3(n_items, 3);
+          // (status[4]: failure injection for tests -- that segment's flag is never raised)
+          if (reinterpret_cast<const volatile unsigned int*>(p.status)[4] != (unsigned int)slot + 1u)
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.flags + slot * kFlagStride), "r"(one) : "memory");
         }
       }
     }
@@ -1153,24 +1057,6 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
 
 }  // namespace
 
-#ifdef GF_PROFILE
-extern "C" int gformer_debug_read_profile2(unsigned long long* host_dst) {
-  return (int)cudaMemcpyFromSymbol(host_dst, g_prof2, sizeof(g_prof2));
-}
-extern "C" int gformer_debug_read_waits(unsigned long long* host_dst) {
-  return (int)cudaMemcpyFromSymbol(host_dst, g_wait, sizeof(g_wait));
-}
-extern "C" int gformer_debug_reset_waits() {
-  static unsigned long long zeros[160 * 1024];
-  return (int)cudaMemcpyToSymbol(g_wait, zeros, sizeof(g_wait));
-}
-extern "C" int gformer_debug_read_profile3(unsigned long long* host_dst) {
-  return (int)cudaMemcpyFromSymbol(host_dst, g_prof3, sizeof(g_prof3));
-}
-extern "C" int gformer_debug_read_profile(unsigned long long* host_dst) {
-  return (int)cudaMemcpyFromSymbol(host_dst, g_prof, sizeof(g_prof));
-}
-#endif
 
 bool tc_linear_supported(int N, int d, int dtype) {
   (void)N;

@@ -103,9 +103,9 @@ __device__ __forceinline__ bool win_wait_epoch(const int* counter, int target, u
                                                unsigned int where) {
   const volatile int* c = counter;
   if (*c >= target) { __threadfence_block(); return true; }
-  const long long t0 = clock64();
+  const long long t0 = clock64(), limit = wait_limit_cycles(status);
   while (*c < target) {
-    if (clock64() - t0 > 4000000000LL) {
+    if (clock64() - t0 > limit) {
       if (atomicCAS(status, 0u, 1u) == 0u) status[1] = where;
       return false;
     }
@@ -344,9 +344,9 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
                 const int half = j & 1;
                 if (t == 1) {  // bounded: stream 0's next S must lie behind this half tile
                   if (*front <= n) {
-                    const long long t0 = clock64();
+                    const long long t0 = clock64(), limit = wait_limit_cycles(p.status);
                     while (*front <= n) {
-                      if (clock64() - t0 > 4000000000LL) {
+                      if (clock64() - t0 > limit) {
                         if (atomicCAS(p.status, 0u, 1u) == 0u) p.status[1] = 26;
                         return;
                       }

@@ -17,10 +17,24 @@ Inputs are seeded Gaussians generated on the device (timing only)."""
 import argparse
 import json
 
+import numpy as np
 import torch
 
 from . import binding as gf
-from .sweep import time_call
+
+
+def time_call(fn, iters, warm=3):
+    """Median microseconds of `iters` calls (CUDA events on the current stream, after `warm` calls)."""
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    evs[0].record()
+    for i in range(iters):
+        fn()
+        evs[i + 1].record()
+    torch.cuda.synchronize()
+    return float(np.median([evs[i].elapsed_time(evs[i + 1]) * 1e3 for i in range(iters)]))
 
 
 def measure(B, H, N, d, w, self_layer=False, iters=5, seed=0):
@@ -39,11 +53,8 @@ def measure(B, H, N, d, w, self_layer=False, iters=5, seed=0):
 
     t_window = layer_us(H) * 1e-6 / H  # every head windowed
     t_linear = layer_us(0) * 1e-6 / H  # every head linear
-    p = gf.partition_balance(t_window, t_linear, 1.0, 1.0)
-    h0 = min(H, max(0, round(p * H)))
-    # the section's FLOP model with the rates the two micro-benchmarks achieved under it
-    perf_sparse = 5.0 * B * N * w / t_window
-    perf_linear = 8.0 * B * N * float(H * d) ** 2 / (H * t_linear)  # the model is quadratic in the linear head count
+    # Algorithm 2 on the measured times, and the section's FLOP model with the rates they imply
+    p, h0, perf_sparse, perf_linear = gf.partition_from_times(B, H, N, d, w, t_window, t_linear)
     h0_model, lat_s, lat_l = gf.partition_heads(B, H, N, d, w, perf_sparse, perf_linear)
     return {"B": B, "H": H, "N": N, "d": d, "w": w, "layer": "self" if self_layer else "causal",
             "s_per_window_head": t_window, "s_per_linear_head": t_linear, "p_balanced": p, "h_sparse_balanced": h0,

@@ -312,3 +312,22 @@ def test_self_layer_argument_errors():
     for chains, N, d in ((1, 128, 64), (26, 32768, 128), (832, 4096, 64), (3, 100000, 128)):
         ws = gf.workspace_bytes(1, chains, N, d, 1, 0, gf.GF_BF16)
         assert ws >= 256 + chains * 2 * (d * d + d) * 4  # at least one segment slot per chain plus the totals
+
+
+def test_partition_from_times_against_the_oracle():
+    # seconds per head of either kind in, Algorithm 2's share and the section's rates out
+    from oracle import partition as op
+
+    B, H, N, E, W = 2, 16, 4096, 64, 128
+    tw, tl = 3.0e-6, 1.0e-6
+    p, h0, ps, pl = gf.partition_from_times(B, H, N, E, W, tw, tl)
+    assert p == pytest.approx(op.balance(1.0, tw, tl, 1.0, 1.0), abs=1e-12)
+    assert h0 == 4  # p' = 1/4 of 16 heads
+    # the rates are the model's work for what was timed over the measured times: with them the model
+    # gives back the measurements (one windowed head alone; all H heads linear)
+    s1, _ = op.model_latencies(B, H, N, E, W, 1, ps, pl)
+    _, lall = op.model_latencies(B, H, N, E, W, 0, ps, pl)
+    assert s1 == pytest.approx(tw, rel=1e-12) and lall == pytest.approx(H * tl, rel=1e-12)
+    for bad in ((0, H, N, E, W, tw, tl), (B, H, N, E, W, 0.0, tl), (B, H, N, E, W, tw, float("inf"))):
+        with pytest.raises(gf.GformerError):
+            gf.partition_from_times(*bad)

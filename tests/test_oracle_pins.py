@@ -318,7 +318,7 @@ def test_prefill_export_then_decode_equals_one_long_sequence(N0, w):
 
 
 # ----------------------------------------------------------------------------- "self" (bidirectional) layer
-# The next row of the scope table has its oracle first; these pins are what fixes it.
+# The bidirectional layer's oracle functions and what fixes them.
 def test_self_window_covering_the_sequence_is_library_softmax_attention():
     q, k, v = rnd((2, 2, 37, 16), 501), rnd((2, 2, 37, 16), 502), rnd((2, 2, 37, 16), 503)
     for w in (37, 38, 500):  # |i - j| < w holds for every pair: plain Eq. 1, no mask

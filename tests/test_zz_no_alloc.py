@@ -1,4 +1,4 @@
-"""The allocation-free entry point against the regular one (collected last on purpose).
+"""The allocation-free entry point against the oracle and the regular one (collected last on purpose).
 
 Callers that may not allocate device memory (a plug-in inside a framework's memory pool, a
 real-time or capture-time path) use gformer_causal_linear_attn_noalloc, whose scratch is a fixed
@@ -8,7 +8,8 @@ although every call reuses the same scratch with the previous call's leftovers i
 import pytest
 import torch
 
-from gates import assert_parity
+import oracle
+from gates import assert_parity, errors
 from paper_2412_19829_b200 import binding as gf
 from paper_2412_19829_b200 import synth
 
@@ -32,6 +33,15 @@ def test_noalloc_matches_regular_entry_point_twice_in_a_row():
         got = gf.causal_linear_attn_noalloc(q, k, v, out, S, z)
         torch.cuda.synchronize()
         f64 = lambda t: t.cpu().to(torch.float64).numpy()
+        assert gf.lib().gformer_noalloc_last_device_status(None) == gf.GF_OK
+        # the answer itself: the fp64 oracle on the same rounded inputs (output and final state)
+        import numpy as np
+        S_want, z_want = np.zeros((B, H, d, d)), np.zeros((B, H, d))
+        want = oracle.causal_linear_attn(f64(q), f64(k), f64(v), S_want, z_want)  # leaves the final state in S_want, z_want
+        assert_parity(f64(got), want, "bf16", f"no-alloc call {call} against the oracle")
+        # (the state sums thousands of terms: the relative gate applies to it)
+        assert errors(f64(S), S_want)["rel_l2"] <= 1e-2 and errors(f64(z), z_want)["rel_l2"] <= 1e-2
+        # and the regular entry point, which uses a caller-owned workspace
         assert_parity(f64(got), f64(ref), "bf16", f"no-alloc call {call}")
         assert_parity(f64(S), f64(S_ref), "bf16", f"no-alloc state S, call {call}")
         assert_parity(f64(z), f64(z_ref), "bf16", f"no-alloc state z, call {call}")
