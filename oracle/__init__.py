@@ -69,6 +69,29 @@ def phi(x):
     return y
 
 
+def phi_favor(x, W):
+    """Positive random features of the vectors x [..., d] under the projection W [d, d] (rows w_a):
+    exp(<w_a, x> - |x|^2 / 2) / sqrt(d)  (Sec. III-A / III-C; the formula is the cited Performer paper's)."""
+    x, W = _f64(x), _f64(W)
+    d = x.shape[-1]
+    assert W.shape == (d, d)
+    y = np.empty_like(x)
+    xs, ys = x.reshape(-1, d), y.reshape(-1, d)
+    lib = _load()
+    for i in range(xs.shape[0]):
+        lib.gfo_phi_favor(_p(xs[i]), _p(W), ctypes.c_int(d), _p(ys[i]))
+    return y
+
+
+def _proj(W, heads, d):
+    """W [heads, d, d] (float64, contiguous) or None: the projection of the linear heads' feature map."""
+    if W is None:
+        return None
+    W = _f64(W)
+    assert W.shape == (heads, d, d), (W.shape, (heads, d, d))
+    return W
+
+
 def default_scale(d: int) -> float:
     """Eq. 1 divides the logits by sqrt(D)."""
     return 1.0 / float(np.sqrt(float(d)))
@@ -90,9 +113,10 @@ def window_attn(q, k, v, w: int, scale: float | None = None):
     return o
 
 
-def causal_linear_attn(q, k, v, S=None, z=None):
+def causal_linear_attn(q, k, v, S=None, z=None, W=None):
     """Returns o; if S [B,H,d,d] / z [B,H,d] are given they are the initial state and are
-    overwritten in place with the final state."""
+    overwritten in place with the final state.  W [H, d, d]: positive random features under these
+    projections instead of elu + 1."""
     q, k, v = _f64(q), _f64(k), _f64(v)
     B, H, N, d = q.shape
     o = np.empty_like(q)
@@ -101,11 +125,11 @@ def causal_linear_attn(q, k, v, S=None, z=None):
     if S is not None:
         assert S.shape == (B, H, d, d) and z.shape == (B, H, d)
     _load().gfo_causal_linear_attn(_p(q), _p(k), _p(v), _p(o), ctypes.c_long(B), ctypes.c_long(H),
-                                   ctypes.c_long(N), ctypes.c_int(d), _p(S), _p(z))
+                                   ctypes.c_long(N), ctypes.c_int(d), _p(S), _p(z), _p(_proj(W, H, d)))
     return o
 
 
-def hybrid_attn_self(q, k, v, w: int, h_sparse: int | None = None, scale: float | None = None):
+def hybrid_attn_self(q, k, v, w: int, h_sparse: int | None = None, scale: float | None = None, W=None):
     """The bidirectional ("self") layer: heads [0, h_sparse) see the keys with |i - j| < w,
     the others run global linear attention phi(Q)(phi(K)^T V) with row normalisation."""
     q, k, v = _f64(q), _f64(k), _f64(v)
@@ -115,7 +139,8 @@ def hybrid_attn_self(q, k, v, w: int, h_sparse: int | None = None, scale: float 
     s = default_scale(d) if scale is None else float(scale)
     o = np.empty_like(q)
     _load().gfo_hybrid_attn_self(_p(q), _p(k), _p(v), _p(o), ctypes.c_long(B), ctypes.c_long(H), ctypes.c_long(N),
-                                 ctypes.c_int(d), ctypes.c_long(w), ctypes.c_long(h0), ctypes.c_double(s))
+                                 ctypes.c_int(d), ctypes.c_long(w), ctypes.c_long(h0), ctypes.c_double(s),
+                                 _p(_proj(W, H - h0, d)))
     return o
 
 
@@ -123,8 +148,8 @@ def window_attn_self(q, k, v, w: int, scale: float | None = None):
     return hybrid_attn_self(q, k, v, w, h_sparse=np.asarray(q).shape[1], scale=scale)
 
 
-def linear_attn_self(q, k, v):
-    return hybrid_attn_self(q, k, v, 1, h_sparse=0)
+def linear_attn_self(q, k, v, W=None):
+    return hybrid_attn_self(q, k, v, 1, h_sparse=0, W=W)
 
 
 class DecodeState:
@@ -138,10 +163,11 @@ class DecodeState:
         self.S = np.zeros((B, H1, d, d))
         self.z = np.zeros((B, H1, d))
         self.t = 0
+        self.W = None  # [H1, d, d]: projections of the positive random features, None: elu + 1
 
 
 def hybrid_attn(q, k, v, w: int, h_sparse: int | None = None, scale: float | None = None,
-                export_state: bool = False):
+                export_state: bool = False, W=None):
     q, k, v = _f64(q), _f64(k), _f64(v)
     B, H, N, d = q.shape
     h0 = default_h_sparse(H) if h_sparse is None else int(h_sparse)
@@ -153,9 +179,10 @@ def hybrid_attn(q, k, v, w: int, h_sparse: int | None = None, scale: float | Non
         _p(q), _p(k), _p(v), _p(o), ctypes.c_long(B), ctypes.c_long(H), ctypes.c_long(N),
         ctypes.c_int(d), ctypes.c_long(w), ctypes.c_long(h0), ctypes.c_double(s),
         _p(st.k_cache if st else None), _p(st.v_cache if st else None),
-        _p(st.S if st else None), _p(st.z if st else None))
+        _p(st.S if st else None), _p(st.z if st else None), _p(_proj(W, H - h0, d)))
     if st is not None:
         st.t = N
+        st.W = _proj(W, H - h0, d)
         return o, st
     return o
 
@@ -169,6 +196,6 @@ def decode_step(q, k, v, st: DecodeState, scale: float | None = None):
     _load().gfo_decode_step(
         _p(q), _p(k), _p(v), _p(o), _p(st.k_cache), _p(st.v_cache), _p(st.S), _p(st.z),
         ctypes.c_long(st.t), ctypes.c_long(B), ctypes.c_long(H), ctypes.c_int(d),
-        ctypes.c_long(st.w), ctypes.c_long(st.h_sparse), ctypes.c_double(s))
+        ctypes.c_long(st.w), ctypes.c_long(st.h_sparse), ctypes.c_double(s), _p(_proj(st.W, H - st.h_sparse, d)))
     st.t += 1
     return o

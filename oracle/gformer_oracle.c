@@ -19,7 +19,16 @@
  *                 Z += phi(K_i), readout H_i = phi(Q_i)^T A / (phi(Q_i) . Z) taken
  *                 AFTER the two updates of step i (inclusive prefix).  The readout
  *                 line is garbled in print; this is the repaired reading.
- *   phi           Sec. II-B: phi(x) = elu(x) + 1.
+ *   phi           Sec. II-B: phi(x) = elu(x) + 1 (element by element).
+ *   phi_W         Sec. III-A / III-C name "positive orthogonal random features" as the feature map of
+ *                 the linear heads without printing a formula; the formula is the cited Performer
+ *                 paper's positive random feature map of the softmax kernel,
+ *                     phi_W(x)[a] = exp(<w_a, x> - |x|^2 / 2) / sqrt(m),   a = 0 .. m-1,
+ *                 with a caller-supplied projection W = (w_a) per head.  m = d, because the state of
+ *                 Algorithm 1 is E x E.  No stabiliser is subtracted and no extra scale is applied
+ *                 to x (the linear heads carry no 1/sqrt(D), reading P3): what the caller passes
+ *                 is what is projected.  Whether the rows of W are orthogonal is the caller's
+ *                 business (a property of the input, generated outside this file).
  *   hybrid        Sec. III-A: heads are split along H; the first h_sparse heads are
  *                 windowed, the rest linear; every head writes its own slot of O.
  *   decode        Algorithm 1 advanced one token at a time plus the window rule on a
@@ -59,6 +68,24 @@ void gfo_phi_array(const double* x, double* y, long n) {
   for (long i = 0; i < n; ++i) y[i] = gfo_phi(x[i]);
 }
 
+/* The positive random feature map of one vector: out[a] = exp(<W[a], x> - |x|^2 / 2) / sqrt(d),
+ * W is d x d row-major (row a = projection vector w_a). */
+void gfo_phi_favor(const double* x, const double* W, int d, double* out) {
+  double n2 = 0.0;
+  for (int c = 0; c < d; ++c) n2 += x[c] * x[c];
+  for (int a = 0; a < d; ++a) {
+    double proj = 0.0;
+    for (int c = 0; c < d; ++c) proj += W[(size_t)a * d + c] * x[c];
+    out[a] = exp(proj - 0.5 * n2) / sqrt((double)d);
+  }
+}
+
+/* Feature map of the linear heads: elu + 1 element by element (W == NULL), or phi_W. */
+static void feature_map(const double* x, const double* W, int d, double* out) {
+  if (W) gfo_phi_favor(x, W, d, out);
+  else for (int a = 0; a < d; ++a) out[a] = gfo_phi(x[a]);
+}
+
 /* One windowed head: q, k, v, o are N x d. */
 static void window_head(const double* q, const double* k, const double* v, double* o,
                         long N, int d, long w, double scale, double* e /* >= min(w,N) */) {
@@ -93,12 +120,10 @@ static void window_head(const double* q, const double* k, const double* v, doubl
  * phi(k), c = value index), z is d.  Both are read as the initial state and left
  * holding the final state. */
 static void linear_head(const double* q, const double* k, const double* v, double* o,
-                        long N, int d, double* S, double* z, double* qp, double* kp) {
+                        long N, int d, double* S, double* z, double* qp, double* kp, const double* W) {
   for (long i = 0; i < N; ++i) {
-    for (int a = 0; a < d; ++a) {
-      qp[a] = gfo_phi(q[i * d + a]);
-      kp[a] = gfo_phi(k[i * d + a]);
-    }
+    feature_map(q + i * d, W, d, qp);
+    feature_map(k + i * d, W, d, kp);
     for (int a = 0; a < d; ++a) {
       for (int c = 0; c < d; ++c) S[a * d + c] += kp[a] * v[i * d + c];
       z[a] += kp[a];
@@ -144,21 +169,20 @@ static void window_head_sym(const double* q, const double* k, const double* v, d
 /* One global (unmasked) linear head, Sec. II-B: S = sum_j phi(K_j) (x) V_j and z = sum_j
  * phi(K_j) over the whole sequence first, then H_i = phi(Q_i)^T S / (phi(Q_i) . z). */
 static void linear_head_global(const double* q, const double* k, const double* v, double* o,
-                               long N, int d, double* S, double* z, double* qp) {
+                               long N, int d, double* S, double* z, double* qp, const double* W) {
   memset(S, 0, sizeof(double) * (size_t)d * (size_t)d);
   memset(z, 0, sizeof(double) * (size_t)d);
-  for (long j = 0; j < N; ++j)
+  for (long j = 0; j < N; ++j) {
+    feature_map(k + j * d, W, d, qp);
     for (int a = 0; a < d; ++a) {
-      double kp = gfo_phi(k[j * d + a]);
-      for (int c = 0; c < d; ++c) S[a * d + c] += kp * v[j * d + c];
-      z[a] += kp;
+      for (int c = 0; c < d; ++c) S[a * d + c] += qp[a] * v[j * d + c];
+      z[a] += qp[a];
     }
+  }
   for (long i = 0; i < N; ++i) {
     double den = 0.0;
-    for (int a = 0; a < d; ++a) {
-      qp[a] = gfo_phi(q[i * d + a]);
-      den += qp[a] * z[a];
-    }
+    feature_map(q + i * d, W, d, qp);
+    for (int a = 0; a < d; ++a) den += qp[a] * z[a];
     for (int c = 0; c < d; ++c) {
       double num = 0.0;
       for (int a = 0; a < d; ++a) num += qp[a] * S[a * d + c];
@@ -170,7 +194,8 @@ static void linear_head_global(const double* q, const double* k, const double* v
 /* The "self" hybrid layer: heads [0, h_sparse) two-sided windowed, heads [h_sparse, H) global
  * linear (Sec. III-A routing, unchanged). */
 void gfo_hybrid_attn_self(const double* q, const double* k, const double* v, double* o,
-                          long B, long H, long N, int d, long w, long h_sparse, double scale) {
+                          long B, long H, long N, int d, long w, long h_sparse, double scale,
+                          const double* W /* [H - h_sparse, d, d] or NULL: elu + 1 */) {
   long span = 2 * w - 1 < N ? 2 * w - 1 : N;
 #pragma omp parallel
   {
@@ -180,7 +205,8 @@ void gfo_hybrid_attn_self(const double* q, const double* k, const double* v, dou
     for (long bh = 0; bh < B * H; ++bh) {
       size_t off = (size_t)bh * (size_t)N * (size_t)d;
       if (bh % H < h_sparse) window_head_sym(q + off, k + off, v + off, o + off, N, d, w, scale, e);
-      else linear_head_global(q + off, k + off, v + off, o + off, N, d, S, S + (size_t)d * d, S + (size_t)d * d + d);
+      else linear_head_global(q + off, k + off, v + off, o + off, N, d, S, S + (size_t)d * d, S + (size_t)d * d + d,
+                              W ? W + (size_t)(bh % H - h_sparse) * d * d : NULL);
     }
     free(e);
     free(S);
@@ -206,7 +232,8 @@ void gfo_window_attn(const double* q, const double* k, const double* v, double* 
 /* Causal linear attention on all B*H heads.  S_io [B,H,d,d] and z_io [B,H,d] may be
  * NULL (fresh zero state, final state discarded). */
 void gfo_causal_linear_attn(const double* q, const double* k, const double* v, double* o,
-                            long B, long H, long N, int d, double* S_io, double* z_io) {
+                            long B, long H, long N, int d, double* S_io, double* z_io,
+                            const double* W /* [H, d, d] or NULL: elu + 1 */) {
 #pragma omp parallel
   {
     double* S = (double*)malloc(sizeof(double) * (size_t)d * (size_t)d);
@@ -218,7 +245,8 @@ void gfo_causal_linear_attn(const double* q, const double* k, const double* v, d
       else memset(S, 0, sizeof(double) * (size_t)d * d);
       if (z_io) memcpy(z, z_io + (size_t)bh * d, sizeof(double) * (size_t)d);
       else memset(z, 0, sizeof(double) * (size_t)d);
-      linear_head(q + off, k + off, v + off, o + off, N, d, S, z, z + d, z + 2 * d);
+      linear_head(q + off, k + off, v + off, o + off, N, d, S, z, z + d, z + 2 * d,
+                  W ? W + (size_t)(bh % H) * d * d : NULL);
       if (S_io) memcpy(S_io + (size_t)bh * d * d, S, sizeof(double) * (size_t)d * d);
       if (z_io) memcpy(z_io + (size_t)bh * d, z, sizeof(double) * (size_t)d);
     }
@@ -234,7 +262,8 @@ void gfo_causal_linear_attn(const double* q, const double* k, const double* v, d
  *   S_out [B, H - h_sparse, d, d], z_out [B, H - h_sparse, d]: final linear state. */
 void gfo_hybrid_attn(const double* q, const double* k, const double* v, double* o,
                      long B, long H, long N, int d, long w, long h_sparse, double scale,
-                     double* k_cache, double* v_cache, double* S_out, double* z_out) {
+                     double* k_cache, double* v_cache, double* S_out, double* z_out,
+                     const double* W /* [H - h_sparse, d, d] or NULL: elu + 1 */) {
   long H1 = H - h_sparse;
   long wn = w < N ? w : N;
 #pragma omp parallel
@@ -259,7 +288,8 @@ void gfo_hybrid_attn(const double* q, const double* k, const double* v, double* 
       } else {
         memset(S, 0, sizeof(double) * (size_t)d * d);
         memset(z, 0, sizeof(double) * (size_t)d);
-        linear_head(q + off, k + off, v + off, o + off, N, d, S, z, z + d, z + 2 * d);
+        linear_head(q + off, k + off, v + off, o + off, N, d, S, z, z + d, z + 2 * d,
+                    W ? W + (size_t)(h - h_sparse) * d * d : NULL);
         size_t soff = (size_t)b * H1 + (h - h_sparse);
         if (S_out) memcpy(S_out + soff * d * d, S, sizeof(double) * (size_t)d * d);
         if (z_out) memcpy(z_out + soff * d, z, sizeof(double) * (size_t)d);
@@ -277,7 +307,8 @@ void gfo_hybrid_attn(const double* q, const double* k, const double* v, double* 
  * Algorithm 1 on the carried (S, z). */
 void gfo_decode_step(const double* q, const double* k, const double* v, double* o,
                      double* k_cache, double* v_cache, double* S, double* z, long t,
-                     long B, long H, int d, long w, long h_sparse, double scale) {
+                     long B, long H, int d, long w, long h_sparse, double scale,
+                     const double* W /* [H - h_sparse, d, d] or NULL: elu + 1 */) {
   long H1 = H - h_sparse;
 #pragma omp parallel
   {
@@ -318,7 +349,8 @@ void gfo_decode_step(const double* q, const double* k, const double* v, double* 
         }
       } else {
         size_t soff = (size_t)b * H1 + (h - h_sparse);
-        linear_head(qi, ki, vi, oi, 1, d, S + soff * d * d, z + soff * d, qp, qp + d);
+        linear_head(qi, ki, vi, oi, 1, d, S + soff * d * d, z + soff * d, qp, qp + d,
+                    W ? W + (size_t)(h - h_sparse) * d * d : NULL);
       }
     }
     free(e);

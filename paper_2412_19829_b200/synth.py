@@ -65,3 +65,24 @@ def decode_tokens(steps, B, H, d, dtype="bf16", seed=0, gain=None):
         x = torch.randn(steps, B, H, d, generator=g, dtype=torch.float32) * gain
         out.append(x.to(torch_dtype(dtype)))
     return tuple(out)
+
+
+def favor_projection(heads, d, seed=0, orthogonal=True, dtype="f32"):
+    """Projection matrices W [heads, d, d] of the positive random feature map (rows = projection
+    vectors): i.i.d. N(0,1) entries drawn from a CPU generator; with orthogonal=True the rows of
+    every matrix are made orthogonal (QR of the Gaussian matrix) and given back the norms of
+    independent Gaussian vectors, so that each row is still N(0, I) on its own.  Rounded to `dtype`.
+    This is the random draw of the method, handed to it as an input."""
+    g = torch.Generator(device="cpu").manual_seed(int(seed) + 104729)
+    out = []
+    for _ in range(heads):
+        G = torch.randn(d, d, generator=g, dtype=torch.float64)
+        if orthogonal:
+            Q, _ = torch.linalg.qr(G.T)            # columns orthonormal -> rows of Q.T orthonormal
+            norms = torch.randn(d, d, generator=g, dtype=torch.float64).norm(dim=1)
+            # the factorisation fixes the signs of its columns: random signs make every row a
+            # direction uniform on the sphere again
+            signs = torch.where(torch.rand(d, generator=g, dtype=torch.float64) < 0.5, -1.0, 1.0)
+            G = Q.T * (norms * signs)[:, None]
+        out.append(G)
+    return torch.stack(out).to(torch.float32).to(torch_dtype(dtype))

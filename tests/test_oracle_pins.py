@@ -456,3 +456,113 @@ def test_partition_printed_example_is_not_what_the_printed_model_gives():
 
     counts = [op.partition_heads(1, 16, 4096, 64, W, 2.31e12, 13.37e12) for W in (16, 32, 64, 128, 256, 512, 1024)]
     assert counts == [16, 16, 15, 15, 14, 14, 13]
+
+
+# ----------------------------------------------------------------------------- positive random features
+# (Sec. III-A / III-C: the feature map the linear heads use; formula of the cited Performer paper)
+def _num(x):
+    if isinstance(x, str):
+        return {"0.5+ln2": 0.5 + math.log(2.0), "0.5+ln3": 0.5 + math.log(3.0)}[x]
+    return float(x)
+
+
+def _favor_golden():
+    with open(os.path.join(HERE, "golden", "hand_worked.json")) as f:
+        g = json.load(f)["favor"]
+    W = np.array([[[_num(x) for x in row] for row in m] for m in g["W"]])
+    return g, W
+
+
+def test_favor_features_hand_worked():
+    g, W = _favor_golden()
+    got = oracle.phi_favor(np.array(g["x"]), W[0]) * math.sqrt(2.0)
+    np.testing.assert_allclose(got, np.array(g["phi_times_sqrt2"]), rtol=1e-14)
+
+
+def test_favor_linear_attention_hand_worked():
+    g, W = _favor_golden()
+    k, v = np.array(g["k"])[None, None], np.array(g["v"])[None, None]
+    for q, want in ((g["q_a"], g["expected_a"]), (g["q_b"], g["expected_b"])):
+        S, z = np.zeros((1, 1, 2, 2)), np.zeros((1, 1, 2))
+        o = oracle.causal_linear_attn(np.array(q)[None, None], k, v, S, z, W=W)
+        np.testing.assert_allclose(o[0, 0], np.array(want), rtol=1e-13)
+        np.testing.assert_allclose(S[0, 0] * math.sqrt(2.0), np.array(g["expected_S_times_sqrt2"]), rtol=1e-13)
+        np.testing.assert_allclose(z[0, 0] * math.sqrt(2.0), np.array(g["expected_z_times_sqrt2"]), rtol=1e-13)
+
+
+def test_favor_features_are_positive_and_fall_with_the_norm():
+    W = rnd((8, 8), 601)
+    x = rnd((50, 8), 602, 2.0)
+    f = oracle.phi_favor(x, W)
+    assert (f > 0).all()
+    # a vector orthogonal to every projection direction only sees the -|x|^2/2 term: with W = 0 the
+    # features are the Gaussian exp(-|x|^2/2)/sqrt(d), the same in every coordinate
+    f0 = oracle.phi_favor(x, np.zeros((8, 8)))
+    np.testing.assert_allclose(f0, np.repeat(np.exp(-0.5 * (x ** 2).sum(1, keepdims=True)) / math.sqrt(8.0), 8, 1), rtol=1e-13)
+
+
+@pytest.mark.parametrize("orthogonal", [False, True])
+def test_favor_features_estimate_the_softmax_kernel(orthogonal):
+    # E_W[ phi_W(q) . phi_W(k) ] = exp(q . k) for Gaussian projection rows (each row on its own is N(0, I)
+    # also in the orthogonal draw): the mean over many independent draws converges to the kernel.
+    from paper_2412_19829_b200 import synth  # input generators only: no attention arithmetic in there
+
+    d, draws = 4, 6000
+    q, k = rnd((3, d), 611, 0.5), rnd((3, d), 612, 0.5)
+    Ws = synth.favor_projection(draws, d, seed=613, orthogonal=orthogonal).double().numpy()
+    est = np.zeros((3, 3))
+    for W in Ws:
+        est += oracle.phi_favor(q, W) @ oracle.phi_favor(k, W).T
+    est /= draws
+    want = np.exp(q @ k.T)
+    # Monte-Carlo: relative standard error of the mean is a few per cent per draw^(1/2) ~ 1.3 %; five sigma
+    np.testing.assert_allclose(est, want, rtol=0.08)
+    if orthogonal:  # the draw really is orthogonal, with Gaussian-like row norms
+        G = Ws[0] @ Ws[0].T
+        assert np.abs(G - np.diag(np.diag(G))).max() < 1e-5 * np.diag(G).max()
+
+
+def test_favor_with_zero_projection_weights_keys_by_their_gaussian():
+    # W = 0: phi(k_j) = exp(-|k_j|^2/2)/sqrt(d) in every coordinate, so row i is the mean of v_0..v_i
+    # weighted by exp(-|k_j|^2/2); keys of equal norm give the plain cumulative mean
+    B, H, N, d = 1, 2, 9, 4
+    q, k, v = rnd((B, H, N, d), 621), rnd((B, H, N, d), 622), rnd((B, H, N, d), 623)
+    W0 = np.zeros((H, d, d))
+    o = oracle.causal_linear_attn(q, k, v, W=W0)
+    wts = np.exp(-0.5 * (k ** 2).sum(-1))  # [B, H, N]
+    want = np.cumsum(wts[..., None] * v, axis=2) / np.cumsum(wts, axis=2)[..., None]
+    np.testing.assert_allclose(o, want, rtol=1e-12)
+    k1 = k / np.linalg.norm(k, axis=-1, keepdims=True)
+    o1 = oracle.causal_linear_attn(q, k1, v, W=W0)
+    np.testing.assert_allclose(o1, np.cumsum(v, axis=2) / np.arange(1, N + 1)[None, None, :, None], rtol=1e-12)
+
+
+def test_favor_linear_attention_equals_the_masked_quadratic_form_and_its_variants_agree():
+    B, H, N, d, w, h0 = 2, 3, 12, 4, 5, 1
+    q, k, v = rnd((B, H, N, d), 631, 0.7), rnd((B, H, N, d), 632, 0.7), rnd((B, H, N, d), 633)
+    W = rnd((H, d, d), 634)
+    o = oracle.causal_linear_attn(q, k, v, W=W)
+    for b in range(B):
+        for h in range(H):
+            fq, fk = oracle.phi_favor(q[b, h], W[h]), oracle.phi_favor(k[b, h], W[h])
+            A = np.tril(fq @ fk.T)  # weights of key j for query i, j <= i
+            np.testing.assert_allclose(o[b, h], (A @ v[b, h]) / A.sum(1, keepdims=True), rtol=1e-11)
+            # the bidirectional layer's global form: no mask
+            A2 = fq @ fk.T
+            og = oracle.linear_attn_self(q[b:b + 1, h:h + 1], k[b:b + 1, h:h + 1], v[b:b + 1, h:h + 1], W=W[h:h + 1])
+            np.testing.assert_allclose(og[0, 0], (A2 @ v[b, h]) / A2.sum(1, keepdims=True), rtol=1e-11)
+    # a per-row factor of phi(q) cancels: the -|q|^2/2 term and the 1/sqrt(m) do not matter for q, so
+    # moving q along a direction orthogonal to every projection row (here: W has rank < d) changes nothing
+    Wr = W.copy()
+    Wr[:, :, -1] = 0.0  # no projection row sees the last coordinate
+    q2 = q.copy()
+    q2[..., -1] += 3.0
+    np.testing.assert_allclose(oracle.causal_linear_attn(q2, k, v, W=Wr), oracle.causal_linear_attn(q, k, v, W=Wr), rtol=1e-11)
+    # hybrid routing and decoding carry the projection of the linear heads only
+    ref, st = oracle.hybrid_attn(q[:, :, :8], k[:, :, :8], v[:, :, :8], w, h_sparse=h0, export_state=True, W=W[h0:])
+    full = oracle.hybrid_attn(q, k, v, w, h_sparse=h0, W=W[h0:])
+    np.testing.assert_allclose(ref, full[:, :, :8], rtol=1e-12)
+    np.testing.assert_allclose(full[:, h0:], o[:, h0:], rtol=1e-12)
+    for t in range(8, N):
+        ot = oracle.decode_step(q[:, :, t], k[:, :, t], v[:, :, t], st)
+        np.testing.assert_allclose(ot, full[:, :, t], rtol=1e-10, atol=1e-12)
