@@ -337,7 +337,9 @@ def run_ours(args, c, rank, world, local_rank):
     ho = torch.empty_like(hq).pin_memory()
     dq, dk, dv = [t.cuda() for t in (hq, hk, hv)]
     do = torch.empty_like(dq)
-    ws = gf.Workspace.for_problem(B, H, N, d, w, h0)
+    favor = args.phi == "favor"
+    Wd = synth.favor_projection(H - h0, d, seed=c["seed"], orthogonal=True, dtype="bf16").cuda() if favor else None
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0, phi=gf.GF_PHI_FAVOR_POS if favor else gf.GF_PHI_ELU1)
     stream = torch.cuda.Stream()
 
     def barrier():
@@ -347,7 +349,10 @@ def run_ours(args, c, rank, world, local_rank):
         torch.cuda.synchronize()
 
     self_layer = bool(c.get("self_layer"))
-    layer = gf.hybrid_attn_self if self_layer else gf.hybrid_attn
+    base_layer = gf.hybrid_attn_self if self_layer else gf.hybrid_attn
+
+    def layer(*a, **kw):
+        return base_layer(*a, W=Wd, **kw)
 
     # Inputs that fit the L2 are rotated over several buffer sets, so that every step reads its
     # inputs from HBM; the L2-resident figure (one set, back to back) is reported beside it.
@@ -491,7 +496,7 @@ def run_ours(args, c, rank, world, local_rank):
     # The two kernels of a step, each timed alone over the same number of launches (B = 1 makes the
     # head slices contiguous): the dominant one carries the roofline entry.
     kern = {}
-    if B == 1 and 0 < h0 < H:
+    if B == 1 and 0 < h0 < H and not favor:
         lq, lk, lv, lo_ = dq[:, h0:], dk[:, h0:], dv[:, h0:], do[:, h0:]
         wq, wk, wv, wo_ = dq[:, :h0], dk[:, :h0], dv[:, :h0], do[:, :h0]
         ws_l = gf.Workspace.for_problem(B, H - h0, N, d, 1, 0)
@@ -533,6 +538,8 @@ def run_ours(args, c, rank, world, local_rank):
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": args.workload, "B": B, "H": H, "N": N, "d": d, "w": w, "h_sparse": h0,
+                       "phi": "positive random features (features of Q and K written to the workspace first)" if favor
+                       else "elu + 1",
                        "global_batch": world * B, "seq_len": N,
                        "parallelism": "replicas only (one batch element per GPU, no collective)",
                        "l2": ("inputs larger than L2 (Q+K+V+O = %.0f MB per step, L2 %.0f MB)" % (set_bytes / 1e6, l2 / 1e6))
@@ -808,6 +815,8 @@ def main():
     ap.add_argument("--workload", default="long32k", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-sustained", action="store_true", help="skip the one-second sustained run")
+    ap.add_argument("--phi", choices=["elu1", "favor"], default="elu1",
+                    help="feature map of the linear heads: elu + 1, or positive random features (seeded projections)")
     ap.add_argument("--kernel-only", choices=["linear", "window"], default=None,
                     help="run only that head group's kernel (no timing): a driver for profilers")
     args = ap.parse_args()

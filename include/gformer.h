@@ -45,8 +45,18 @@ typedef enum {
 
 typedef enum { GF_F32 = 0, GF_BF16 = 1 } gf_dtype;
 typedef enum { GF_BHND = 0, GF_BNHD = 1 } gf_layout;
-/* Feature map of the linear heads.  GF_PHI_ELU1: phi(x) = elu(x) + 1 (Sec. II-B). */
-typedef enum { GF_PHI_ELU1 = 0 } gf_phi;
+/* Feature map of the linear heads.
+ * GF_PHI_ELU1: phi(x) = elu(x) + 1, element by element (Sec. II-B).
+ * GF_PHI_FAVOR_POS: the positive random features Sec. III-A and III-C name ("positive orthogonal
+ *   random features"; the paper prints no formula, this is the cited Performer paper's):
+ *       phi_W(x)[a] = exp(<w_a, x> - |x|^2 / 2) / sqrt(d),   a = 0 .. d-1,
+ *   with d features because the state of Algorithm 1 is d x d.  The projection vectors w_a are the
+ *   caller's (argument W of the ..._w entry points): one d x d matrix per linear head, row a = w_a,
+ *   in the storage dtype of q.  x is taken as passed (no extra scale, no stabiliser): the state S, z is
+ *   the definition's.  The kernels use the fact that a factor common to all features of one query
+ *   cancels in the output (they take the query features relative to the row's largest projection), so
+ *   only the key features must be representable: |k|^2 / 2 - <w_a, k> up to about 85 (fp32) is fine. */
+typedef enum { GF_PHI_ELU1 = 0, GF_PHI_FAVOR_POS = 1 } gf_phi;
 
 /* Process-wide knobs for tests and benchmarks (gformer_set_tuning). */
 typedef enum {
@@ -144,6 +154,10 @@ unsigned long long gformer_launch_count(void);
 
 /* Scratch bytes the attention entry points need for this problem (never 0). */
 size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, int dtype);
+/* The same for a given feature map of the linear heads: with GF_PHI_FAVOR_POS on the tensor-core path
+ * the features of Q and K are written to the workspace first (two bf16 tensors of the linear heads'
+ * size), so more is needed; with GF_PHI_ELU1 this is gformer_workspace_bytes. */
+size_t gformer_workspace_bytes_phi(int B, int H, int N, int d, int w, int h_sparse, int dtype, int phi);
 
 /* Synchronises `cuda_stream`, reads the device status word kept in ws and returns
  * GF_OK, GF_ERR_TIMEOUT (a bounded wait inside a tensor-core kernel gave up; outputs of
@@ -187,6 +201,15 @@ int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void
                                int B, int H, int N, int d, int phi, int chunk,
                                float* S_io, float* z_io,
                                int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* gformer_causal_linear_attn with the feature map's parameter: W is null for GF_PHI_ELU1 and, for
+ * GF_PHI_FAVOR_POS (Sec. III-A / III-C), a device pointer to the projections [H, d, d] in the storage
+ * dtype of q (16-byte aligned; row a of head h's matrix is w_a).  Workspace: gformer_workspace_bytes_phi.
+ * GF_ERR_INVALID_ARG when W and phi do not go together. */
+int gformer_causal_linear_attn_w(const void* q, const void* k, const void* v, void* o,
+                                 int B, int H, int N, int d, int phi, const void* W, int chunk,
+                                 float* S_io, float* z_io,
+                                 int dtype, int layout, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * gformer_causal_linear_attn for callers that cannot allocate device memory (no counterpart
@@ -282,6 +305,22 @@ int gformer_decode_step(const void* q, const void* k, const void* v, void* o,
 int gformer_decode_step_ragged(const void* q, const void* k, const void* v, void* o,
                                gf_decode_state* st, long long* t_seq, float scale, int phi,
                                void* cuda_stream);
+
+/* The three layer-level entry points with the feature map's parameter (see gformer_causal_linear_attn_w):
+ * W [H - h_sparse, d, d] holds the projections of the linear heads only, in head order; null for
+ * GF_PHI_ELU1.  Everything else as in gformer_hybrid_attn, gformer_hybrid_attn_self and
+ * gformer_decode_step (a decode state filled by gformer_hybrid_attn_w must be advanced with the same phi
+ * and W).  Workspace of the first two: gformer_workspace_bytes_phi. */
+int gformer_hybrid_attn_w(const void* q, const void* k, const void* v, void* o,
+                          int B, int H, int N, int d, int w, int h_sparse, float scale,
+                          int phi, const void* W, int chunk, int dtype, int layout, gf_decode_state* state_out,
+                          void* ws, size_t ws_bytes, void* cuda_stream);
+int gformer_hybrid_attn_self_w(const void* q, const void* k, const void* v, void* o,
+                               int B, int H, int N, int d, int w, int h_sparse, float scale,
+                               int phi, const void* W, int dtype, int layout,
+                               void* ws, size_t ws_bytes, void* cuda_stream);
+int gformer_decode_step_w(const void* q, const void* k, const void* v, void* o,
+                          gf_decode_state* st, float scale, int phi, const void* W, void* cuda_stream);
 
 #ifdef __cplusplus
 }

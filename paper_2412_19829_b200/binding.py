@@ -14,7 +14,7 @@ import torch
 GF_OK, GF_ERR_INVALID_ARG, GF_ERR_UNSUPPORTED, GF_ERR_WORKSPACE, GF_ERR_CUDA, GF_ERR_TIMEOUT = range(6)
 GF_F32, GF_BF16 = 0, 1
 GF_BHND, GF_BNHD = 0, 1
-GF_PHI_ELU1 = 0
+GF_PHI_ELU1, GF_PHI_FAVOR_POS = 0, 1
 GF_TUNE_FORCE_SIMT, GF_TUNE_LINEAR_SPLIT, GF_TUNE_LINEAR_CTAS, GF_TUNE_WAIT_KCYCLES, GF_TUNE_TEST_DROP_FLAG = 0, 1, 2, 3, 4
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -67,6 +67,17 @@ def lib() -> ctypes.CDLL:
         L.gformer_linear_plan_parts.argtypes = [i, i, i, i, pint, pint, pint]
         L.gformer_workspace_bytes.restype = sz
         L.gformer_workspace_bytes.argtypes = [i] * 7
+        L.gformer_workspace_bytes_phi.restype = sz
+        L.gformer_workspace_bytes_phi.argtypes = [i] * 8
+        L.gformer_causal_linear_attn_w.restype = i
+        L.gformer_causal_linear_attn_w.argtypes = [vp, vp, vp, vp, i, i, i, i, i, vp, i, vp, vp, i, i, vp, sz, vp]
+        L.gformer_hybrid_attn_w.restype = i
+        L.gformer_hybrid_attn_w.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, f, i, vp, i, i, i,
+                                            ctypes.POINTER(DecodeStateC), vp, sz, vp]
+        L.gformer_hybrid_attn_self_w.restype = i
+        L.gformer_hybrid_attn_self_w.argtypes = [vp, vp, vp, vp, i, i, i, i, i, i, f, i, vp, i, i, vp, sz, vp]
+        L.gformer_decode_step_w.restype = i
+        L.gformer_decode_step_w.argtypes = [vp, vp, vp, vp, ctypes.POINTER(DecodeStateC), f, i, vp, vp]
         L.gformer_last_device_status.restype = i
         L.gformer_last_device_status.argtypes = [vp, vp]
         L.gformer_window_attn.restype = i
@@ -167,8 +178,18 @@ def partition_heads(B: int, H: int, N: int, E: int, W: int, perf_sparse: float, 
     return h0.value, ls.value, ll.value
 
 
-def workspace_bytes(B, H, N, d, w, h_sparse, dtype) -> int:
-    return int(lib().gformer_workspace_bytes(B, H, N, d, w, h_sparse, dtype))
+def workspace_bytes(B, H, N, d, w, h_sparse, dtype, phi: int = GF_PHI_ELU1) -> int:
+    return int(lib().gformer_workspace_bytes_phi(B, H, N, d, w, h_sparse, dtype, phi))
+
+
+def _phi_args(W, q, heads, d):
+    """(phi, pointer) of the linear heads' feature map: W None = elu + 1, else the projections [heads, d, d]
+    of the positive random features, a contiguous CUDA tensor of q's dtype."""
+    if W is None:
+        return GF_PHI_ELU1, None
+    if not (W.is_cuda and W.is_contiguous() and W.dtype == q.dtype and tuple(W.shape) == (heads, d, d)):
+        raise ValueError(f"W must be a contiguous CUDA tensor [{heads}, {d}, {d}] of dtype {q.dtype}")
+    return GF_PHI_FAVOR_POS, W.data_ptr()
 
 
 def _dtype_code(t: torch.Tensor) -> int:
@@ -213,9 +234,9 @@ class Workspace:
         self.nbytes = self.buf.numel() - off
 
     @classmethod
-    def for_problem(cls, B, H, N, d, w=1, h_sparse=0, dtype=GF_BF16, device=None):
-        """Scratch sized by gformer_workspace_bytes for this problem."""
-        return cls(workspace_bytes(B, H, N, d, w, h_sparse, dtype), device)
+    def for_problem(cls, B, H, N, d, w=1, h_sparse=0, dtype=GF_BF16, device=None, phi=GF_PHI_ELU1):
+        """Scratch sized by gformer_workspace_bytes_phi for this problem."""
+        return cls(workspace_bytes(B, H, N, d, w, h_sparse, dtype, phi), device)
 
     def last_device_status(self, stream=None) -> int:
         return int(lib().gformer_last_device_status(self.ptr, _stream_ptr(stream)))
@@ -264,24 +285,28 @@ def window_attn_self(q, k, v, w: int, scale: float = 0.0, layout: int = GF_BHND,
 
 
 def hybrid_attn_self(q, k, v, w: int, h_sparse: int = -1, scale: float = 0.0, layout: int = GF_BHND, out=None,
-                     ws=None, stream=None):
-    """gformer_hybrid_attn_self: the bidirectional layer (two-sided windowed heads, global linear heads)."""
+                     ws=None, stream=None, W=None):
+    """gformer_hybrid_attn_self(_w): the bidirectional layer (two-sided windowed heads, global linear heads).
+    W [H - h_sparse, d, d]: positive random features under these projections instead of elu + 1."""
     _check_qkv(q, k, v)
     B, H, N, d = _dims(q, layout)
     o = torch.empty_like(q) if out is None else out
     dt = _dtype_code(q)
-    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, h_sparse, dt))
-    rc = lib().gformer_hybrid_attn_self(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, int(w),
-                                        int(h_sparse), float(scale), GF_PHI_ELU1, dt, layout, W.ptr, W.nbytes,
-                                        _stream_ptr(stream))
+    h0 = default_h_sparse(H) if h_sparse < 0 else h_sparse
+    phi, wp = _phi_args(W, q, H - h0, d)
+    wsp = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, h_sparse, dt, phi))
+    rc = lib().gformer_hybrid_attn_self_w(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, int(w),
+                                          int(h_sparse), float(scale), phi, wp, dt, layout, wsp.ptr, wsp.nbytes,
+                                          _stream_ptr(stream))
     if rc != GF_OK:
-        raise GformerError(rc, "gformer_hybrid_attn_self")
+        raise GformerError(rc, "gformer_hybrid_attn_self_w")
     return o
 
 
 def causal_linear_attn(q, k, v, S=None, z=None, chunk: int = 0, layout: int = GF_BHND, out=None, ws=None,
-                       stream=None):
-    """gformer_causal_linear_attn: Algorithm 1 with phi = elu + 1; S, z (fp32) updated in place."""
+                       stream=None, W=None):
+    """gformer_causal_linear_attn(_w): Algorithm 1 with phi = elu + 1, or with the positive random features
+    under the projections W [H, d, d]; S, z (fp32) updated in place."""
     _check_qkv(q, k, v)
     B, H, N, d = _dims(q, layout)
     o = torch.empty_like(q) if out is None else out
@@ -289,13 +314,14 @@ def causal_linear_attn(q, k, v, S=None, z=None, chunk: int = 0, layout: int = GF
     if S is not None:
         assert S.dtype == torch.float32 and S.is_contiguous() and tuple(S.shape) == (B, H, d, d)
         assert z.dtype == torch.float32 and z.is_contiguous() and tuple(z.shape) == (B, H, d)
-    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, 1, 0, dt))
-    rc = lib().gformer_causal_linear_attn(
-        q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, GF_PHI_ELU1, int(chunk),
+    phi, wp = _phi_args(W, q, H, d)
+    wsp = _ws_for(q, ws, workspace_bytes(B, H, N, d, 1, 0, dt, phi))
+    rc = lib().gformer_causal_linear_attn_w(
+        q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, phi, wp, int(chunk),
         S.data_ptr() if S is not None else None, z.data_ptr() if z is not None else None,
-        dt, layout, W.ptr, W.nbytes, _stream_ptr(stream))
+        dt, layout, wsp.ptr, wsp.nbytes, _stream_ptr(stream))
     if rc != GF_OK:
-        raise GformerError(rc, "gformer_causal_linear_attn")
+        raise GformerError(rc, "gformer_causal_linear_attn_w")
     return o
 
 
@@ -337,32 +363,36 @@ class DecodeState:
 
 
 def hybrid_attn(q, k, v, w: int, h_sparse: int = -1, scale: float = 0.0, chunk: int = 0,
-                layout: int = GF_BHND, state_out: DecodeState | None = None, out=None, ws=None, stream=None):
-    """gformer_hybrid_attn: heads [0, h_sparse) windowed, the rest linear, merged by head."""
+                layout: int = GF_BHND, state_out: DecodeState | None = None, out=None, ws=None, stream=None, W=None):
+    """gformer_hybrid_attn(_w): heads [0, h_sparse) windowed, the rest linear, merged by head.
+    W [H - h_sparse, d, d]: positive random features under these projections instead of elu + 1."""
     _check_qkv(q, k, v)
     B, H, N, d = _dims(q, layout)
     o = torch.empty_like(q) if out is None else out
     dt = _dtype_code(q)
-    W = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, h_sparse, dt))
-    rc = lib().gformer_hybrid_attn(
+    h0 = default_h_sparse(H) if h_sparse < 0 else h_sparse
+    phi, wp = _phi_args(W, q, H - h0, d)
+    wsp = _ws_for(q, ws, workspace_bytes(B, H, N, d, w, h_sparse, dt, phi))
+    rc = lib().gformer_hybrid_attn_w(
         q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), B, H, N, d, int(w), int(h_sparse), float(scale),
-        GF_PHI_ELU1, int(chunk), dt, layout, ctypes.byref(state_out.c) if state_out is not None else None,
-        W.ptr, W.nbytes, _stream_ptr(stream))
+        phi, wp, int(chunk), dt, layout, ctypes.byref(state_out.c) if state_out is not None else None,
+        wsp.ptr, wsp.nbytes, _stream_ptr(stream))
     if rc != GF_OK:
-        raise GformerError(rc, "gformer_hybrid_attn")
+        raise GformerError(rc, "gformer_hybrid_attn_w")
     return o
 
 
-def decode_step(q, k, v, st: DecodeState, scale: float = 0.0, out=None, stream=None):
-    """gformer_decode_step: q, k, v are [B, H, d]; st is advanced by one token."""
+def decode_step(q, k, v, st: DecodeState, scale: float = 0.0, out=None, stream=None, W=None):
+    """gformer_decode_step(_w): q, k, v are [B, H, d]; st is advanced by one token.  W as in hybrid_attn."""
     for t in (q, k, v):
         if not (t.is_cuda and t.is_contiguous() and t.dim() == 3):
             raise ValueError("q, k, v must be contiguous [B, H, d] CUDA tensors")
     o = torch.empty_like(q) if out is None else out
-    rc = lib().gformer_decode_step(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), ctypes.byref(st.c),
-                                   float(scale), GF_PHI_ELU1, _stream_ptr(stream))
+    phi, wp = _phi_args(W, q, st.c.H - st.c.h_sparse, st.c.d)
+    rc = lib().gformer_decode_step_w(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(), ctypes.byref(st.c),
+                                     float(scale), phi, wp, _stream_ptr(stream))
     if rc != GF_OK:
-        raise GformerError(rc, "gformer_decode_step")
+        raise GformerError(rc, "gformer_decode_step_w")
     return o
 
 

@@ -14,7 +14,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "libgformer.so")
-SOURCES = ["api.cu", "simt_kernels.cu", "tma_host.cu", "tc_window.cu", "tc_linear.cu", "tc_linear_self.cu", "noalloc.cu", "partition.cu"]
+SOURCES = ["api.cu", "simt_kernels.cu", "tma_host.cu", "tc_window.cu", "tc_linear.cu", "tc_linear_self.cu", "noalloc.cu", "partition.cu", "tc_favor.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

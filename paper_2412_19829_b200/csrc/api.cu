@@ -114,15 +114,41 @@ int run_window(const Tuning& tn, const void* q, const void* k, const void* v, vo
                                             gf::make_strides(layout, H, N, d), h_begin, h_count, stream));
 }
 
+// Feature map of the linear heads of one call: elu + 1 (W null), or positive random features under
+// the projections W [h_count, d, d].  On the tensor-core path those are computed first, into the two
+// feature tensors at the end of the workspace (feat_offset bytes in).
+struct Phi {
+  const void* W = nullptr;
+  size_t feat_offset = 0;
+};
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+size_t feature_bytes(int B, int h_lin, int N, int d) { return align256((size_t)B * h_lin * N * d * 2); }
+
+int check_phi(int phi, const void* W) {
+  if (phi == GF_PHI_ELU1) return W == nullptr ? GF_OK : GF_ERR_INVALID_ARG;
+  if (phi == GF_PHI_FAVOR_POS) return (W != nullptr && aligned16(W)) ? GF_OK : GF_ERR_INVALID_ARG;
+  return GF_ERR_UNSUPPORTED;
+}
+
 int run_linear(const Tuning& tn, const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
                int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init, int max_ctas,
-               WsHeader* ws, cudaStream_t stream, bool shared = false) {
+               WsHeader* ws, cudaStream_t stream, bool shared = false, const Phi& phi = Phi()) {
   if (h_count <= 0) return GF_OK;
-  if (!tn.force_simt && gf::tc_linear_supported(N, d, dtype))
+  if (!tn.force_simt && gf::tc_linear_supported(N, d, dtype)) {
+    void *fq = nullptr, *fk = nullptr;
+    if (phi.W != nullptr) {
+      fq = reinterpret_cast<uint8_t*>(ws) + phi.feat_offset;
+      fk = reinterpret_cast<uint8_t*>(fq) + feature_bytes(B, h_count, N, d);
+      const int rc = cuda_status(gf::launch_favor_features_tc(q, k, phi.W, fq, fk, B, H, N, d, layout, h_begin,
+                                                              h_count, ws, stream));
+      if (rc != GF_OK) return rc;
+    }
     return cuda_status(gf::launch_linear_tc(q, k, v, o, B, H, N, d, layout, h_begin, h_count, S_io, z_io,
-                                            zero_init, tn.linear_split, max_ctas, ws, stream, shared));
+                                            zero_init, tn.linear_split, max_ctas, ws, stream, shared, fq, fk));
+  }
   return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d),
-                                            h_begin, h_count, S_io, z_io, zero_init, stream));
+                                            h_begin, h_count, S_io, z_io, zero_init, stream, false, phi.W));
 }
 
 // Zeroes the workspace header and, for a call that runs the tensor-core linear kernel on n_lin
@@ -138,7 +164,8 @@ int clear_ws(const Tuning& tn, void* ws, cudaStream_t stream, int n_lin = 0, int
   return GF_OK;
 }
 
-size_t workspace_bytes(const Tuning& tn, int B, int H, int N, int d, int h_sparse, int dtype);
+size_t workspace_bytes(const Tuning& tn, int B, int H, int N, int d, int h_sparse, int dtype, int phi = GF_PHI_ELU1,
+                       size_t* feat_offset = nullptr);
 
 }  // namespace
 
@@ -214,11 +241,18 @@ size_t gformer_workspace_bytes(int B, int H, int N, int d, int w, int h_sparse, 
   (void)w;
   return workspace_bytes(tuning_now(), B, H, N, d, h_sparse, dtype);
 }
+
+size_t gformer_workspace_bytes_phi(int B, int H, int N, int d, int w, int h_sparse, int dtype, int phi) {
+  (void)w;
+  return workspace_bytes(tuning_now(), B, H, N, d, h_sparse, dtype, phi);
+}
 }  // extern "C"
 
 namespace {
-size_t workspace_bytes(const Tuning& tn, int B, int H, int N, int d, int h_sparse, int dtype) {
+size_t workspace_bytes(const Tuning& tn, int B, int H, int N, int d, int h_sparse, int dtype, int phi,
+                       size_t* feat_offset) {
   size_t bytes = sizeof(WsHeader);
+  if (feat_offset) *feat_offset = 0;
   if (B < 1 || H < 1 || N < 1) return bytes;
   if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
   if (h_sparse > H) h_sparse = H;
@@ -228,6 +262,11 @@ size_t workspace_bytes(const Tuning& tn, int B, int H, int N, int d, int h_spars
     const size_t causal = gf::linear_tc_workspace_bytes(B * h_lin, N, d, tn.linear_split);
     const size_t self = gf::linear_self_workspace_bytes(B * h_lin, N, d);
     bytes += causal > self ? causal : self;
+    if (phi == GF_PHI_FAVOR_POS) {  // the features of Q and K of the linear heads, behind everything else
+      bytes = align256(bytes);
+      if (feat_offset) *feat_offset = bytes;
+      bytes += 2 * feature_bytes(B, h_lin, N, d);
+    }
   }
   return bytes;
 }
@@ -278,20 +317,36 @@ int gformer_window_attn_self(const void* q, const void* k, const void* v, void* 
 int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int w, int h_sparse, float scale, int phi, int dtype, int layout, void* ws,
                              size_t ws_bytes, void* cuda_stream) {
+  if (phi == GF_PHI_FAVOR_POS) return GF_ERR_INVALID_ARG;  // needs its projections: gformer_hybrid_attn_self_w
+  return gformer_hybrid_attn_self_w(q, k, v, o, B, H, N, d, w, h_sparse, scale, phi, nullptr, dtype, layout, ws, ws_bytes,
+                                    cuda_stream);
+}
+
+int gformer_hybrid_attn_self_w(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                               int w, int h_sparse, float scale, int phi, const void* W, int dtype, int layout,
+                               void* ws, size_t ws_bytes, void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
   const Tuning tn = tuning_now();
   if (w < 1) return GF_ERR_INVALID_ARG;
-  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  if ((rc = check_phi(phi, W)) != GF_OK) return rc;
+  size_t feat_offset = 0;
   if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
   if (h_sparse > H) return GF_ERR_INVALID_ARG;
-  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, h_sparse, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, h_sparse, dtype, phi, &feat_offset));
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   rc = clear_ws(tn, ws, stream);
   if (rc != GF_OK) return rc;
   const bool tc_linear = !tn.force_simt && gf::tc_linear_supported(N, d, dtype);
+  // positive random features: computed first (on the stream the linear kernels run on), then read in
+  // place of Q and K
+  void *fq = nullptr, *fk = nullptr;
+  if (W != nullptr && tc_linear && h_sparse < H) {
+    fq = reinterpret_cast<uint8_t*>(ws) + feat_offset;
+    fk = reinterpret_cast<uint8_t*>(fq) + feature_bytes(B, H - h_sparse, N, d);
+  }
   if (h_sparse > 0 && h_sparse < H && tc_linear) {
     // Both head groups on tensor-core kernels: the three launches of the linear heads go to the
     // library's high-priority stream, the windowed heads to its side stream a few microseconds
@@ -303,8 +358,12 @@ int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* 
     if (cudaEventRecord(f->fork, stream) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(f->side, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(f->first, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
-    rc = cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
-                                               sizeof(WsHeader), f->first));
+    if (fq != nullptr)
+      rc = cuda_status(gf::launch_favor_features_tc(q, k, W, fq, fk, B, H, N, d, layout, h_sparse, H - h_sparse,
+                                                    (WsHeader*)ws, f->first));
+    if (rc == GF_OK)
+      rc = cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
+                                                 sizeof(WsHeader), f->first, fq, fk));
     if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
     int rc2 = cuda_status(gf::launch_delay(8000, f->side));
@@ -317,40 +376,67 @@ int gformer_hybrid_attn_self(const void* q, const void* k, const void* v, void* 
   rc = run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, stream, true);
   if (rc != GF_OK) return rc;
   if (h_sparse == H) return GF_OK;
-  if (tc_linear)
+  if (tc_linear) {
+    if (fq != nullptr) {
+      rc = cuda_status(gf::launch_favor_features_tc(q, k, W, fq, fk, B, H, N, d, layout, h_sparse, H - h_sparse,
+                                                    (WsHeader*)ws, stream));
+      if (rc != GF_OK) return rc;
+    }
     return cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
-                                                 sizeof(WsHeader), stream));
+                                                 sizeof(WsHeader), stream, fq, fk));
+  }
   // fp32 storage (or the CUDA-core knob): token by token, a summing sweep and a readout sweep
   return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d), h_sparse,
-                                            H - h_sparse, nullptr, nullptr, true, stream, true));
+                                            H - h_sparse, nullptr, nullptr, true, stream, true, W));
 }
 
 int gformer_causal_linear_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                                int phi, int chunk, float* S_io, float* z_io, int dtype, int layout, void* ws,
                                size_t ws_bytes, void* cuda_stream) {
+  if (phi == GF_PHI_FAVOR_POS) return GF_ERR_INVALID_ARG;  // needs its projections: gformer_causal_linear_attn_w
+  return gformer_causal_linear_attn_w(q, k, v, o, B, H, N, d, phi, nullptr, chunk, S_io, z_io, dtype, layout, ws,
+                                      ws_bytes, cuda_stream);
+}
+
+int gformer_causal_linear_attn_w(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
+                                 int phi, const void* W, int chunk, float* S_io, float* z_io, int dtype, int layout,
+                                 void* ws, size_t ws_bytes, void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
   const Tuning tn = tuning_now();
-  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  if ((rc = check_phi(phi, W)) != GF_OK) return rc;
+  Phi fm;
+  fm.W = W;
   if (chunk != 0 && chunk != 128) return chunk < 0 || chunk % 64 ? GF_ERR_INVALID_ARG : GF_ERR_UNSUPPORTED;
   if ((S_io == nullptr) != (z_io == nullptr)) return GF_ERR_INVALID_ARG;
   if (S_io && (!aligned16(S_io) || !aligned16(z_io))) return GF_ERR_INVALID_ARG;
-  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, 0, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, 0, dtype, phi, &fm.feat_offset));
   if (rc != GF_OK) return rc;
   cudaStream_t stream = (cudaStream_t)cuda_stream;
   rc = clear_ws(tn, ws, stream, B * H, N, d, dtype);
   if (rc != GF_OK) return rc;
-  return run_linear(tn, q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, 0, (WsHeader*)ws, stream);
+  return run_linear(tn, q, k, v, o, B, H, N, d, dtype, layout, 0, H, S_io, z_io, false, 0, (WsHeader*)ws, stream, false,
+                    fm);
 }
 
 int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
                         int h_sparse, float scale, int phi, int chunk, int dtype, int layout,
                         gf_decode_state* state_out, void* ws, size_t ws_bytes, void* cuda_stream) {
+  if (phi == GF_PHI_FAVOR_POS) return GF_ERR_INVALID_ARG;  // needs its projections: gformer_hybrid_attn_w
+  return gformer_hybrid_attn_w(q, k, v, o, B, H, N, d, w, h_sparse, scale, phi, nullptr, chunk, dtype, layout, state_out,
+                               ws, ws_bytes, cuda_stream);
+}
+
+int gformer_hybrid_attn_w(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int w,
+                          int h_sparse, float scale, int phi, const void* W, int chunk, int dtype, int layout,
+                          gf_decode_state* state_out, void* ws, size_t ws_bytes, void* cuda_stream) {
   int rc = check_common(q, k, v, o, B, H, N, d, dtype, layout);
   if (rc != GF_OK) return rc;
   const Tuning tn = tuning_now();
   if (w < 1) return GF_ERR_INVALID_ARG;
-  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  if ((rc = check_phi(phi, W)) != GF_OK) return rc;
+  Phi fm;
+  fm.W = W;
   if (chunk != 0 && chunk != 128) return chunk < 0 || chunk % 64 ? GF_ERR_INVALID_ARG : GF_ERR_UNSUPPORTED;
   if (h_sparse < 0) h_sparse = gformer_default_h_sparse(H);
   if (h_sparse > H) return GF_ERR_INVALID_ARG;
@@ -363,7 +449,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
       return GF_ERR_INVALID_ARG;
     if (h_lin > 0 && (!s->S || !s->z || !aligned16(s->S) || !aligned16(s->z))) return GF_ERR_INVALID_ARG;
   }
-  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, h_sparse, dtype));
+  rc = check_ws(ws, ws_bytes, workspace_bytes(tn, B, H, N, d, h_sparse, dtype, phi, &fm.feat_offset));
   if (rc != GF_OK) return rc;
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)d);
   cudaStream_t stream = (cudaStream_t)cuda_stream;
@@ -404,7 +490,7 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
   const bool lin_first = both && lin_ctas > 0;
   if (lin_first && cudaStreamWaitEvent(f->first, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
   rc = run_linear(tn, q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, lin_ctas,
-                  (WsHeader*)ws, lin_first ? f->first : stream, both);
+                  (WsHeader*)ws, lin_first ? f->first : stream, both, fm);
   if (lin_first) {
     if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
@@ -430,25 +516,35 @@ int gformer_hybrid_attn(const void* q, const void* k, const void* v, void* o, in
 }
 
 static int decode_step_impl(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
-                            long long* t_seq, float scale, int phi, void* cuda_stream);
+                            long long* t_seq, float scale, int phi, const void* W, void* cuda_stream);
 
 int gformer_decode_step(const void* q, const void* k, const void* v, void* o, gf_decode_state* st, float scale,
                         int phi, void* cuda_stream) {
-  return decode_step_impl(q, k, v, o, st, nullptr, scale, phi, cuda_stream);
+  if (phi == GF_PHI_FAVOR_POS) return GF_ERR_INVALID_ARG;  // needs its projections: gformer_decode_step_w
+  return decode_step_impl(q, k, v, o, st, nullptr, scale, phi, nullptr, cuda_stream);
+}
+
+int gformer_decode_step_w(const void* q, const void* k, const void* v, void* o, gf_decode_state* st, float scale,
+                          int phi, const void* W, void* cuda_stream) {
+  return decode_step_impl(q, k, v, o, st, nullptr, scale, phi, W, cuda_stream);
 }
 
 int gformer_decode_step_ragged(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
                                long long* t_seq, float scale, int phi, void* cuda_stream) {
   if (!t_seq || (reinterpret_cast<uintptr_t>(t_seq) & 7u) != 0) return GF_ERR_INVALID_ARG;
   if (st && st->H > 4096) return GF_ERR_UNSUPPORTED;  // the arrival count of a sequence's heads has 15 bits
-  return decode_step_impl(q, k, v, o, st, t_seq, scale, phi, cuda_stream);
+  if (phi == GF_PHI_FAVOR_POS) return GF_ERR_INVALID_ARG;
+  return decode_step_impl(q, k, v, o, st, t_seq, scale, phi, nullptr, cuda_stream);
 }
 
 static int decode_step_impl(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
-                            long long* t_seq, float scale, int phi, void* cuda_stream) {
+                            long long* t_seq, float scale, int phi, const void* W, void* cuda_stream) {
   if (!q || !k || !v || !o || !st) return GF_ERR_INVALID_ARG;
   if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(o)) return GF_ERR_INVALID_ARG;
-  if (phi != GF_PHI_ELU1) return GF_ERR_UNSUPPORTED;
+  {
+    const int rc = check_phi(phi, W);
+    if (rc != GF_OK) return rc;
+  }
   if (st->B < 1 || st->H < 1 || st->w < 1 || st->h_sparse < 0 || st->h_sparse > st->H || st->t < 0)
     return GF_ERR_INVALID_ARG;
   if (st->dtype != GF_F32 && st->dtype != GF_BF16) return GF_ERR_INVALID_ARG;
@@ -465,7 +561,7 @@ static int decode_step_impl(const void* q, const void* k, const void* v, void* o
   if (!(scale > 0.f)) scale = 1.0f / sqrtf((float)st->d);
   cudaError_t e = gf::launch_decode_step(q, k, v, o, st->k_cache, st->v_cache, st->S, st->z, st->t, t_seq, st->B,
                                          st->H, st->d, st->w, st->h_sparse, scale, st->dtype,
-                                         (cudaStream_t)cuda_stream);
+                                         (cudaStream_t)cuda_stream, W);
   if (e != cudaSuccess) return GF_ERR_CUDA;
   if (t_seq == nullptr) st->t += 1;
   return GF_OK;

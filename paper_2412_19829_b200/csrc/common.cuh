@@ -53,14 +53,16 @@ cudaError_t launch_window_simt(const void* q, const void* k, const void* v, void
 // global_sum: the unmasked linear attention of the bidirectional layer (sum over all tokens, then readout).
 cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
                                int dtype, Strides st, int h_begin, int h_count, float* S_io, float* z_io,
-                               bool zero_init, cudaStream_t stream, bool global_sum = false);
+                               bool zero_init, cudaStream_t stream, bool global_sum = false,
+                               const void* W = nullptr /* [h_count, d, d] storage dtype: positive random features */);
 cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void* v_cache, int B, int N, int d,
                                int w, int dtype, Strides st, int h_sparse, cudaStream_t stream);
 // t_seq == nullptr: every sequence is at position t; else sequence b is at t_seq[b] (device array,
 // negative = idle slot, otherwise below 2^48) and the kernel itself moves the positions on.
 cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
                                void* v_cache, float* S, float* z, long long t, long long* t_seq, int B, int H,
-                               int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream);
+                               int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream,
+                               const void* W = nullptr /* [H - h_sparse, d, d] storage dtype */);
 
 // Writes the two test knobs into a workspace header that has just been cleared.
 cudaError_t launch_set_header(WsHeader* ws, unsigned int wait_kcycles, unsigned int drop_flag, cudaStream_t stream);
@@ -80,7 +82,7 @@ cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* 
 size_t linear_self_workspace_bytes(int nchains, int N, int d);
 cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                                   int layout, int h_begin, int h_count, WsHeader* ws, size_t scratch_offset,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, const void* fq = nullptr, const void* fk = nullptr);
 // Segmentation used by the tensor-core linear kernel (split: 0 = automatic, else chunks per segment;
 // ctas: CTAs the kernel will run with, 0 = one per SM of a B200) and the scratch it needs beyond
 // the workspace header (sized for the largest segment count the plan may pick for any ctas).
@@ -97,7 +99,15 @@ size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split);
 size_t linear_tc_flag_bytes(int nchains, int N, int split);
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared = false);
+                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared = false,
+                             const void* fq = nullptr, const void* fk = nullptr);
+// Positive random features phi_W of Q and K of heads [h_begin, h_begin + h_count) (bf16 storage) into the
+// contiguous bf16 tensors fq, fk [B, h_count, N, d]; W: [h_count, d, d] bf16, row a of a head's matrix is
+// its projection vector w_a.  With fq, fk given, the two linear-attention launchers read them in place
+// of Q and K and leave their own feature map out.
+cudaError_t launch_favor_features_tc(const void* q, const void* k, const void* W, void* fq, void* fk, int B, int H,
+                                     int N, int d, int layout, int h_begin, int h_count, WsHeader* ws,
+                                     cudaStream_t stream);
 
 // ---- device helpers
 // Cycles a bounded wait may take; `status` points at the first word of the workspace header.

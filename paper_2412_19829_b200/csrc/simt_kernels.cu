@@ -132,11 +132,13 @@ template <typename T, int D>
 __global__ void __launch_bounds__(256)
 linear_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                    T* __restrict__ o, int N, Strides st, int h_begin, int h_count,
-                   float* __restrict__ S_io, float* __restrict__ z_io, int zero_init, int global_sum) {
+                   float* __restrict__ S_io, float* __restrict__ z_io, int zero_init, int global_sum,
+                   const T* __restrict__ W /* [h_count, D, D] or null: elu + 1 */) {
   constexpr int TB = 16;
   constexpr int AR = D / 8;
   __shared__ float qs[TB][D];
   __shared__ float ks[TB][D];
+  __shared__ float xr[TB][D + 1];  // raw rows while the positive random features are taken (W != null)
   __shared__ float vs[TB][32];
   __shared__ float red[TB][8][33];
   __shared__ float redden[TB][8];
@@ -165,16 +167,61 @@ linear_simt_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
   const bool accumulate = !global_sum || sweep == 0, readout = !global_sum || sweep == 1;
   for (int n0 = 0; n0 < N; n0 += TB) {
     __syncthreads();
-    for (int idx = tid; idx < TB * D; idx += 256) {
-      const int tok = idx / D, a = idx % D;
-      const int n = n0 + tok;
-      float qq = 0.f, kk = 0.f;
-      if (n < N) {
-        qq = phi_elu1(to_f32(q[base + (long long)n * st.n + a]));
-        kk = phi_elu1(to_f32(k[base + (long long)n * st.n + a]));
+    if (W == nullptr) {
+      for (int idx = tid; idx < TB * D; idx += 256) {
+        const int tok = idx / D, a = idx % D;
+        const int n = n0 + tok;
+        float qq = 0.f, kk = 0.f;
+        if (n < N) {
+          qq = phi_elu1(to_f32(q[base + (long long)n * st.n + a]));
+          kk = phi_elu1(to_f32(k[base + (long long)n * st.n + a]));
+        }
+        qs[tok][a] = qq;
+        ks[tok][a] = kk;  // 0 for rows past N: they must not enter the state
       }
-      qs[tok][a] = qq;
-      ks[tok][a] = kk;  // 0 for rows past N: they must not enter the state
+    } else {
+      // phi_W(x)[a] = exp(<w_a, x> - |x|^2 / 2) / sqrt(D) (Sec. III-A / III-C), Q rows first, then K rows.
+      // A factor common to all features of a query cancels in the output: the query features are taken
+      // relative to the row's largest projection, exp(<w_a, q> - max_a <w_a, q>), which keeps their
+      // products with the state inside the range of fp32.
+      const T* Wh = W + (long long)hl * D * D;
+      for (int which = 0; which < 2; ++which) {
+        const T* src = which ? k : q;
+        float (*dst)[D] = which ? ks : qs;
+        for (int idx = tid; idx < TB * D; idx += 256) {
+          const int tok = idx / D, a = idx % D;
+          const int n = n0 + tok;
+          xr[tok][a] = (n < N) ? to_f32(src[base + (long long)n * st.n + a]) : 0.f;
+        }
+        __syncthreads();
+        for (int idx = tid; idx < TB * D; idx += 256) {
+          const int tok = idx / D, a = idx % D;
+          float proj = 0.f, n2 = 0.f;
+          for (int cc = 0; cc < D; ++cc) {
+            const float x = xr[tok][cc];
+            proj = fmaf(to_f32(Wh[(long long)a * D + cc]), x, proj);
+            n2 = fmaf(x, x, n2);
+          }
+          if (which) dst[tok][a] = (n0 + tok < N) ? expf(proj - 0.5f * n2) * rsqrtf((float)D) : 0.f;
+          else dst[tok][a] = proj;
+        }
+        __syncthreads();
+        if (which == 0) {  // queries: relative to the row maximum
+          float e[TB * D / 256];
+          for (int i = 0; i < TB * D / 256; ++i) {
+            const int idx = tid + 256 * i, tok = idx / D, a = idx % D;
+            float mx = -INFINITY;
+            for (int cc = 0; cc < D; ++cc) mx = fmaxf(mx, qs[tok][cc]);
+            e[i] = expf(qs[tok][a] - mx);
+          }
+          __syncthreads();
+          for (int i = 0; i < TB * D / 256; ++i) {
+            const int idx = tid + 256 * i;
+            qs[idx / D][idx % D] = e[i];
+          }
+          __syncthreads();
+        }
+      }
     }
     for (int idx = tid; idx < TB * 32; idx += 256) {
       const int tok = idx >> 5, cc = idx & 31;
@@ -281,7 +328,7 @@ __global__ void __launch_bounds__(256, 7)
 decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __restrict__ v,
                    T* __restrict__ o, T* __restrict__ kc, T* __restrict__ vc, float* __restrict__ S,
                    float* __restrict__ z, long long t_all, long long* __restrict__ t_seq, int H, int w,
-                   int h_sparse, float scale) {
+                   int h_sparse, float scale, const T* __restrict__ W /* [H - h_sparse, D, D] or null: elu + 1 */) {
   constexpr int D4 = D / 4;
   constexpr int G = 256 / D4;  // thread groups along the reduced dimension
   extern __shared__ __align__(16) float dyn[];  // window heads: w scores
@@ -394,9 +441,42 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
     float* Sb = S + sidx * D * D;
     float* zb = z + sidx * D;
     float denloc = 0.f;
+    if (W != nullptr) {
+      // positive random features of q_t and k_t (Sec. III-A / III-C): exp(<w_a, x> - |x|^2 / 2) / sqrt(D)
+      // for the key; for the query exp(<w_a, q> - max_a <w_a, q>) (a factor common to its features cancels
+      // in the output).  A warp per feature, lanes along the input dimension.
+      if (tid < D) {
+        part[0][tid] = qv;
+        part[1][tid] = to_f32(kin);
+      }
+      const float n2k = block_reduce(tid < D ? to_f32(kin) * to_f32(kin) : 0.f, false, scratch);  // barriers inside publish part[]
+      const T* Wh = W + (long long)(h - h_sparse) * D * D;
+      const int lane = tid & 31, wid = tid >> 5;
+      for (int a = wid; a < D; a += 8) {
+        float pq = 0.f, pk = 0.f;
+        for (int cc = lane; cc < D; cc += 32) {
+          const float wv = to_f32(Wh[(long long)a * D + cc]);
+          pq = fmaf(wv, part[0][cc], pq);
+          pk = fmaf(wv, part[1][cc], pk);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+          pq += __shfl_xor_sync(0xffffffffu, pq, off);
+          pk += __shfl_xor_sync(0xffffffffu, pk, off);
+        }
+        if (lane == 0) {
+          qs[a] = pq;
+          ks[a] = expf(pk - 0.5f * n2k) * rsqrtf((float)D);
+        }
+      }
+      __syncthreads();
+      const float pmax = block_reduce(tid < D ? qs[tid] : -INFINITY, true, scratch);
+      if (tid < D) qs[tid] = expf(qs[tid] - pmax);
+      __syncthreads();
+    }
     if (tid < D) {
-      const float qp = phi_elu1(qv);
-      const float kp = phi_elu1(to_f32(kin));
+      const float qp = W != nullptr ? qs[tid] : phi_elu1(qv);
+      const float kp = W != nullptr ? ks[tid] : phi_elu1(to_f32(kin));
       qs[tid] = qp;
       ks[tid] = kp;
       const float zn = zb[tid] + kp;
@@ -447,14 +527,16 @@ cudaError_t window_dispatch(const void* q, const void* k, const void* v, void* o
 template <typename T>
 cudaError_t linear_dispatch(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
                             Strides st, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                            bool global_sum, cudaStream_t stream) {
+                            bool global_sum, cudaStream_t stream, const void* W) {
   dim3 grid(d / 32, h_count, B);
   if (d == 64)
     linear_simt_kernel<T, 64><<<grid, 256, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, st, h_begin,
-                                                        h_count, S_io, z_io, zero_init ? 1 : 0, global_sum ? 1 : 0);
+                                                        h_count, S_io, z_io, zero_init ? 1 : 0, global_sum ? 1 : 0,
+                                                        (const T*)W);
   else
     linear_simt_kernel<T, 128><<<grid, 256, 0, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, N, st, h_begin,
-                                                         h_count, S_io, z_io, zero_init ? 1 : 0, global_sum ? 1 : 0);
+                                                         h_count, S_io, z_io, zero_init ? 1 : 0, global_sum ? 1 : 0,
+                                                         (const T*)W);
   note_launch();
   return cudaGetLastError();
 }
@@ -462,7 +544,7 @@ cudaError_t linear_dispatch(const void* q, const void* k, const void* v, void* o
 template <typename T>
 cudaError_t decode_dispatch(const void* q, const void* k, const void* v, void* o, void* kc, void* vc, float* S,
                             float* z, long long t, long long* t_seq, int B, int H, int d, int w, int h_sparse,
-                            float scale, cudaStream_t stream) {
+                            float scale, cudaStream_t stream, const void* W) {
   dim3 grid(H, B);
   const size_t dyn = (size_t)w * sizeof(float);
   if (d == 64) {
@@ -472,7 +554,7 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, void* o
       if (e != cudaSuccess) return e;
     }
     kern<<<grid, 256, dyn, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, (T*)kc, (T*)vc, S, z, t, t_seq,
-                                     H, w, h_sparse, scale);
+                                     H, w, h_sparse, scale, (const T*)W);
   } else {
     auto kern = decode_step_kernel<T, 128>;
     if (dyn > 40 * 1024) {
@@ -480,7 +562,7 @@ cudaError_t decode_dispatch(const void* q, const void* k, const void* v, void* o
       if (e != cudaSuccess) return e;
     }
     kern<<<grid, 256, dyn, stream>>>((const T*)q, (const T*)k, (const T*)v, (T*)o, (T*)kc, (T*)vc, S, z, t, t_seq,
-                                     H, w, h_sparse, scale);
+                                     H, w, h_sparse, scale, (const T*)W);
   }
   note_launch();
   return cudaGetLastError();
@@ -499,13 +581,13 @@ cudaError_t launch_window_simt(const void* q, const void* k, const void* v, void
 
 cudaError_t launch_linear_simt(const void* q, const void* k, const void* v, void* o, int B, int N, int d,
                                int dtype, Strides st, int h_begin, int h_count, float* S_io, float* z_io,
-                               bool zero_init, cudaStream_t stream, bool global_sum) {
+                               bool zero_init, cudaStream_t stream, bool global_sum, const void* W) {
   if (h_count <= 0 || B <= 0) return cudaSuccess;
   if (dtype == GF_F32)
     return linear_dispatch<float>(q, k, v, o, B, N, d, st, h_begin, h_count, S_io, z_io, zero_init, global_sum,
-                                  stream);
+                                  stream, W);
   return linear_dispatch<__nv_bfloat16>(q, k, v, o, B, N, d, st, h_begin, h_count, S_io, z_io, zero_init, global_sum,
-                                        stream);
+                                        stream, W);
 }
 
 cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void* v_cache, int B, int N, int d,
@@ -557,12 +639,13 @@ cudaError_t launch_delay(unsigned int ns, cudaStream_t stream) {
 
 cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void* o, void* k_cache,
                                void* v_cache, float* S, float* z, long long t, long long* t_seq, int B, int H,
-                               int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream) {
+                               int d, int w, int h_sparse, float scale, int dtype, cudaStream_t stream,
+                               const void* W) {
   if (dtype == GF_F32)
     return decode_dispatch<float>(q, k, v, o, k_cache, v_cache, S, z, t, t_seq, B, H, d, w, h_sparse, scale,
-                                  stream);
+                                  stream, W);
   return decode_dispatch<__nv_bfloat16>(q, k, v, o, k_cache, v_cache, S, z, t, t_seq, B, H, d, w, h_sparse, scale,
-                                        stream);
+                                        stream, W);
 }
 
 }  // namespace gf

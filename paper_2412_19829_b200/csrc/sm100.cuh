@@ -313,5 +313,9 @@ EncodeTiledFn get_encode_tiled();
 // Tensor map over a logical [B, H, N, d] bf16 tensor, dims innermost-first {d, N, H, B}, box
 // {64, box_rows, 1, 1}, 128-byte swizzle, out-of-range reads give zeros.
 bool make_qkv_tensor_map(CUtensorMap* map, const void* base, int B, int H, int N, int d, int layout, int box_rows);
+// The same for a contiguous [B, h_count, N, d] tensor that holds heads [h_begin, h_begin + h_count) only,
+// addressed by the call's head coordinate.
+bool make_feature_tensor_map(CUtensorMap* map, const void* base, int B, int H, int N, int d, int h_begin,
+                             int h_count, int box_rows);
 
 }  // namespace gf

@@ -215,8 +215,17 @@ __device__ __forceinline__ uint32_t phi_bf16x2(uint32_t w) {
   return *reinterpret_cast<const uint32_t*>(&f);
 }
 
+// kId: the tensors the kernel reads as Q and K already hold features (positive random features
+// computed by a kernel of their own): the feature map here is the identity.
+template <bool kId>
+__device__ __forceinline__ uint32_t phi_sel(uint32_t w) {
+  if constexpr (kId) return w;
+  else return phi_bf16x2(w);
+}
+
 // phi on 64 rows (four groups of 16 from k8_begin on) x one 16-byte column chunk of a K tile, in
 // place in shared memory (128B swizzle); rows past the end of the sequence become zero.
+template <bool kId>
 __device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane16, int k8_begin, int n_valid) {
   uint4 rawv[4];
 #pragma unroll
@@ -228,10 +237,10 @@ __device__ __forceinline__ void transform_k_rows(uint8_t* kb, int cin, int lane1
   for (int k = 0; k < 4; ++k) {
     const int row = lane16 + 16 * (k8_begin + k);
     const uint32_t keep = (row < n_valid) ? 0xffffffffu : 0u;
-    rawv[k].x = phi_bf16x2(rawv[k].x) & keep;
-    rawv[k].y = phi_bf16x2(rawv[k].y) & keep;
-    rawv[k].z = phi_bf16x2(rawv[k].z) & keep;
-    rawv[k].w = phi_bf16x2(rawv[k].w) & keep;
+    rawv[k].x = phi_sel<kId>(rawv[k].x) & keep;
+    rawv[k].y = phi_sel<kId>(rawv[k].y) & keep;
+    rawv[k].z = phi_sel<kId>(rawv[k].z) & keep;
+    rawv[k].w = phi_sel<kId>(rawv[k].w) & keep;
   }
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
@@ -301,7 +310,7 @@ __device__ __forceinline__ bool publish_inclusive(const LinParams& p, const LinI
   return ok;
 }
 
-template <int D, bool kDirect>
+template <int D, bool kDirect, bool kId>
 __global__ void __launch_bounds__(kThreads, 1)
 linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mk,
                  const __grid_constant__ CUtensorMap mv, const __grid_constant__ CUtensorMap mo,
@@ -769,7 +778,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         ok = ok && mbar_wait(&bar.k_full[sl], (idx / KS) & 1, p.status, 430);
         const int cc = tt >> 4;
         if (ok && tt < 2 * D)
-          transform_k_rows(sK + sl * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
+          transform_k_rows<kId>(sK + sl * C::kTile + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
                            p.N - (it.c_begin + jrow) * 128);
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kd_phi[sl]);
@@ -781,7 +790,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
         ok = ok && mbar_wait(&bar.ka_full[sk], (ta / KA) & 1, p.status, 410);
         const int cc = tt >> 4;  // logical 16-byte column chunk 0 .. D/8-1
         if (ok && tt < 2 * D)
-          transform_k_rows(a_kslot(sk) + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
+          transform_k_rows<kId>(a_kslot(sk) + (cc >> 3) * C::kBoxBytes, cc & 7, tt & 15, kgrp ? 0 : 4,
                            p.N - (it.c_begin + j) * 128);
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(&bar.kphi_full[sk]);  // the tile may go to the tensor core and be parked
@@ -956,7 +965,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
               }
             }
 #pragma unroll
-            for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_bf16x2(pk[w]);
+            for (int w = 0; w < kChunksPerHalf * 4; ++w) pk[w] = phi_sel<kId>(pk[w]);
             if (nq >= QS)  // MMA1/MMA2 of the slot's previous chunk are done with it
               ok = mbar_wait(&bar.qphi_free[sq], ((nq / QS) + 1) & 1, p.status, 401);
             tc_fence_after_sync();
@@ -1232,11 +1241,18 @@ size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
 
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
-                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared) {
+                             int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared,
+                             const void* fq, const void* fk) {
   if (h_count <= 0) return cudaSuccess;
+  // fq, fk: feature tensors [B, h_count, N, d] that stand in for Q and K (feature map: identity)
+  const bool features = fq != nullptr;
   CUtensorMap mq, mk, mv, mo;
-  if (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128) ||
-      !make_qkv_tensor_map(&mv, v, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mo, o, B, H, N, d, layout, 128))
+  if (features ? (!make_feature_tensor_map(&mq, fq, B, H, N, d, h_begin, h_count, 128) ||
+                  !make_feature_tensor_map(&mk, fk, B, H, N, d, h_begin, h_count, 128))
+               : (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) ||
+                  !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128)))
+    return cudaErrorInvalidValue;
+  if (!make_qkv_tensor_map(&mv, v, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mo, o, B, H, N, d, layout, 128))
     return cudaErrorInvalidValue;
   LinParams p;
   p.N = N;
@@ -1277,11 +1293,18 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
     p.seg_base = p.nch / g;
     p.seg_rem = p.nch % g;
     p.nitems = count * g;
+    if (features) {
+      if (d == 64)
+        return direct ? launch(linear_tc_kernel<64, true, true>, LinCfg<64>::kBytes)
+                      : launch(linear_tc_kernel<64, false, true>, LinCfg<64>::kBytes);
+      return direct ? launch(linear_tc_kernel<128, true, true>, LinCfg<128>::kBytes)
+                    : launch(linear_tc_kernel<128, false, true>, LinCfg<128>::kBytes);
+    }
     if (d == 64)
-      return direct ? launch(linear_tc_kernel<64, true>, LinCfg<64>::kBytes)
-                    : launch(linear_tc_kernel<64, false>, LinCfg<64>::kBytes);
-    return direct ? launch(linear_tc_kernel<128, true>, LinCfg<128>::kBytes)
-                  : launch(linear_tc_kernel<128, false>, LinCfg<128>::kBytes);
+      return direct ? launch(linear_tc_kernel<64, true, false>, LinCfg<64>::kBytes)
+                    : launch(linear_tc_kernel<64, false, false>, LinCfg<64>::kBytes);
+    return direct ? launch(linear_tc_kernel<128, true, false>, LinCfg<128>::kBytes)
+                  : launch(linear_tc_kernel<128, false, false>, LinCfg<128>::kBytes);
   };
   // `whole` leading chains uncut (automatic plan only: a segment length asked for by the caller always takes
   // the two-pass form, also when it covers the whole chain), the others cut into G segments behind them

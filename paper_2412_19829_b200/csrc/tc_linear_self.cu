@@ -39,6 +39,13 @@ __device__ __forceinline__ uint32_t phi2(uint32_t w) {
   return *reinterpret_cast<const uint32_t*>(&f);
 }
 
+// kId: the tensors read as Q and K already hold features: the feature map here is the identity.
+template <bool kId>
+__device__ __forceinline__ uint32_t phi_sel(uint32_t w) {
+  if constexpr (kId) return w;
+  else return phi2(w);
+}
+
 struct SelfParams {
   int N, nch, h_begin, h_count, nchains;
   int G, seg_base, seg_rem, nitems;  // segments per chain (balanced lengths), nchains * G
@@ -80,7 +87,7 @@ struct RedCfg {
   static constexpr int kThreads = 22 * 32;
 };
 
-template <int D>
+template <int D, bool kId>
 __global__ void __launch_bounds__(RedCfg<D>::kThreads, 1)
 linear_self_reduce_kernel(const __grid_constant__ CUtensorMap mk, const __grid_constant__ CUtensorMap mv,
                           const SelfParams p) {
@@ -242,10 +249,10 @@ linear_self_reduce_kernel(const __grid_constant__ CUtensorMap mk, const __grid_c
           for (int k = 0; k < 4; ++k) {
             const int row = l16 + 16 * ((grp ? 0 : 4) + k);
             const uint32_t keep = (row < n_valid) ? 0xffffffffu : 0u;  // rows past the end contribute nothing
-            rawv[k].x = phi2(rawv[k].x) & keep;
-            rawv[k].y = phi2(rawv[k].y) & keep;
-            rawv[k].z = phi2(rawv[k].z) & keep;
-            rawv[k].w = phi2(rawv[k].w) & keep;
+            rawv[k].x = phi_sel<kId>(rawv[k].x) & keep;
+            rawv[k].y = phi_sel<kId>(rawv[k].y) & keep;
+            rawv[k].z = phi_sel<kId>(rawv[k].z) & keep;
+            rawv[k].w = phi_sel<kId>(rawv[k].w) & keep;
             *reinterpret_cast<uint4*>(kb + row * 128 + ((cin ^ (row & 7)) << 4)) = rawv[k];
           }
           fence_proxy_async_smem();
@@ -295,7 +302,7 @@ struct OutCfg {
   static constexpr int kThreads = 15 * 32;
 };
 
-template <int D>
+template <int D, bool kId>
 __global__ void __launch_bounds__(OutCfg<D>::kThreads, 1)
 linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__ CUtensorMap mo,
                            const SelfParams p) {
@@ -486,7 +493,7 @@ linear_self_readout_kernel(const __grid_constant__ CUtensorMap mq, const __grid_
         if (ok && lane == 0) mbar_arrive(&q_free[s]);  // this warp has its part of the raw tile in registers
         if (ok) {
 #pragma unroll
-          for (int w = 0; w < kChunks * 4; ++w) pk[w] = phi2(pk[w]);
+          for (int w = 0; w < kChunks * 4; ++w) pk[w] = phi_sel<kId>(pk[w]);
           if (nq >= 2) ok = mbar_wait(&tq_free[s], ((nq >> 1) + 1) & 1, p.status, 831);
         }
         tc_fence_after_sync();
@@ -568,11 +575,17 @@ size_t linear_self_workspace_bytes(int nchains, int N, int d) {
 
 cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                                   int layout, int h_begin, int h_count, WsHeader* ws, size_t scratch_offset,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, const void* fq, const void* fk) {
   if (h_count <= 0) return cudaSuccess;
+  // fq, fk: feature tensors [B, h_count, N, d] that stand in for Q and K (feature map: identity)
+  const bool features = fq != nullptr;
   CUtensorMap mq, mk, mv, mo;
-  if (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128) ||
-      !make_qkv_tensor_map(&mv, v, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mo, o, B, H, N, d, layout, 128))
+  if (features ? (!make_feature_tensor_map(&mq, fq, B, H, N, d, h_begin, h_count, 128) ||
+                  !make_feature_tensor_map(&mk, fk, B, H, N, d, h_begin, h_count, 128))
+               : (!make_qkv_tensor_map(&mq, q, B, H, N, d, layout, 128) ||
+                  !make_qkv_tensor_map(&mk, k, B, H, N, d, layout, 128)))
+    return cudaErrorInvalidValue;
+  if (!make_qkv_tensor_map(&mv, v, B, H, N, d, layout, 128) || !make_qkv_tensor_map(&mo, o, B, H, N, d, layout, 128))
     return cudaErrorInvalidValue;
   SelfParams p;
   p.N = N;
@@ -605,15 +618,23 @@ cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, v
     kern<<<grid, threads, smem, stream>>>(mq, mo, p);
     return cudaSuccess;
   };
-  e = (d == 64) ? launch_red(linear_self_reduce_kernel<64>, RedCfg<64>::kBytes, RedCfg<64>::kThreads)
-                : launch_red(linear_self_reduce_kernel<128>, RedCfg<128>::kBytes, RedCfg<128>::kThreads);
+  if (features)
+    e = (d == 64) ? launch_red(linear_self_reduce_kernel<64, true>, RedCfg<64>::kBytes, RedCfg<64>::kThreads)
+                  : launch_red(linear_self_reduce_kernel<128, true>, RedCfg<128>::kBytes, RedCfg<128>::kThreads);
+  else
+    e = (d == 64) ? launch_red(linear_self_reduce_kernel<64, false>, RedCfg<64>::kBytes, RedCfg<64>::kThreads)
+                  : launch_red(linear_self_reduce_kernel<128, false>, RedCfg<128>::kBytes, RedCfg<128>::kThreads);
   if (e != cudaSuccess) return e;
   note_launch();
   linear_self_sum_kernel<<<dim3((state_floats / 4 + 255) / 256, p.nchains), 256, 0, stream>>>(p.partial, p.total, p.G,
                                                                                               state_floats);
   note_launch();
-  e = (d == 64) ? launch_out(linear_self_readout_kernel<64>, OutCfg<64>::kBytes, OutCfg<64>::kThreads)
-                : launch_out(linear_self_readout_kernel<128>, OutCfg<128>::kBytes, OutCfg<128>::kThreads);
+  if (features)
+    e = (d == 64) ? launch_out(linear_self_readout_kernel<64, true>, OutCfg<64>::kBytes, OutCfg<64>::kThreads)
+                  : launch_out(linear_self_readout_kernel<128, true>, OutCfg<128>::kBytes, OutCfg<128>::kThreads);
+  else
+    e = (d == 64) ? launch_out(linear_self_readout_kernel<64, false>, OutCfg<64>::kBytes, OutCfg<64>::kThreads)
+                  : launch_out(linear_self_readout_kernel<128, false>, OutCfg<128>::kBytes, OutCfg<128>::kThreads);
   if (e != cudaSuccess) return e;
   note_launch();
   return cudaGetLastError();

@@ -305,7 +305,8 @@ def test_self_layer_argument_errors():
     assert call(w=0) == gf.GF_ERR_INVALID_ARG
     assert call(h_sparse=5) == gf.GF_ERR_INVALID_ARG
     assert call(d=96) == gf.GF_ERR_UNSUPPORTED
-    assert call(phi=1) == gf.GF_ERR_UNSUPPORTED
+    assert call(phi=1) == gf.GF_ERR_INVALID_ARG  # positive random features need their projections: the _w entry point
+    assert call(phi=7) == gf.GF_ERR_UNSUPPORTED
     assert call(ws_bytes=8) == gf.GF_ERR_WORKSPACE
     assert call(ws=0) == gf.GF_ERR_WORKSPACE
     # the bidirectional layer's segment sums fit the workspace the size query reports
@@ -331,3 +332,30 @@ def test_partition_from_times_against_the_oracle():
     for bad in ((0, H, N, E, W, tw, tl), (B, H, N, E, W, 0.0, tl), (B, H, N, E, W, tw, float("inf"))):
         with pytest.raises(gf.GformerError):
             gf.partition_from_times(*bad)
+
+
+def test_feature_map_argument_errors():
+    # the positive random features (Sec. III-A / III-C) come with a projection pointer; elu + 1 must not have one
+    L = gf.lib()
+    q, k, v, o, ws, W = FAKE, FAKE + (1 << 30), FAKE + (2 << 30), FAKE + (3 << 30), FAKE + (4 << 30), FAKE + (5 << 30)
+    big = 1 << 30
+    lin = lambda phi, Wp: L.gformer_causal_linear_attn_w(q, k, v, o, 1, 4, 64, 64, phi, Wp, 0, None, None, gf.GF_BF16, 0,
+                                                         ws, big, None)
+    assert lin(gf.GF_PHI_FAVOR_POS, None) == gf.GF_ERR_INVALID_ARG
+    assert lin(gf.GF_PHI_ELU1, W) == gf.GF_ERR_INVALID_ARG
+    assert lin(gf.GF_PHI_FAVOR_POS, W + 4) == gf.GF_ERR_INVALID_ARG  # misaligned
+    assert lin(5, W) == gf.GF_ERR_UNSUPPORTED
+    hyb = lambda phi, Wp: L.gformer_hybrid_attn_w(q, k, v, o, 1, 4, 64, 64, 32, 1, 0.0, phi, Wp, 0, gf.GF_BF16, 0, None,
+                                                  ws, big, None)
+    assert hyb(gf.GF_PHI_FAVOR_POS, None) == gf.GF_ERR_INVALID_ARG
+    assert hyb(gf.GF_PHI_ELU1, W) == gf.GF_ERR_INVALID_ARG
+    st = gf.DecodeStateC(FAKE, FAKE, FAKE, FAKE, 0, 2, 4, 64, 32, 1, gf.GF_BF16)
+    assert L.gformer_decode_step_w(q, k, v, o, ctypes.byref(st), 0.0, gf.GF_PHI_FAVOR_POS, None, None) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_decode_step(q, k, v, o, ctypes.byref(st), 0.0, gf.GF_PHI_FAVOR_POS, None) == gf.GF_ERR_INVALID_ARG
+    assert st.t == 0
+    # the features of Q and K live in the workspace on the tensor-core path: two bf16 tensors of the linear heads
+    B, H, N, d, h0 = 2, 8, 4096, 128, 2
+    plain = gf.workspace_bytes(B, H, N, d, 1, h0, gf.GF_BF16)
+    favor = gf.workspace_bytes(B, H, N, d, 1, h0, gf.GF_BF16, gf.GF_PHI_FAVOR_POS)
+    assert favor >= plain + 2 * B * (H - h0) * N * d * 2
+    assert hyb(gf.GF_PHI_FAVOR_POS, W) in (gf.GF_OK, gf.GF_ERR_CUDA)  # arguments are fine (no device here: the launch fails)

@@ -937,3 +937,106 @@ def test_a_wait_that_runs_out_is_reported_and_the_next_call_is_fine():
     o = gf.causal_linear_attn(qd, kd, vd, ws=ws)
     assert ws.last_device_status() == gf.GF_OK
     assert_parity(f64(o), ref, "bf16", "call after a timed-out one")
+
+
+# ------------------------------------------------------------------ positive random features (Sec. III-A / III-C)
+def _proj(heads, d, dtype, seed):
+    return synth.favor_projection(heads, d, seed=seed, orthogonal=True, dtype="f32" if dtype == "f32" else "bf16")
+
+
+def assert_parity_by_scale(got, ref, kind, what):
+    """The gates on outputs brought to unit scale.  The absolute gates are stated for the benchmark's inputs
+    (N(0,1)/sqrt(d): outputs well below 1).  Under the unscaled stress distribution these feature maps give
+    peaked attention, so an output row is close to single value rows of size 2 to 4, where one bf16
+    rounding of the output alone is up to 8e-3 or 1.6e-2: the absolute gates are then applied to
+    got / s and ref / s with s = max(1, max |ref|); the relative-L2 gate is unchanged by s."""
+    s = max(1.0, float(np.abs(ref).max()))
+    return assert_parity(got / s, ref / s, kind, what)
+
+
+@pytest.mark.parametrize("gain", [None, 1.0])
+@pytest.mark.parametrize("N,d", [(128, 64), (300, 128), (1000, 64), (4096, 128), (4001, 64)])
+def test_favor_causal_linear_tensor_core(N, d, gain):
+    B, H = 2, 3
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=300 + N + d, gain=gain)
+    W = _proj(H, d, "bf16", seed=N + d)
+    S_ref, z_ref = np.zeros((B, H, d, d)), np.zeros((B, H, d))
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v), S_ref, z_ref, W=f64(W))
+    S, z = torch.zeros(B, H, d, d, device="cuda"), torch.zeros(B, H, d, device="cuda")
+    ws = gf.Workspace.for_problem(B, H, N, d, 1, 0, phi=gf.GF_PHI_FAVOR_POS)
+    o = gf.causal_linear_attn(*dev(q, k, v), S, z, W=W.cuda(), ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    (assert_parity if gain is None else assert_parity_by_scale)(f64(o), ref, "bf16", f"favor linear N={N} d={d} gain={gain}")
+    assert errors(f64(S), S_ref)["rel_l2"] <= 1e-2 and errors(f64(z), z_ref)["rel_l2"] <= 1e-2
+
+
+@pytest.mark.parametrize("split", [-1, 2])
+def test_favor_causal_linear_both_forms_and_bnhd(split):
+    # whole chains (one-pass form) and chains cut into segments, under the [B, N, H, d] layout
+    B, H, N, d = 2, 4, 1500, 128
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=812)
+    W = _proj(H, d, "bf16", seed=813)
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v), W=f64(W))
+    ins = [t.permute(0, 2, 1, 3).contiguous().cuda() for t in (q, k, v)]
+    ws = gf.Workspace.for_problem(B, H, N, d, 1, 0, phi=gf.GF_PHI_FAVOR_POS)
+    o = gf.causal_linear_attn(*ins, W=W.cuda(), layout=gf.GF_BNHD, ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    assert_parity(f64(o.permute(0, 2, 1, 3)), ref, "bf16", f"favor linear bnhd split={split}")
+
+
+@pytest.mark.parametrize("dtype,force_simt", [("f32", 0), ("bf16", 1)])
+@pytest.mark.parametrize("N,d", [(1, 64), (130, 64), (300, 128)])
+def test_favor_causal_linear_cuda_core_path(dtype, force_simt, N, d):
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, force_simt)
+    B, H = 1, 2
+    q, k, v = synth.qkv(B, H, N, d, dtype, seed=820 + N)
+    W = _proj(H, d, dtype, seed=821)
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v), W=f64(W))
+    o = gf.causal_linear_attn(*dev(q, k, v), W=W.cuda())
+    assert_parity(f64(o), ref, kind_of(dtype), f"favor linear cuda cores {dtype} N={N} d={d}")
+
+
+@pytest.mark.parametrize("B,H,N,d,w,h0", [(2, 4, 700, 64, 100, 1), (1, 8, 2048, 128, 256, 2), (2, 3, 333, 128, 64, 0)])
+def test_favor_hybrid_layer_prefill_then_decode(B, H, N, d, w, h0):
+    steps = 6
+    q, k, v = synth.qkv(B, H, N + steps, d, "bf16", seed=830 + N, gain=1.0 if d == 64 else None)
+    W = _proj(H - h0, d, "bf16", seed=831)
+    ref = oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0, W=f64(W))
+    qd, kd, vd = dev(q, k, v)
+    Wd = W.cuda()
+    st = gf.DecodeState(B, H, d, w, h0)
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0, phi=gf.GF_PHI_FAVOR_POS)
+    o = gf.hybrid_attn(qd[:, :, :N].contiguous(), kd[:, :, :N].contiguous(), vd[:, :, :N].contiguous(), w,
+                       h_sparse=h0, state_out=st, W=Wd, ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    check = assert_parity_by_scale if d == 64 else assert_parity  # d = 64 runs the unscaled stress distribution
+    check(f64(o), ref[:, :, :N], "bf16", "favor hybrid prefill")
+    for t in range(N, N + steps):
+        ot = gf.decode_step(qd[:, :, t].contiguous(), kd[:, :, t].contiguous(), vd[:, :, t].contiguous(), st, W=Wd)
+        check(f64(ot), ref[:, :, t], "bf16", f"favor decode step {t - N}")
+
+
+@pytest.mark.parametrize("B,H,N,d,w,h0", [(1, 4, 1000, 128, 128, 1), (2, 3, 300, 64, 40, 1), (1, 2, 4096, 64, 64, 0)])
+def test_favor_self_layer(B, H, N, d, w, h0):
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=840 + N)
+    W = _proj(H - h0, d, "bf16", seed=841)
+    ref = oracle.hybrid_attn_self(f64(q), f64(k), f64(v), w, h_sparse=h0, W=f64(W))
+    ws = gf.Workspace.for_problem(B, H, N, d, w, h0, phi=gf.GF_PHI_FAVOR_POS)
+    o = gf.hybrid_attn_self(*dev(q, k, v), w, h_sparse=h0, W=W.cuda(), ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    assert_parity(f64(o), ref, "bf16", "favor self layer")
+
+
+def test_favor_is_not_elu_and_needs_its_projection():
+    B, H, N, d = 1, 2, 256, 64
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=850, gain=1.0)
+    W = _proj(H, d, "bf16", seed=851)
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v), W=f64(W))
+    o_elu = gf.causal_linear_attn(*dev(q, k, v))
+    assert not passes(f64(o_elu), ref, "bf16")  # negative control: the other feature map fails the gates
+    qd = q.cuda()
+    rc = gf.lib().gformer_causal_linear_attn(qd.data_ptr(), qd.data_ptr(), qd.data_ptr(), torch.empty_like(qd).data_ptr(),
+                                             B, H, N, d, gf.GF_PHI_FAVOR_POS, 0, None, None, gf.GF_BF16, gf.GF_BHND,
+                                             gf.Workspace(1 << 20).ptr, 1 << 20, None)
+    assert rc == gf.GF_ERR_INVALID_ARG
