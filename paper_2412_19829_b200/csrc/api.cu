@@ -35,6 +35,7 @@ Tuning tuning_now() {
 }
 
 constexpr int kMaxDevices = 64;
+constexpr unsigned int kPlacedWaitNs = 20000;  // longest the windowed heads are held back for the linear kernel's CTAs
 struct Fork {
   cudaStream_t side = nullptr, first = nullptr;  // lowest / highest stream priority
   cudaEvent_t fork = nullptr, join = nullptr, join_first = nullptr;
@@ -133,7 +134,7 @@ int check_phi(int phi, const void* W) {
 
 int run_linear(const Tuning& tn, const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d, int dtype,
                int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init, int max_ctas,
-               WsHeader* ws, cudaStream_t stream, bool shared = false, const Phi& phi = Phi()) {
+               WsHeader* ws, cudaStream_t stream, bool shared = false, const Phi& phi = Phi(), int* first_grid = nullptr) {
   if (h_count <= 0) return GF_OK;
   if (!tn.force_simt && gf::tc_linear_supported(N, d, dtype)) {
     void *fq = nullptr, *fk = nullptr;
@@ -145,7 +146,7 @@ int run_linear(const Tuning& tn, const void* q, const void* k, const void* v, vo
       if (rc != GF_OK) return rc;
     }
     return cuda_status(gf::launch_linear_tc(q, k, v, o, B, H, N, d, layout, h_begin, h_count, S_io, z_io,
-                                            zero_init, tn.linear_split, max_ctas, ws, stream, shared, fq, fk));
+                                            zero_init, tn.linear_split, max_ctas, ws, stream, shared, fq, fk, first_grid));
   }
   return cuda_status(gf::launch_linear_simt(q, k, v, o, B, N, d, dtype, gf::make_strides(layout, H, N, d),
                                             h_begin, h_count, S_io, z_io, zero_init, stream, false, phi.W));
@@ -361,12 +362,16 @@ int gformer_hybrid_attn_self_w(const void* q, const void* k, const void* v, void
     if (fq != nullptr)
       rc = cuda_status(gf::launch_favor_features_tc(q, k, W, fq, fk, B, H, N, d, layout, h_sparse, H - h_sparse,
                                                     (WsHeader*)ws, f->first));
+    int lin_grid = 0;
     if (rc == GF_OK)
       rc = cuda_status(gf::launch_linear_self_tc(q, k, v, o, B, H, N, d, layout, h_sparse, H - h_sparse, (WsHeader*)ws,
-                                                 sizeof(WsHeader), f->first, fq, fk));
+                                                 sizeof(WsHeader), f->first, fq, fk, &lin_grid));
     if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
-    int rc2 = cuda_status(gf::launch_delay(8000, f->side));
+    // the windowed heads start once the CTAs of the first linear kernel have all started
+    int rc2 = (rc == GF_OK && lin_grid > 0)
+                  ? cuda_status(gf::launch_wait_placed((WsHeader*)ws, (unsigned int)lin_grid, kPlacedWaitNs, f->side))
+                  : GF_OK;
     if (rc2 == GF_OK)
       rc2 = run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, f->side, true);
     if (cudaEventRecord(f->join, f->side) != cudaSuccess) return GF_ERR_CUDA;
@@ -469,8 +474,7 @@ int gformer_hybrid_attn_w(const void* q, const void* k, const void* v, void* o, 
     int L = 0, G = 0, whole = 0, dev = 0, sms = 0;
     gf::linear_tc_plan_parts(B * h_lin, N, d, tn.linear_split, 0, &whole, &L, &G, true);
     if (whole > 0) G = 1;  // items of the first launch: the chains left whole
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-      return GF_ERR_CUDA;
+    if (gf::device_info(&dev, &sms) != cudaSuccess) return GF_ERR_CUDA;
     if ((long long)B * h_lin * G >= sms) {
       lin_ctas = (tn.linear_ctas > 0 && tn.linear_ctas < sms) ? tn.linear_ctas : sms;
     }
@@ -489,8 +493,9 @@ int gformer_hybrid_attn_w(const void* q, const void* k, const void* v, void* o, 
   // (the caller's stream may well have the lowest, like the side stream).
   const bool lin_first = both && lin_ctas > 0;
   if (lin_first && cudaStreamWaitEvent(f->first, f->fork, 0) != cudaSuccess) return GF_ERR_CUDA;
+  int lin_grid = 0;
   rc = run_linear(tn, q, k, v, o, B, H, N, d, dtype, layout, h_sparse, h_lin, S_out, z_out, true, lin_ctas,
-                  (WsHeader*)ws, lin_first ? f->first : stream, both, fm);
+                  (WsHeader*)ws, lin_first ? f->first : stream, both, fm, &lin_grid);
   if (lin_first) {
     if (cudaEventRecord(f->join_first, f->first) != cudaSuccess) return GF_ERR_CUDA;
     if (cudaStreamWaitEvent(stream, f->join_first, 0) != cudaSuccess) return GF_ERR_CUDA;
@@ -498,9 +503,11 @@ int gformer_hybrid_attn_w(const void* q, const void* k, const void* v, void* o, 
   cudaStream_t wstream = both ? f->side : stream;
   // Both kernels become runnable at the fork.  CTAs of the persistent linear kernel wait for one
   // another and want every SM from the start, while a windowed-heads CTA that got onto an SM first
-  // keeps it for many tiles: hold the side stream back for a few microseconds, until the linear
-  // kernel's CTAs have been placed.
-  if (lin_first && cuda_status(gf::launch_delay(8000, wstream)) != GF_OK) return GF_ERR_CUDA;
+  // keeps it for many tiles: the side stream is held back until the linear kernel's CTAs have all
+  // started (they count themselves in the workspace header), 20 microseconds at most.
+  if (lin_first && rc == GF_OK && lin_grid > 0 &&
+      cuda_status(gf::launch_wait_placed((WsHeader*)ws, (unsigned int)lin_grid, kPlacedWaitNs, wstream)) != GF_OK)
+    return GF_ERR_CUDA;
   int rc2 = run_window(tn, q, k, v, o, B, H, N, d, w, scale, dtype, layout, 0, h_sparse, (WsHeader*)ws, wstream);
   if (rc2 == GF_OK && state_out && h_sparse > 0)
     rc2 = cuda_status(gf::launch_export_ring(k, v, state_out->k_cache, state_out->v_cache, B, N, d, w, dtype,

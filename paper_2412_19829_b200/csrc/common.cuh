@@ -36,7 +36,8 @@ struct WsHeader {
   unsigned int ticket;   // work counter of the persistent kernels
   unsigned int wait_kcycles;  // limit of every bounded wait in units of 1024 cycles; 0 = default (about 2 s)
   unsigned int drop_flag;     // failure injection for tests: the linear kernel skips the flag of segment n - 1
-  unsigned int pad[59];
+  unsigned int placed;        // CTAs of the call's linear-attention kernels that have started (see launch_wait_placed)
+  unsigned int pad[58];
 };
 static_assert(sizeof(WsHeader) == 256, "workspace header is 256 bytes");
 
@@ -67,9 +68,16 @@ cudaError_t launch_decode_step(const void* q, const void* k, const void* v, void
 // Writes the two test knobs into a workspace header that has just been cleared.
 cudaError_t launch_set_header(WsHeader* ws, unsigned int wait_kcycles, unsigned int drop_flag, cudaStream_t stream);
 
-// One tiny CTA that returns after about `ns` nanoseconds: holds back the work queued behind it
-// in its stream without occupying an SM's shared memory or tensor memory.
-cudaError_t launch_delay(unsigned int ns, cudaStream_t stream);
+// One tiny CTA that returns once `target` CTAs of the call's linear-attention kernel have started
+// (WsHeader::placed), or after max_ns nanoseconds whichever comes first: holds back the work queued
+// behind it in its stream without occupying an SM's shared memory or tensor memory.  Never an error:
+// when the limit ends the wait, the work behind it simply starts.
+cudaError_t launch_wait_placed(WsHeader* ws, unsigned int target, unsigned int max_ns, cudaStream_t stream);
+
+// The current device and its SM count (asked of the driver once per device).
+cudaError_t device_info(int* dev, int* sms);
+// cudaFuncAttributeMaxDynamicSharedMemorySize of a kernel, set once per kernel and device.
+cudaError_t ensure_dynamic_smem(const void* kernel, int dev, int bytes);
 
 // ---- tensor-core (tcgen05 / TMEM / TMA) path: bf16 storage, d in {64,128}.
 bool tc_window_supported(int N, int d, int w, int dtype);
@@ -82,7 +90,8 @@ cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* 
 size_t linear_self_workspace_bytes(int nchains, int N, int d);
 cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                                   int layout, int h_begin, int h_count, WsHeader* ws, size_t scratch_offset,
-                                  cudaStream_t stream, const void* fq = nullptr, const void* fk = nullptr);
+                                  cudaStream_t stream, const void* fq = nullptr, const void* fk = nullptr,
+                                  int* first_grid = nullptr /* CTAs of the first launch */);
 // Segmentation used by the tensor-core linear kernel (split: 0 = automatic, else chunks per segment;
 // ctas: CTAs the kernel will run with, 0 = one per SM of a B200) and the scratch it needs beyond
 // the workspace header (sized for the largest segment count the plan may pick for any ctas).
@@ -100,7 +109,8 @@ size_t linear_tc_flag_bytes(int nchains, int N, int split);
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
                              int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared = false,
-                             const void* fq = nullptr, const void* fk = nullptr);
+                             const void* fq = nullptr, const void* fk = nullptr,
+                             int* first_grid = nullptr /* CTAs of the first launch */);
 // Positive random features phi_W of Q and K of heads [h_begin, h_begin + h_count) (bf16 storage) into the
 // contiguous bf16 tensors fq, fk [B, h_count, N, d]; W: [h_count, d, d] bf16, row a of a head's matrix is
 // its projection vector w_a.  With fq, fk given, the two linear-attention launchers read them in place

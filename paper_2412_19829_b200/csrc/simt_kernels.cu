@@ -609,13 +609,16 @@ cudaError_t launch_export_ring(const void* k, const void* v, void* k_cache, void
 }
 
 namespace {
-__global__ void delay_kernel(unsigned int ns) {
+__global__ void wait_placed_kernel(const unsigned int* placed, unsigned int target, unsigned int max_ns) {
   unsigned long long t0, t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
   for (int i = 0; i < 100000; ++i) {  // bounded whatever the timer does
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(placed) : "memory");
+    if (v >= target) break;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    if (t - t0 >= ns) break;
-    __nanosleep(200);
+    if (t - t0 >= max_ns) break;
+    __nanosleep(100);
   }
 }
 }  // namespace
@@ -631,8 +634,8 @@ cudaError_t launch_set_header(WsHeader* ws, unsigned int wait_kcycles, unsigned 
   return cudaGetLastError();
 }
 
-cudaError_t launch_delay(unsigned int ns, cudaStream_t stream) {
-  delay_kernel<<<1, 32, 0, stream>>>(ns);
+cudaError_t launch_wait_placed(WsHeader* ws, unsigned int target, unsigned int max_ns, cudaStream_t stream) {
+  wait_placed_kernel<<<1, 1, 0, stream>>>(&ws->placed, target, max_ns);
   note_launch();
   return cudaGetLastError();
 }

@@ -173,7 +173,9 @@ cudaError_t launch_favor_features_tc(const void* q, const void* k, const void* W
   if (rows > 65535) return cudaErrorInvalidValue;
   dim3 grid((unsigned)((N + 127) / 128), (unsigned)rows, 2);
   auto launch = [&](auto kern, int smem) -> cudaError_t {
-    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    int dev = 0, sms = 0;
+    cudaError_t err = device_info(&dev, &sms);
+    if (err == cudaSuccess) err = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), dev, smem);
     if (err != cudaSuccess) return err;
     kern<<<grid, kFavorThreads, smem, stream>>>(mxq, mxk, mw, mfq, mfk, p);
     note_launch();

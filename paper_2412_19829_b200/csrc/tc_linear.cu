@@ -336,6 +336,7 @@ linear_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
+    atomicAdd(&p.status[5], 1u);  // WsHeader::placed: this CTA has an SM
     mbar_init(&bar.q_full[0], 1);
     mbar_init(&bar.q_full[1], 1);
     for (int s = 0; s < 5; ++s) {
@@ -1242,7 +1243,8 @@ size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
                              int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared,
-                             const void* fq, const void* fk) {
+                             const void* fq, const void* fk, int* first_grid) {
+  if (first_grid) *first_grid = 0;
   if (h_count <= 0) return cudaSuccess;
   // fq, fk: feature tensors [B, h_count, N, d] that stand in for Q and K (feature map: identity)
   const bool features = fq != nullptr;
@@ -1262,8 +1264,7 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   const int nchains = B * h_count;
   int dev = 0, sms = 0;
   cudaError_t e;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = device_info(&dev, &sms)) != cudaSuccess) return e;
   // One CTA per SM at most: every CTA must be resident for the segment hand-over to make progress.
   // (max_ctas > 0 leaves SMs to a kernel running beside this one.)
   if (max_ctas > 0 && max_ctas < sms) sms = max_ctas;
@@ -1277,9 +1278,10 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
   p.flags = reinterpret_cast<unsigned int*>(scratch);  // zeroed by the caller
   p.prefix = reinterpret_cast<float*>(scratch + linear_tc_flag_bytes(nchains, N, split));
   auto launch = [&](auto kern, size_t smem) -> cudaError_t {
-    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), dev, (int)smem);
     if (err != cudaSuccess) return err;
     dim3 grid(p.nitems < sms ? p.nitems : sms);
+    if (first_grid && *first_grid == 0) *first_grid = (int)grid.x;
     kern<<<grid, kThreads, smem, stream>>>(mq, mk, mv, mo, p);
     note_launch();
     return cudaGetLastError();

@@ -102,6 +102,7 @@ linear_self_reduce_kernel(const __grid_constant__ CUtensorMap mk, const __grid_c
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
+    atomicAdd(&p.status[5], 1u);  // WsHeader::placed: this CTA has an SM
     for (int i = 0; i < KS; ++i) {
       mbar_init(&k_full[i], 1);
       mbar_init(&kphi[i], 16);
@@ -575,7 +576,8 @@ size_t linear_self_workspace_bytes(int nchains, int N, int d) {
 
 cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                                   int layout, int h_begin, int h_count, WsHeader* ws, size_t scratch_offset,
-                                  cudaStream_t stream, const void* fq, const void* fk) {
+                                  cudaStream_t stream, const void* fq, const void* fk, int* first_grid) {
+  if (first_grid) *first_grid = 0;
   if (h_count <= 0) return cudaSuccess;
   // fq, fk: feature tensors [B, h_count, N, d] that stand in for Q and K (feature map: identity)
   const bool features = fq != nullptr;
@@ -603,17 +605,17 @@ cudaError_t launch_linear_self_tc(const void* q, const void* k, const void* v, v
   p.status = &ws->status;
   int dev = 0, sms = 0;
   cudaError_t e;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+  if ((e = device_info(&dev, &sms)) != cudaSuccess) return e;
   dim3 grid(p.nitems < sms ? p.nitems : sms);
+  if (first_grid) *first_grid = (int)grid.x;
   auto launch_red = [&](auto kern, int smem, int threads) -> cudaError_t {
-    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), dev, smem);
     if (err != cudaSuccess) return err;
     kern<<<grid, threads, smem, stream>>>(mk, mv, p);
     return cudaSuccess;
   };
   auto launch_out = [&](auto kern, int smem, int threads) -> cudaError_t {
-    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), dev, smem);
     if (err != cudaSuccess) return err;
     kern<<<grid, threads, smem, stream>>>(mq, mo, p);
     return cudaSuccess;

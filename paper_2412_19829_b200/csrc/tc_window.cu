@@ -551,19 +551,6 @@ window_tc_kernel(const __grid_constant__ CUtensorMap mq, const __grid_constant__
   if (warp == kWarpMma) tmem_dealloc(tmem, 512);
 }
 
-// Per device: the SM count, and whether a kernel instantiation already has its shared-memory limit.
-constexpr int kMaxDev = 64;
-int g_sms[kMaxDev];
-template <int D, bool kTwoSided>
-cudaError_t prepare_kernel(int dev) {
-  static bool done[kMaxDev];
-  if (done[dev]) return cudaSuccess;
-  cudaError_t e = cudaFuncSetAttribute(window_tc_kernel<D, kTwoSided>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       WinSmem<D>::kBytes);
-  if (e == cudaSuccess) done[dev] = true;
-  return e;
-}
-
 }  // namespace
 
 bool tc_window_supported(int N, int d, int w, int dtype) {
@@ -596,30 +583,23 @@ cudaError_t launch_window_tc(const void* q, const void* k, const void* v, void* 
   p.total = (int)total;
   p.status = &ws->status;
   p.ticket = &ws->ticket;  // zeroed with the workspace header by the caller
-  int dev = 0;
+  int dev = 0, sms = 0;
   cudaError_t e;
-  if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
-  if (dev < 0 || dev >= kMaxDev) return cudaErrorInvalidDevice;
-  if (g_sms[dev] == 0) {
-    int sms = 0;
-    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-    g_sms[dev] = sms;
-  }
+  if ((e = device_info(&dev, &sms)) != cudaSuccess) return e;
   // one persistent CTA per SM (it takes the SM's whole tensor memory); CTAs never wait for one
   // another, so it does not matter how many of them are resident at a time
-  const int sms = g_sms[dev];
   dim3 grid((unsigned)(total < sms ? total : sms));
-  auto launch = [&](auto kern, cudaError_t prepared, int smem) -> cudaError_t {
-    if (prepared != cudaSuccess) return prepared;
+  auto launch = [&](auto kern, int smem) -> cudaError_t {
+    cudaError_t err = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), dev, smem);
+    if (err != cudaSuccess) return err;
     kern<<<grid, kThreads, smem, stream>>>(mq, mk, mv, mo, p);
     return cudaSuccess;
   };
   if (d == 64)
-    e = fwd > 0 ? launch(window_tc_kernel<64, true>, prepare_kernel<64, true>(dev), WinSmem<64>::kBytes)
-                : launch(window_tc_kernel<64, false>, prepare_kernel<64, false>(dev), WinSmem<64>::kBytes);
+    e = fwd > 0 ? launch(window_tc_kernel<64, true>, WinSmem<64>::kBytes) : launch(window_tc_kernel<64, false>, WinSmem<64>::kBytes);
   else
-    e = fwd > 0 ? launch(window_tc_kernel<128, true>, prepare_kernel<128, true>(dev), WinSmem<128>::kBytes)
-                : launch(window_tc_kernel<128, false>, prepare_kernel<128, false>(dev), WinSmem<128>::kBytes);
+    e = fwd > 0 ? launch(window_tc_kernel<128, true>, WinSmem<128>::kBytes)
+                : launch(window_tc_kernel<128, false>, WinSmem<128>::kBytes);
   if (e != cudaSuccess) return e;
   note_launch();
   return cudaGetLastError();
