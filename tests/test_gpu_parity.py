@@ -283,6 +283,48 @@ def test_hybrid_with_whole_and_cut_linear_chains_and_state_export():
     assert errors(f64(st.z[:, idx].cpu()), zr)["rel_l2"] <= 1e-2
 
 
+@pytest.mark.parametrize("d", [64, 128])
+def test_linear_chunk_size_invariance(d):
+    """Algorithm 1 regrouped in different ways gives the same values up to rounding: token by token
+    (the CUDA-core path: a chunk of one row), 128 rows at a time with every chain whole, and 128-row
+    chunks in segments of 1, 2 and 5 chunks with the state handed over between CTAs.  (128 is the only
+    chunk height of the tensor-core path -- the M of a one-CTA tcgen05 product -- so the `chunk` argument
+    takes 0 or 128 and answers GF_ERR_UNSUPPORTED to 64 and 256; what varies is the regrouping around it.)"""
+    B, H, N = 2, 3, 10 * 128 - 37
+    q, k, v = synth.qkv(B, H, N, d, "bf16", seed=640 + d, gain=1.0)
+    S_ref, z_ref = np.zeros((B, H, d, d)), np.zeros((B, H, d))
+    ref = oracle.causal_linear_attn(f64(q), f64(k), f64(v), S_ref, z_ref)
+    outs, states = {}, {}
+
+    def run(name):
+        S = torch.zeros(B, H, d, d, device="cuda"); z = torch.zeros(B, H, d, device="cuda")
+        ws = gf.Workspace.for_problem(B, H, N, d, 1, 0)
+        o = gf.causal_linear_attn(*dev(q, k, v), S, z, chunk=128, ws=ws)
+        assert ws.last_device_status() == gf.GF_OK
+        assert_parity(f64(o), ref, "bf16", f"linear d={d} regrouping {name}")
+        assert errors(f64(S), S_ref)["rel_l2"] <= 1e-2 and errors(f64(z), z_ref)["rel_l2"] <= 1e-2
+        outs[name], states[name] = f64(o), f64(S)
+
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 1)
+    run("token by token")
+    gf.set_tuning(gf.GF_TUNE_FORCE_SIMT, 0)
+    for split, name in ((-1, "whole chains"), (1, "segments of 1"), (2, "segments of 2"), (5, "segments of 5")):
+        gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
+        run(name)
+    base = outs["whole chains"]
+    for name, o in outs.items():
+        assert errors(o, base)["max_abs"] <= 2e-2, name
+        # (the tensor-core forms round phi(K) to bf16 before the products, the token-wise form keeps fp32:
+        # their states differ by that rounding, a few 1e-3; among the tensor-core forms far less)
+        assert errors(states[name], states["whole chains"])["rel_l2"] <= (5e-3 if name == "token by token" else 1e-3), name
+    # other chunk heights are refused, not silently replaced
+    ws = gf.Workspace.for_problem(B, H, N, d, 1, 0)
+    for chunk in (64, 256):
+        with pytest.raises(gf.GformerError) as e:
+            gf.causal_linear_attn(*dev(q, k, v), chunk=chunk, ws=ws)
+        assert e.value.status == gf.GF_ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("split", [1, 2, 4])
 def test_linear_tensor_core_split_invariance(split):
     gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, split)
