@@ -24,6 +24,21 @@
  *     library clears what it needs inside the call, so ws may hold anything on entry, but
  *     two calls that run concurrently must not share one ws.
  *   - o must not alias an input.
+ *   - Precondition of every call that runs causal linear attention on the tensor-core path
+ *     (gformer_causal_linear_attn*, gformer_hybrid_attn*): when the plan cuts a chain into
+ *     segments (gformer_linear_plan reports more than one), the kernel's CTAs -- at most one per
+ *     SM, never more than the device has SMs -- wait for one another's states, so all of them
+ *     must get an SM while the kernel runs.  On a device that is otherwise idle, or shared with
+ *     kernels that end by themselves, they do.  Two such calls on different streams (or from two
+ *     host threads) may overlap: each kernel's CTAs then start as the other's finish, and a
+ *     segment's predecessor always belongs to a CTA with a lower index, which the hardware
+ *     starts first (observed on B200; CUDA does not promise an order), so the waits still end.
+ *     What must not run beside such a call is work that
+ *     holds SMs until the call has finished (a persistent kernel that itself waits for this
+ *     call's results): the waits are bounded, so the outcome is GF_ERR_TIMEOUT from
+ *     gformer_last_device_status and undefined outputs, not a hang.  Whole chains (one segment),
+ *     the windowed heads and the bidirectional layer have no such precondition: their CTAs
+ *     never wait for other CTAs.
  */
 #ifndef GFORMER_H_
 #define GFORMER_H_
