@@ -84,7 +84,7 @@ def measured_peaks():
 
 
 def recorded_traffic(workload):
-    """DRAM bytes per launch from the committed ncu capture, if one is recorded."""
+    """DRAM bytes per launch of the workload's kernels ({kernel: bytes}) from the committed ncu captures, if recorded."""
     p = os.path.join(ROOT, "profiles", "traffic.json")
     if os.path.exists(p):
         with open(p) as f:
@@ -533,6 +533,8 @@ def run_ours(args, c, rank, world, local_rank):
         else:
             dom, dom_bytes, achieved = "gformer_hybrid_attn step", abytes, step_gbs
             dom_desc = "whole step (both kernels)"
+        traffic = recorded_traffic(args.workload) or {}
+        step_traffic = sum(traffic.values()) if traffic and not favor and all(v is not None for v in traffic.values()) else None
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -546,11 +548,20 @@ def run_ours(args, c, rank, world, local_rank):
                        if n_sets == 1 else
                        ("inputs fit the L2 (%.0f MB of %.0f MB): steps rotate over %d buffer sets so that they read HBM; "
                         "the L2-resident figure is in l2_resident" % (set_bytes / 1e6, l2 / 1e6, n_sets))},
-            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                         "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
-                         "traffic": recorded_traffic(args.workload),
-                         "peak_source": which + " copy bandwidth", "algorithmic_bytes": dom_bytes,
-                         "kernel": dom_desc, "kernels": kern,
+            # The headline figure is the whole layer's (what the target is phrased for): its algorithmic
+            # bytes over the step time.  The kernel that takes most of the step, timed alone, is the
+            # sub-entry `dominant_kernel`; `traffic` is the DRAM bytes of a step's kernels from the
+            # committed ncu captures.
+            "roofline": {"bound": "hbm", "achieved": step_gbs, "peak": peak, "unit": "GB/s",
+                         "frac": step_gbs / peak, "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS,
+                         "traffic": step_traffic, "peak_source": which + " copy bandwidth",
+                         "algorithmic_bytes": abytes,
+                         "kernel": "whole layer: every kernel of a step (see kernels), CUDA events around the step",
+                         "tflops_algorithmic": algorithmic_flops(c, h0) / mean_launch_s / 1e12,
+                         "dominant_kernel": {"name": dom, "how": dom_desc, "achieved": achieved, "frac": achieved / peak,
+                                             "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+                                             "algorithmic_bytes": dom_bytes, "traffic": traffic.get(dom)},
+                         "kernels": kern,
                          "step": {"achieved": step_gbs, "frac": step_gbs / peak,
                                   "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS, "algorithmic_bytes": abytes,
                                   "tflops_algorithmic": algorithmic_flops(c, h0) / mean_launch_s / 1e12}},
