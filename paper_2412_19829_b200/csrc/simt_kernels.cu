@@ -299,6 +299,54 @@ __global__ void export_ring_kernel(const T* __restrict__ k, const T* __restrict_
 // ------------------------------------------------------------------------------------
 // Decode step: one CTA per (b, h).
 // ------------------------------------------------------------------------------------
+// A 16-byte load that stays where it is written: two of them in a row are both in flight before the
+// first use (left to itself the compiler, short of registers, pairs every load with its use).
+__device__ __forceinline__ uint4 ld16_in_order(const void* p) {
+  uint4 r;
+  asm volatile("ld.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p) : "memory");
+  return r;
+}
+// 16 bytes of a ring row (4 floats or 8 bf16) against the matching entries of a vector in shared memory
+template <typename T> struct Row16;
+template <> struct Row16<float> {
+  static constexpr int kElems = 4;
+  static __device__ __forceinline__ float dot(uint4 raw, const float* qv) {
+    const float4 q4 = *reinterpret_cast<const float4*>(qv);
+    return __uint_as_float(raw.x) * q4.x + __uint_as_float(raw.y) * q4.y + __uint_as_float(raw.z) * q4.z +
+           __uint_as_float(raw.w) * q4.w;
+  }
+  static __device__ __forceinline__ void axpy(uint4 raw, float p, float* acc) {
+    acc[0] = fmaf(p, __uint_as_float(raw.x), acc[0]);
+    acc[1] = fmaf(p, __uint_as_float(raw.y), acc[1]);
+    acc[2] = fmaf(p, __uint_as_float(raw.z), acc[2]);
+    acc[3] = fmaf(p, __uint_as_float(raw.w), acc[3]);
+  }
+};
+template <> struct Row16<__nv_bfloat16> {
+  static constexpr int kElems = 8;
+  static __device__ __forceinline__ float dot(uint4 raw, const float* qv) {
+    const float4 qa = *reinterpret_cast<const float4*>(qv), qb = *reinterpret_cast<const float4*>(qv + 4);
+    float a0 = __uint_as_float(raw.x << 16) * qa.x, a1 = __uint_as_float(raw.x & 0xffff0000u) * qa.y;
+    a0 = fmaf(__uint_as_float(raw.y << 16), qa.z, a0);
+    a1 = fmaf(__uint_as_float(raw.y & 0xffff0000u), qa.w, a1);
+    a0 = fmaf(__uint_as_float(raw.z << 16), qb.x, a0);
+    a1 = fmaf(__uint_as_float(raw.z & 0xffff0000u), qb.y, a1);
+    a0 = fmaf(__uint_as_float(raw.w << 16), qb.z, a0);
+    a1 = fmaf(__uint_as_float(raw.w & 0xffff0000u), qb.w, a1);
+    return a0 + a1;
+  }
+  static __device__ __forceinline__ void axpy(uint4 raw, float p, float* acc) {
+    acc[0] = fmaf(p, __uint_as_float(raw.x << 16), acc[0]);
+    acc[1] = fmaf(p, __uint_as_float(raw.x & 0xffff0000u), acc[1]);
+    acc[2] = fmaf(p, __uint_as_float(raw.y << 16), acc[2]);
+    acc[3] = fmaf(p, __uint_as_float(raw.y & 0xffff0000u), acc[3]);
+    acc[4] = fmaf(p, __uint_as_float(raw.z << 16), acc[4]);
+    acc[5] = fmaf(p, __uint_as_float(raw.z & 0xffff0000u), acc[5]);
+    acc[6] = fmaf(p, __uint_as_float(raw.w << 16), acc[6]);
+    acc[7] = fmaf(p, __uint_as_float(raw.w & 0xffff0000u), acc[7]);
+  }
+};
+
 __device__ __forceinline__ float block_reduce(float x, bool is_max, float* scratch /* 33 floats */) {
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
 #pragma unroll
@@ -331,11 +379,14 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
                    int h_sparse, float scale, const T* __restrict__ W /* [H - h_sparse, D, D] or null: elu + 1 */) {
   constexpr int D4 = D / 4;
   constexpr int G = 256 / D4;  // thread groups along the reduced dimension
+  // windowed heads: a ring row is read 16 bytes per thread (a slot's round trip to L2 is what a step
+  // waits for, so the fewer rounds the better): TPS threads per slot, GW slots per round
+  constexpr int EPT = Row16<T>::kElems, TPS = D / EPT, GW = 256 / TPS;
   extern __shared__ __align__(16) float dyn[];  // window heads: w scores
   __shared__ __align__(16) float qs[D];
   __shared__ __align__(16) float ks[D];
   __shared__ float scratch[33];
-  __shared__ __align__(16) float part[G][D];
+  __shared__ __align__(16) float part[GW][D];  // GW >= G
 
   const int h = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const long long io = ((long long)b * H + h) * D;
@@ -389,25 +440,33 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
       vcb[(long long)cur * D + tid] = vin;
     }
     __syncthreads();
-    // scores: D/4 threads per slot (a warp reads whole cache lines of the ring), partial dot
-    // products reduced over the group by shuffles; slot `cur` is read from the step input (same
-    // values).  D/4 is 16 or 32, so a group never straddles a warp.
+    // scores: TPS threads per slot (a warp reads whole cache lines of the ring), partial dot products
+    // reduced over the group by shuffles; slot `cur` is read from the step input (same values).  TPS is
+    // 8, 16 or 32, so a group never straddles a warp.
+    const int cw = tid % TPS, gw = tid / TPS;
     float mloc = -INFINITY;
-    const float4 qq = *reinterpret_cast<const float4*>(&qs[4 * c4]);
-    for (int s0 = 0; s0 < nvalid; s0 += G) {  // uniform trip count: the shuffles below are warp-wide
-      const int s = s0 + grp;
-      float acc = 0.f;
-      if (s < nvalid) {
-        const T* kr = (s == cur) ? (k + io) : (kcb + (long long)s * D);
-        const float4 kk = Vec4<T>::load(kr + 4 * c4);
-        acc = qq.x * kk.x + qq.y * kk.y + qq.z * kk.z + qq.w * kk.w;
-      }
+    for (int s0 = 0; s0 < nvalid; s0 += 2 * GW) {  // uniform trip count: the shuffles below are warp-wide
+      const int sa = s0 + gw, sb = s0 + GW + gw;
+      uint4 ra = make_uint4(0u, 0u, 0u, 0u), rb = ra;
+      if (sa < nvalid) ra = ld16_in_order(((sa == cur) ? (k + io) : (kcb + (long long)sa * D)) + EPT * cw);
+      if (sb < nvalid) rb = ld16_in_order(((sb == cur) ? (k + io) : (kcb + (long long)sb * D)) + EPT * cw);
+      float acc_a = Row16<T>::dot(ra, &qs[EPT * cw]), acc_b = Row16<T>::dot(rb, &qs[EPT * cw]);
 #pragma unroll
-      for (int off = D4 / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
-      if (s < nvalid && c4 == 0) {
-        acc *= scale;
-        dyn[s] = acc;
-        mloc = fmaxf(mloc, acc);
+      for (int off = TPS / 2; off > 0; off >>= 1) {
+        acc_a += __shfl_xor_sync(0xffffffffu, acc_a, off);
+        acc_b += __shfl_xor_sync(0xffffffffu, acc_b, off);
+      }
+      if (cw == 0) {
+        if (sa < nvalid) {
+          acc_a *= scale;
+          dyn[sa] = acc_a;
+          mloc = fmaxf(mloc, acc_a);
+        }
+        if (sb < nvalid) {
+          acc_b *= scale;
+          dyn[sb] = acc_b;
+          mloc = fmaxf(mloc, acc_b);
+        }
       }
     }
     const float mx = block_reduce(mloc, true, scratch);
@@ -418,22 +477,24 @@ decode_step_kernel(const T* __restrict__ q, const T* __restrict__ k, const T* __
       lloc += p;
     }
     const float lsum = block_reduce(lloc, false, scratch);  // barriers inside publish dyn[]
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s = grp; s < nvalid; s += G) {
-      const T* vr = (s == cur) ? (v + io) : (vcb + (long long)s * D);
-      const float4 vv = Vec4<T>::load(vr + 4 * c4);
-      const float p = dyn[s];
-      acc.x += p * vv.x;
-      acc.y += p * vv.y;
-      acc.z += p * vv.z;
-      acc.w += p * vv.w;
+    float accv[EPT];
+#pragma unroll
+    for (int e = 0; e < EPT; ++e) accv[e] = 0.f;
+    for (int sa = gw; sa < nvalid; sa += 2 * GW) {
+      const int sb = sa + GW;
+      uint4 ra = ld16_in_order(((sa == cur) ? (v + io) : (vcb + (long long)sa * D)) + EPT * cw), rb = make_uint4(0u, 0u, 0u, 0u);
+      if (sb < nvalid) rb = ld16_in_order(((sb == cur) ? (v + io) : (vcb + (long long)sb * D)) + EPT * cw);
+      Row16<T>::axpy(ra, dyn[sa], accv);
+      Row16<T>::axpy(rb, sb < nvalid ? dyn[sb] : 0.f, accv);
     }
-    *reinterpret_cast<float4*>(&part[grp][4 * c4]) = acc;
+#pragma unroll
+    for (int e = 0; e < EPT; e += 4)
+      *reinterpret_cast<float4*>(&part[gw][EPT * cw + e]) = make_float4(accv[e], accv[e + 1], accv[e + 2], accv[e + 3]);
     __syncthreads();
     if (tid < D) {
       float sum = 0.f;
 #pragma unroll
-      for (int gi = 0; gi < G; ++gi) sum += part[gi][tid];
+      for (int gi = 0; gi < GW; ++gi) sum += part[gi][tid];
       o[io + tid] = from_f32<T>(sum / lsum);
     }
   } else {
