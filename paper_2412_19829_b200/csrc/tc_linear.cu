@@ -1112,6 +1112,21 @@ void plan_range(int nchains, int nch, int* g_min_out, int* g_max_out) {
 }  // namespace
 
 namespace {
+// Bytes of parked tiles that stay in L2 while a round of items runs: about 0.6 of the cache (80 MB of
+// a B200's 126 MiB).  Asked of the current device once; the B200 figure when there is no device (the
+// plan can be queried on a machine without one).
+double l2_park_bytes() {
+  static double cached = 0.0;  // (a benign race: every writer stores the same value)
+  if (cached == 0.0) {
+    int dev = 0, l2 = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev) == cudaSuccess &&
+        l2 > 0)
+      cached = 0.6056 * (double)l2;
+    else
+      cached = 80e6;
+  }
+  return cached;
+}
 // Best two-pass plan for nchains chains of nch chunks: its cost in two-pass chunks (1e300 and
 // *G_out = 1 when the chains are too short to cut).
 double best_cut(int nchains, int nch, int d, int kPlanSMs, int* G_out) {
@@ -1123,10 +1138,10 @@ double best_cut(int nchains, int nch, int d, int kPlanSMs, int* G_out) {
       const long long items = (long long)nchains * g;
       const long long rounds = (items + kPlanSMs - 1) / kPlanSMs;
       const double L = (double)nch / g;
-      // What the running CTAs park at one time should stay in L2 (about 80 MB of its 126 MB): of a
+      // What the running CTAs park at one time should stay in L2 (l2_park_bytes): of a
       // longer segment the excess comes back from DRAM, up to 40 % more time per chunk when the
       // rounds bound the time (when the serial chain does, DRAM has slack and nothing is charged).
-      const double l_cap = 80e6 / ((double)(items < kPlanSMs ? items : kPlanSMs) * 4.0 * 128.0 * d);
+      const double l_cap = l2_park_bytes() / ((double)(items < kPlanSMs ? items : kPlanSMs) * 4.0 * 128.0 * d);
       const double spill = L > l_cap ? 1.0 + 0.4 * (1.0 - l_cap / L) : 1.0;
       const double by_rounds = (double)rounds * (L + handover_cost(d)) * spill, by_chain = L + 0.65 * g;
       const double cost = by_rounds > by_chain ? by_rounds : by_chain;
