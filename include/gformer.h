@@ -336,6 +336,10 @@ int gformer_hybrid_attn_self_w(const void* q, const void* k, const void* v, void
                                void* ws, size_t ws_bytes, void* cuda_stream);
 int gformer_decode_step_w(const void* q, const void* k, const void* v, void* o,
                           gf_decode_state* st, float scale, int phi, const void* W, void* cuda_stream);
+/* gformer_decode_step_ragged with the feature map's parameter (W as above). */
+int gformer_decode_step_ragged_w(const void* q, const void* k, const void* v, void* o,
+                                 gf_decode_state* st, long long* t_seq, float scale, int phi, const void* W,
+                                 void* cuda_stream);
 
 #ifdef __cplusplus
 }

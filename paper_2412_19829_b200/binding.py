@@ -100,6 +100,8 @@ def lib() -> ctypes.CDLL:
         L.gformer_decode_step.argtypes = [vp, vp, vp, vp, ctypes.POINTER(DecodeStateC), f, i, vp]
         L.gformer_decode_step_ragged.restype = i
         L.gformer_decode_step_ragged.argtypes = [vp, vp, vp, vp, ctypes.POINTER(DecodeStateC), vp, f, i, vp]
+        L.gformer_decode_step_ragged_w.restype = i
+        L.gformer_decode_step_ragged_w.argtypes = [vp, vp, vp, vp, ctypes.POINTER(DecodeStateC), vp, f, i, vp, vp]
         _lib = L
     return _lib
 
@@ -396,18 +398,20 @@ def decode_step(q, k, v, st: DecodeState, scale: float = 0.0, out=None, stream=N
     return o
 
 
-def decode_step_ragged(q, k, v, st: DecodeState, t_seq: torch.Tensor, scale: float = 0.0, out=None, stream=None):
-    """gformer_decode_step_ragged: sequence b of the batch is at position t_seq[b] (int64 CUDA
-    tensor of B entries, negative = idle slot); the positions are advanced on the device."""
+def decode_step_ragged(q, k, v, st: DecodeState, t_seq: torch.Tensor, scale: float = 0.0, out=None, stream=None,
+                       W=None):
+    """gformer_decode_step_ragged(_w): sequence b of the batch is at position t_seq[b] (int64 CUDA
+    tensor of B entries, negative = idle slot); the positions are advanced on the device.  W as in hybrid_attn."""
     for t in (q, k, v):
         if not (t.is_cuda and t.is_contiguous() and t.dim() == 3):
             raise ValueError("q, k, v must be contiguous [B, H, d] CUDA tensors")
     if not (t_seq.is_cuda and t_seq.dtype == torch.int64 and t_seq.is_contiguous() and t_seq.numel() == q.shape[0]):
         raise ValueError("t_seq must be a contiguous int64 CUDA tensor with one entry per sequence")
     o = torch.empty_like(q) if out is None else out
-    rc = lib().gformer_decode_step_ragged(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
-                                          ctypes.byref(st.c), t_seq.data_ptr(), float(scale), GF_PHI_ELU1,
-                                          _stream_ptr(stream))
+    phi, wp = _phi_args(W, q, st.c.H - st.c.h_sparse, st.c.d)
+    rc = lib().gformer_decode_step_ragged_w(q.data_ptr(), k.data_ptr(), v.data_ptr(), o.data_ptr(),
+                                            ctypes.byref(st.c), t_seq.data_ptr(), float(scale), phi, wp,
+                                            _stream_ptr(stream))
     if rc != GF_OK:
-        raise GformerError(rc, "gformer_decode_step_ragged")
+        raise GformerError(rc, "gformer_decode_step_ragged_w")
     return o

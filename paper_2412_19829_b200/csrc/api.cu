@@ -538,10 +538,15 @@ int gformer_decode_step_w(const void* q, const void* k, const void* v, void* o, 
 
 int gformer_decode_step_ragged(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
                                long long* t_seq, float scale, int phi, void* cuda_stream) {
+  if (phi == GF_PHI_FAVOR_POS) return GF_ERR_INVALID_ARG;  // needs its projections: gformer_decode_step_ragged_w
+  return gformer_decode_step_ragged_w(q, k, v, o, st, t_seq, scale, phi, nullptr, cuda_stream);
+}
+
+int gformer_decode_step_ragged_w(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,
+                                 long long* t_seq, float scale, int phi, const void* W, void* cuda_stream) {
   if (!t_seq || (reinterpret_cast<uintptr_t>(t_seq) & 7u) != 0) return GF_ERR_INVALID_ARG;
   if (st && st->H > 4096) return GF_ERR_UNSUPPORTED;  // the arrival count of a sequence's heads has 15 bits
-  if (phi == GF_PHI_FAVOR_POS) return GF_ERR_INVALID_ARG;
-  return decode_step_impl(q, k, v, o, st, t_seq, scale, phi, nullptr, cuda_stream);
+  return decode_step_impl(q, k, v, o, st, t_seq, scale, phi, W, cuda_stream);
 }
 
 static int decode_step_impl(const void* q, const void* k, const void* v, void* o, gf_decode_state* st,

@@ -287,6 +287,15 @@ def test_ragged_decode_argument_errors():
         gf.GF_ERR_INVALID_ARG
     assert L.gformer_decode_step_ragged(a[0], a[1], a[2], 0, ctypes.byref(st), FAKE + (8 << 20), 0.0, gf.GF_PHI_ELU1,
                                         None) == gf.GF_ERR_INVALID_ARG
+    # the feature map and its parameter go together, here as everywhere
+    assert L.gformer_decode_step_ragged(*a, ctypes.byref(st), FAKE + (8 << 20), 0.0, gf.GF_PHI_FAVOR_POS, None) == \
+        gf.GF_ERR_INVALID_ARG
+    assert L.gformer_decode_step_ragged_w(*a, ctypes.byref(st), FAKE + (8 << 20), 0.0, gf.GF_PHI_FAVOR_POS, None,
+                                          None) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_decode_step_ragged_w(*a, ctypes.byref(st), FAKE + (8 << 20), 0.0, gf.GF_PHI_ELU1, FAKE + (9 << 20),
+                                          None) == gf.GF_ERR_INVALID_ARG
+    assert L.gformer_decode_step_ragged_w(*a, ctypes.byref(st), None, 0.0, gf.GF_PHI_FAVOR_POS, FAKE + (9 << 20),
+                                          None) == gf.GF_ERR_INVALID_ARG
     assert st.t == 0
 
 

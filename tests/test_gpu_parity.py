@@ -1059,6 +1059,37 @@ def test_favor_hybrid_layer_prefill_then_decode(B, H, N, d, w, h0):
         check(f64(ot), ref[:, :, t], "bf16", f"favor decode step {t - N}")
 
 
+def test_favor_ragged_decode_matches_every_sequence_alone():
+    # three slots at different positions (one prefilled past the window, one from scratch, one idle) under the
+    # positive random features: every sequence against the oracle's layer on that sequence alone
+    B, H, d, w, h0, steps = 3, 4, 64, 24, 1, 12
+    W = _proj(H - h0, d, "bf16", seed=871)
+    Wd = W.cuda()
+    lens = [steps, 70 + steps, 0]
+    seqs = [synth.qkv(1, H, max(n, 1), d, "bf16", seed=872 + i) for i, n in enumerate(lens)]
+    refs = [oracle.hybrid_attn(f64(q), f64(k), f64(v), w, h_sparse=h0, W=f64(W)) for q, k, v in seqs]
+    st = gf.DecodeState(B, H, d, w, h0)
+    t_seq = torch.tensor([0, 70, -1], dtype=torch.int64, device="cuda")
+    q1, k1, v1 = dev(*seqs[1])
+    ws = gf.Workspace.for_problem(1, H, 70, d, w, h0, phi=gf.GF_PHI_FAVOR_POS)
+    gf.hybrid_attn(q1[:, :, :70].contiguous(), k1[:, :, :70].contiguous(), v1[:, :, :70].contiguous(), w, h_sparse=h0,
+                   state_out=_alias_state(st, 1), W=Wd, ws=ws)
+    assert ws.last_device_status() == gf.GF_OK
+    pos, got = [0, 70, 0], [[], [], []]
+    for step in range(steps):
+        qs = torch.zeros(B, H, d, dtype=torch.bfloat16); ks = torch.zeros_like(qs); vs = torch.zeros_like(qs)
+        for b in range(2):
+            qs[b], ks[b], vs[b] = (x[0, :, pos[b]] for x in seqs[b])
+        o = gf.decode_step_ragged(qs.cuda(), ks.cuda(), vs.cuda(), st, t_seq, W=Wd)
+        for b in range(2):
+            got[b].append(o[b].cpu()); pos[b] += 1
+        assert torch.count_nonzero(o[2]) == 0
+    assert t_seq.tolist() == [steps, 70 + steps, -1]
+    for b, first in ((0, 0), (1, 70)):
+        out = torch.stack(got[b], dim=1).unsqueeze(0)
+        assert_parity(f64(out), refs[b][:, :, first:lens[b]], "bf16", f"favor ragged decode, slot {b}")
+
+
 @pytest.mark.parametrize("B,H,N,d,w,h0", [(1, 4, 1000, 128, 128, 1), (2, 3, 300, 64, 40, 1), (1, 2, 4096, 64, 64, 0)])
 def test_favor_self_layer(B, H, N, d, w, h0):
     q, k, v = synth.qkv(B, H, N, d, "bf16", seed=840 + N)
