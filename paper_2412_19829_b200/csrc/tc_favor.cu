@@ -43,8 +43,9 @@ favor_tc_kernel(const __grid_constant__ CUtensorMap mxq, const __grid_constant__
   __shared__ __align__(8) uint64_t full, done;
   __shared__ uint32_t tmem_base_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int i0 = blockIdx.x * 128;
-  const int hl = blockIdx.y % p.h_count, b = blockIdx.y / p.h_count;
+  // (the (batch, head) index is the x coordinate of the grid, which has the range for it)
+  const int i0 = blockIdx.y * 128;
+  const int hl = blockIdx.x % p.h_count, b = blockIdx.x / p.h_count;
   const bool is_k = blockIdx.z != 0;
   const CUtensorMap* mx = is_k ? &mxk : &mxq;
   const CUtensorMap* mf = is_k ? &mfk : &mfq;
@@ -169,9 +170,9 @@ cudaError_t launch_favor_features_tc(const void* q, const void* k, const void* W
   p.h_begin = h_begin;
   p.h_count = h_count;
   p.status = &ws->status;
-  const long long rows = (long long)B * h_count;
-  if (rows > 65535) return cudaErrorInvalidValue;
-  dim3 grid((unsigned)((N + 127) / 128), (unsigned)rows, 2);
+  const long long rows = (long long)B * h_count, tiles = ((long long)N + 127) / 128;
+  if (rows > 0x7fffffffLL || tiles > 65535) return cudaErrorInvalidValue;  // (tiles: more than 8 million tokens)
+  dim3 grid((unsigned)rows, (unsigned)tiles, 2);
   auto launch = [&](auto kern, int smem) -> cudaError_t {
     int dev = 0, sms = 0;
     cudaError_t err = device_info(&dev, &sms);
