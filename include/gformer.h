@@ -29,13 +29,14 @@
  *     segments (gformer_linear_plan reports more than one), the kernel's CTAs -- at most one per
  *     SM, never more than the device has SMs -- wait for one another's states, so all of them
  *     must get an SM while the kernel runs.  On a device that is otherwise idle, or shared with
- *     kernels that end by themselves, they do.  Two such calls on different streams (or from two
- *     host threads) may overlap: each kernel's CTAs then start as the other's finish, and a
- *     segment's predecessor always belongs to a CTA with a lower index, which the hardware
- *     starts first (observed on B200; CUDA does not promise an order), so the waits still end.
- *     What must not run beside such a call is work that
- *     holds SMs until the call has finished (a persistent kernel that itself waits for this
- *     call's results): the waits are bounded, so the outcome is GF_ERR_TIMEOUT from
+ *     kernels that end by themselves, they do.  Two such kernels side by side could each hold a
+ *     part of the SMs and wait for the rest, so the library orders them per device: such a kernel
+ *     starts only when the previous one -- from whatever stream or host thread -- has finished
+ *     (an event wait in front of the launch).  Inside a stream capture that wait is not possible:
+ *     graphs that contain such a call must not be replayed side by side on one device.  What must
+ *     not run beside such a call is work that holds SMs until the call has finished (a persistent
+ *     kernel that itself waits for this call's results): the waits are bounded, so the outcome is
+ *     GF_ERR_TIMEOUT from
  *     gformer_last_device_status and undefined outputs, not a hang.  Whole chains (one segment),
  *     the windowed heads and the bidirectional layer have no such precondition: their CTAs
  *     never wait for other CTAs.

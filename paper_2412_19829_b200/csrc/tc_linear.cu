@@ -43,6 +43,8 @@
 // no parking and no hand-over; the phi warps transform each K tile in place one chunk ahead of
 // the chunk pipeline (four K slots at D = 64).
 // Every wait is bounded; on expiry the kernel records a status word and drains.
+#include <mutex>
+
 #include "common.cuh"
 #include "sm100.cuh"
 
@@ -1255,6 +1257,19 @@ size_t linear_tc_workspace_bytes(int nchains, int N, int d, int split) {
          (size_t)plan_slots_max(nchains, N, split) * ((size_t)128 * d + d) * sizeof(float);
 }
 
+namespace {
+// The CTAs of a cut-chain launch wait for one another, so two such kernels must not share the SMs: each
+// could hold some of them while its own unplaced CTAs wait for the rest.  Per device the launches are
+// therefore chained by an event: a cut-chain kernel starts only when the previous one, from whatever
+// stream or host thread, has finished.  (Not inside a stream capture, where an outside event cannot be
+// waited for: there the order of the caller's graphs applies.)
+struct CutChainOrder {
+  std::mutex mu;
+  cudaEvent_t last[64] = {};
+};
+CutChainOrder g_cut_order;
+}  // namespace
+
 cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* o, int B, int H, int N, int d,
                              int layout, int h_begin, int h_count, float* S_io, float* z_io, bool zero_init,
                              int split, int max_ctas, WsHeader* ws, cudaStream_t stream, bool shared,
@@ -1297,9 +1312,24 @@ cudaError_t launch_linear_tc(const void* q, const void* k, const void* v, void* 
     if (err != cudaSuccess) return err;
     dim3 grid(p.nitems < sms ? p.nitems : sms);
     if (first_grid && *first_grid == 0) *first_grid = (int)grid.x;
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (p.G > 1 && (err = cudaStreamIsCapturing(stream, &capturing)) != cudaSuccess) return err;
+    const bool chained = p.G > 1 && capturing == cudaStreamCaptureStatusNone;
+    std::unique_lock<std::mutex> order;
+    if (chained) {
+      order = std::unique_lock<std::mutex>(g_cut_order.mu);
+      cudaEvent_t& ev = g_cut_order.last[dev];
+      if (ev == nullptr) {
+        if ((err = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming)) != cudaSuccess) return err;
+      } else if ((err = cudaStreamWaitEvent(stream, ev, 0)) != cudaSuccess) {
+        return err;
+      }
+    }
     kern<<<grid, kThreads, smem, stream>>>(mq, mk, mv, mo, p);
     note_launch();
-    return cudaGetLastError();
+    err = cudaGetLastError();
+    if (chained && err == cudaSuccess) err = cudaEventRecord(g_cut_order.last[dev], stream);
+    return err;
   };
   // Chains [chain0, chain0 + count) of the call in one launch: whole (the one-pass form of the kernel) or cut
   // into g segments (the two-pass form).  The one-pass form neither reads nor writes the hand-over scratch.

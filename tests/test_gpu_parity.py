@@ -283,6 +283,41 @@ def test_hybrid_with_whole_and_cut_linear_chains_and_state_export():
     assert errors(f64(st.z[:, idx].cpu()), zr)["rel_l2"] <= 1e-2
 
 
+def test_cut_chain_calls_from_two_streams_and_two_threads():
+    """Calls whose chains are cut into segments (CTAs that wait for one another) issued at the same time from
+    two host threads on two streams: the library runs such kernels one after the other on a device, so every
+    call ends with a clean status and the oracle's values, with nothing to synchronise on the caller's side."""
+    import threading
+    B, H, N, d = 1, 10, 4 * 1024, 128
+    gf.set_tuning(gf.GF_TUNE_LINEAR_SPLIT, 1)  # 32 segments per chain: 320 items, more than two rounds of the CTAs
+    assert gf.linear_plan(B * H, N, d) == (32, 1)
+    data = [synth.qkv(B, H, N, d, "bf16", seed=660 + i, gain=1.0) for i in range(2)]
+    refs = [oracle.causal_linear_attn(f64(q), f64(k), f64(v)) for q, k, v in data]
+    devs = [dev(*x) for x in data]
+    outs = [[None] * 6 for _ in range(2)]
+    status = [None, None]
+
+    def worker(i):
+        torch.cuda.set_device(0)
+        stream = torch.cuda.Stream()
+        ws = [gf.Workspace.for_problem(B, H, N, d, 1, 0) for _ in range(6)]
+        with torch.cuda.stream(stream):
+            for r in range(6):
+                outs[i][r] = gf.causal_linear_attn(*devs[i], ws=ws[r], stream=stream)
+        stream.synchronize()
+        status[i] = [w.last_device_status(stream) for w in ws]
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    for i in range(2):
+        assert status[i] == [gf.GF_OK] * 6
+        for r in range(6):
+            assert_parity(f64(outs[i][r]), refs[i], "bf16", f"thread {i}, call {r}")
+
+
 @pytest.mark.parametrize("d", [64, 128])
 def test_linear_chunk_size_invariance(d):
     """Algorithm 1 regrouped in different ways gives the same values up to rounding: token by token
